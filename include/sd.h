@@ -1,0 +1,241 @@
+/*
+ * sd.h - C ABI of the speculative-decoding hot path for one B200 (sm_100a).
+ *
+ * The library runs the online half of task-routed heterogeneous speculative
+ * decoding: route a prompt to one of several draft models, let that draft
+ * propose gamma tokens one after the other, score them with one parallel pass
+ * of the target model, accept or reject them, and forget the rejected part of
+ * both KV caches.  Notation follows the paper: gamma = tokens drafted per
+ * iteration, alpha = draft/target agreement, c = cost of one draft pass over
+ * one target pass (Eq. 1), tau = tokens emitted per target pass (Sec. 3.1).
+ *
+ * Conventions that hold for every call:
+ *  - the return value is an sd_status; argument and capacity errors are found
+ *    on the host before anything is launched;
+ *  - work is enqueued on the CUDA stream given at sd_create and the call
+ *    returns without waiting, unless its comment says "synchronises";
+ *  - "device" pointers are CUDA device addresses valid on the current device,
+ *    "host" pointers are ordinary memory; the caller owns every buffer it
+ *    passes and the library keeps no pointer past the call, except the arena
+ *    and the stream handed to sd_create;
+ *  - the library owns its weight copies, KV caches and per-sequence state, all
+ *    carved out of the caller's arena; it never allocates device memory;
+ *  - nothing traps: a kernel that meets an impossible value (a token id out of
+ *    range, a position past the cache) skips the access and sets a bit in a
+ *    status word that sd_device_status returns.
+ */
+#ifndef SD_H
+#define SD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd_ctx sd_ctx;
+
+typedef enum {
+    SD_OK = 0,
+    SD_ERR_INVALID_ARG = 1,
+    SD_ERR_STATE = 2,        /* call out of order for that sequence */
+    SD_ERR_CAPACITY = 3,     /* KV cache, batch or row limit would be exceeded */
+    SD_ERR_OOM = 4,          /* arena too small */
+    SD_ERR_CUDA = 5,
+    SD_ERR_TIMEOUT = 6,
+    SD_ERR_UNSUPPORTED = 7
+} sd_status;
+
+enum { SD_F32 = 0, SD_BF16 = 1 };
+
+#define SD_MAX_BATCH 64      /* sequences per call */
+#define SD_MAX_ROWS 256      /* query rows per forward pass: n_seq * (gamma + 1) */
+#define SD_MAX_GAMMA 15
+
+/* bits of the device status word */
+#define SD_DEV_BAD_TOKEN 1u      /* token id outside [0, vocab) */
+#define SD_DEV_BAD_POS 2u        /* position outside the KV cache */
+#define SD_DEV_BAD_NACC 4u       /* n_acc outside [0, gamma] at rollback */
+#define SD_DEV_WAIT_EXPIRED 8u   /* a bounded wait inside a kernel gave up */
+
+/* Decoder-only transformer of the LLaMA family (the paper's target and drafts,
+ * Sec. 3.1): RMSNorm, rotary position embedding (pairs (i, i + head_dim/2)),
+ * grouped-query attention, SwiGLU feed-forward, no biases, untied lm_head. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t dtype;           /* SD_F32 or SD_BF16: storage of weights, activations, KV */
+    float rms_eps;
+    float rope_base;
+} sd_model_desc;
+
+typedef struct {
+    int32_t max_seqs;        /* sequence slots, <= SD_MAX_BATCH */
+    int32_t max_ctx;         /* KV positions per sequence */
+    int32_t max_gamma;       /* <= SD_MAX_GAMMA */
+    int32_t n_drafts;        /* K heterogeneous drafts; models[0] is the target, models[1..K] the drafts */
+    float temperature;       /* same for draft and target; 0 = greedy */
+    uint64_t seed;           /* Philox4x32-10 key */
+    int32_t clf_d_hidden;    /* prompt classifier d_model(target) -> clf_d_hidden -> n_drafts; 0 = none */
+    int32_t reserved;
+} sd_config;
+
+typedef struct {
+    int64_t iterations, drafted, accepted, emitted;   /* Eq. 2: accepted / drafted; tau = emitted / iterations */
+} sd_counters;
+
+/* tensor kinds for sd_load_tensor; matrices are row-major [out_features][in_features] */
+enum {
+    SD_T_EMBED = 0, SD_T_LM_HEAD = 1, SD_T_FINAL_NORM = 2,
+    SD_T_WQ = 3, SD_T_WK = 4, SD_T_WV = 5, SD_T_WO = 6, SD_T_WG = 7, SD_T_WU = 8, SD_T_WD = 9,
+    SD_T_NORM1 = 10, SD_T_NORM2 = 11
+};
+
+/* ---------------------------------------------------------------- lifecycle */
+
+/* Bytes of device memory sd_create needs for this configuration (weights, KV
+ * caches, state, scratch).  models: 1 + n_drafts descriptors.  0 on bad input. */
+size_t sd_arena_bytes(const sd_config* cfg, const sd_model_desc* models);
+
+/* Creates a context on the current device.  arena: device memory of at least
+ * sd_arena_bytes, 256-byte aligned, owned by the caller and left alone by it
+ * until sd_destroy.  cuda_stream: a cudaStream_t (NULL = legacy default).
+ * Zeroes the state; weights are undefined until loaded.  Synchronises. */
+sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cuda_stream,
+                    void* arena_device, size_t arena_bytes, sd_ctx** out);
+sd_status sd_destroy(sd_ctx* ctx);
+
+/* Copies one tensor into the library's own layout.  model_id 0 = target,
+ * 1..K = drafts.  layer is ignored for SD_T_EMBED / LM_HEAD / FINAL_NORM.
+ * Matrices are in the model's dtype (bf16 as raw 16-bit patterns), norm gains
+ * are fp32.  src may be host (src_on_device = 0) or device memory. */
+sd_status sd_load_tensor(sd_ctx* ctx, int model_id, int kind, int layer, const void* src, int src_on_device);
+
+/* Prompt classifier, MLP variant of Sec. 3.3.3: fp32 w1 [h][d], b1 [h], w2 [K][h], b2 [K]. */
+sd_status sd_load_classifier(sd_ctx* ctx, const float* w1, const float* b1, const float* w2, const float* b2,
+                             int src_on_device);
+
+/* Starts sequence slot `seq` with a prompt (host, n_prompt >= 2 token ids) and
+ * a Philox stream id; resets its lengths, iteration counter and counters. */
+sd_status sd_seq_begin(sd_ctx* ctx, int seq, const int32_t* prompt_host, int n_prompt, uint32_t seq_id);
+
+/* Runs prompt tokens [0, n_prompt - 1) of each listed sequence through the
+ * target and through the sequence's routed draft so that both KV caches hold
+ * everything but the last prompt token.  Needs sd_route_prompt first. */
+sd_status sd_prefill(sd_ctx* ctx, const int32_t* seqs_host, int n_seq);
+
+/* ------------------------------------------------------- the five hot calls */
+
+/* Sec. 2.1 / 2.4: picks the draft model for each listed sequence.  A
+ * forced_task_host[i] >= 0 (task type given by the user) is taken as is; -1 (or
+ * a NULL array) runs the classifier on the prompt: mean of the target's
+ * embedding rows over the prompt -> FC + ReLU -> FC -> argmax (lowest index
+ * on ties).  draft_id_out_host may be NULL.  Synchronises (the draft id selects
+ * which weights later calls launch on). */
+sd_status sd_route_prompt(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, const int32_t* forced_task_host,
+                          int32_t* draft_id_out_host);
+
+/* Fig. 1(a): the routed draft proposes gamma tokens for each listed sequence,
+ * one autoregressive step after the other.  x_dev [n_seq][gamma] receives the
+ * tokens, q_dev [n_seq][gamma][vocab] the fp32 distributions they were drawn
+ * from (softmax(logits / T); one-hot when T = 0).  Sequences are grouped by
+ * draft internally; the first step also feeds the token the draft missed after
+ * a fully accepted iteration. */
+sd_status sd_draft_steps(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                         int32_t* x_dev, float* q_dev);
+
+/* Fig. 1(b): one pass of the target over [last token, x_0 .. x_{gamma-1}] of
+ * every listed sequence against its KV cache (keys/values of the gamma+1 rows
+ * are appended).  logits_dev [n_seq][gamma+1][vocab] fp32: row j is the
+ * target's prediction for the token after row j's input. */
+sd_status sd_verify(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                    const int32_t* x_dev, float* logits_dev);
+
+/* Sec. 3.1 (the stochastic verification rule of Leviathan et al. that the paper
+ * adopts): with p_j the target distribution of row j and q_s the draft's, slot s
+ * is accepted iff u_s * q_s(x_s) <= p_s(x_s) (one rounded fp32 multiply, u_s in
+ * (0,1] from Philox); n = number of leading accepted slots; the next token y is
+ * drawn from norm(max(0, p_n - q_n)) when n < gamma, from p_gamma otherwise,
+ * by an exact integer inverse CDF.  A pure function of its buffers. */
+typedef struct {
+    const float* target;     /* device [B][gamma+1][V]: logits (target_is_logits) or probabilities */
+    int32_t target_is_logits;/* 1: p = softmax(target / temperature) is computed inside the kernel */
+    const float* q;          /* device [B][gamma][V] draft probabilities */
+    const int32_t* x;        /* device [B][gamma] draft tokens */
+    int32_t B, gamma, V;
+    float temperature;       /* used with logits only; 0 = one-hot argmax */
+    uint64_t seed;           /* Philox key */
+    const uint32_t* iter;    /* device [B]: Philox counter word 0 of each row */
+    const uint32_t* seq_id;  /* device [B]: Philox counter word 2 of each row */
+    int32_t* n_acc;          /* device [B] out */
+    int32_t* out_tok;        /* device [B][gamma+1] out: x_0..x_{n-1}, y, then -1 */
+    void* cuda_stream;
+} sd_accept_args;
+sd_status sd_accept(const sd_accept_args* args);
+
+/* The same rule for sequences of a context: temperature, seed, iteration and
+ * stream ids come from the context's per-sequence state on the device. */
+sd_status sd_accept_seqs(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                         const float* target_logits_dev, const float* q_dev, const int32_t* x_dev,
+                         int32_t* n_acc_dev, int32_t* out_tok_dev);
+
+/* Commits an iteration: appends out_tok[0..n_acc] to each sequence, sets the
+ * target cache length to L + n_acc and the draft cache length to
+ * min(L + n_acc, L + gamma - 1) (L = length before the iteration), advances the
+ * iteration counter and the counters of Eq. 2.  No KV data moves: rejected
+ * positions stay where they are and the next append overwrites them. */
+sd_status sd_kv_rollback(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                         const int32_t* n_acc_dev, const int32_t* out_tok_dev);
+
+/* -------------------------------------------------------------- observation */
+
+/* Copies the sequence's tokens (up to cap) and counters to the host; also
+ * refreshes the host's capacity bookkeeping with the true length.  Synchronises. */
+sd_status sd_seq_read(sd_ctx* ctx, int seq, int32_t* tokens_host, int cap, int32_t* len_out, sd_counters* counters_out);
+
+/* Overrides a sequence's token history (host) so that a test can replay another
+ * run's iterations: keeps the KV caches, sets length to n_tokens, target cache
+ * length to n_tokens - 1 and the draft cache length to draft_kv_len. */
+sd_status sd_seq_force(sd_ctx* ctx, int seq, const int32_t* tokens_host, int n_tokens, int draft_kv_len, uint32_t iter);
+
+/* Reads and clears the device status word.  Synchronises. */
+sd_status sd_device_status(sd_ctx* ctx, uint32_t* flags_out);
+
+/* Plain autoregressive pass of the target over the last token of each listed
+ * sequence (the baseline that defines c in Eq. 1): logits_dev [n_seq][vocab].
+ * Appends one KV position but does not commit a token. */
+sd_status sd_target_step(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, float* logits_dev);
+
+/* ------------------------------------------- single operators (for testing) */
+
+/* y[rows][n_out] (fp32) = x[rows][n_in] * W[n_out][n_in]^T; x and W in `dtype`.
+ * impl: 0 = automatic, 1 = plain CUDA-core kernel, 2 = tensor-core kernel
+ * (SD_ERR_UNSUPPORTED if the shape does not fit it).  All pointers device. */
+sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype,
+                       int impl, void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl);
+
+/* Attention of `rows` query rows against a cache laid out as the library lays
+ * it out: k_cache/v_cache [n_slots][n_kv_heads][max_ctx][head_dim], q
+ * [rows][n_heads][head_dim], row r belongs to slot row_slot[r] and sees
+ * positions 0..row_pos[r]; out [rows][n_heads][head_dim].  dtype as above. */
+sd_status sd_op_attention(const void* q, const void* k_cache, const void* v_cache, void* out,
+                          const int32_t* row_slot, const int32_t* row_pos, int rows,
+                          int n_heads, int n_kv_heads, int head_dim, int max_ctx, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx);
+
+/* Philox4x32-10 on the device: out[i][0..3] for ctr[i][0..3], one key.  For tests. */
+sd_status sd_op_philox(const uint32_t* ctr_dev, int n, uint32_t key0, uint32_t key1, uint32_t* out_dev, void* cuda_stream);
+
+/* softmax(logits / T) and one draw per row by the integer inverse CDF:
+ * probs_dev [rows][V] out, tok_dev [rows] out, u_int in [1, 2^24] per row (device). */
+sd_status sd_op_softmax_sample(const float* logits_dev, int rows, int V, float temperature,
+                               const uint32_t* u_int_dev, float* probs_dev, int32_t* tok_dev, void* cuda_stream);
+
+const char* sd_status_str(sd_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SD_H */

@@ -93,6 +93,8 @@ def lib():
         L.orc_silu.restype = C.c_double
         L.orc_linear.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_linear.restype = None
+        L.orc_attention_head.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
+        L.orc_attention_head.restype = None
         L.orc_route_prompt.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int,
                                        C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                        C.c_int, C.c_int, C.c_void_p]
@@ -215,6 +217,25 @@ class OracleCache:
         if rc != 0:
             raise ValueError("oracle cache capacity exceeded")
         return out
+
+
+def attention_head(q, K, V):
+    """q [hd], K, V [n_ctx, hd] (float64) -> softmax(q K^T / sqrt(hd)) V."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    out = np.empty(q.shape[0], dtype=np.float64)
+    lib().orc_attention_head(_ptr(q), _ptr(K), _ptr(V), K.shape[0], q.shape[0], K.shape[1], _ptr(out))
+    return out
+
+
+def linear(W, X):
+    """X [rows, n_in] float64, W [n_out, n_in] fp32 or uint16 bf16 bits -> X W^T (float64)."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    W = np.ascontiguousarray(W)
+    Y = np.empty((X.shape[0], W.shape[0]), dtype=np.float64)
+    lib().orc_linear(_ptr(W), 1 if W.dtype == np.uint16 else 0, W.shape[0], W.shape[1], _ptr(X), X.shape[0], _ptr(Y))
+    return Y
 
 
 def route_prompt(embed, tokens, w1, b1, w2, b2, forced_task=-1):

@@ -399,6 +399,27 @@ int orc_forward_full(const orc_model* m, const int32_t* tokens, int n, double* l
     return 0;
 }
 
+/* softmax(q K^T / sqrt(hd)) V for one query vector over n_ctx cached positions of one head;
+ * K, V: [n_ctx][hd] with row stride `stride` doubles.  The definition, written out. */
+void orc_attention_head(const double* q, const double* K, const double* V, int n_ctx, int hd, int stride, double* out)
+{
+    double* s = malloc(sizeof(double) * (size_t)n_ctx);
+    double mx = -INFINITY, den = 0.0;
+    for (int p = 0; p < n_ctx; ++p) {
+        double acc = 0.0;
+        for (int i = 0; i < hd; ++i) acc += q[i] * K[(size_t)p * stride + i];
+        s[p] = acc / sqrt((double)hd);
+        if (s[p] > mx) mx = s[p];
+    }
+    for (int p = 0; p < n_ctx; ++p) { s[p] = exp(s[p] - mx); den += s[p]; }
+    for (int i = 0; i < hd; ++i) {
+        double acc = 0.0;
+        for (int p = 0; p < n_ctx; ++p) acc += s[p] / den * V[(size_t)p * stride + i];
+        out[i] = acc;
+    }
+    free(s);
+}
+
 /* Single primitives exported so that tests can pin them one by one. */
 void orc_rmsnorm(const double* x, const float* gain, int d, double eps, double* y) { rmsnorm(x, gain, d, eps, y); }
 void orc_rope(double* vec, int n_heads, int head_dim, int pos, double base) { rope(vec, n_heads, head_dim, pos, base); }

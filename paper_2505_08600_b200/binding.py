@@ -1,0 +1,275 @@
+"""Thin ctypes binding of libsd.so: same names as include/sd.h, argument marshalling only.
+
+PyTorch appears here for device memory and streams alone; every step of the path runs in
+the library's kernels.  Importing this module without the built library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsd.so")
+
+SD_F32, SD_BF16 = 0, 1
+SD_MAX_BATCH, SD_MAX_ROWS, SD_MAX_GAMMA = 64, 256, 15
+T_EMBED, T_LM_HEAD, T_FINAL_NORM, T_WQ, T_WK, T_WV, T_WO, T_WG, T_WU, T_WD, T_NORM1, T_NORM2 = range(12)
+TENSOR_KIND = dict(embed=T_EMBED, lm_head=T_LM_HEAD, final_norm=T_FINAL_NORM, wq=T_WQ, wk=T_WK, wv=T_WV,
+                   wo=T_WO, wg=T_WG, wu=T_WU, wd=T_WD, norm1=T_NORM1, norm2=T_NORM2)
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "dtype")] + \
+               [("rms_eps", C.c_float), ("rope_base", C.c_float)]
+
+
+class Config(C.Structure):
+    _fields_ = [("max_seqs", C.c_int32), ("max_ctx", C.c_int32), ("max_gamma", C.c_int32), ("n_drafts", C.c_int32),
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("clf_d_hidden", C.c_int32), ("reserved", C.c_int32)]
+
+
+class Counters(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("iterations", "drafted", "accepted", "emitted")]
+
+
+class AcceptArgs(C.Structure):
+    _fields_ = [("target", C.c_void_p), ("target_is_logits", C.c_int32), ("q", C.c_void_p), ("x", C.c_void_p),
+                ("B", C.c_int32), ("gamma", C.c_int32), ("V", C.c_int32), ("temperature", C.c_float),
+                ("seed", C.c_uint64), ("iter", C.c_void_p), ("seq_id", C.c_void_p), ("n_acc", C.c_void_p),
+                ("out_tok", C.c_void_p), ("cuda_stream", C.c_void_p)]
+
+
+class SdError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {lib().sd_status_str(status).decode()} ({status})")
+
+
+_lib = None
+_vp, _i, _sz = C.c_void_p, C.c_int, C.c_size_t
+
+_PROTOS = {
+    "sd_arena_bytes": (_sz, [C.POINTER(Config), C.POINTER(ModelDesc)]),
+    "sd_create": (_i, [C.POINTER(Config), C.POINTER(ModelDesc), _vp, _vp, _sz, C.POINTER(_vp)]),
+    "sd_destroy": (_i, [_vp]),
+    "sd_load_tensor": (_i, [_vp, _i, _i, _i, _vp, _i]),
+    "sd_load_classifier": (_i, [_vp, _vp, _vp, _vp, _vp, _i]),
+    "sd_seq_begin": (_i, [_vp, _i, _vp, _i, C.c_uint32]),
+    "sd_prefill": (_i, [_vp, _vp, _i]),
+    "sd_route_prompt": (_i, [_vp, _vp, _i, _vp, _vp]),
+    "sd_draft_steps": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
+    "sd_verify": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
+    "sd_accept": (_i, [C.POINTER(AcceptArgs)]),
+    "sd_accept_seqs": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "sd_kv_rollback": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
+    "sd_seq_read": (_i, [_vp, _i, _vp, _i, C.POINTER(C.c_int32), C.POINTER(Counters)]),
+    "sd_seq_force": (_i, [_vp, _i, _vp, _i, _i, C.c_uint32]),
+    "sd_device_status": (_i, [_vp, C.POINTER(C.c_uint32)]),
+    "sd_target_step": (_i, [_vp, _vp, _i, _vp]),
+    "sd_op_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "sd_op_linear_workspace": (_sz, [_i, _i, _i, _i, _i]),
+    "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "sd_op_attention_workspace": (_sz, [_i, _i, _i, _i]),
+    "sd_op_philox": (_i, [_vp, _i, C.c_uint32, C.c_uint32, _vp, _vp]),
+    "sd_op_softmax_sample": (_i, [_vp, _i, _i, C.c_float, _vp, _vp, _vp, _vp]),
+    "sd_status_str": (C.c_char_p, [_i]),
+}
+
+
+def lib():
+    """Loads libsd.so; there is no fallback of any kind when it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is not built: run `python -m paper_2505_08600_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in _PROTOS.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    return sorted(_PROTOS)
+
+
+def _check(status, where):
+    if status != 0:
+        raise SdError(status, where)
+
+
+def _stream_ptr(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dp(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _seqs(seqs):
+    a = np.ascontiguousarray(seqs, dtype=np.int32)
+    return a, a.ctypes.data_as(C.c_void_p), int(a.shape[0])
+
+
+def _desc(dims, dtype, rms_eps=1e-5, rope_base=10000.0):
+    return ModelDesc(dims["n_layers"], dims["d_model"], dims["n_heads"], dims["n_kv_heads"], dims["head_dim"],
+                     dims["d_ffn"], dims["vocab"], SD_BF16 if dtype == "bf16" else SD_F32, rms_eps, rope_base)
+
+
+class Context:
+    """Owns one sd_ctx and the torch-allocated arena behind it.  Methods carry the names of
+    the C calls and do nothing but marshal their arguments."""
+
+    def __init__(self, target_dims, draft_dims, dtype, max_seqs, max_ctx, max_gamma, temperature, seed,
+                 clf_d_hidden=0, device="cuda:0", stream=None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: this library has no CPU path")
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.L = lib()
+        self.dtype = dtype
+        self.dims = [target_dims] + list(draft_dims)
+        self.vocab = target_dims["vocab"]
+        n = len(self.dims)
+        self._descs = (ModelDesc * n)(*[_desc(d, dtype) for d in self.dims])
+        self.cfg = Config(max_seqs, max_ctx, max_gamma, n - 1, float(temperature), int(seed), int(clf_d_hidden), 0)
+        need = self.L.sd_arena_bytes(C.byref(self.cfg), self._descs)
+        if need == 0:
+            raise SdError(1, "sd_arena_bytes")
+        self.arena = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+        base = (self.arena.data_ptr() + 255) & ~255
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        h = C.c_void_p()
+        _check(self.L.sd_create(C.byref(self.cfg), self._descs, _stream_ptr(self.stream), C.c_void_p(base), need, C.byref(h)), "sd_create")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.L.sd_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- loading
+    def sd_load_tensor(self, model_id, kind, layer, src):
+        """src: numpy array (host) or torch CUDA tensor, already in the model's dtype
+        (bf16 as uint16 bit patterns or torch.bfloat16)."""
+        if isinstance(src, np.ndarray):
+            src = np.ascontiguousarray(src)
+            _check(self.L.sd_load_tensor(self.h, model_id, kind, layer, src.ctypes.data_as(C.c_void_p), 0), "sd_load_tensor")
+        else:
+            assert src.is_cuda and src.is_contiguous()
+            _check(self.L.sd_load_tensor(self.h, model_id, kind, layer, _dp(src), 1), "sd_load_tensor")
+
+    def load_weights(self, model_id, weights):
+        for name, val in weights.items():
+            kind = TENSOR_KIND[name]
+            if isinstance(val, (list, tuple)):
+                for l, a in enumerate(val):
+                    self.sd_load_tensor(model_id, kind, l, a)
+            else:
+                self.sd_load_tensor(model_id, kind, 0, val)
+
+    def sd_load_classifier(self, w1, b1, w2, b2):
+        arrs = [np.ascontiguousarray(a, dtype=np.float32) for a in (w1, b1, w2, b2)]
+        _check(self.L.sd_load_classifier(self.h, *[a.ctypes.data_as(C.c_void_p) for a in arrs], 0), "sd_load_classifier")
+
+    # ---- sequences
+    def sd_seq_begin(self, seq, prompt, seq_id=None):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        _check(self.L.sd_seq_begin(self.h, seq, p.ctypes.data_as(C.c_void_p), p.shape[0], seq if seq_id is None else seq_id), "sd_seq_begin")
+
+    def sd_route_prompt(self, seqs, forced_task=None):
+        a, p, n = _seqs(seqs)
+        out = np.zeros(n, dtype=np.int32)
+        f = np.ascontiguousarray(forced_task, dtype=np.int32) if forced_task is not None else None
+        _check(self.L.sd_route_prompt(self.h, p, n, f.ctypes.data_as(C.c_void_p) if f is not None else None,
+                                      out.ctypes.data_as(C.c_void_p)), "sd_route_prompt")
+        return out
+
+    def sd_prefill(self, seqs):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_prefill(self.h, p, n), "sd_prefill")
+
+    # ---- the hot calls; tensors are preallocated CUDA tensors owned by the caller
+    def sd_draft_steps(self, seqs, gamma, x, q):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_draft_steps(self.h, p, n, gamma, _dp(x), _dp(q)), "sd_draft_steps")
+
+    def sd_verify(self, seqs, gamma, x, logits):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_verify(self.h, p, n, gamma, _dp(x), _dp(logits)), "sd_verify")
+
+    def sd_accept_seqs(self, seqs, gamma, logits, q, x, n_acc, out_tok):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_accept_seqs(self.h, p, n, gamma, _dp(logits), _dp(q), _dp(x), _dp(n_acc), _dp(out_tok)), "sd_accept_seqs")
+
+    def sd_kv_rollback(self, seqs, gamma, n_acc, out_tok):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_kv_rollback(self.h, p, n, gamma, _dp(n_acc), _dp(out_tok)), "sd_kv_rollback")
+
+    def sd_target_step(self, seqs, logits):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_target_step(self.h, p, n, _dp(logits)), "sd_target_step")
+
+    # ---- observation
+    def sd_seq_read(self, seq, cap=None):
+        cap = self.cfg.max_ctx + 1 if cap is None else cap
+        toks = np.zeros(cap, dtype=np.int32)
+        ln = C.c_int32()
+        cnt = Counters()
+        _check(self.L.sd_seq_read(self.h, seq, toks.ctypes.data_as(C.c_void_p), cap, C.byref(ln), C.byref(cnt)), "sd_seq_read")
+        return toks[: min(cap, ln.value)].copy(), {k: getattr(cnt, k) for k in ("iterations", "drafted", "accepted", "emitted")}
+
+    def sd_seq_force(self, seq, tokens, draft_kv_len, it):
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        _check(self.L.sd_seq_force(self.h, seq, t.ctypes.data_as(C.c_void_p), t.shape[0], int(draft_kv_len), int(it)), "sd_seq_force")
+
+    def sd_device_status(self):
+        f = C.c_uint32()
+        _check(self.L.sd_device_status(self.h, C.byref(f)), "sd_device_status")
+        return f.value
+
+
+def sd_accept(target, q, x, temperature, seed, it, seq_id, n_acc, out_tok, target_is_logits, stream=None):
+    """Stateless accept/reject: all arguments are CUDA tensors except the scalars."""
+    B, g1, V = target.shape
+    a = AcceptArgs(target.data_ptr(), int(target_is_logits), q.data_ptr() if q is not None else None,
+                   x.data_ptr() if x is not None else None, B, g1 - 1, V, float(temperature), int(seed),
+                   it.data_ptr(), seq_id.data_ptr(), n_acc.data_ptr(), out_tok.data_ptr(), _stream_ptr(stream).value)
+    _check(lib().sd_accept(C.byref(a)), "sd_accept")
+
+
+def sd_op_linear(x, w, y, dtype, impl=0, stream=None):
+    rows, n_in = x.shape
+    n_out = w.shape[0]
+    need = lib().sd_op_linear_workspace(rows, n_out, n_in, dtype, impl)
+    ws = torch.empty(max(need, 1), dtype=torch.uint8, device=x.device)
+    _check(lib().sd_op_linear(_dp(x), _dp(w), _dp(y), rows, n_out, n_in, dtype, impl, _dp(ws), need, _stream_ptr(stream)), "sd_op_linear")
+
+
+def sd_op_attention(q, kc, vc, out, row_slot, row_pos, n_heads, n_kv_heads, head_dim, max_ctx, dtype, stream=None):
+    rows = q.shape[0]
+    need = lib().sd_op_attention_workspace(rows, n_heads, head_dim, max_ctx)
+    ws = torch.empty(max(need, 1), dtype=torch.uint8, device=q.device)
+    _check(lib().sd_op_attention(_dp(q), _dp(kc), _dp(vc), _dp(out), _dp(row_slot), _dp(row_pos), rows, n_heads,
+                                 n_kv_heads, head_dim, max_ctx, dtype, _dp(ws), need, _stream_ptr(stream)), "sd_op_attention")
+
+
+def sd_op_philox(ctr, key0, key1, out, stream=None):
+    _check(lib().sd_op_philox(_dp(ctr), ctr.shape[0], key0, key1, _dp(out), _stream_ptr(stream)), "sd_op_philox")
+
+
+def sd_op_softmax_sample(logits, temperature, u_int, probs, tok, stream=None):
+    rows, V = logits.shape
+    _check(lib().sd_op_softmax_sample(_dp(logits), rows, V, float(temperature), _dp(u_int), _dp(probs), _dp(tok),
+                                      _stream_ptr(stream)), "sd_op_softmax_sample")

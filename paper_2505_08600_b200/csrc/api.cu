@@ -1,0 +1,593 @@
+// Host runtime behind the C ABI: arena layout, model tables, per-sequence bookkeeping and
+// the launch sequences of the five hot calls.  Nothing here allocates device memory; all of
+// it is carved out of the arena handed to sd_create.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <vector>
+
+#include "kernels.h"
+
+using namespace sd;
+
+namespace {
+
+struct Bump {                       // bump allocator over the arena; base == nullptr just measures
+    char* base;
+    size_t off;
+    void* take(size_t bytes) {
+        off = (off + 255) & ~(size_t)255;
+        void* p = base ? base + off : nullptr;
+        off += bytes;
+        return p;
+    }
+};
+
+struct Layer {
+    void* wqkv;                     // [(H + 2 Hkv) hd][d]: query rows, then key rows, then value rows
+    void* wo;                       // [d][H hd]
+    void* wgu;                      // [2F][d]: gate rows, then up rows
+    void* wd;                       // [d][F]
+    float* norm1;
+    float* norm2;
+};
+
+struct Model {
+    sd_model_desc d;
+    size_t esz;
+    void* embed;
+    void* lm_head;
+    float* final_norm;
+    std::vector<Layer> layers;
+    char* kcache;                   // [layer][slot][kv_head][position][head_dim]
+    char* vcache;
+    size_t kv_layer_bytes;
+    float* rope_cos;                // [max_ctx][head_dim / 2]
+    float* rope_sin;
+    int n_qkv() const { return (d.n_heads + 2 * d.n_kv_heads) * d.head_dim; }
+};
+
+enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
+
+}  // namespace
+
+struct sd_ctx {
+    sd_config cfg;
+    std::vector<Model> models;
+    cudaStream_t st;
+    SeqState S;
+    // scratch of one forward pass
+    float* h; void* xn; void* q; void* attn; void* act; float* lin; float* draft_logits;
+    int32_t* row_slot; int32_t* row_pos;
+    void* attn_ws; size_t attn_ws_bytes;
+    // classifier
+    float* clf_w1; float* clf_b1; float* clf_w2; float* clf_b2; bool clf_loaded;
+    // host bookkeeping
+    std::vector<int> phase, len_ub, n_prompt, draft_id;
+    size_t arena_used;
+};
+
+namespace {
+
+size_t esize(int dtype) { return dtype == SD_BF16 ? 2 : 4; }
+
+bool valid_desc(const sd_model_desc& m) {
+    if (m.n_layers < 1 || m.d_model < 8 || m.n_heads < 1 || m.n_kv_heads < 1 || m.d_ffn < 8 || m.vocab < 2) return false;
+    if (m.n_heads % m.n_kv_heads) return false;
+    if (m.head_dim < 8 || m.head_dim > 256 || (m.head_dim & 7)) return false;
+    if (m.dtype != SD_F32 && m.dtype != SD_BF16) return false;
+    if ((m.d_model & 7) || (m.d_ffn & 7)) return false;
+    return true;
+}
+
+bool valid_cfg(const sd_config* c, const sd_model_desc* ms) {
+    if (!c || !ms) return false;
+    if (c->max_seqs < 1 || c->max_seqs > SD_MAX_BATCH || c->max_ctx < 4 || c->max_gamma < 0 || c->max_gamma > SD_MAX_GAMMA) return false;
+    if (c->n_drafts < 0 || c->n_drafts > 16 || !(c->temperature >= 0.f) || c->clf_d_hidden < 0) return false;
+    for (int i = 0; i <= c->n_drafts; ++i) {
+        if (!valid_desc(ms[i])) return false;
+        if (ms[i].vocab != ms[0].vocab) return false;        // draft and target share the vocabulary
+    }
+    return true;
+}
+
+// The single place that decides where everything lives.  Run once with a null base to size
+// the arena, once more with the real base to place the pointers.
+void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
+    const sd_config& cfg = c->cfg;
+    const int S = cfg.max_seqs, nm = 1 + cfg.n_drafts;
+    c->models.resize(nm);
+    int d_max = 0, f_max = 0, qkv_max = 0, dq_max = 0, lin_max = 0;
+    for (int i = 0; i < nm; ++i) {
+        Model& M = c->models[i];
+        M.d = ms[i];
+        M.esz = esize(ms[i].dtype);
+        const sd_model_desc& m = M.d;
+        const size_t dq = (size_t)m.n_heads * m.head_dim, dkv = (size_t)m.n_kv_heads * m.head_dim;
+        M.embed = B.take((size_t)m.vocab * m.d_model * M.esz);
+        M.lm_head = B.take((size_t)m.vocab * m.d_model * M.esz);
+        M.final_norm = (float*)B.take(sizeof(float) * m.d_model);
+        M.layers.resize(m.n_layers);
+        for (int l = 0; l < m.n_layers; ++l) {
+            Layer& L = M.layers[l];
+            L.wqkv = B.take((dq + 2 * dkv) * m.d_model * M.esz);
+            L.wo = B.take((size_t)m.d_model * dq * M.esz);
+            L.wgu = B.take((size_t)2 * m.d_ffn * m.d_model * M.esz);
+            L.wd = B.take((size_t)m.d_model * m.d_ffn * M.esz);
+            L.norm1 = (float*)B.take(sizeof(float) * m.d_model);
+            L.norm2 = (float*)B.take(sizeof(float) * m.d_model);
+        }
+        M.kv_layer_bytes = (size_t)S * dkv * cfg.max_ctx * M.esz;
+        M.kcache = (char*)B.take(M.kv_layer_bytes * m.n_layers);
+        M.vcache = (char*)B.take(M.kv_layer_bytes * m.n_layers);
+        M.rope_cos = (float*)B.take(sizeof(float) * (size_t)cfg.max_ctx * (m.head_dim / 2));
+        M.rope_sin = (float*)B.take(sizeof(float) * (size_t)cfg.max_ctx * (m.head_dim / 2));
+        d_max = std::max(d_max, m.d_model);
+        f_max = std::max(f_max, m.d_ffn);
+        qkv_max = std::max(qkv_max, M.n_qkv());
+        dq_max = std::max(dq_max, (int)dq);
+        lin_max = std::max(lin_max, std::max(std::max(M.n_qkv(), 2 * m.d_ffn), m.d_model));
+    }
+    const size_t R = SD_MAX_ROWS;
+    c->S.len = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->S.tkv = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->S.dkv = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->S.iter = (uint32_t*)B.take(sizeof(uint32_t) * S);
+    c->S.seq_id = (uint32_t*)B.take(sizeof(uint32_t) * S);
+    c->S.draft_id = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->S.n_prompt = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->S.counters = (int64_t*)B.take(sizeof(int64_t) * 4 * S);
+    c->S.tok_stride = cfg.max_ctx + 1;
+    c->S.max_ctx = cfg.max_ctx;
+    c->S.tokens = (int32_t*)B.take(sizeof(int32_t) * (size_t)S * c->S.tok_stride);
+    c->S.status = (uint32_t*)B.take(sizeof(uint32_t));
+    c->h = (float*)B.take(sizeof(float) * R * d_max);
+    c->xn = B.take(4 * R * d_max);
+    c->q = B.take(4 * R * dq_max);
+    c->attn = B.take(4 * R * dq_max);
+    c->act = B.take(4 * R * f_max);
+    c->lin = (float*)B.take(sizeof(float) * R * lin_max);
+    c->draft_logits = (float*)B.take(sizeof(float) * (size_t)SD_MAX_BATCH * ms[0].vocab);
+    c->row_slot = (int32_t*)B.take(sizeof(int32_t) * R);
+    c->row_pos = (int32_t*)B.take(sizeof(int32_t) * R);
+    c->attn_ws_bytes = 0;
+    for (int i = 0; i < nm; ++i)
+        c->attn_ws_bytes = std::max(c->attn_ws_bytes, attention_workspace_bytes((int)R, ms[i].n_heads, ms[i].head_dim, cfg.max_ctx));
+    c->attn_ws = B.take(c->attn_ws_bytes);
+    if (cfg.clf_d_hidden > 0 && cfg.n_drafts > 0) {
+        c->clf_w1 = (float*)B.take(sizeof(float) * (size_t)cfg.clf_d_hidden * ms[0].d_model);
+        c->clf_b1 = (float*)B.take(sizeof(float) * cfg.clf_d_hidden);
+        c->clf_w2 = (float*)B.take(sizeof(float) * (size_t)cfg.n_drafts * cfg.clf_d_hidden);
+        c->clf_b2 = (float*)B.take(sizeof(float) * cfg.n_drafts);
+    } else {
+        c->clf_w1 = c->clf_b1 = c->clf_w2 = c->clf_b2 = nullptr;
+    }
+}
+
+#define CUDA_TRY(expr)                                                                     \
+    do {                                                                                   \
+        cudaError_t e__ = (expr);                                                          \
+        if (e__ != cudaSuccess) {                                                          \
+            fprintf(stderr, "[sd] CUDA error %s at %s:%d\n", cudaGetErrorString(e__), __FILE__, __LINE__); \
+            return SD_ERR_CUDA;                                                            \
+        }                                                                                  \
+    } while (0)
+#define SD_TRY(expr)                      \
+    do {                                  \
+        sd_status s__ = (expr);           \
+        if (s__ != SD_OK) return s__;     \
+    } while (0)
+
+sd_status linear(sd_ctx* c, const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype) {
+    CUDA_TRY(launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, c->st));
+    return SD_OK;
+}
+
+enum LogitsMode { LOGITS_NONE = 0, LOGITS_ALL = 1, LOGITS_LAST = 2 };
+
+// One pass of a model over n_rows query rows described by `plan`.
+sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
+    const sd_model_desc& m = M.d;
+    const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
+    cudaStream_t st = c->st;
+    CUDA_TRY(launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
+    for (int l = 0; l < m.n_layers; ++l) {
+        const Layer& L = M.layers[l];
+        void* kc = M.kcache + M.kv_layer_bytes * l;
+        void* vc = M.vcache + M.kv_layer_bytes * l;
+        CUDA_TRY(launch_rmsnorm(c->h, L.norm1, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        SD_TRY(linear(c, c->xn, L.wqkv, c->lin, n_rows, M.n_qkv(), d, dt));
+        CUDA_TRY(launch_rope_kv(c->lin, c->q, kc, vc, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
+                                M.rope_cos, M.rope_sin, c->S.status, st));
+        CUDA_TRY(launch_attention(c->q, kc, vc, c->attn, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
+                                  c->attn_ws, c->attn_ws_bytes, st));
+        SD_TRY(linear(c, c->attn, L.wo, c->lin, n_rows, d, H * hd, dt));
+        CUDA_TRY(launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
+        CUDA_TRY(launch_rmsnorm(c->h, L.norm2, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        SD_TRY(linear(c, c->xn, L.wgu, c->lin, n_rows, 2 * F, d, dt));
+        CUDA_TRY(launch_swiglu(c->lin, c->act, dt, n_rows, F, st));
+        SD_TRY(linear(c, c->act, L.wd, c->lin, n_rows, d, F, dt));
+        CUDA_TRY(launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
+    }
+    if (mode == LOGITS_ALL) {
+        CUDA_TRY(launch_rmsnorm(c->h, M.final_norm, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        SD_TRY(linear(c, c->xn, M.lm_head, logits_out, n_rows, m.vocab, d, dt));
+    } else if (mode == LOGITS_LAST) {
+        const int R = plan.rows_per_seq;
+        CUDA_TRY(launch_rmsnorm(c->h, M.final_norm, c->xn, dt, list.n, d, m.rms_eps, R, R - 1, st));
+        SD_TRY(linear(c, c->xn, M.lm_head, logits_out, list.n, m.vocab, d, dt));
+    }
+    return SD_OK;
+}
+
+sd_status make_list(sd_ctx* c, const int32_t* seqs, int n_seq, int min_phase, SeqList& list) {
+    if (!c || !seqs || n_seq < 1 || n_seq > SD_MAX_BATCH) return SD_ERR_INVALID_ARG;
+    list.n = n_seq;
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i];
+        if (s < 0 || s >= c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j) if (seqs[j] == s) return SD_ERR_INVALID_ARG;
+        if (c->phase[s] < min_phase) return SD_ERR_STATE;
+        list.ids[i] = s;
+        list.out[i] = i;
+    }
+    for (int i = n_seq; i < SD_MAX_BATCH; ++i) { list.ids[i] = 0; list.out[i] = 0; }
+    return SD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sd_status_str(sd_status s) {
+    switch (s) {
+        case SD_OK: return "ok";
+        case SD_ERR_INVALID_ARG: return "invalid argument";
+        case SD_ERR_STATE: return "call out of order for this sequence";
+        case SD_ERR_CAPACITY: return "capacity exceeded";
+        case SD_ERR_OOM: return "arena too small";
+        case SD_ERR_CUDA: return "CUDA error";
+        case SD_ERR_TIMEOUT: return "timeout";
+        case SD_ERR_UNSUPPORTED: return "unsupported";
+    }
+    return "unknown";
+}
+
+size_t sd_arena_bytes(const sd_config* cfg, const sd_model_desc* models) {
+    if (!valid_cfg(cfg, models)) return 0;
+    sd_ctx tmp;
+    tmp.cfg = *cfg;
+    Bump B{nullptr, 0};
+    layout(&tmp, models, B);
+    return B.off + 256;
+}
+
+sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cuda_stream, void* arena, size_t arena_bytes,
+                    sd_ctx** out) {
+    if (!out) return SD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!valid_cfg(cfg, models) || !arena || ((uintptr_t)arena & 255)) return SD_ERR_INVALID_ARG;
+    if (cfg->clf_d_hidden > 0 && cfg->n_drafts < 1) return SD_ERR_INVALID_ARG;
+    const size_t need = sd_arena_bytes(cfg, models);
+    if (arena_bytes < need) return SD_ERR_OOM;
+    sd_ctx* c = new sd_ctx();
+    c->cfg = *cfg;
+    c->st = (cudaStream_t)cuda_stream;
+    Bump B{(char*)arena, 0};
+    layout(c, models, B);
+    c->arena_used = B.off;
+    c->clf_loaded = false;
+    c->phase.assign(cfg->max_seqs, PH_FREE);
+    c->len_ub.assign(cfg->max_seqs, 0);
+    c->n_prompt.assign(cfg->max_seqs, 0);
+    c->draft_id.assign(cfg->max_seqs, -1);
+    cudaStream_t st = c->st;
+    auto fail = [&](sd_status s) { delete c; return s; };
+    // state starts at zero; rotary tables are computed here in double and stored as fp32
+    if (cudaMemsetAsync(c->S.len, 0, (char*)c->S.status + sizeof(uint32_t) - (char*)c->S.len, st) != cudaSuccess) return fail(SD_ERR_CUDA);
+    for (size_t i = 0; i < c->models.size(); ++i) {
+        Model& M = c->models[i];
+        const int half = M.d.head_dim / 2;
+        std::vector<float> cs((size_t)cfg->max_ctx * half), sn((size_t)cfg->max_ctx * half);
+        for (int i2 = 0; i2 < half; ++i2) {
+            const double inv_freq = pow((double)M.d.rope_base, -2.0 * i2 / M.d.head_dim);
+            for (int p = 0; p < cfg->max_ctx; ++p) {
+                cs[(size_t)p * half + i2] = (float)cos(p * inv_freq);
+                sn[(size_t)p * half + i2] = (float)sin(p * inv_freq);
+            }
+        }
+        if (cudaMemcpyAsync(M.rope_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(M.rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return fail(SD_ERR_CUDA);
+    }
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
+    *out = c;
+    return SD_OK;
+}
+
+sd_status sd_destroy(sd_ctx* c) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    cudaStreamSynchronize(c->st);
+    delete c;
+    return SD_OK;
+}
+
+sd_status sd_load_tensor(sd_ctx* c, int model_id, int kind, int layer, const void* src, int on_dev) {
+    if (!c || !src || model_id < 0 || model_id >= (int)c->models.size()) return SD_ERR_INVALID_ARG;
+    Model& M = c->models[model_id];
+    const sd_model_desc& m = M.d;
+    const size_t dq = (size_t)m.n_heads * m.head_dim, dkv = (size_t)m.n_kv_heads * m.head_dim, d = m.d_model, F = m.d_ffn;
+    const bool per_layer = kind >= SD_T_WQ;
+    if (per_layer && (layer < 0 || layer >= m.n_layers)) return SD_ERR_INVALID_ARG;
+    void* dst = nullptr;
+    size_t bytes = 0;
+    Layer* L = per_layer ? &M.layers[layer] : nullptr;
+    switch (kind) {
+        case SD_T_EMBED: dst = M.embed; bytes = (size_t)m.vocab * d * M.esz; break;
+        case SD_T_LM_HEAD: dst = M.lm_head; bytes = (size_t)m.vocab * d * M.esz; break;
+        case SD_T_FINAL_NORM: dst = M.final_norm; bytes = d * 4; break;
+        case SD_T_WQ: dst = L->wqkv; bytes = dq * d * M.esz; break;
+        case SD_T_WK: dst = (char*)L->wqkv + dq * d * M.esz; bytes = dkv * d * M.esz; break;
+        case SD_T_WV: dst = (char*)L->wqkv + (dq + dkv) * d * M.esz; bytes = dkv * d * M.esz; break;
+        case SD_T_WO: dst = L->wo; bytes = d * dq * M.esz; break;
+        case SD_T_WG: dst = L->wgu; bytes = F * d * M.esz; break;
+        case SD_T_WU: dst = (char*)L->wgu + F * d * M.esz; bytes = F * d * M.esz; break;
+        case SD_T_WD: dst = L->wd; bytes = d * F * M.esz; break;
+        case SD_T_NORM1: dst = L->norm1; bytes = d * 4; break;
+        case SD_T_NORM2: dst = L->norm2; bytes = d * 4; break;
+        default: return SD_ERR_INVALID_ARG;
+    }
+    CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->st));
+    if (!on_dev) CUDA_TRY(cudaStreamSynchronize(c->st));     // the host buffer may go away after the call
+    return SD_OK;
+}
+
+sd_status sd_load_classifier(sd_ctx* c, const float* w1, const float* b1, const float* w2, const float* b2, int on_dev) {
+    if (!c || !w1 || !b1 || !w2 || !b2) return SD_ERR_INVALID_ARG;
+    if (!c->clf_w1) return SD_ERR_STATE;
+    const size_t dh = c->cfg.clf_d_hidden, d = c->models[0].d.d_model, K = c->cfg.n_drafts;
+    cudaMemcpyKind kd = on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    CUDA_TRY(cudaMemcpyAsync(c->clf_w1, w1, dh * d * 4, kd, c->st));
+    CUDA_TRY(cudaMemcpyAsync(c->clf_b1, b1, dh * 4, kd, c->st));
+    CUDA_TRY(cudaMemcpyAsync(c->clf_w2, w2, K * dh * 4, kd, c->st));
+    CUDA_TRY(cudaMemcpyAsync(c->clf_b2, b2, K * 4, kd, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    c->clf_loaded = true;
+    return SD_OK;
+}
+
+sd_status sd_seq_begin(sd_ctx* c, int seq, const int32_t* prompt, int n_prompt, uint32_t seq_id) {
+    if (!c || !prompt || seq < 0 || seq >= c->cfg.max_seqs || n_prompt < 2) return SD_ERR_INVALID_ARG;
+    if (n_prompt > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    const int V = c->models[0].d.vocab;
+    for (int i = 0; i < n_prompt; ++i) if (prompt[i] < 0 || prompt[i] >= V) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaMemcpyAsync(c->S.tokens + (size_t)seq * c->S.tok_stride, prompt, sizeof(int32_t) * n_prompt,
+                             cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(launch_set_state(c->S, seq, n_prompt, 0, 0, 0u, seq_id, 1, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    c->phase[seq] = PH_BEGUN;
+    c->len_ub[seq] = n_prompt;
+    c->n_prompt[seq] = n_prompt;
+    c->draft_id[seq] = -1;
+    return SD_OK;
+}
+
+sd_status sd_route_prompt(sd_ctx* c, const int32_t* seqs, int n_seq, const int32_t* forced, int32_t* draft_out) {
+    SeqList list, fl;
+    SD_TRY(make_list(c, seqs, n_seq, PH_BEGUN, list));
+    const int K = c->cfg.n_drafts;
+    if (K < 1) return SD_ERR_STATE;
+    fl = list;
+    bool need_clf = false;
+    for (int i = 0; i < n_seq; ++i) {
+        int f = forced ? forced[i] : -1;
+        if (f >= K) return SD_ERR_INVALID_ARG;
+        fl.ids[i] = f < 0 ? -1 : f;
+        need_clf |= f < 0;
+    }
+    if (need_clf && !c->clf_loaded) return SD_ERR_STATE;
+    Model& T = c->models[0];
+    CUDA_TRY(launch_classifier(c->S, list, fl, T.embed, T.d.dtype, T.d.d_model, T.d.vocab, c->clf_w1, c->clf_b1,
+                               c->cfg.clf_d_hidden, c->clf_w2, c->clf_b2, K, c->st));
+    std::vector<int32_t> ids(c->cfg.max_seqs);
+    CUDA_TRY(cudaMemcpyAsync(ids.data(), c->S.draft_id, sizeof(int32_t) * ids.size(), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i];
+        c->draft_id[s] = ids[s];
+        if (c->phase[s] == PH_BEGUN) c->phase[s] = PH_ROUTED;
+        if (draft_out) draft_out[i] = ids[s];
+    }
+    return SD_OK;
+}
+
+sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
+    SeqList all;
+    SD_TRY(make_list(c, seqs, n_seq, c->cfg.n_drafts > 0 ? PH_ROUTED : PH_BEGUN, all));
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i], n = c->n_prompt[s] - 1;
+        SeqList one = all;
+        one.n = 1; one.ids[0] = s; one.out[0] = 0;
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass == 1 && c->cfg.n_drafts < 1) break;
+            Model& M = c->models[pass == 0 ? 0 : 1 + c->draft_id[s]];
+            for (int p0 = 0; p0 < n; p0 += SD_MAX_ROWS) {
+                const int rows = std::min(SD_MAX_ROWS, n - p0);
+                RowPlan plan{PLAN_PREFILL, rows, p0, 0, 0, nullptr};
+                SD_TRY(forward(c, M, one, plan, rows, LOGITS_NONE, nullptr));
+            }
+        }
+        CUDA_TRY(launch_set_state(c->S, s, n + 1, n, n, 0u, 0u, 0, c->st));
+        c->phase[s] = PH_READY;
+    }
+    return SD_OK;
+}
+
+sd_status sd_draft_steps(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, int32_t* x_dev, float* q_dev) {
+    SeqList all;
+    SD_TRY(make_list(c, seqs, n_seq, PH_READY, all));
+    if (gamma < 1 || gamma > c->cfg.max_gamma || !x_dev || !q_dev) return SD_ERR_INVALID_ARG;
+    if (c->cfg.n_drafts < 1) return SD_ERR_STATE;
+    for (int i = 0; i < n_seq; ++i)
+        if (c->len_ub[seqs[i]] + gamma - 1 > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    const int V = c->models[0].d.vocab;
+    for (int k = 0; k < c->cfg.n_drafts; ++k) {             // sequences grouped per routed draft
+        SeqList g = all;
+        g.n = 0;
+        for (int i = 0; i < n_seq; ++i)
+            if (c->draft_id[seqs[i]] == k) { g.ids[g.n] = seqs[i]; g.out[g.n] = i; ++g.n; }
+        if (g.n == 0) continue;
+        Model& M = c->models[1 + k];
+        for (int s = 0; s < gamma; ++s) {
+            if (s == 0) {
+                RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_dev};
+                SD_TRY(forward(c, M, g, plan, 2 * g.n, LOGITS_LAST, c->draft_logits));
+            } else {
+                RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_dev};
+                SD_TRY(forward(c, M, g, plan, g.n, LOGITS_ALL, c->draft_logits));
+            }
+            CUDA_TRY(launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
+        }
+    }
+    return SD_OK;
+}
+
+sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_dev, float* logits_dev) {
+    SeqList list;
+    SD_TRY(make_list(c, seqs, n_seq, PH_READY, list));
+    if (gamma < 0 || gamma > c->cfg.max_gamma || !logits_dev || (gamma > 0 && !x_dev)) return SD_ERR_INVALID_ARG;
+    if (n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_CAPACITY;
+    for (int i = 0; i < n_seq; ++i)
+        if (c->len_ub[seqs[i]] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev};
+    return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev);
+}
+
+sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logits_dev) {
+    SeqList list;
+    SD_TRY(make_list(c, seqs, n_seq, PH_READY, list));
+    if (!logits_dev) return SD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_seq; ++i)
+        if (c->len_ub[seqs[i]] > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr};
+    return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev);
+}
+
+sd_status sd_accept(const sd_accept_args* a) {
+    if (!a || !a->target || !a->n_acc || !a->out_tok || !a->iter || !a->seq_id) return SD_ERR_INVALID_ARG;
+    if (a->B < 1 || a->gamma < 0 || a->gamma > SD_MAX_GAMMA || a->V < 2 || !(a->temperature >= 0.f)) return SD_ERR_INVALID_ARG;
+    if (a->gamma > 0 && (!a->q || !a->x)) return SD_ERR_INVALID_ARG;
+    AcceptParams p;
+    memset(&p, 0, sizeof(p));
+    p.target = a->target; p.target_is_logits = a->target_is_logits; p.q = a->q; p.x = a->x;
+    p.B = a->B; p.gamma = a->gamma; p.V = a->V; p.T = a->temperature; p.seed = a->seed;
+    p.iter = a->iter; p.seq_id = a->seq_id; p.use_list = 0; p.n_acc = a->n_acc; p.out_tok = a->out_tok;
+    CUDA_TRY(launch_accept(p, (cudaStream_t)a->cuda_stream));
+    return SD_OK;
+}
+
+sd_status sd_accept_seqs(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const float* logits_dev, const float* q_dev,
+                         const int32_t* x_dev, int32_t* n_acc_dev, int32_t* out_tok_dev) {
+    AcceptParams p;
+    memset(&p, 0, sizeof(p));
+    SD_TRY(make_list(c, seqs, n_seq, PH_READY, p.list));
+    if (gamma < 0 || gamma > c->cfg.max_gamma || !logits_dev || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!q_dev || !x_dev)) return SD_ERR_INVALID_ARG;
+    p.target = logits_dev; p.target_is_logits = 1; p.q = q_dev; p.x = x_dev;
+    p.B = n_seq; p.gamma = gamma; p.V = c->models[0].d.vocab; p.T = c->cfg.temperature; p.seed = c->cfg.seed;
+    p.iter = c->S.iter; p.seq_id = c->S.seq_id; p.use_list = 1; p.n_acc = n_acc_dev; p.out_tok = out_tok_dev;
+    CUDA_TRY(launch_accept(p, c->st));
+    return SD_OK;
+}
+
+sd_status sd_kv_rollback(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* n_acc_dev, const int32_t* out_tok_dev) {
+    SeqList list;
+    SD_TRY(make_list(c, seqs, n_seq, PH_READY, list));
+    if (gamma < 0 || gamma > c->cfg.max_gamma || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_seq; ++i)
+        if (c->len_ub[seqs[i]] + gamma + 1 > c->S.tok_stride) return SD_ERR_CAPACITY;
+    CUDA_TRY(launch_rollback(c->S, list, gamma, n_acc_dev, out_tok_dev, c->st));
+    for (int i = 0; i < n_seq; ++i) c->len_ub[seqs[i]] += gamma + 1;
+    return SD_OK;
+}
+
+sd_status sd_seq_read(sd_ctx* c, int seq, int32_t* tokens, int cap, int32_t* len_out, sd_counters* cnt) {
+    if (!c || seq < 0 || seq >= c->cfg.max_seqs || cap < 0 || (cap > 0 && !tokens)) return SD_ERR_INVALID_ARG;
+    if (c->phase[seq] == PH_FREE) return SD_ERR_STATE;
+    int32_t len = 0;
+    CUDA_TRY(cudaMemcpyAsync(&len, c->S.len + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    const int n = std::min(cap, (int)len);
+    if (n > 0) CUDA_TRY(cudaMemcpyAsync(tokens, c->S.tokens + (size_t)seq * c->S.tok_stride, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, c->st));
+    if (cnt) CUDA_TRY(cudaMemcpyAsync(cnt, c->S.counters + 4 * seq, sizeof(int64_t) * 4, cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    if (len_out) *len_out = len;
+    c->len_ub[seq] = len;
+    return SD_OK;
+}
+
+sd_status sd_seq_force(sd_ctx* c, int seq, const int32_t* tokens, int n_tokens, int draft_kv_len, uint32_t iter) {
+    if (!c || !tokens || seq < 0 || seq >= c->cfg.max_seqs || n_tokens < 2 || draft_kv_len < 0 || draft_kv_len >= n_tokens) return SD_ERR_INVALID_ARG;
+    if (c->phase[seq] < PH_READY) return SD_ERR_STATE;
+    if (n_tokens > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    CUDA_TRY(cudaMemcpyAsync(c->S.tokens + (size_t)seq * c->S.tok_stride, tokens, sizeof(int32_t) * n_tokens, cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(launch_set_state(c->S, seq, n_tokens, n_tokens - 1, draft_kv_len, iter, 0u, 0, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    c->len_ub[seq] = n_tokens;
+    return SD_OK;
+}
+
+sd_status sd_device_status(sd_ctx* c, uint32_t* flags) {
+    if (!c || !flags) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaMemcpyAsync(flags, c->S.status, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaMemsetAsync(c->S.status, 0, sizeof(uint32_t), c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+// ------------------------------------------------------------------ single operators
+size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl) {
+    (void)rows; (void)n_out; (void)n_in; (void)dtype; (void)impl;
+    return 0;
+}
+
+sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype, int impl,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    (void)workspace; (void)workspace_bytes;
+    if (!x || !w || !y || rows < 1 || n_out < 1 || n_in < 1 || (dtype != SD_F32 && dtype != SD_BF16)) return SD_ERR_INVALID_ARG;
+    if (impl == 2) return SD_ERR_UNSUPPORTED;
+    if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;
+    CUDA_TRY(launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, (cudaStream_t)stream));
+    return SD_OK;
+}
+
+size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx) {
+    return attention_workspace_bytes(rows, n_heads, head_dim, max_ctx);
+}
+
+sd_status sd_op_attention(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
+                          const int32_t* row_pos, int rows, int H, int Hkv, int hd, int max_ctx, int dtype,
+                          void* ws, size_t ws_bytes, void* stream) {
+    if (!q || !kc || !vc || !out || !row_slot || !row_pos || rows < 1 || H < 1 || Hkv < 1 || H % Hkv) return SD_ERR_INVALID_ARG;
+    if (hd < 8 || hd > 256 || (hd & 7) || max_ctx < 1 || (dtype != SD_F32 && dtype != SD_BF16)) return SD_ERR_INVALID_ARG;
+    if (ws_bytes < attention_workspace_bytes(rows, H, hd, max_ctx)) return SD_ERR_OOM;
+    CUDA_TRY(launch_attention(q, kc, vc, out, dtype, row_slot, row_pos, rows, H, Hkv, hd, max_ctx, ws, ws_bytes, (cudaStream_t)stream));
+    return SD_OK;
+}
+
+sd_status sd_op_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, void* stream) {
+    if (!ctr || !out || n < 0) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(launch_philox(ctr, n, k0, k1, out, (cudaStream_t)stream));
+    return SD_OK;
+}
+
+sd_status sd_op_softmax_sample(const float* logits, int rows, int V, float T, const uint32_t* u_int, float* probs,
+                               int32_t* tok, void* stream) {
+    if (!logits || !u_int || !probs || !tok || rows < 1 || V < 2 || !(T >= 0.f)) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(launch_softmax_sample_explicit(logits, rows, V, T, u_int, probs, tok, (cudaStream_t)stream));
+    return SD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,241 @@
+// Vocabulary-wide kernels: softmax with temperature, the exact integer inverse-CDF draw, the
+// draft's per-step sampler and the fused accept / reject / resample kernel.
+#include "kernels.h"
+
+namespace sd {
+
+__global__ void k_philox(const uint32_t* __restrict__ ctr, int n, uint32_t k0, uint32_t k1, uint32_t* __restrict__ out) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t o[4];
+    philox4x32_10(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3], k0, k1, o);
+    for (int j = 0; j < 4; ++j) out[4 * i + j] = o[j];
+}
+cudaError_t launch_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    k_philox<<<(n + 127) / 128, 128, 0, st>>>(ctr, n, k0, k1, out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- block-wide helpers
+struct BlockScratch {
+    float red[32];
+    unsigned long long scan[32];
+    unsigned long long total;
+    int tok;
+    int idx;
+};
+
+__device__ __forceinline__ int block_min_int(int v, BlockScratch& sh) {
+    int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    int* r = reinterpret_cast<int*>(sh.red);
+    if (lane == 0) r[w] = v;
+    __syncthreads();
+    int x = (threadIdx.x < nw) ? r[threadIdx.x] : 0x7fffffff;
+    if (w == 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x = min(x, __shfl_xor_sync(0xffffffffu, x, o));
+        if (lane == 0) sh.idx = x;
+    }
+    __syncthreads();
+    return sh.idx;
+}
+
+// lowest index of the maximum of f(k), k in [0, V)
+template <class F>
+__device__ __forceinline__ int block_argmax(F f, int V, BlockScratch& sh, float* max_out) {
+    float m = -INFINITY;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, f(k));
+    m = block_max(m, sh.red);
+    int best = 0x7fffffff;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) if (f(k) == m) { best = k; break; }
+    if (max_out) *max_out = m;
+    return block_min_int(best, sh);
+}
+
+// Exact inverse CDF over integer weights floor(w(k) * 2^32): returns the first k whose running
+// sum reaches ceil(u_int * total / 2^24), or -1 when every weight is zero.  Each thread owns a
+// contiguous chunk; integer addition is associative, so the split cannot change the answer.
+template <class F>
+__device__ __forceinline__ int block_icdf(F w, int V, uint32_t u_int, BlockScratch& sh) {
+    const int t = threadIdx.x, lane = t & 31, wid = t >> 5, nw = (blockDim.x + 31) >> 5;
+    const int chunk = (V + blockDim.x - 1) / blockDim.x;
+    const int k0 = min(V, t * chunk), k1 = min(V, k0 + chunk);
+    unsigned long long local = 0;
+    for (int k = k0; k < k1; ++k) local += __float2ull_rz(w(k) * 4294967296.0f);
+    unsigned long long incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    __syncthreads();
+    if (lane == 31) sh.scan[wid] = incl;
+    if (t == 0) sh.tok = -1;
+    __syncthreads();
+    if (wid == 0) {
+        unsigned long long v = lane < nw ? sh.scan[lane] : 0ull, s = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            unsigned long long u = __shfl_up_sync(0xffffffffu, s, o);
+            if (lane >= o) s += u;
+        }
+        sh.scan[lane] = s - v;                       // exclusive prefix of each warp
+        if (lane == 31) sh.total = s;
+    }
+    __syncthreads();
+    const unsigned long long tot = sh.total;
+    if (tot == 0ull) return -1;
+    incl += sh.scan[wid];
+    const unsigned long long excl = incl - local;
+    const unsigned long long thr = ((unsigned long long)u_int * tot + 16777215ull) >> 24;
+    if (excl < thr && thr <= incl) {
+        unsigned long long run = excl;
+        for (int k = k0; k < k1; ++k) {
+            run += __float2ull_rz(w(k) * 4294967296.0f);
+            if (run >= thr) { sh.tok = k; break; }
+        }
+    }
+    __syncthreads();
+    return sh.tok;
+}
+
+// ---------------------------------------------------------------- softmax + draw (draft steps)
+// One block per row.  probs = softmax(logits / T) (one-hot argmax when T == 0) is written out,
+// then one token is drawn from the written fp32 values.
+__device__ __forceinline__ int softmax_sample_row(const float* __restrict__ l, int V, float T, uint32_t u_int,
+                                                  float* __restrict__ probs, BlockScratch& sh) {
+    if (T == 0.f) {
+        int a = block_argmax([&](int k) { return l[k]; }, V, sh, nullptr);
+        for (int k = threadIdx.x; k < V; k += blockDim.x) probs[k] = (k == a) ? 1.f : 0.f;
+        return a;
+    }
+    float m = -INFINITY;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, l[k]);
+    m = block_max(m, sh.red);
+    float s = 0.f;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) / T);
+    s = block_sum(s, sh.red);
+    for (int k = threadIdx.x; k < V; k += blockDim.x) probs[k] = expf((l[k] - m) / T) / s;
+    __syncthreads();
+    int tok = block_icdf([&](int k) { return probs[k]; }, V, u_int, sh);
+    if (tok < 0) tok = block_argmax([&](int k) { return probs[k]; }, V, sh, nullptr);
+    return tok;
+}
+
+__global__ void __launch_bounds__(1024) k_softmax_sample_explicit(const float* __restrict__ logits, int V, float T,
+                                                                  const uint32_t* __restrict__ u_int,
+                                                                  float* __restrict__ probs, int32_t* __restrict__ tok) {
+    __shared__ BlockScratch sh;
+    const int r = blockIdx.x;
+    int k = softmax_sample_row(logits + (size_t)r * V, V, T, u_int[r], probs + (size_t)r * V, sh);
+    if (threadIdx.x == 0) tok[r] = k;
+}
+cudaError_t launch_softmax_sample_explicit(const float* logits, int rows, int V, float T, const uint32_t* u_int,
+                                           float* probs, int32_t* tok, cudaStream_t st) {
+    if (rows <= 0) return cudaSuccess;
+    k_softmax_sample_explicit<<<rows, 1024, 0, st>>>(logits, V, T, u_int, probs, tok);
+    return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(1024) k_draft_sample(const float* __restrict__ logits, SeqState S, SeqList list, int V, float T,
+                                                       uint64_t seed, int step, int gamma, float* __restrict__ q_out,
+                                                       int32_t* __restrict__ x_out) {
+    __shared__ BlockScratch sh;
+    const int i = blockIdx.x, slot = list.ids[i], b = list.out[i];
+    const uint32_t u = uniform24(seed, S.iter[slot], (uint32_t)step, S.seq_id[slot], DRAW_DRAFT);
+    int k = softmax_sample_row(logits + (size_t)i * V, V, T, u, q_out + ((size_t)b * gamma + step) * V, sh);
+    if (threadIdx.x == 0) x_out[(size_t)b * gamma + step] = k;
+}
+cudaError_t launch_draft_sample(const float* logits, const SeqState& S, const SeqList& list, int V, float T,
+                                uint64_t seed, int step, int gamma, float* q_out, int32_t* x_out, cudaStream_t st) {
+    if (list.n <= 0) return cudaSuccess;
+    k_draft_sample<<<list.n, 1024, 0, st>>>(logits, S, list, V, T, seed, step, gamma, q_out, x_out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- accept / reject / resample
+// One block per sequence.  Slot s is accepted iff u_s * q_s(x_s) <= p_s(x_s) with a single
+// rounded fp32 multiply; the first rejected slot n (or gamma) picks the row the next token is
+// drawn from: the residual max(0, p_n - q_n) or, after gamma accepts, p_gamma itself.
+__global__ void __launch_bounds__(1024) k_accept(AcceptParams P) {
+    __shared__ BlockScratch sh;
+    __shared__ float row_max[SD_MAX_GAMMA + 1], row_sum[SD_MAX_GAMMA + 1];
+    __shared__ int row_arg[SD_MAX_GAMMA + 1];
+    __shared__ int n_sh;
+    const int i = blockIdx.x;
+    const int idx = P.use_list ? P.list.ids[i] : i;
+    const int b = P.use_list ? P.list.out[i] : i;
+    const int V = P.V, gamma = P.gamma;
+    const float T = P.T;
+    const float* tgt = P.target + (size_t)b * (gamma + 1) * V;
+    const float* q = P.q + (size_t)b * gamma * V;
+    const int32_t* x = P.x + (size_t)b * gamma;
+    const bool logits = P.target_is_logits != 0;
+
+    if (logits) {
+        for (int j = 0; j <= gamma; ++j) {
+            const float* l = tgt + (size_t)j * V;
+            if (T == 0.f) {
+                int a = block_argmax([&](int k) { return l[k]; }, V, sh, nullptr);
+                if (threadIdx.x == 0) row_arg[j] = a;
+            } else {
+                float m = -INFINITY;
+                for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, l[k]);
+                m = block_max(m, sh.red);
+                float s = 0.f;
+                for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) / T);
+                s = block_sum(s, sh.red);
+                if (threadIdx.x == 0) { row_max[j] = m; row_sum[j] = s; }
+            }
+        }
+        __syncthreads();
+    }
+    auto prob = [&](int j, int k) -> float {
+        const float v = tgt[(size_t)j * V + k];
+        if (!logits) return v;
+        if (T == 0.f) return k == row_arg[j] ? 1.f : 0.f;
+        return expf((v - row_max[j]) / T) / row_sum[j];
+    };
+
+    if (threadIdx.x == 0) {
+        const uint32_t it = P.iter[idx], sid = P.seq_id[idx];
+        int n = 0;
+        while (n < gamma) {
+            int xs = x[n];
+            if (xs < 0 || xs >= V) break;                        // impossible token: treat as rejected
+            const uint32_t ui = uniform24(P.seed, it, (uint32_t)n, sid, DRAW_ACCEPT);
+            const float u = (float)ui * (1.0f / 16777216.0f);
+            const float lhs = __fmul_rn(u, q[(size_t)n * V + xs]);
+            if (!(lhs <= prob(n, xs))) break;
+            ++n;
+        }
+        n_sh = n;
+    }
+    __syncthreads();
+    const int n = n_sh;
+    const uint32_t ui = uniform24(P.seed, P.iter[idx], (uint32_t)n, P.seq_id[idx], DRAW_RESAMPLE);
+    int y;
+    if (n < gamma) {
+        const float* qn = q + (size_t)n * V;
+        y = block_icdf([&](int k) { return fmaxf(__fsub_rn(prob(n, k), qn[k]), 0.f); }, V, ui, sh);
+        if (y < 0) y = block_icdf([&](int k) { return prob(n, k); }, V, ui, sh);
+    } else {
+        y = block_icdf([&](int k) { return prob(n, k); }, V, ui, sh);
+    }
+    if (y < 0) y = block_argmax([&](int k) { return prob(n, k); }, V, sh, nullptr);
+    if (threadIdx.x == 0) P.n_acc[b] = n;
+    for (int s = threadIdx.x; s <= gamma; s += blockDim.x)
+        P.out_tok[(size_t)b * (gamma + 1) + s] = s < n ? x[s] : (s == n ? y : -1);
+}
+
+cudaError_t launch_accept(const AcceptParams& p, cudaStream_t st) {
+    if (p.B <= 0) return cudaSuccess;
+    k_accept<<<p.B, 1024, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace sd

@@ -1,0 +1,126 @@
+"""Single-operator parity of the CUDA library against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_08600_b200 import synth
+from gpu_util import DEV, quantize, to_dev, widen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sd():
+    from paper_2505_08600_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_philox_known_answers_on_device(sd, golden_dir):
+    rows = [[int(t, 16) for t in l.split()] for l in open(f"{golden_dir}/philox4x32_10_kat.txt") if not l.startswith("#")]
+    for r in rows:
+        ctr = to_dev(np.array([r[:4]], dtype=np.uint32))
+        out = torch.zeros((1, 4), dtype=torch.int32, device=DEV)
+        sd.sd_op_philox(ctr, r[4], r[5], out)
+        assert out.cpu().numpy().view(np.uint32)[0].tolist() == r[6:]
+    # a batch of counters against the oracle's generator
+    rng = np.random.default_rng(0)
+    ctr = rng.integers(0, 2**32, size=(257, 4), dtype=np.uint64).astype(np.uint32)
+    out = torch.zeros((257, 4), dtype=torch.int32, device=DEV)
+    sd.sd_op_philox(to_dev(ctr), 0xDEADBEEF, 0x12345678, out)
+    got = out.cpu().numpy().view(np.uint32)
+    for i in range(257):
+        assert got[i].tolist() == oracle.philox4x32_10(ctr[i], [0xDEADBEEF, 0x12345678]).tolist()
+
+
+LINEAR_SHAPES = [  # rows, n_out, n_in
+    (1, 8, 8), (5, 37, 64), (6, 1024, 256), (8, 688, 256), (9, 256, 688), (17, 130, 344), (6, 300, 1000),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rows,n_out,n_in", LINEAR_SHAPES)
+def test_linear_plain_kernel(sd, dtype, rows, n_out, n_in):
+    x = quantize(synth.make_logits((rows, n_in), seed=11, stream=rows), dtype)
+    w = quantize(synth.make_logits((n_out, n_in), seed=12, stream=n_out, std=0.05), dtype)
+    ref = oracle.linear(w, widen(x))
+    y = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    sd.sd_op_linear(to_dev(x), to_dev(w), y, sd.SD_BF16 if dtype == "bf16" else sd.SD_F32, impl=1)
+    got = y.cpu().numpy().astype(np.float64)
+    # fp32 accumulation of n_in products of magnitude ~0.05: a few 1e-6 at most
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-5 * np.sqrt(n_in / 64))
+
+
+ATTN_CASES = [  # H, Hkv, hd, max_ctx, positions of the rows
+    (4, 4, 64, 40, [0, 1, 7, 39]),
+    (4, 2, 64, 300, [5, 128, 129, 255, 299]),
+    (8, 2, 128, 700, [0, 63, 64, 65, 511, 699]),
+    (2, 1, 16, 33, [32, 31, 0]),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("H,Hkv,hd,max_ctx,positions", ATTN_CASES)
+def test_attention_over_cache(sd, dtype, H, Hkv, hd, max_ctx, positions):
+    n_slots, rows = 3, len(positions)
+    q = quantize(synth.make_logits((rows, H, hd), seed=21, stream=hd), dtype)
+    kc = quantize(synth.make_logits((n_slots, Hkv, max_ctx, hd), seed=22, stream=hd), dtype)
+    vc = quantize(synth.make_logits((n_slots, Hkv, max_ctx, hd), seed=23, stream=hd), dtype)
+    row_slot = np.array([(2 * r + 1) % n_slots for r in range(rows)], dtype=np.int32)
+    row_pos = np.array(positions, dtype=np.int32)
+    out = torch.zeros((rows, H, hd), dtype=torch.bfloat16 if dtype == "bf16" else torch.float32, device=DEV)
+    sd.sd_op_attention(to_dev(q), to_dev(kc), to_dev(vc), out, to_dev(row_slot), to_dev(row_pos), H, Hkv, hd, max_ctx,
+                       sd.SD_BF16 if dtype == "bf16" else sd.SD_F32)
+    got = out.float().cpu().numpy().astype(np.float64)
+    qf, kf, vf = widen(q), widen(kc), widen(vc)
+    for r in range(rows):
+        for h in range(H):
+            kvh = h // (H // Hkv)
+            n_ctx = positions[r] + 1
+            ref = oracle.attention_head(qf[r, h], kf[row_slot[r], kvh, :n_ctx], vf[row_slot[r], kvh, :n_ctx])
+            tol = 2e-2 if dtype == "bf16" else 2e-5          # bf16 output rounding: 2^-9 relative on values up to ~3
+            np.testing.assert_allclose(got[r, h], ref, rtol=0, atol=tol)
+
+
+def test_attention_inactive_row_gives_zeros(sd):
+    H, hd, max_ctx = 2, 64, 16
+    q = synth.make_logits((2, H, hd), seed=1)
+    kc = synth.make_logits((1, H, max_ctx, hd), seed=2)
+    out = torch.ones((2, H, hd), dtype=torch.float32, device=DEV)
+    sd.sd_op_attention(to_dev(q), to_dev(kc), to_dev(kc), out, to_dev(np.zeros(2, dtype=np.int32)),
+                       to_dev(np.array([-1, 3], dtype=np.int32)), H, H, hd, max_ctx, sd.SD_F32)
+    o = out.cpu().numpy()
+    assert (o[0] == 0).all() and np.abs(o[1]).max() > 0
+
+
+@pytest.mark.parametrize("V", [8, 1000, 1024, 32000])
+@pytest.mark.parametrize("T", [1.0, 0.7, 0.0])
+def test_softmax_and_draw(sd, V, T):
+    rows = 7
+    logits = synth.make_logits((rows, V), seed=31, stream=V, std=2.0)
+    u = np.array([oracle.uniform24(3, r, 0, 0, 0) for r in range(rows)], dtype=np.uint32)
+    u[0], u[1] = 1, 2**24
+    probs = torch.zeros((rows, V), dtype=torch.float32, device=DEV)
+    tok = torch.full((rows,), -7, dtype=torch.int32, device=DEV)
+    sd.sd_op_softmax_sample(to_dev(logits), T, to_dev(u), probs, tok)
+    p_ref = oracle.softmax_T(logits.astype(np.float64), T)
+    p_gpu = probs.cpu().numpy()
+    assert np.abs(p_gpu.astype(np.float64) - p_ref).max() <= 1e-3          # the stated probability tolerance
+    assert np.abs(p_gpu.astype(np.float64) - p_ref).max() <= 2e-6          # what fp32 arithmetic actually gives
+    t_gpu = tok.cpu().numpy()
+    same = 0
+    for r in range(rows):
+        t_ref = oracle.sample_icdf(p_ref[r], int(u[r]))
+        same += int(t_ref == t_gpu[r])
+        # the draw must be right for the oracle's CDF up to the rounding of the probabilities
+        cdf = np.cumsum(p_ref[r].astype(np.float64))
+        uu = u[r] / 2**24
+        k = int(t_gpu[r])
+        assert 0 <= k < V and p_ref[r][k] > 0
+        assert (cdf[k - 1] if k else 0.0) - 1e-4 < uu <= cdf[k] + 1e-4
+    if T == 0.0:
+        assert same == rows
+        assert (t_gpu == np.argmax(logits, axis=1)).all()
+    else:
+        assert same >= rows - 1

@@ -257,3 +257,13 @@ def test_linear_against_library_matmul_both_dtypes():
     one = np.array([[0x3F80, 0xC000]], dtype=np.uint16); x = np.array([[3.0, 0.5]]); y = np.empty((1, 1))
     oracle.lib().orc_linear(one.ctypes.data, 1, 1, 2, x.ctypes.data, 1, y.ctypes.data)
     assert y[0, 0] == 2.0
+
+
+def test_attention_head_against_library_softmax():
+    rng = np.random.default_rng(6)
+    q = rng.standard_normal(32); K = rng.standard_normal((19, 32)); V = rng.standard_normal((19, 32))
+    ref = scipy.special.softmax(K @ q / math.sqrt(32)) @ V
+    np.testing.assert_allclose(oracle.attention_head(q, K, V), ref, rtol=1e-12, atol=1e-14)
+    # one position: the value itself; identical keys: the mean of the values
+    np.testing.assert_allclose(oracle.attention_head(q, K[:1], V[:1]), V[0], atol=1e-15)
+    np.testing.assert_allclose(oracle.attention_head(q, np.tile(K[:1], (5, 1)), V[:5]), V[:5].mean(axis=0), atol=1e-14)
