@@ -144,6 +144,12 @@ sd_status sd_route_prompt(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, cons
 sd_status sd_draft_steps(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
                          int32_t* x_dev, float* q_dev);
 
+/* The same, but step s > 0 feeds x_forced_dev[.][s-1] instead of the token the draft drew
+ * at step s-1 (x_sampled_dev still receives the draws).  It lets a caller replay a recorded
+ * run step by step; sd_draft_steps is this call with both arrays the same. */
+sd_status sd_draft_steps_replay(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                                const int32_t* x_forced_dev, int32_t* x_sampled_dev, float* q_dev);
+
 /* Fig. 1(b): one pass of the target over [last token, x_0 .. x_{gamma-1}] of
  * every listed sequence against its KV cache (keys/values of the gamma+1 rows
  * are appended).  logits_dev [n_seq][gamma+1][vocab] fp32: row j is the

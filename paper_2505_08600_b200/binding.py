@@ -61,6 +61,7 @@ _PROTOS = {
     "sd_prefill": (_i, [_vp, _vp, _i]),
     "sd_route_prompt": (_i, [_vp, _vp, _i, _vp, _vp]),
     "sd_draft_steps": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
+    "sd_draft_steps_replay": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp]),
     "sd_verify": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "sd_accept": (_i, [C.POINTER(AcceptArgs)]),
     "sd_accept_seqs": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
@@ -204,6 +205,10 @@ class Context:
     def sd_draft_steps(self, seqs, gamma, x, q):
         a, p, n = _seqs(seqs)
         _check(self.L.sd_draft_steps(self.h, p, n, gamma, _dp(x), _dp(q)), "sd_draft_steps")
+
+    def sd_draft_steps_replay(self, seqs, gamma, x_forced, x_sampled, q):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_draft_steps_replay(self.h, p, n, gamma, _dp(x_forced), _dp(x_sampled), _dp(q)), "sd_draft_steps_replay")
 
     def sd_verify(self, seqs, gamma, x, logits):
         a, p, n = _seqs(seqs)

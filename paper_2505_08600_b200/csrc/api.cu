@@ -426,9 +426,14 @@ sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
 }
 
 sd_status sd_draft_steps(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, int32_t* x_dev, float* q_dev) {
+    return sd_draft_steps_replay(c, seqs, n_seq, gamma, x_dev, x_dev, q_dev);
+}
+
+sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_in,
+                                int32_t* x_dev, float* q_dev) {
     SeqList all;
     SD_TRY(make_list(c, seqs, n_seq, PH_READY, all));
-    if (gamma < 1 || gamma > c->cfg.max_gamma || !x_dev || !q_dev) return SD_ERR_INVALID_ARG;
+    if (gamma < 1 || gamma > c->cfg.max_gamma || !x_dev || !q_dev || !x_in) return SD_ERR_INVALID_ARG;
     if (c->cfg.n_drafts < 1) return SD_ERR_STATE;
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] + gamma - 1 > c->cfg.max_ctx) return SD_ERR_CAPACITY;
@@ -442,10 +447,10 @@ sd_status sd_draft_steps(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, i
         Model& M = c->models[1 + k];
         for (int s = 0; s < gamma; ++s) {
             if (s == 0) {
-                RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_dev};
+                RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_in};
                 SD_TRY(forward(c, M, g, plan, 2 * g.n, LOGITS_LAST, c->draft_logits));
             } else {
-                RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_dev};
+                RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_in};
                 SD_TRY(forward(c, M, g, plan, g.n, LOGITS_ALL, c->draft_logits));
             }
             CUDA_TRY(launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
