@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the verify step (target pass over gamma+1 rows + accept/reject + KV rollback).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 7b] [--impl reference]
+
+One JSON line on stdout.  `value` is verify-step tokens/s: B * (gamma + 1) query positions per
+sd_verify + sd_accept_seqs + sd_kv_rollback, timed with CUDA events on the library's stream with
+inputs resident in HBM.  The path does not shard: with N > 1 every rank runs an independent replica.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_08600_b200 import synth  # noqa: E402
+
+METRIC = "verify_step_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def eq1_speedup(alpha, gamma, c):
+    return (1 - alpha ** (gamma + 1)) / ((1 - alpha) * (gamma * c + 1))
+
+
+# ------------------------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on a bounded sample of the same verify step
+# ------------------------------------------------------------------------------------------
+def oracle_sample(cfg_name, sample_layers=1, reps=1):
+    """Times the oracle's cached forward over gamma+1 rows at the config's shapes with only
+    `sample_layers` of the layers, and the lm_head alone, then scales to the full depth."""
+    import oracle
+    cfg = synth.CONFIGS[cfg_name]
+    wl, t = cfg["workload"], dict(cfg["target"])
+    gamma = wl["gamma"]
+    n_prompt = wl["prompt"] if isinstance(wl["prompt"], int) else (wl["prompt"][0] + wl["prompt"][1]) // 2
+    B = wl["batch"]
+    full_layers = t["n_layers"]
+    t["n_layers"] = sample_layers
+    w = synth.make_weights(t, seed=0, model_index=0, dtype=cfg["dtype"])
+    m = oracle.OracleModel(t, w)
+    cache = m.new_cache(n_prompt + gamma + 1)
+    rng = np.random.default_rng(0)
+    cache.k[:] = rng.standard_normal(cache.k.shape[0])          # attention cost does not depend on the values
+    cache.v[:] = rng.standard_normal(cache.v.shape[0])
+    toks = synth.make_prompt(t["vocab"], gamma + 1, seed=1)
+    cores = len(os.sched_getaffinity(0))
+    t_with, t_layers = [], []
+    for _ in range(reps):
+        t0 = time.perf_counter(); cache.forward(toks, n_prompt - 1, want_logits=True); t_with.append(time.perf_counter() - t0)
+        t0 = time.perf_counter(); cache.forward(toks, n_prompt - 1, want_logits=False); t_layers.append(time.perf_counter() - t0)
+    tl, tw = min(t_layers), min(t_with)
+    step_s = B * (tl / sample_layers * full_layers + (tw - tl))  # sequences are independent: B of them cost B times one
+    return dict(value=B * (gamma + 1) / step_s, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{sample_layers} of {full_layers} layers + lm_head at full width, {gamma + 1} rows, context {n_prompt}, "
+                       f"one sequence; scaled by layers and batch {B}",
+                seconds_measured=round(sum(t_with) + sum(t_layers), 2), step_seconds_scaled=round(step_s, 2))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        oracle_sample(args.config)
+    for _ in range(max(1, min(args.steps, 5))):
+        vals.append(oracle_sample(args.config))
+    v = statistics.median(x["value"] for x in vals)
+    cb = dict(vals[0]); cb["value"] = v
+    wl = synth.CONFIGS[args.config]["workload"]
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+        "warmup": args.warmup, "ms_per_step": 1000.0 * wl["batch"] * (wl["gamma"] + 1) / v, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.config}: verify step, oracle on host cores, bounded sample"},
+        "cpu_baseline": cb, "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------
+def device_weights(torch, dims, dtype, seed, model_index, dev):
+    """Random-init weights generated on the device, tensor by tensor (N(0, 0.02), gains 1)."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed * 1000003 + model_index)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    shapes = synth.mat_shapes(dims)
+
+    def normal(shape):
+        return (torch.randn(shape, generator=g, device=dev, dtype=torch.float32) * 0.02).to(td).contiguous()
+
+    yield "embed", 0, normal((dims["vocab"], dims["d_model"]))
+    yield "lm_head", 0, normal((dims["vocab"], dims["d_model"]))
+    ones = torch.ones(dims["d_model"], device=dev, dtype=torch.float32)
+    yield "final_norm", 0, ones
+    for l in range(dims["n_layers"]):
+        for name in synth.LAYER_MATS:
+            yield name, l, normal(shapes[name])
+        yield "norm1", l, ones
+        yield "norm2", l, ones
+
+
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, gpu_id):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_id), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_08600_b200 import binding as sd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)      # only for the barrier and the max over ranks
+    cfg = synth.CONFIGS[args.config]
+    wl, tdims = cfg["workload"], cfg["target"]
+    gamma = args.gamma if args.gamma is not None else wl["gamma"]
+    B, V, T, seed = wl["batch"], tdims["vocab"], wl["temperature"], wl["seed"]
+    K, W = args.steps, args.warmup
+    n_iter_phase = min(10, K)
+    total_steps = 2 * (K + W) + args.profile_steps + n_iter_phase + 8
+    if isinstance(wl["prompt"], int):
+        lens = [wl["prompt"]] * B
+    else:
+        lens = synth.make_prompt_lengths(B, wl["prompt"][0], wl["prompt"][1], seed=seed).tolist()
+    max_ctx = max(wl["max_ctx"], max(lens) + (gamma + 1) * total_steps + 8)
+
+    ctx = sd.Context(tdims, cfg["drafts"], cfg["dtype"], B, max_ctx, max(gamma, 1), T, seed, clf_d_hidden=cfg["classifier"][1], device=dev)
+    for mid, dims in enumerate([tdims] + list(cfg["drafts"])):
+        for name, l, tensor in device_weights(torch, dims, cfg["dtype"], 0, mid, dev):
+            ctx.sd_load_tensor(mid, sd.TENSOR_KIND[name], l, tensor)
+    clf = synth.make_classifier(*cfg["classifier"], seed=0)
+    ctx.sd_load_classifier(clf["w1"], clf["b1"], clf["w2"], clf["b2"])
+    torch.cuda.synchronize()
+
+    seqs = list(range(B))
+    for s in seqs:
+        ctx.sd_seq_begin(s, synth.make_prompt(V, lens[s], seed=seed, seq=s), s)
+    n_drafts = len(cfg["drafts"])
+    routed = ctx.sd_route_prompt(seqs) if B == 1 else ctx.sd_route_prompt(seqs, forced_task=[s % n_drafts for s in seqs])
+    ctx.sd_prefill(seqs)
+
+    x = torch.zeros((B, gamma), dtype=torch.int32, device=dev)
+    q = torch.zeros((B, gamma, V), dtype=torch.float32, device=dev)
+    logits = torch.zeros((B, gamma + 1, V), dtype=torch.float32, device=dev)
+    n_acc = torch.zeros((B,), dtype=torch.int32, device=dev)
+    out_tok = torch.zeros((B, gamma + 1), dtype=torch.int32, device=dev)
+    ctx.sd_draft_steps(seqs, gamma, x, q)          # the drafts every timed verify step scores (values do not change its cost)
+    torch.cuda.synchronize()
+
+    def verify_step():
+        ctx.sd_verify(seqs, gamma, x, logits)
+        ctx.sd_accept_seqs(seqs, gamma, logits, q, x, n_acc, out_tok)
+        ctx.sd_kv_rollback(seqs, gamma, n_acc, out_tok)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    stream = torch.cuda.current_stream(dev)
+    # ---- phase A: the headline, device-resident inputs
+    for _ in range(W):
+        verify_step()
+    l0 = ctx.sd_launch_count()
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(dev).uuid)
+        gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(K):
+        verify_step()
+    ev1.record(stream)
+    barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    clocks = sampler.stop()
+    launches = ctx.sd_launch_count() - l0
+    ms_step = ms_total / K
+    value = world * B * (gamma + 1) / (ms_step * 1e-3)
+    ctx.sd_seq_read(0)
+
+    # ---- per-kernel split of the same step (events between launches; separate from the timed run)
+    ctx.sd_profile(1)
+    for _ in range(args.profile_steps):
+        verify_step()
+    prof = ctx.sd_profile_read()
+    ctx.sd_profile(0)
+    lin_ms = prof["linear"]["ms"] / args.profile_steps
+    n_ctx = [int(ctx.sd_seq_read(s)[0].shape[0]) for s in seqs]
+    esz = 2 if cfg["dtype"] == "bf16" else 4
+    weight_bytes = synth.param_count(tdims, streamed_only=True) * esz
+    kv_bytes = sum(n_ctx) * 2 * tdims["n_layers"] * tdims["n_kv_heads"] * tdims["head_dim"] * esz
+    peak, peak_kind = _peaks()
+    achieved = weight_bytes / (lin_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "weight GEMMs (all launches of one verify step)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "algorithmic_bytes_per_step": weight_bytes, "kernel_ms_per_step": lin_ms,
+                "whole_step": {"bytes": weight_bytes + kv_bytes, "gbs": (weight_bytes + kv_bytes) / (ms_step * 1e-3) / 1e9,
+                               "frac_of_peak": (weight_bytes + kv_bytes) / (ms_step * 1e-3) / 1e9 / peak,
+                               "frac_of_nominal_8tbs": (weight_bytes + kv_bytes) / (ms_step * 1e-3) / 1e9 / 8000.0},
+                "split_ms_per_step": {k: v["ms"] / args.profile_steps for k, v in prof.items()}}
+
+    # ---- e2e: drafts and results in pinned host memory, copies inside the timed region
+    xh = x.cpu().pin_memory(); qh = q.cpu().pin_memory()
+    nh = torch.zeros((B,), dtype=torch.int32).pin_memory(); oh = torch.zeros((B, gamma + 1), dtype=torch.int32).pin_memory()
+    for _ in range(W):
+        ctx.sd_verify_accept_host(seqs, gamma, xh, qh, nh, oh)
+    barrier()
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for _ in range(K):
+        ctx.sd_verify_accept_host(seqs, gamma, xh, qh, nh, oh)
+    ev1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)) / K
+    e2e = {"value": world * B * (gamma + 1) / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": int(xh.numel() * 4 + qh.numel() * 4), "d2h_bytes_per_step": int(nh.numel() * 4 + oh.numel() * 4)}
+    ctx.sd_seq_read(0)
+
+    # ---- whole iterations and the cost ratio c of Eq. 1
+    def timed(fn, n):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    def iteration():
+        ctx.sd_draft_steps(seqs, gamma, x, q)
+        verify_step()
+
+    ctx.sd_draft_steps(seqs, gamma, x, q)
+    draft_ms = timed(lambda: ctx.sd_draft_steps(seqs, gamma, x, q), 3) / gamma
+    l1 = torch.zeros((B, 1, V), dtype=torch.float32, device=dev)
+    ctx.sd_target_step(seqs, l1)
+    decode_ms = timed(lambda: ctx.sd_target_step(seqs, l1), 3)
+    iter_ms = timed(iteration, n_iter_phase)
+    c = draft_ms / decode_ms
+    extras = {"draft_step_ms": draft_ms, "target_decode_step_ms": decode_ms, "iteration_ms": iter_ms, "c": c,
+              "verify_over_decode": ms_step / decode_ms,
+              "eq1_speedup": {f"alpha={a}": eq1_speedup(a, gamma, c) for a in (0.6, 0.8)},
+              "routed_drafts": [int(r) for r in routed]}
+    status = ctx.sd_device_status()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_sample(args.config)
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
+            "config": {"workload": f"{args.config}: batch {B}, gamma {gamma}, prompt {lens if B > 1 else lens[0]}, "
+                                   f"target {tdims['n_layers']}x{tdims['d_model']}, verify step = sd_verify + sd_accept_seqs + sd_kv_rollback",
+                       "l2": "weights (>= 2 GB per step) far exceed the 126 MB L2; no flush", "replicas": world,
+                       "device_status": status},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras,
+        }))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="7b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--gamma", type=int, default=None)
+    ap.add_argument("--profile-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -193,7 +193,28 @@ sd_status sd_accept_seqs(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int g
 sd_status sd_kv_rollback(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
                          const int32_t* n_acc_dev, const int32_t* out_tok_dev);
 
+/* One verify step for a caller whose drafts live in host memory: copies x_host [n_seq][gamma]
+ * and q_host [n_seq][gamma][vocab] to the device, runs sd_verify, sd_accept_seqs and
+ * sd_kv_rollback on them and copies n_acc [n_seq] and out_tok [n_seq][gamma+1] back.
+ * Pinned host memory makes the copies asynchronous.  Synchronises before returning. */
+sd_status sd_verify_accept_host(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                                const int32_t* x_host, const float* q_host,
+                                int32_t* n_acc_host, int32_t* out_tok_host);
+
 /* -------------------------------------------------------------- observation */
+
+/* Number of kernels this context has launched since sd_create. */
+sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);
+
+/* Per-kernel timing for measurements: while enabled, a CUDA event is recorded in front of
+ * every launch.  sd_profile_read synchronises, adds the time between consecutive events to
+ * the category of the launch that followed the first one, and clears the record.
+ * Categories: 0 weight GEMMs, 1 attention, 2 norm/rotary/elementwise, 3 sampling and
+ * accept, 4 state updates. */
+#define SD_PROF_NCAT 5
+sd_status sd_profile(sd_ctx* ctx, int enable);
+sd_status sd_profile_read(sd_ctx* ctx, float* ms_by_cat, uint32_t* launches_by_cat);
+
 
 /* Copies the sequence's tokens (up to cap) and counters to the host; also
  * refreshes the host's capacity bookkeeping with the true length.  Synchronises. */

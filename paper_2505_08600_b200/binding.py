@@ -66,6 +66,10 @@ _PROTOS = {
     "sd_accept": (_i, [C.POINTER(AcceptArgs)]),
     "sd_accept_seqs": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_kv_rollback": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
+    "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
+    "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
+    "sd_profile": (_i, [_vp, _i]),
+    "sd_profile_read": (_i, [_vp, _vp, _vp]),
     "sd_seq_read": (_i, [_vp, _i, _vp, _i, C.POINTER(C.c_int32), C.POINTER(Counters)]),
     "sd_seq_force": (_i, [_vp, _i, _vp, _i, _i, C.c_uint32]),
     "sd_device_status": (_i, [_vp, C.POINTER(C.c_uint32)]),
@@ -225,6 +229,27 @@ class Context:
     def sd_target_step(self, seqs, logits):
         a, p, n = _seqs(seqs)
         _check(self.L.sd_target_step(self.h, p, n, _dp(logits)), "sd_target_step")
+
+    def sd_verify_accept_host(self, seqs, gamma, x_host, q_host, n_acc_host, out_tok_host):
+        """x_host, q_host, n_acc_host, out_tok_host: CPU tensors (pinned for asynchronous copies)."""
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_verify_accept_host(self.h, p, n, gamma, _dp(x_host), _dp(q_host), _dp(n_acc_host), _dp(out_tok_host)),
+               "sd_verify_accept_host")
+
+    def sd_launch_count(self):
+        v = C.c_uint64()
+        _check(self.L.sd_launch_count(self.h, C.byref(v)), "sd_launch_count")
+        return v.value
+
+    def sd_profile(self, enable):
+        _check(self.L.sd_profile(self.h, int(enable)), "sd_profile")
+
+    def sd_profile_read(self):
+        ms = (C.c_float * 5)()
+        n = (C.c_uint32 * 5)()
+        _check(self.L.sd_profile_read(self.h, ms, n), "sd_profile_read")
+        names = ("linear", "attention", "elementwise", "sampling", "state")
+        return {k: dict(ms=float(ms[i]), launches=int(n[i])) for i, k in enumerate(names)}
 
     # ---- observation
     def sd_seq_read(self, seq, cap=None):

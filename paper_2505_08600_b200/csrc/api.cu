@@ -66,6 +66,14 @@ struct sd_ctx {
     // host bookkeeping
     std::vector<int> phase, len_ub, n_prompt, draft_id;
     size_t arena_used;
+    // staging for the host-buffer entry point
+    int32_t* st_x; float* st_q; float* st_logits; int32_t* st_nacc; int32_t* st_out;
+    // launch accounting and optional per-category timing
+    uint64_t launches;
+    bool prof_on;
+    std::vector<cudaEvent_t> prof_ev;
+    std::vector<int> prof_cat;
+    size_t prof_used;
 };
 
 namespace {
@@ -155,6 +163,12 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     for (int i = 0; i < nm; ++i)
         c->attn_ws_bytes = std::max(c->attn_ws_bytes, attention_workspace_bytes((int)R, ms[i].n_heads, ms[i].head_dim, cfg.max_ctx));
     c->attn_ws = B.take(c->attn_ws_bytes);
+    const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
+    c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
+    c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
+    c->st_logits = (float*)B.take(sizeof(float) * std::min((size_t)SD_MAX_ROWS, (size_t)S * (cfg.max_gamma + 1)) * V0);
+    c->st_nacc = (int32_t*)B.take(sizeof(int32_t) * S);
+    c->st_out = (int32_t*)B.take(sizeof(int32_t) * S * (cfg.max_gamma + 1));
     if (cfg.clf_d_hidden > 0 && cfg.n_drafts > 0) {
         c->clf_w1 = (float*)B.take(sizeof(float) * (size_t)cfg.clf_d_hidden * ms[0].d_model);
         c->clf_b1 = (float*)B.take(sizeof(float) * cfg.clf_d_hidden);
@@ -179,8 +193,33 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
         if (s__ != SD_OK) return s__;     \
     } while (0)
 
+// Categories of the optional per-kernel timing (sd_profile).
+enum { CAT_LINEAR = 0, CAT_ATTENTION = 1, CAT_ELEMENTWISE = 2, CAT_SAMPLING = 3, CAT_STATE = 4, CAT_NONE = 5 };
+
+// When profiling is on, an event is recorded in front of every launch and tagged with the
+// category of that launch; sd_profile_read adds up the gaps between consecutive events.
+cudaError_t prof_mark(sd_ctx* c, int cat) {
+    if (!c->prof_on) return cudaSuccess;
+    if (c->prof_used == c->prof_ev.size()) {
+        cudaEvent_t e;
+        cudaError_t err = cudaEventCreate(&e);
+        if (err != cudaSuccess) return err;
+        c->prof_ev.push_back(e);
+        c->prof_cat.push_back(CAT_NONE);
+    }
+    c->prof_cat[c->prof_used] = cat;
+    return cudaEventRecord(c->prof_ev[c->prof_used++], c->st);
+}
+
+#define LAUNCH(cat, expr)                 \
+    do {                                  \
+        CUDA_TRY(prof_mark(c, cat));      \
+        CUDA_TRY(expr);                   \
+        c->launches += 1;                 \
+    } while (0)
+
 sd_status linear(sd_ctx* c, const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype) {
-    CUDA_TRY(launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, c->st));
+    LAUNCH(CAT_LINEAR, launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, c->st));
     return SD_OK;
 }
 
@@ -191,33 +230,34 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
-    CUDA_TRY(launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
         void* vc = M.vcache + M.kv_layer_bytes * l;
-        CUDA_TRY(launch_rmsnorm(c->h, L.norm1, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, L.norm1, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
         SD_TRY(linear(c, c->xn, L.wqkv, c->lin, n_rows, M.n_qkv(), d, dt));
-        CUDA_TRY(launch_rope_kv(c->lin, c->q, kc, vc, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
+        LAUNCH(CAT_ELEMENTWISE, launch_rope_kv(c->lin, c->q, kc, vc, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
                                 M.rope_cos, M.rope_sin, c->S.status, st));
-        CUDA_TRY(launch_attention(c->q, kc, vc, c->attn, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
+        LAUNCH(CAT_ATTENTION, launch_attention(c->q, kc, vc, c->attn, dt, c->row_slot, c->row_pos, n_rows, H, Hkv, hd, c->cfg.max_ctx,
                                   c->attn_ws, c->attn_ws_bytes, st));
         SD_TRY(linear(c, c->attn, L.wo, c->lin, n_rows, d, H * hd, dt));
-        CUDA_TRY(launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
-        CUDA_TRY(launch_rmsnorm(c->h, L.norm2, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, L.norm2, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
         SD_TRY(linear(c, c->xn, L.wgu, c->lin, n_rows, 2 * F, d, dt));
-        CUDA_TRY(launch_swiglu(c->lin, c->act, dt, n_rows, F, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_swiglu(c->lin, c->act, dt, n_rows, F, st));
         SD_TRY(linear(c, c->act, L.wd, c->lin, n_rows, d, F, dt));
-        CUDA_TRY(launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
     }
     if (mode == LOGITS_ALL) {
-        CUDA_TRY(launch_rmsnorm(c->h, M.final_norm, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, M.final_norm, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
         SD_TRY(linear(c, c->xn, M.lm_head, logits_out, n_rows, m.vocab, d, dt));
     } else if (mode == LOGITS_LAST) {
         const int R = plan.rows_per_seq;
-        CUDA_TRY(launch_rmsnorm(c->h, M.final_norm, c->xn, dt, list.n, d, m.rms_eps, R, R - 1, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, M.final_norm, c->xn, dt, list.n, d, m.rms_eps, R, R - 1, st));
         SD_TRY(linear(c, c->xn, M.lm_head, logits_out, list.n, m.vocab, d, dt));
     }
+    CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
 
@@ -278,6 +318,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     layout(c, models, B);
     c->arena_used = B.off;
     c->clf_loaded = false;
+    c->launches = 0; c->prof_on = false; c->prof_used = 0;
     c->phase.assign(cfg->max_seqs, PH_FREE);
     c->len_ub.assign(cfg->max_seqs, 0);
     c->n_prompt.assign(cfg->max_seqs, 0);
@@ -310,6 +351,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
 sd_status sd_destroy(sd_ctx* c) {
     if (!c) return SD_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->st);
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     delete c;
     return SD_OK;
 }
@@ -365,7 +407,7 @@ sd_status sd_seq_begin(sd_ctx* c, int seq, const int32_t* prompt, int n_prompt, 
     for (int i = 0; i < n_prompt; ++i) if (prompt[i] < 0 || prompt[i] >= V) return SD_ERR_INVALID_ARG;
     CUDA_TRY(cudaMemcpyAsync(c->S.tokens + (size_t)seq * c->S.tok_stride, prompt, sizeof(int32_t) * n_prompt,
                              cudaMemcpyHostToDevice, c->st));
-    CUDA_TRY(launch_set_state(c->S, seq, n_prompt, 0, 0, 0u, seq_id, 1, c->st));
+    LAUNCH(CAT_STATE, launch_set_state(c->S, seq, n_prompt, 0, 0, 0u, seq_id, 1, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
     c->phase[seq] = PH_BEGUN;
     c->len_ub[seq] = n_prompt;
@@ -389,7 +431,7 @@ sd_status sd_route_prompt(sd_ctx* c, const int32_t* seqs, int n_seq, const int32
     }
     if (need_clf && !c->clf_loaded) return SD_ERR_STATE;
     Model& T = c->models[0];
-    CUDA_TRY(launch_classifier(c->S, list, fl, T.embed, T.d.dtype, T.d.d_model, T.d.vocab, c->clf_w1, c->clf_b1,
+    LAUNCH(CAT_ELEMENTWISE, launch_classifier(c->S, list, fl, T.embed, T.d.dtype, T.d.d_model, T.d.vocab, c->clf_w1, c->clf_b1,
                                c->cfg.clf_d_hidden, c->clf_w2, c->clf_b2, K, c->st));
     std::vector<int32_t> ids(c->cfg.max_seqs);
     CUDA_TRY(cudaMemcpyAsync(ids.data(), c->S.draft_id, sizeof(int32_t) * ids.size(), cudaMemcpyDeviceToHost, c->st));
@@ -419,7 +461,7 @@ sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
                 SD_TRY(forward(c, M, one, plan, rows, LOGITS_NONE, nullptr));
             }
         }
-        CUDA_TRY(launch_set_state(c->S, s, n + 1, n, n, 0u, 0u, 0, c->st));
+        LAUNCH(CAT_STATE, launch_set_state(c->S, s, n + 1, n, n, 0u, 0u, 0, c->st));
         c->phase[s] = PH_READY;
     }
     return SD_OK;
@@ -453,7 +495,7 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
                 RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_in};
                 SD_TRY(forward(c, M, g, plan, g.n, LOGITS_ALL, c->draft_logits));
             }
-            CUDA_TRY(launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
+            LAUNCH(CAT_SAMPLING, launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
         }
     }
     return SD_OK;
@@ -503,7 +545,8 @@ sd_status sd_accept_seqs(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, c
     p.target = logits_dev; p.target_is_logits = 1; p.q = q_dev; p.x = x_dev;
     p.B = n_seq; p.gamma = gamma; p.V = c->models[0].d.vocab; p.T = c->cfg.temperature; p.seed = c->cfg.seed;
     p.iter = c->S.iter; p.seq_id = c->S.seq_id; p.use_list = 1; p.n_acc = n_acc_dev; p.out_tok = out_tok_dev;
-    CUDA_TRY(launch_accept(p, c->st));
+    LAUNCH(CAT_SAMPLING, launch_accept(p, c->st));
+    CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
 
@@ -513,7 +556,8 @@ sd_status sd_kv_rollback(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, c
     if (gamma < 0 || gamma > c->cfg.max_gamma || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] + gamma + 1 > c->S.tok_stride) return SD_ERR_CAPACITY;
-    CUDA_TRY(launch_rollback(c->S, list, gamma, n_acc_dev, out_tok_dev, c->st));
+    LAUNCH(CAT_STATE, launch_rollback(c->S, list, gamma, n_acc_dev, out_tok_dev, c->st));
+    CUDA_TRY(prof_mark(c, CAT_NONE));
     for (int i = 0; i < n_seq; ++i) c->len_ub[seqs[i]] += gamma + 1;
     return SD_OK;
 }
@@ -538,7 +582,7 @@ sd_status sd_seq_force(sd_ctx* c, int seq, const int32_t* tokens, int n_tokens, 
     if (c->phase[seq] < PH_READY) return SD_ERR_STATE;
     if (n_tokens > c->cfg.max_ctx) return SD_ERR_CAPACITY;
     CUDA_TRY(cudaMemcpyAsync(c->S.tokens + (size_t)seq * c->S.tok_stride, tokens, sizeof(int32_t) * n_tokens, cudaMemcpyHostToDevice, c->st));
-    CUDA_TRY(launch_set_state(c->S, seq, n_tokens, n_tokens - 1, draft_kv_len, iter, 0u, 0, c->st));
+    LAUNCH(CAT_STATE, launch_set_state(c->S, seq, n_tokens, n_tokens - 1, draft_kv_len, iter, 0u, 0, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
     c->len_ub[seq] = n_tokens;
     return SD_OK;
@@ -549,6 +593,55 @@ sd_status sd_device_status(sd_ctx* c, uint32_t* flags) {
     CUDA_TRY(cudaMemcpyAsync(flags, c->S.status, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaMemsetAsync(c->S.status, 0, sizeof(uint32_t), c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_verify_accept_host(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_host,
+                                const float* q_host, int32_t* n_acc_host, int32_t* out_tok_host) {
+    if (!c || !seqs || n_seq < 1 || n_seq > c->cfg.max_seqs || gamma < 0 || gamma > c->cfg.max_gamma) return SD_ERR_INVALID_ARG;
+    if (!n_acc_host || !out_tok_host || (gamma > 0 && (!x_host || !q_host))) return SD_ERR_INVALID_ARG;
+    if (n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_CAPACITY;
+    const size_t V = c->models[0].d.vocab;
+    if (gamma > 0) {
+        CUDA_TRY(cudaMemcpyAsync(c->st_x, x_host, sizeof(int32_t) * n_seq * gamma, cudaMemcpyHostToDevice, c->st));
+        CUDA_TRY(cudaMemcpyAsync(c->st_q, q_host, sizeof(float) * n_seq * gamma * V, cudaMemcpyHostToDevice, c->st));
+    }
+    SD_TRY(sd_verify(c, seqs, n_seq, gamma, c->st_x, c->st_logits));
+    SD_TRY(sd_accept_seqs(c, seqs, n_seq, gamma, c->st_logits, c->st_q, c->st_x, c->st_nacc, c->st_out));
+    SD_TRY(sd_kv_rollback(c, seqs, n_seq, gamma, c->st_nacc, c->st_out));
+    CUDA_TRY(cudaMemcpyAsync(n_acc_host, c->st_nacc, sizeof(int32_t) * n_seq, cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaMemcpyAsync(out_tok_host, c->st_out, sizeof(int32_t) * n_seq * (gamma + 1), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_launch_count(sd_ctx* c, uint64_t* out) {
+    if (!c || !out) return SD_ERR_INVALID_ARG;
+    *out = c->launches;
+    return SD_OK;
+}
+
+sd_status sd_profile(sd_ctx* c, int enable) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    c->prof_on = enable != 0;
+    c->prof_used = 0;
+    return SD_OK;
+}
+
+sd_status sd_profile_read(sd_ctx* c, float* ms_by_cat, uint32_t* launches_by_cat) {
+    if (!c || !ms_by_cat || !launches_by_cat) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (int i = 0; i < SD_PROF_NCAT; ++i) { ms_by_cat[i] = 0.f; launches_by_cat[i] = 0; }
+    for (size_t i = 0; i + 1 < c->prof_used; ++i) {
+        const int cat = c->prof_cat[i];
+        if (cat < 0 || cat >= SD_PROF_NCAT) continue;
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]));
+        ms_by_cat[cat] += ms;
+        launches_by_cat[cat] += 1;
+    }
+    c->prof_used = 0;
     return SD_OK;
 }
 
