@@ -7,6 +7,7 @@
 
 #include <vector>
 
+#include "gemm_tc.h"
 #include "kernels.h"
 
 using namespace sd;
@@ -646,16 +647,36 @@ sd_status sd_profile_read(sd_ctx* c, float* ms_by_cat, uint32_t* launches_by_cat
 }
 
 // ------------------------------------------------------------------ single operators
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else return 148;
+    }
+    return n;
+}
+
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl) {
-    (void)rows; (void)n_out; (void)n_in; (void)dtype; (void)impl;
-    return 0;
+    if (impl == 1 || dtype != SD_BF16 || !gemm_tc_supported(rows, n_out, n_in)) return 0;
+    return gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
 }
 
 sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype, int impl,
                        void* workspace, size_t workspace_bytes, void* stream) {
-    (void)workspace; (void)workspace_bytes;
     if (!x || !w || !y || rows < 1 || n_out < 1 || n_in < 1 || (dtype != SD_F32 && dtype != SD_BF16)) return SD_ERR_INVALID_ARG;
-    if (impl == 2) return SD_ERR_UNSUPPORTED;
+    if (impl < 0 || impl > 2) return SD_ERR_INVALID_ARG;
+    const bool tc_ok = dtype == SD_BF16 && gemm_tc_supported(rows, n_out, n_in);
+    if (impl == 2 && !tc_ok) return SD_ERR_UNSUPPORTED;
+    if (impl == 2 || (impl == 0 && tc_ok)) {
+        const GemmGeom g = gemm_geometry(rows, n_out, n_in, sm_count());
+        if (!workspace || workspace_bytes < gemm_partials_bytes(g)) return SD_ERR_OOM;
+        TensorMap tw, tx;
+        if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
+        CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, (cudaStream_t)stream));
+        CUDA_TRY(launch_reduce_plain((const float*)workspace, g, y, (cudaStream_t)stream));
+        return SD_OK;
+    }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;
     CUDA_TRY(launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, (cudaStream_t)stream));
     return SD_OK;

@@ -1,0 +1,313 @@
+// Weight-streaming GEMM on the fifth-generation tensor cores (tcgen05 + TMEM + TMA), bf16.
+//
+//   P = X[m_tok][K] * W[n_out][K]^T          (fp32 accumulation)
+//
+// The weight matrix is the 128-row operand (A, K-major), the handful of token rows is the
+// narrow one (B, N = m_pad = m_tok rounded up to 16), so one tcgen05.mma covers 128 weight
+// rows x m_pad tokens x 16 reduction elements and the accumulator lives in TMEM as
+// 128 lanes x m_pad fp32 columns.  The kernel is bound by the one pass over W from HBM:
+//   - tiles of 128 rows x 64 k (16 KB, 128-byte swizzle) arrive by TMA into a ring of stages;
+//   - work is cut stream-K style: the (row tile, k block) pairs are numbered row-tile-major
+//     and split evenly over the grid, so that every SM streams the same number of bytes
+//     whatever the matrix shape; a CTA whose range crosses a tile boundary produces one
+//     partial accumulator ("segment") per tile it touches;
+//   - segments are written to a workspace as fp32 [slot][token][128]; the consumer kernels
+//     add the segments of a tile in a fixed order, which keeps results run-to-run identical.
+// Roles: warp 0 issues TMA, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM.
+// Every wait is bounded; on expiry the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
+#include <cuda.h>
+
+#include "gemm_tc.h"
+
+namespace sd {
+
+namespace {
+
+constexpr int TILE_N = 128;                 // weight rows per tile (UMMA M)
+constexpr int TILE_K = 64;                  // bf16 elements per k block = one 128-byte swizzle row
+constexpr int A_BYTES = TILE_N * TILE_K * 2;
+constexpr int NUM_THREADS = 192;
+constexpr int MAX_STAGES = 12;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after about two seconds, or as soon as another role has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > 2000000000ull) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);      // start address
+    d |= (uint64_t)1 << 16;                             // leading byte offset (unused for this layout)
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                             // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t r[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
+struct Shared {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, GemmGeom g,
+               float* __restrict__ partials, uint32_t* status) {
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ Shared sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tiles0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;        // 1024-byte aligned stage ring
+    const uint32_t stage_bytes = A_BYTES + (uint32_t)g.m_pad * 128u;
+    volatile int* abort_flag = &sh.abort_flag;
+
+    // this CTA's share of the (row tile, k block) pairs
+    const uint32_t T = (uint32_t)g.n_tiles * (uint32_t)g.kb_per_tile;
+    const uint32_t u0 = (uint32_t)(((uint64_t)blockIdx.x * T) / gridDim.x);
+    const uint32_t u1 = (uint32_t)(((uint64_t)(blockIdx.x + 1) * T) / gridDim.x);
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * (uint32_t)g.m_pad) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; ++s) { mbar_init(smem_u32(&sh.full[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint64_t pol_stream, pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            uint32_t it = 0;
+            for (uint32_t u = u0; u < u1; ++u, ++it) {
+                const int s = it % g.stages;
+                const uint32_t ph = (it / g.stages) & 1u;
+                if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag)) break;
+                const int tile = u / g.kb_per_tile, kb = u % g.kb_per_tile;
+                const uint32_t a = tiles0 + s * stage_bytes, b = a + A_BYTES, bar = smem_u32(&sh.full[s]);
+                mbar_expect_tx(bar, stage_bytes);
+                tma_load_2d(a, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
+                tma_load_2d(b, &tm_x, kb * TILE_K, 0, bar, pol_keep);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.m_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+            uint32_t it = 0, seg = 0;
+            bool ok = true;
+            for (uint32_t u = u0; u < u1 && ok; ++seg) {
+                const uint32_t kb0 = u % g.kb_per_tile;
+                const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
+                const uint32_t buf = seg & 1u;
+                if (!mbar_wait(smem_u32(&sh.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, abort_flag)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)g.m_pad;
+                for (uint32_t j = 0; j < n_kb; ++j, ++it) {
+                    const int s = it % g.stages;
+                    const uint32_t ph = (it / g.stages) & 1u;
+                    if (!mbar_wait(smem_u32(&sh.full[s]), ph, abort_flag)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a = tiles0 + s * stage_bytes;
+                    const uint64_t da = umma_desc(a), db = umma_desc(a + A_BYTES);
+#pragma unroll
+                    for (uint32_t k = 0; k < TILE_K / 16; ++k)     // 16 elements = 32 bytes further along the swizzled row
+                        umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (j | k) != 0u);
+                    umma_commit(smem_u32(&sh.empty[s]));           // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(smem_u32(&sh.tmem_full[buf]));
+                u += n_kb;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: TMEM -> partials
+        const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
+        const int row = quarter * 32 + lane;                               // weight row inside the tile
+        uint32_t seg = 0;
+        for (uint32_t u = u0; u < u1; ++seg) {
+            const uint32_t kb0 = u % g.kb_per_tile;
+            const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
+            const uint32_t buf = seg & 1u;
+            if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
+            for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (c0 + j < g.m_tok) out[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+            u += n_kb;
+        }
+    }
+
+    // ---------------------------------------------------------------------- wind-down
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (sh.abort_flag) {
+        if (threadIdx.x == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
+        const uint64_t t0 = global_ns();                   // let copies in flight land before the CTA goes away
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+// bf16 matrix [rows][K] row-major as a 2-D tensor map with boxes of box_rows x 64 elements,
+// 128-byte swizzle; reads outside the matrix return zeros.
+bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || ((uintptr_t)base & 15) || (K & 7) || box_rows < 1 || box_rows > 256) return false;
+    static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "tensor map size");
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)TILE_K, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
+    GemmGeom g;
+    g.m_tok = m_tok;
+    g.m_pad = (m_tok + 15) & ~15;
+    g.n_out = n_out;
+    g.K = K;
+    g.n_tiles = (n_out + TILE_N - 1) / TILE_N;
+    g.kb_per_tile = (K + TILE_K - 1) / TILE_K;
+    const long long T = (long long)g.n_tiles * g.kb_per_tile;
+    g.grid = (int)std::min<long long>(n_sm, T);
+    const int per_cta = (int)((T + g.grid - 1) / g.grid);
+    g.max_seg = (per_cta + g.kb_per_tile - 2) / g.kb_per_tile + 1;
+    const int stage_bytes = A_BYTES + g.m_pad * 128;
+    g.stages = std::max(2, std::min(MAX_STAGES, (200 * 1024) / stage_bytes));
+    return g;
+}
+
+size_t gemm_partials_bytes(const GemmGeom& g) { return sizeof(float) * (size_t)g.grid * g.max_seg * g.m_pad * TILE_N; }
+
+bool gemm_tc_supported(int m_tok, int n_out, int K) { return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0; }
+
+cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials,
+                                uint32_t* status, cudaStream_t st) {
+    const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_streamk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 512);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    k_gemm_streamk<<<g.grid, NUM_THREADS, smem, st>>>(*(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, partials, status);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------- plain consumer
+// y[m][n] = sum of the segments of n's tile, in the fixed order of the CTAs that produced them.
+__global__ void k_reduce_plain(const float* __restrict__ partials, GemmGeom g, float* __restrict__ y) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x, m = blockIdx.y;
+    if (n >= g.n_out) return;
+    y[(size_t)m * g.n_out + n] = gemm_reduce(partials, g, m, n);
+}
+
+cudaError_t launch_reduce_plain(const float* partials, const GemmGeom& g, float* y, cudaStream_t st) {
+    dim3 grid((g.n_out + 255) / 256, g.m_tok);
+    k_reduce_plain<<<grid, 256, 0, st>>>(partials, g, y);
+    return cudaGetLastError();
+}
+
+}  // namespace sd

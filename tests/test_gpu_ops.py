@@ -124,3 +124,31 @@ def test_softmax_and_draw(sd, V, T):
         assert (t_gpu == np.argmax(logits, axis=1)).all()
     else:
         assert same >= rows - 1
+
+
+TC_SHAPES = [  # rows, n_out, n_in: single tile, several tiles + ragged tail, split tiles, wide token counts
+    (6, 128, 64), (6, 128, 4096), (1, 256, 512), (6, 1024, 256), (16, 300, 1000), (6, 4096, 4096),
+    (5, 12288, 1024), (17, 640, 2304), (96, 1152, 768), (72, 4096, 1024), (200, 256, 512), (256, 384, 320),
+    (6, 32000, 512), (2, 11008, 1024), (6, 1024, 11008),
+]
+
+
+@pytest.mark.parametrize("rows,n_out,n_in", TC_SHAPES)
+def test_linear_tensor_core_kernel(sd, rows, n_out, n_in):
+    x = quantize(synth.make_logits((rows, n_in), seed=13, stream=rows), "bf16")
+    w = quantize(synth.make_logits((n_out, n_in), seed=14, stream=n_out % 1000, std=0.05), "bf16")
+    y = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    sd.sd_op_linear(to_dev(x), to_dev(w), y, sd.SD_BF16, impl=2)
+    torch.cuda.synchronize()
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    # the oracle computes sampled rows and columns one by one at the larger sizes
+    rng = np.random.default_rng(rows * 7 + n_out)
+    cols = np.arange(n_out) if n_out * n_in <= 2**22 else np.unique(np.concatenate(
+        [rng.integers(0, n_out, 192), [0, 127, 128, n_out - 1, n_out - 129 if n_out > 129 else 0]]))
+    ref = oracle.linear(np.ascontiguousarray(w[cols]), widen(x))
+    np.testing.assert_allclose(got[:, cols], ref, rtol=0, atol=2e-5 * np.sqrt(n_in / 64))
+    # same answer on a second run: the reduction order is fixed
+    y2 = torch.zeros_like(y)
+    sd.sd_op_linear(to_dev(x), to_dev(w), y2, sd.SD_BF16, impl=2)
+    assert torch.equal(y, y2)
