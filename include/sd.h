@@ -203,6 +203,10 @@ sd_status sd_verify_accept_host(sd_ctx* ctx, const int32_t* seqs_host, int n_seq
 
 /* -------------------------------------------------------------- observation */
 
+/* bf16 models run on the tensor-core kernels by default; on != 0 makes the context use the
+ * plain CUDA-core kernels instead (the two paths check each other in the tests). */
+sd_status sd_force_plain_path(sd_ctx* ctx, int on);
+
 /* Number of kernels this context has launched since sd_create. */
 sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);
 

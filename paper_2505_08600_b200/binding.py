@@ -67,6 +67,7 @@ _PROTOS = {
     "sd_accept_seqs": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_kv_rollback": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
+    "sd_force_plain_path": (_i, [_vp, _i]),
     "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
     "sd_profile": (_i, [_vp, _i]),
     "sd_profile_read": (_i, [_vp, _vp, _vp]),
@@ -235,6 +236,9 @@ class Context:
         a, p, n = _seqs(seqs)
         _check(self.L.sd_verify_accept_host(self.h, p, n, gamma, _dp(x_host), _dp(q_host), _dp(n_acc_host), _dp(out_tok_host)),
                "sd_verify_accept_host")
+
+    def sd_force_plain_path(self, on):
+        _check(self.L.sd_force_plain_path(self.h, int(on)), "sd_force_plain_path")
 
     def sd_launch_count(self):
         v = C.c_uint64()

@@ -32,6 +32,7 @@ struct Layer {
     void* wd;                       // [d][F]
     float* norm1;
     float* norm2;
+    TensorMap tm_qkv, tm_wo, tm_gu, tm_wd;   // TMA descriptors of the four matrices (bf16 models)
 };
 
 struct Model {
@@ -46,6 +47,8 @@ struct Model {
     size_t kv_layer_bytes;
     float* rope_cos;                // [max_ctx][head_dim / 2]
     float* rope_sin;
+    TensorMap tm_lm;
+    bool tc;                        // the tensor-core path applies (bf16, shapes fit)
     int n_qkv() const { return (d.n_heads + 2 * d.n_kv_heads) * d.head_dim; }
 };
 
@@ -62,6 +65,9 @@ struct sd_ctx {
     float* h; void* xn; void* q; void* attn; void* act; float* lin; float* draft_logits;
     int32_t* row_slot; int32_t* row_pos;
     void* attn_ws; size_t attn_ws_bytes;
+    float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
+    float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
+    bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     // classifier
     float* clf_w1; float* clf_b1; float* clf_w2; float* clf_b2; bool clf_loaded;
     // host bookkeeping
@@ -80,6 +86,16 @@ struct sd_ctx {
 namespace {
 
 size_t esize(int dtype) { return dtype == SD_BF16 ? 2 : 4; }
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else return 148;
+    }
+    return n;
+}
 
 bool valid_desc(const sd_model_desc& m) {
     if (m.n_layers < 1 || m.d_model < 8 || m.n_heads < 1 || m.n_kv_heads < 1 || m.d_ffn < 8 || m.vocab < 2) return false;
@@ -162,8 +178,21 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->row_pos = (int32_t*)B.take(sizeof(int32_t) * R);
     c->attn_ws_bytes = 0;
     for (int i = 0; i < nm; ++i)
-        c->attn_ws_bytes = std::max(c->attn_ws_bytes, attention_workspace_bytes((int)R, ms[i].n_heads, ms[i].head_dim, cfg.max_ctx));
+        c->attn_ws_bytes = std::max(c->attn_ws_bytes, attention_split_supported(ms[i].dtype, ms[i].n_heads, ms[i].n_kv_heads, ms[i].head_dim)
+                                        ? attention_split_workspace((int)R, ms[i].n_heads, ms[i].head_dim, cfg.max_ctx)
+                                        : attention_workspace_bytes((int)R, ms[i].n_heads, ms[i].head_dim, cfg.max_ctx));
     c->attn_ws = B.take(c->attn_ws_bytes);
+    c->partials_bytes = 0;
+    for (int i = 0; i < nm; ++i) {
+        const sd_model_desc& m = ms[i];
+        if (m.dtype != SD_BF16) continue;
+        const int shapes[5][2] = {{(m.n_heads + 2 * m.n_kv_heads) * m.head_dim, m.d_model}, {m.d_model, m.n_heads * m.head_dim},
+                                  {2 * m.d_ffn, m.d_model}, {m.d_model, m.d_ffn}, {m.vocab, m.d_model}};
+        for (auto& s : shapes)
+            c->partials_bytes = std::max(c->partials_bytes, gemm_partials_bytes(gemm_geometry(SD_MAX_ROWS, s[0], s[1], sm_count())));
+    }
+    c->partials = (float*)B.take(c->partials_bytes);
+    c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
     const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
@@ -227,7 +256,10 @@ sd_status linear(sd_ctx* c, const void* x, const void* w, float* y, int rows, in
 enum LogitsMode { LOGITS_NONE = 0, LOGITS_ALL = 1, LOGITS_LAST = 2 };
 
 // One pass of a model over n_rows query rows described by `plan`.
+sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out);
+
 sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
+    if (M.tc && !c->force_plain) return forward_tc(c, M, list, plan, n_rows, mode, logits_out);
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
@@ -258,6 +290,57 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
         LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, M.final_norm, c->xn, dt, list.n, d, m.rms_eps, R, R - 1, st));
         SD_TRY(linear(c, c->xn, M.lm_head, logits_out, list.n, m.vocab, d, dt));
     }
+    CUDA_TRY(prof_mark(c, CAT_NONE));
+    return SD_OK;
+}
+
+sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, GemmGeom& g) {
+    g = gemm_geometry(rows, n_out, K, sm_count());
+    if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
+    TensorMap tx;
+    if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
+    LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, c->S.status, c->st));
+    return SD_OK;
+}
+
+// The same pass on the tensor-core path (bf16 models): every GEMM leaves split accumulators
+// in the workspace and the kernel after it folds the reduction into its own work.
+sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
+    const sd_model_desc& m = M.d;
+    const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
+    cudaStream_t st = c->st;
+    GemmGeom g;
+    RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
+    RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
+    RowScale none{nullptr, 0, 0.f, 0.f};
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
+    LAUNCH(CAT_ELEMENTWISE, launch_prep_norm(c->h, M.layers[0].norm1, c->xn, c->ssq, n_rows, d, st));
+    for (int l = 0; l < m.n_layers; ++l) {
+        const Layer& L = M.layers[l];
+        void* kc = M.kcache + M.kv_layer_bytes * l;
+        void* vc = M.vcache + M.kv_layer_bytes * l;
+        SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, g));
+        LAUNCH(CAT_ELEMENTWISE, launch_cons_qkv_rope(c->partials, g, l == 0 ? first : tiled, c->q, kc, vc, c->row_slot, c->row_pos,
+                                                     n_rows, H, Hkv, hd, c->cfg.max_ctx, M.rope_cos, M.rope_sin, st));
+        LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
+                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, st));
+        c->launches += 1;
+        SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, g));
+        LAUNCH(CAT_ELEMENTWISE, launch_cons_residual(c->partials, g, c->h, L.norm2, c->xn, c->ssq, n_rows, st));
+        SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, g));
+        LAUNCH(CAT_ELEMENTWISE, launch_cons_swiglu(c->partials, g, tiled, c->act, n_rows, F, st));
+        SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, g));
+        const float* next_gain = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
+        LAUNCH(CAT_ELEMENTWISE, launch_cons_residual(c->partials, g, c->h, next_gain, c->xn, c->ssq, n_rows, st));
+    }
+    if (mode != LOGITS_NONE) {
+        // the lm_head GEMM runs over all rows (they share the one pass over the weights); only the wanted rows are reduced
+        const int R = plan.rows_per_seq;
+        SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, g));
+        if (mode == LOGITS_ALL) LAUNCH(CAT_LINEAR, launch_reduce_plain(c->partials, g, logits_out, n_rows, 1, 0, tiled, st));
+        else LAUNCH(CAT_LINEAR, launch_reduce_plain(c->partials, g, logits_out, list.n, R, R - 1, tiled, st));
+    }
+    (void)none;
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
@@ -345,6 +428,22 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
             return fail(SD_ERR_CUDA);
     }
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
+    c->force_plain = false;
+    for (Model& M : c->models) {
+        const sd_model_desc& m = M.d;
+        M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE &&
+               attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim);
+        if (!M.tc) continue;
+        const int dq = m.n_heads * m.head_dim;
+        bool ok = make_tensor_map_bf16(&M.tm_lm, M.lm_head, m.vocab, m.d_model, 128);
+        for (Layer& L : M.layers) {
+            ok = ok && make_tensor_map_bf16(&L.tm_qkv, L.wqkv, M.n_qkv(), m.d_model, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_wo, L.wo, m.d_model, dq, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_gu, L.wgu, 2 * m.d_ffn, m.d_model, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_wd, L.wd, m.d_model, m.d_ffn, 128);
+        }
+        if (!ok) return fail(SD_ERR_CUDA);
+    }
     *out = c;
     return SD_OK;
 }
@@ -458,7 +557,7 @@ sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
             Model& M = c->models[pass == 0 ? 0 : 1 + c->draft_id[s]];
             for (int p0 = 0; p0 < n; p0 += SD_MAX_ROWS) {
                 const int rows = std::min(SD_MAX_ROWS, n - p0);
-                RowPlan plan{PLAN_PREFILL, rows, p0, 0, 0, nullptr};
+                RowPlan plan{PLAN_PREFILL, rows, p0, 0, 0, nullptr, p0 + rows};
                 SD_TRY(forward(c, M, one, plan, rows, LOGITS_NONE, nullptr));
             }
         }
@@ -481,6 +580,8 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] + gamma - 1 > c->cfg.max_ctx) return SD_ERR_CAPACITY;
     const int V = c->models[0].d.vocab;
+    int bound = 0;
+    for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     for (int k = 0; k < c->cfg.n_drafts; ++k) {             // sequences grouped per routed draft
         SeqList g = all;
         g.n = 0;
@@ -490,10 +591,10 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
         Model& M = c->models[1 + k];
         for (int s = 0; s < gamma; ++s) {
             if (s == 0) {
-                RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_in};
+                RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_in, bound};
                 SD_TRY(forward(c, M, g, plan, 2 * g.n, LOGITS_LAST, c->draft_logits));
             } else {
-                RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_in};
+                RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_in, bound + s};
                 SD_TRY(forward(c, M, g, plan, g.n, LOGITS_ALL, c->draft_logits));
             }
             LAUNCH(CAT_SAMPLING, launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
@@ -509,7 +610,9 @@ sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const 
     if (n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_CAPACITY;
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
-    RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev};
+    int bound = 0;
+    for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
+    RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound};
     return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev);
 }
 
@@ -519,7 +622,9 @@ sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logit
     if (!logits_dev) return SD_ERR_INVALID_ARG;
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] > c->cfg.max_ctx) return SD_ERR_CAPACITY;
-    RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr};
+    int bound = 0;
+    for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
+    RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr, bound};
     return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev);
 }
 
@@ -616,6 +721,12 @@ sd_status sd_verify_accept_host(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     return SD_OK;
 }
 
+sd_status sd_force_plain_path(sd_ctx* c, int on) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    c->force_plain = on != 0;
+    return SD_OK;
+}
+
 sd_status sd_launch_count(sd_ctx* c, uint64_t* out) {
     if (!c || !out) return SD_ERR_INVALID_ARG;
     *out = c->launches;
@@ -647,16 +758,6 @@ sd_status sd_profile_read(sd_ctx* c, float* ms_by_cat, uint32_t* launches_by_cat
 }
 
 // ------------------------------------------------------------------ single operators
-static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl) {
     if (impl == 1 || dtype != SD_BF16 || !gemm_tc_supported(rows, n_out, n_in)) return 0;
     return gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
@@ -674,7 +775,8 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
         TensorMap tw, tx;
         if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
         CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, (cudaStream_t)stream));
-        CUDA_TRY(launch_reduce_plain((const float*)workspace, g, y, (cudaStream_t)stream));
+        RowScale none{nullptr, 0, 0.f, 0.f};
+        CUDA_TRY(launch_reduce_plain((const float*)workspace, g, y, rows, 1, 0, none, (cudaStream_t)stream));
         return SD_OK;
     }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;
@@ -683,7 +785,8 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
 }
 
 size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx) {
-    return attention_workspace_bytes(rows, n_heads, head_dim, max_ctx);
+    return std::max(attention_workspace_bytes(rows, n_heads, head_dim, max_ctx),
+                    (head_dim == 64 || head_dim == 128) ? attention_split_workspace(rows, n_heads, head_dim, max_ctx) : (size_t)0);
 }
 
 sd_status sd_op_attention(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
@@ -691,7 +794,12 @@ sd_status sd_op_attention(const void* q, const void* kc, const void* vc, void* o
                           void* ws, size_t ws_bytes, void* stream) {
     if (!q || !kc || !vc || !out || !row_slot || !row_pos || rows < 1 || H < 1 || Hkv < 1 || H % Hkv) return SD_ERR_INVALID_ARG;
     if (hd < 8 || hd > 256 || (hd & 7) || max_ctx < 1 || (dtype != SD_F32 && dtype != SD_BF16)) return SD_ERR_INVALID_ARG;
-    if (ws_bytes < attention_workspace_bytes(rows, H, hd, max_ctx)) return SD_ERR_OOM;
+    if (ws_bytes < sd_op_attention_workspace(rows, H, hd, max_ctx)) return SD_ERR_OOM;
+    if (attention_split_supported(dtype, H, Hkv, hd)) {
+        if (!ws) return SD_ERR_INVALID_ARG;
+        CUDA_TRY(launch_attention_split(q, kc, vc, out, row_slot, row_pos, rows, 1, H, Hkv, hd, max_ctx, max_ctx, ws, ws_bytes, (cudaStream_t)stream));
+        return SD_OK;
+    }
     CUDA_TRY(launch_attention(q, kc, vc, out, dtype, row_slot, row_pos, rows, H, Hkv, hd, max_ctx, ws, ws_bytes, (cudaStream_t)stream));
     return SD_OK;
 }

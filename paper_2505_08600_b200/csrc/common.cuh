@@ -41,6 +41,7 @@ struct RowPlan {
     int step;               // PLAN_DRAFT_NEXT: s >= 1
     int gamma;              // row stride of x
     const int32_t* x;       // [n_seq][gamma] draft tokens (device)
+    int ctx_bound;          // host's upper bound on 1 + the largest position any row of the pass sees
 };
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);

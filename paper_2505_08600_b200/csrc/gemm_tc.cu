@@ -274,6 +274,7 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     g.grid = (int)std::min<long long>(n_sm, T);
     const int per_cta = (int)((T + g.grid - 1) / g.grid);
     g.max_seg = (per_cta + g.kb_per_tile - 2) / g.kb_per_tile + 1;
+    if (T * g.grid >= (1ll << 32)) g.grid = 0;          // the consumers' 32-bit index arithmetic would overflow
     const int stage_bytes = A_BYTES + g.m_pad * 128;
     g.stages = std::max(2, std::min(MAX_STAGES, (200 * 1024) / stage_bytes));
     return g;
@@ -281,7 +282,9 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
 
 size_t gemm_partials_bytes(const GemmGeom& g) { return sizeof(float) * (size_t)g.grid * g.max_seg * g.m_pad * TILE_N; }
 
-bool gemm_tc_supported(int m_tok, int n_out, int K) { return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0; }
+bool gemm_tc_supported(int m_tok, int n_out, int K) {
+    return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0 && (long long)((n_out + 127) / 128) * ((K + 63) / 64) < (1ll << 24);
+}
 
 cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials,
                                 uint32_t* status, cudaStream_t st) {
@@ -297,16 +300,19 @@ cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, co
 }
 
 // ---------------------------------------------------------------------------- plain consumer
-// y[m][n] = sum of the segments of n's tile, in the fixed order of the CTAs that produced them.
-__global__ void k_reduce_plain(const float* __restrict__ partials, GemmGeom g, float* __restrict__ y) {
-    const int n = blockIdx.x * blockDim.x + threadIdx.x, m = blockIdx.y;
+// y[i][n] = scale(row) * (sum of the segments of n's tile, in the fixed order of their CTAs).
+__global__ void k_reduce_plain(const float* __restrict__ partials, GemmGeom g, float* __restrict__ y, int row_stride,
+                               int row_offset, RowScale rs) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x, i = blockIdx.y;
     if (n >= g.n_out) return;
-    y[(size_t)m * g.n_out + n] = gemm_reduce(partials, g, m, n);
+    const int m = i * row_stride + row_offset;
+    y[(size_t)i * g.n_out + n] = gemm_reduce(partials, g, m, n) * row_scale(rs, m);
 }
 
-cudaError_t launch_reduce_plain(const float* partials, const GemmGeom& g, float* y, cudaStream_t st) {
-    dim3 grid((g.n_out + 255) / 256, g.m_tok);
-    k_reduce_plain<<<grid, 256, 0, st>>>(partials, g, y);
+cudaError_t launch_reduce_plain(const float* partials, const GemmGeom& g, float* y, int n_out_rows, int row_stride,
+                                int row_offset, const RowScale& rs, cudaStream_t st) {
+    dim3 grid((g.n_out + 255) / 256, n_out_rows);
+    k_reduce_plain<<<grid, 256, 0, st>>>(partials, g, y, row_stride, row_offset, rs);
     return cudaGetLastError();
 }
 

@@ -35,6 +35,13 @@ cudaError_t launch_attention(const void* q, const void* kcache_layer, const void
                              int n_heads, int n_kv_heads, int head_dim, int max_ctx,
                              void* workspace, size_t workspace_bytes, cudaStream_t st);
 
+// ---- attention_split.cu : split-KV kernel for bf16 caches with head_dim 64 / 128
+bool attention_split_supported(int dtype, int H, int Hkv, int hd);
+size_t attention_split_workspace(int rows, int H, int hd, int max_ctx);
+cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
+                                   const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
+                                   int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, cudaStream_t st);
+
 // ---- sampling.cu
 cudaError_t launch_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, cudaStream_t st);
 // probs[r] = softmax(logits[r] / T); tok[r] drawn with u_int[r] (explicit) ...
