@@ -169,6 +169,7 @@ def run_gpu(args):
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    torch.cuda.set_stream(torch.cuda.Stream(dev))           # a capturable (non-default) stream for everything below
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)      # only for the barrier and the max over ranks
     cfg = synth.CONFIGS[args.config]
@@ -207,10 +208,8 @@ def run_gpu(args):
     ctx.sd_draft_steps(seqs, gamma, x, q)          # the drafts every timed verify step scores (values do not change its cost)
     torch.cuda.synchronize()
 
-    def verify_step():
-        ctx.sd_verify(seqs, gamma, x, logits)
-        ctx.sd_accept_seqs(seqs, gamma, logits, q, x, n_acc, out_tok)
-        ctx.sd_kv_rollback(seqs, gamma, n_acc, out_tok)
+    def verify_step():          # sd_verify + sd_accept_seqs + sd_kv_rollback as one captured launch sequence
+        ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
 
     def barrier():
         torch.cuda.synchronize()

@@ -193,6 +193,13 @@ sd_status sd_accept_seqs(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int g
 sd_status sd_kv_rollback(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
                          const int32_t* n_acc_dev, const int32_t* out_tok_dev);
 
+/* sd_verify + sd_accept_seqs + sd_kv_rollback as one call (one captured launch sequence):
+ * logits_dev [n_seq][gamma+1][vocab] is scratch owned by the caller and holds the target's
+ * logits afterwards. */
+sd_status sd_verify_accept(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, int gamma,
+                           const int32_t* x_dev, const float* q_dev, float* logits_dev,
+                           int32_t* n_acc_dev, int32_t* out_tok_dev);
+
 /* One verify step for a caller whose drafts live in host memory: copies x_host [n_seq][gamma]
  * and q_host [n_seq][gamma][vocab] to the device, runs sd_verify, sd_accept_seqs and
  * sd_kv_rollback on them and copies n_acc [n_seq] and out_tok [n_seq][gamma+1] back.
@@ -202,6 +209,10 @@ sd_status sd_verify_accept_host(sd_ctx* ctx, const int32_t* seqs_host, int n_seq
                                 int32_t* n_acc_host, int32_t* out_tok_host);
 
 /* -------------------------------------------------------------- observation */
+
+/* Repeated calls replay captured CUDA graphs by default (keyed by sequences, gamma, buffers
+ * and a 256-token bucket of the context length); on == 0 launches kernel by kernel. */
+sd_status sd_use_graphs(sd_ctx* ctx, int on);
 
 /* bf16 models run on the tensor-core kernels by default; on != 0 makes the context use the
  * plain CUDA-core kernels instead (the two paths check each other in the tests). */

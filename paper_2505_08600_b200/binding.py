@@ -67,6 +67,8 @@ _PROTOS = {
     "sd_accept_seqs": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_kv_rollback": (_i, [_vp, _vp, _i, _i, _vp, _vp]),
     "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
+    "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "sd_use_graphs": (_i, [_vp, _i]),
     "sd_force_plain_path": (_i, [_vp, _i]),
     "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
     "sd_profile": (_i, [_vp, _i]),
@@ -236,6 +238,13 @@ class Context:
         a, p, n = _seqs(seqs)
         _check(self.L.sd_verify_accept_host(self.h, p, n, gamma, _dp(x_host), _dp(q_host), _dp(n_acc_host), _dp(out_tok_host)),
                "sd_verify_accept_host")
+
+    def sd_verify_accept(self, seqs, gamma, x, q, logits, n_acc, out_tok):
+        a, p, n = _seqs(seqs)
+        _check(self.L.sd_verify_accept(self.h, p, n, gamma, _dp(x), _dp(q), _dp(logits), _dp(n_acc), _dp(out_tok)), "sd_verify_accept")
+
+    def sd_use_graphs(self, on):
+        _check(self.L.sd_use_graphs(self.h, int(on)), "sd_use_graphs")
 
     def sd_force_plain_path(self, on):
         _check(self.L.sd_force_plain_path(self.h, int(on)), "sd_force_plain_path")

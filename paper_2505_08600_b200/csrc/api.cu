@@ -68,6 +68,10 @@ struct sd_ctx {
     float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
+    bool graphs_on;                             // replay captured CUDA graphs for repeated calls
+    struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
+    std::vector<CachedGraph> graphs;
+    uint64_t graph_clock;
     // classifier
     float* clf_w1; float* clf_b1; float* clf_w2; float* clf_b2; bool clf_loaded;
     // host bookkeeping
@@ -345,6 +349,62 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     return SD_OK;
 }
 
+// Calls of the hot path repeat with the same shapes and buffers, and all state they depend on
+// lives on the device, so the launch sequence of a call is captured once into a CUDA graph
+// and replayed: one host call instead of hundreds of launches.  The key holds everything that
+// shapes the launches (sequences, gamma, buffers, context-length bucket).
+struct KeyBuilder {
+    std::vector<uint8_t> bytes;
+    template <typename T> KeyBuilder& add(const T& v) {
+        const uint8_t* p = reinterpret_cast<const uint8_t*>(&v);
+        bytes.insert(bytes.end(), p, p + sizeof(T));
+        return *this;
+    }
+    KeyBuilder& add_list(const int32_t* seqs, int n) { add(n); for (int i = 0; i < n; ++i) add(seqs[i]); return *this; }
+};
+
+int bound_bucket(int bound) { return (bound + 255) & ~255; }
+
+template <class Body>
+sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
+    if (!c->graphs_on || c->prof_on) return body();
+    c->graph_clock += 1;
+    for (auto& g : c->graphs)
+        if (g.key == key.bytes) {
+            CUDA_TRY(cudaGraphLaunch(g.exec, c->st));
+            c->launches += g.launches;
+            g.last_use = c->graph_clock;
+            return SD_OK;
+        }
+    const uint64_t l0 = c->launches;
+    if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        (void)cudaGetLastError();                       // e.g. the legacy default stream cannot capture:
+        c->graphs_on = false;                           // launch kernel by kernel from now on
+        return body();
+    }
+    const sd_status s = body();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(c->st, &graph);
+    if (s != SD_OK || e != cudaSuccess) {
+        if (graph) cudaGraphDestroy(graph);
+        c->launches = l0;
+        return s != SD_OK ? s : SD_ERR_CUDA;
+    }
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ei != cudaSuccess) { c->launches = l0; return SD_ERR_CUDA; }
+    if (c->graphs.size() >= 24) {                       // drop the least recently used entry
+        size_t victim = 0;
+        for (size_t i = 1; i < c->graphs.size(); ++i) if (c->graphs[i].last_use < c->graphs[victim].last_use) victim = i;
+        cudaGraphExecDestroy(c->graphs[victim].exec);
+        c->graphs.erase(c->graphs.begin() + victim);
+    }
+    c->graphs.push_back({key.bytes, exec, c->launches - l0, c->graph_clock});
+    CUDA_TRY(cudaGraphLaunch(exec, c->st));
+    return SD_OK;
+}
+
 sd_status make_list(sd_ctx* c, const int32_t* seqs, int n_seq, int min_phase, SeqList& list) {
     if (!c || !seqs || n_seq < 1 || n_seq > SD_MAX_BATCH) return SD_ERR_INVALID_ARG;
     list.n = n_seq;
@@ -429,6 +489,8 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     }
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
     c->force_plain = false;
+    c->graphs_on = true;
+    c->graph_clock = 0;
     for (Model& M : c->models) {
         const sd_model_desc& m = M.d;
         M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE &&
@@ -452,6 +514,7 @@ sd_status sd_destroy(sd_ctx* c) {
     if (!c) return SD_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->st);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
     delete c;
     return SD_OK;
 }
@@ -582,6 +645,11 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     const int V = c->models[0].d.vocab;
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
+    KeyBuilder key;
+    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain);
+    for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
+    bound = bound_bucket(bound + gamma) - gamma;
+    return run_graphed(c, key, [&]() -> sd_status {
     for (int k = 0; k < c->cfg.n_drafts; ++k) {             // sequences grouped per routed draft
         SeqList g = all;
         g.n = 0;
@@ -601,6 +669,7 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
         }
     }
     return SD_OK;
+    });
 }
 
 sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_dev, float* logits_dev) {
@@ -612,8 +681,10 @@ sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const 
         if (c->len_ub[seqs[i]] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
-    RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound};
-    return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev);
+    RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound_bucket(bound)};
+    KeyBuilder key;
+    key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain);
+    return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev); });
 }
 
 sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logits_dev) {
@@ -624,8 +695,10 @@ sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logit
         if (c->len_ub[seqs[i]] > c->cfg.max_ctx) return SD_ERR_CAPACITY;
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
-    RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr, bound};
-    return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev);
+    RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr, bound_bucket(bound)};
+    KeyBuilder key;
+    key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain);
+    return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev); });
 }
 
 sd_status sd_accept(const sd_accept_args* a) {
@@ -702,6 +775,42 @@ sd_status sd_device_status(sd_ctx* c, uint32_t* flags) {
     return SD_OK;
 }
 
+sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_dev, const float* q_dev,
+                           float* logits_dev, int32_t* n_acc_dev, int32_t* out_tok_dev) {
+    if (!c || !seqs || !logits_dev || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
+    const bool saved = c->graphs_on;
+    KeyBuilder key;
+    key.add(4).add_list(seqs, n_seq).add(gamma).add(x_dev).add(q_dev).add(logits_dev).add(n_acc_dev).add(out_tok_dev).add(c->force_plain);
+    int bound = 0;
+    for (int i = 0; i < n_seq && seqs[i] >= 0 && seqs[i] < c->cfg.max_seqs; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
+    key.add(bound_bucket(bound));
+    std::vector<int> ub(c->len_ub);
+    auto body = [&]() -> sd_status {
+        c->graphs_on = false;                    // the three calls below must launch into this capture, not replay their own graphs
+        sd_status s = sd_verify(c, seqs, n_seq, gamma, x_dev, logits_dev);
+        if (s == SD_OK) s = sd_accept_seqs(c, seqs, n_seq, gamma, logits_dev, q_dev, x_dev, n_acc_dev, out_tok_dev);
+        if (s == SD_OK) s = sd_kv_rollback(c, seqs, n_seq, gamma, n_acc_dev, out_tok_dev);
+        c->graphs_on = saved;
+        return s;
+    };
+    // argument and capacity checks must run on every call, captured or replayed
+    if (n_seq < 1 || n_seq > SD_MAX_BATCH || gamma < 0 || gamma > c->cfg.max_gamma || n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i];
+        if (s < 0 || s >= c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
+        if (c->phase[s] < PH_READY) return SD_ERR_STATE;
+        if (c->len_ub[s] + gamma + 1 > c->S.tok_stride || c->len_ub[s] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    }
+    const bool replay = saved && !c->prof_on;
+    bool cached = false;
+    if (replay) for (auto& g : c->graphs) cached |= g.key == key.bytes;
+    const sd_status s = run_graphed(c, key, body);
+    if (s == SD_OK && cached)                    // a replay does not run the host bookkeeping of sd_kv_rollback
+        for (int i = 0; i < n_seq; ++i) c->len_ub[seqs[i]] += gamma + 1;
+    if (s != SD_OK) c->len_ub = ub;
+    return s;
+}
+
 sd_status sd_verify_accept_host(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_host,
                                 const float* q_host, int32_t* n_acc_host, int32_t* out_tok_host) {
     if (!c || !seqs || n_seq < 1 || n_seq > c->cfg.max_seqs || gamma < 0 || gamma > c->cfg.max_gamma) return SD_ERR_INVALID_ARG;
@@ -712,12 +821,16 @@ sd_status sd_verify_accept_host(sd_ctx* c, const int32_t* seqs, int n_seq, int g
         CUDA_TRY(cudaMemcpyAsync(c->st_x, x_host, sizeof(int32_t) * n_seq * gamma, cudaMemcpyHostToDevice, c->st));
         CUDA_TRY(cudaMemcpyAsync(c->st_q, q_host, sizeof(float) * n_seq * gamma * V, cudaMemcpyHostToDevice, c->st));
     }
-    SD_TRY(sd_verify(c, seqs, n_seq, gamma, c->st_x, c->st_logits));
-    SD_TRY(sd_accept_seqs(c, seqs, n_seq, gamma, c->st_logits, c->st_q, c->st_x, c->st_nacc, c->st_out));
-    SD_TRY(sd_kv_rollback(c, seqs, n_seq, gamma, c->st_nacc, c->st_out));
+    SD_TRY(sd_verify_accept(c, seqs, n_seq, gamma, c->st_x, c->st_q, c->st_logits, c->st_nacc, c->st_out));
     CUDA_TRY(cudaMemcpyAsync(n_acc_host, c->st_nacc, sizeof(int32_t) * n_seq, cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaMemcpyAsync(out_tok_host, c->st_out, sizeof(int32_t) * n_seq * (gamma + 1), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_use_graphs(sd_ctx* c, int on) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    c->graphs_on = on != 0;
     return SD_OK;
 }
 

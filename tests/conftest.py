@@ -15,3 +15,17 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(autouse=True)
+def _side_stream(request):
+    """GPU tests run on a non-default CUDA stream: the library captures its launch sequences
+    into CUDA graphs, which the legacy default stream does not allow."""
+    if request.node.get_closest_marker("gpu") is None:
+        yield
+        return
+    import torch
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        yield
+    torch.cuda.synchronize()
