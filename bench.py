@@ -44,9 +44,10 @@ def eq1_speedup(alpha, gamma, c):
 # ------------------------------------------------------------------------------------------
 # CPU baseline: the oracle as it stands, on a bounded sample of the same verify step
 # ------------------------------------------------------------------------------------------
-def oracle_sample(cfg_name, sample_layers=1, reps=1):
+def oracle_sample(cfg_name, sample_layers=2, min_seconds=10.0, max_reps=64):
     """Times the oracle's cached forward over gamma+1 rows at the config's shapes with only
-    `sample_layers` of the layers, and the lm_head alone, then scales to the full depth."""
+    `sample_layers` of the layers, and the lm_head alone, then scales to the full depth.
+    Repeats until about `min_seconds` of CPU work have been timed."""
     import oracle
     cfg = synth.CONFIGS[cfg_name]
     wl, t = cfg["workload"], dict(cfg["target"])
@@ -64,14 +65,14 @@ def oracle_sample(cfg_name, sample_layers=1, reps=1):
     toks = synth.make_prompt(t["vocab"], gamma + 1, seed=1)
     cores = len(os.sched_getaffinity(0))
     t_with, t_layers = [], []
-    for _ in range(reps):
+    while len(t_with) < max_reps and sum(t_with) + sum(t_layers) < min_seconds:
         t0 = time.perf_counter(); cache.forward(toks, n_prompt - 1, want_logits=True); t_with.append(time.perf_counter() - t0)
         t0 = time.perf_counter(); cache.forward(toks, n_prompt - 1, want_logits=False); t_layers.append(time.perf_counter() - t0)
     tl, tw = min(t_layers), min(t_with)
     step_s = B * (tl / sample_layers * full_layers + (tw - tl))  # sequences are independent: B of them cost B times one
     return dict(value=B * (gamma + 1) / step_s, unit=UNIT, cores=cores, kind="oracle",
                 sample=f"{sample_layers} of {full_layers} layers + lm_head at full width, {gamma + 1} rows, context {n_prompt}, "
-                       f"one sequence; scaled by layers and batch {B}",
+                       f"one sequence, best of {len(t_with)} repeats; scaled by layers and batch {B}",
                 seconds_measured=round(sum(t_with) + sum(t_layers), 2), step_seconds_scaled=round(step_s, 2))
 
 
@@ -81,9 +82,9 @@ def run_reference(args):
         return
     vals = []
     for _ in range(args.warmup if args.warmup < 2 else 1):
-        oracle_sample(args.config)
+        oracle_sample(args.config, min_seconds=1.0)
     for _ in range(max(1, min(args.steps, 5))):
-        vals.append(oracle_sample(args.config))
+        vals.append(oracle_sample(args.config, min_seconds=5.0))
     v = statistics.median(x["value"] for x in vals)
     cb = dict(vals[0]); cb["value"] = v
     wl = synth.CONFIGS[args.config]["workload"]
@@ -237,11 +238,13 @@ def run_gpu(args):
     sampler = ClockSampler(gpu_id)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    torch.cuda.profiler.start()                 # a profiler told to wait for this range sees the timed steps only
     ev0.record(stream)
     for _ in range(K):
         verify_step()
     ev1.record(stream)
     barrier()
+    torch.cuda.profiler.stop()
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
     clocks = sampler.stop()
     launches = ctx.sd_launch_count() - l0
