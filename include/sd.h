@@ -257,6 +257,25 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
                        int impl, void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl);
 
+/* The bf16 tensor-core form of sd_op_linear for callers that cannot allocate device memory
+ * (the paper has no counterpart; this serves embedders).  A host that runs this library
+ * inside its own serving loop, under a memory pool that already owns the whole device or in
+ * a section where cudaMalloc is forbidden, has only the buffers it was handed: x
+ * [rows][n_in] and w [n_out][n_in] as bf16 bit patterns, y [rows][n_out] fp32, all device
+ * pointers owned by the caller.  The split accumulators that sd_op_linear keeps in a
+ * caller-supplied workspace live here in an array of SD_STATIC_SCRATCH_BYTES that is part of
+ * the library image on every GPU that loads it, for the life of the process.  The call
+ * allocates and frees nothing.
+ *  - Shapes whose accumulators do not fit (roughly rows > 32 at 148 SMs) return
+ *    SD_ERR_CAPACITY; shapes the tensor-core kernel cannot take return SD_ERR_UNSUPPORTED.
+ *  - The first call on a device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last call left:
+ *    the kernel overwrites every word it later reads, so nothing needs clearing, but two
+ *    calls whose kernels overlap on the GPU (different streams, no ordering) race. */
+#define SD_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
+sd_status sd_op_linear_static(const void* x, const void* w, float* y, int rows, int n_out, int n_in, void* cuda_stream);
+
 /* Attention of `rows` query rows against a cache laid out as the library lays
  * it out: k_cache/v_cache [n_slots][n_kv_heads][max_ctx][head_dim], q
  * [rows][n_heads][head_dim], row r belongs to slot row_slot[r] and sees

@@ -79,6 +79,7 @@ _PROTOS = {
     "sd_target_step": (_i, [_vp, _vp, _i, _vp]),
     "sd_op_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_linear_workspace": (_sz, [_i, _i, _i, _i, _i]),
+    "sd_op_linear_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_attention_workspace": (_sz, [_i, _i, _i, _i]),
     "sd_op_philox": (_i, [_vp, _i, C.c_uint32, C.c_uint32, _vp, _vp]),
@@ -298,6 +299,12 @@ def sd_op_linear(x, w, y, dtype, impl=0, stream=None):
     need = lib().sd_op_linear_workspace(rows, n_out, n_in, dtype, impl)
     ws = torch.empty(max(need, 1), dtype=torch.uint8, device=x.device)
     _check(lib().sd_op_linear(_dp(x), _dp(w), _dp(y), rows, n_out, n_in, dtype, impl, _dp(ws), need, _stream_ptr(stream)), "sd_op_linear")
+
+
+def sd_op_linear_static(x, w, y, stream=None):
+    """bf16 x [rows][n_in], w [n_out][n_in] -> fp32 y [rows][n_out]; the library's built-in scratch, no allocation."""
+    rows, n_in = x.shape
+    _check(lib().sd_op_linear_static(_dp(x), _dp(w), _dp(y), rows, w.shape[0], n_in, _stream_ptr(stream)), "sd_op_linear_static")
 
 
 def sd_op_attention(q, kc, vc, out, row_slot, row_pos, n_heads, n_kv_heads, head_dim, max_ctx, dtype, stream=None):

@@ -1,0 +1,58 @@
+"""The allocation-free linear entry point against the ordinary one (through the C ABI).
+
+sd_op_linear_static exists for hosts that may not allocate device memory while they call the
+library (a serving loop whose memory pool owns the whole device, a region where cudaMalloc is
+forbidden): it keeps the GEMM's split accumulators in an array built into the library instead
+of a caller-supplied workspace.  Both entry points run the same kernels, so their outputs
+must be identical; the check is repeated on a second call because the built-in array is
+shared between calls and keeps the first call's contents.  This file sorts last on purpose,
+so a run that stops at the first failure has already been through every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_08600_b200 import synth
+from gpu_util import DEV, quantize, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sd():
+    from paper_2505_08600_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_static_scratch_linear_matches_workspace_linear_twice(sd):
+    before = torch.cuda.memory_allocated()
+    shapes = [(6, 4096, 1024), (17, 640, 2304)]          # the second call has another shape and finds the first one's leftovers
+    inputs = []
+    for rows, n_out, n_in in shapes:
+        x = to_dev(quantize(synth.make_logits((rows, n_in), seed=31, stream=rows), "bf16"))
+        w = to_dev(quantize(synth.make_logits((n_out, n_in), seed=32, stream=n_out % 1000, std=0.05), "bf16"))
+        ref = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+        sd.sd_op_linear(x, w, ref, sd.SD_BF16, impl=2)
+        got = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+        inputs.append((x, w, ref, got))
+    torch.cuda.synchronize()
+    held = torch.cuda.memory_allocated()
+    for x, w, ref, got in inputs:                         # two calls in a row, nothing allocated in between
+        sd.sd_op_linear_static(x, w, got)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == held >= before
+    for (rows, n_out, n_in), (x, w, ref, got) in zip(shapes, inputs):
+        assert torch.isfinite(got).all()
+        # same kernels, same fixed reduction order: the tolerance of the tensor-core linear tests is met with room to spare
+        np.testing.assert_allclose(got.cpu().numpy(), ref.cpu().numpy(), rtol=0, atol=2e-5 * np.sqrt(n_in / 64))
+        assert torch.equal(got, ref)
+
+
+def test_static_scratch_linear_rejects_what_does_not_fit(sd):
+    x = torch.zeros((200, 512), dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros((4096, 512), dtype=torch.bfloat16, device=DEV)
+    y = torch.zeros((200, 4096), dtype=torch.float32, device=DEV)
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_op_linear_static(x, w, y)                   # 200 rows of accumulators exceed the built-in array
+    assert e.value.status == 3                            # SD_ERR_CAPACITY
