@@ -67,6 +67,8 @@ struct sd_ctx {
     void* attn_ws; size_t attn_ws_bytes;
     float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
+    uint32_t* gemm_counters;                    // arrival counters of the GEMM's output tiles (zero between launches)
+    int pull_units;                             // weight boxes per CTA that a GEMM pulls into L2 for its successor
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
     struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
@@ -197,6 +199,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     }
     c->partials = (float*)B.take(c->partials_bytes);
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
+    c->gemm_counters = (uint32_t*)B.take(GEMM_COUNTER_BYTES);
     const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
@@ -267,7 +270,8 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
-    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
+                                         nullptr, nullptr, nullptr, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -282,7 +286,7 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
         LAUNCH(CAT_ELEMENTWISE, launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
         LAUNCH(CAT_ELEMENTWISE, launch_rmsnorm(c->h, L.norm2, c->xn, dt, n_rows, d, m.rms_eps, 1, 0, st));
         SD_TRY(linear(c, c->xn, L.wgu, c->lin, n_rows, 2 * F, d, dt));
-        LAUNCH(CAT_ELEMENTWISE, launch_swiglu(c->lin, c->act, dt, n_rows, F, st));
+        LAUNCH(CAT_ELEMENTWISE, launch_swiglu(c->lin, c->act, dt, n_rows, F, M.tc ? 1 : 0, st));
         SD_TRY(linear(c, c->act, L.wd, c->lin, n_rows, d, F, dt));
         LAUNCH(CAT_ELEMENTWISE, launch_residual_add(c->h, c->lin, (size_t)n_rows * d, st));
     }
@@ -298,53 +302,75 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     return SD_OK;
 }
 
-sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, GemmGeom& g) {
-    g = gemm_geometry(rows, n_out, K, sm_count());
+// One weight GEMM with its fused epilogue.  `next` names the matrix the following GEMM on the
+// stream will read (nullptr: none), so that this launch can pull its head into L2 while finishing.
+struct NextMat { const TensorMap* tm; int n_out, K; };
+
+sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep,
+                  const NextMat* next) {
+    const GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
-    LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, c->S.status, c->st));
+    NextWeights nw;
+    nw.units = 0;
+    if (next && next->tm && c->pull_units > 0) {
+        const GemmGeom gn = gemm_geometry(rows, next->n_out, next->K, sm_count());
+        nw.tm = *next->tm; nw.n_tiles = gn.n_tiles; nw.kb_per_tile = gn.kb_per_tile; nw.grid = gn.grid; nw.units = c->pull_units;
+    }
+    LAUNCH(CAT_LINEAR, launch_gemm_fused(tw, tx, g, ep, &nw, c->partials, c->gemm_counters, c->S.status, 1, c->st));
     return SD_OK;
 }
 
-// The same pass on the tensor-core path (bf16 models): every GEMM leaves split accumulators
-// in the workspace and the kernel after it folds the reduction into its own work.
+// The same pass on the tensor-core path (bf16 models): five kernels per layer (QKV GEMM,
+// attention, Wo GEMM, gate/up GEMM, down GEMM); each GEMM's finishing CTAs apply the step that
+// follows it, and every kernel is launched as a programmatic dependent of the one before.
 sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
-    GemmGeom g;
-    RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
-    RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
-    RowScale none{nullptr, 0, 0.f, 0.f};
-    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos, st));
-    LAUNCH(CAT_ELEMENTWISE, launch_prep_norm(c->h, M.layers[0].norm1, c->xn, c->ssq, n_rows, d, st));
+    const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
+    const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
+                                         M.layers[0].norm1, c->xn, c->ssq, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
         void* vc = M.vcache + M.kv_layer_bytes * l;
-        SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, g));
-        LAUNCH(CAT_ELEMENTWISE, launch_cons_qkv_rope(c->partials, g, l == 0 ? first : tiled, c->q, kc, vc, c->row_slot, c->row_pos,
-                                                     n_rows, H, Hkv, hd, c->cfg.max_ctx, M.rope_cos, M.rope_sin, st));
+        Epilogue e;
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_QKV_ROPE; e.rs = l == 0 ? first : tiled;
+        e.q_out = (bf16*)c->q; e.kc = (bf16*)kc; e.vc = (bf16*)vc; e.row_slot = c->row_slot; e.row_pos = c->row_pos;
+        e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = M.rope_cos; e.rsin = M.rope_sin;
+        NextMat nx{&L.tm_wo, d, H * hd};
+        SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e, &nx));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
-                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, st));
-        c->launches += 1;
-        SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, g));
-        LAUNCH(CAT_ELEMENTWISE, launch_cons_residual(c->partials, g, c->h, L.norm2, c->xn, c->ssq, n_rows, st));
-        SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, g));
-        LAUNCH(CAT_ELEMENTWISE, launch_cons_swiglu(c->partials, g, tiled, c->act, n_rows, F, st));
-        SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, g));
-        const float* next_gain = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
-        LAUNCH(CAT_ELEMENTWISE, launch_cons_residual(c->partials, g, c->h, next_gain, c->xn, c->ssq, n_rows, st));
+                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st));
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_RESIDUAL; e.h = c->h; e.gain_next = L.norm2; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
+        nx = NextMat{&L.tm_gu, 2 * F, d};
+        SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e, &nx));
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_SWIGLU; e.rs = tiled; e.act = (bf16*)c->act; e.F = F;
+        nx = NextMat{&L.tm_wd, d, F};
+        SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, e, &nx));
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_RESIDUAL; e.h = c->h; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
+        e.gain_next = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
+        if (l + 1 < m.n_layers) nx = NextMat{&M.layers[l + 1].tm_qkv, M.n_qkv(), d};
+        else nx = NextMat{mode != LOGITS_NONE ? &M.tm_lm : nullptr, m.vocab, d};
+        SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, e, &nx));
     }
     if (mode != LOGITS_NONE) {
-        // the lm_head GEMM runs over all rows (they share the one pass over the weights); only the wanted rows are reduced
+        // the lm_head GEMM runs over all rows (they share the one pass over the weights); only the wanted rows are written
         const int R = plan.rows_per_seq;
-        SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, g));
-        if (mode == LOGITS_ALL) LAUNCH(CAT_LINEAR, launch_reduce_plain(c->partials, g, logits_out, n_rows, 1, 0, tiled, st));
-        else LAUNCH(CAT_LINEAR, launch_reduce_plain(c->partials, g, logits_out, list.n, R, R - 1, tiled, st));
+        Epilogue e;
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_PLAIN; e.rs = tiled; e.y = logits_out;
+        if (mode == LOGITS_ALL) { e.n_out_rows = n_rows; e.row_stride = 1; e.row_offset = 0; }
+        else { e.n_out_rows = list.n; e.row_stride = R; e.row_offset = R - 1; }
+        SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, e, nullptr));
     }
-    (void)none;
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
@@ -487,13 +513,18 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
             cudaStreamSynchronize(st) != cudaSuccess)
             return fail(SD_ERR_CUDA);
     }
+    if (cudaMemsetAsync(c->gemm_counters, 0, GEMM_COUNTER_BYTES, st) != cudaSuccess ||
+        cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess)
+        return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
     c->force_plain = false;
+    c->pull_units = 16;
     c->graphs_on = true;
     c->graph_clock = 0;
     for (Model& M : c->models) {
         const sd_model_desc& m = M.d;
-        M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE &&
+        M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE && m.d_ffn % 64 == 0 &&
+               (m.vocab + 127) / 128 <= GEMM_MAX_TILES && (2 * m.d_ffn + 127) / 128 <= GEMM_MAX_TILES &&
                attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim);
         if (!M.tc) continue;
         const int dq = m.n_heads * m.head_dim;
@@ -537,8 +568,18 @@ sd_status sd_load_tensor(sd_ctx* c, int model_id, int kind, int layer, const voi
         case SD_T_WK: dst = (char*)L->wqkv + dq * d * M.esz; bytes = dkv * d * M.esz; break;
         case SD_T_WV: dst = (char*)L->wqkv + (dq + dkv) * d * M.esz; bytes = dkv * d * M.esz; break;
         case SD_T_WO: dst = L->wo; bytes = d * dq * M.esz; break;
-        case SD_T_WG: dst = L->wgu; bytes = F * d * M.esz; break;
-        case SD_T_WU: dst = (char*)L->wgu + F * d * M.esz; bytes = F * d * M.esz; break;
+        case SD_T_WG:
+        case SD_T_WU:
+            if (M.tc) {
+                // tensor-core layout: 128-row tiles of 64 gate rows followed by the 64 up rows of the same features,
+                // so that the CTA finishing a tile holds both halves of SwiGLU
+                const size_t chunk = 64 * d * M.esz;
+                CUDA_TRY(cudaMemcpy2DAsync((char*)L->wgu + (kind == SD_T_WU ? chunk : 0), 2 * chunk, src, chunk, chunk, F / 64,
+                                           on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->st));
+                if (!on_dev) CUDA_TRY(cudaStreamSynchronize(c->st));
+                return SD_OK;
+            }
+            dst = kind == SD_T_WG ? (char*)L->wgu : (char*)L->wgu + F * d * M.esz; bytes = F * d * M.esz; break;
         case SD_T_WD: dst = L->wd; bytes = d * F * M.esz; break;
         case SD_T_NORM1: dst = L->norm1; bytes = d * 4; break;
         case SD_T_NORM2: dst = L->norm2; bytes = d * 4; break;
@@ -710,7 +751,7 @@ sd_status sd_accept(const sd_accept_args* a) {
     p.target = a->target; p.target_is_logits = a->target_is_logits; p.q = a->q; p.x = a->x;
     p.B = a->B; p.gamma = a->gamma; p.V = a->V; p.T = a->temperature; p.seed = a->seed;
     p.iter = a->iter; p.seq_id = a->seq_id; p.use_list = 0; p.n_acc = a->n_acc; p.out_tok = a->out_tok;
-    CUDA_TRY(launch_accept(p, (cudaStream_t)a->cuda_stream));
+    CUDA_TRY(launch_accept(p, 0, (cudaStream_t)a->cuda_stream));
     return SD_OK;
 }
 
@@ -724,7 +765,7 @@ sd_status sd_accept_seqs(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, c
     p.target = logits_dev; p.target_is_logits = 1; p.q = q_dev; p.x = x_dev;
     p.B = n_seq; p.gamma = gamma; p.V = c->models[0].d.vocab; p.T = c->cfg.temperature; p.seed = c->cfg.seed;
     p.iter = c->S.iter; p.seq_id = c->S.seq_id; p.use_list = 1; p.n_acc = n_acc_dev; p.out_tok = out_tok_dev;
-    LAUNCH(CAT_SAMPLING, launch_accept(p, c->st));
+    LAUNCH(CAT_SAMPLING, launch_accept(p, 1, c->st));
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
@@ -873,7 +914,7 @@ sd_status sd_profile_read(sd_ctx* c, float* ms_by_cat, uint32_t* launches_by_cat
 // ------------------------------------------------------------------ single operators
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl) {
     if (impl == 1 || dtype != SD_BF16 || !gemm_tc_supported(rows, n_out, n_in)) return 0;
-    return gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
+    return GEMM_COUNTER_BYTES + gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
 }
 
 sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype, int impl,
@@ -884,12 +925,15 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
     if (impl == 2 && !tc_ok) return SD_ERR_UNSUPPORTED;
     if (impl == 2 || (impl == 0 && tc_ok)) {
         const GemmGeom g = gemm_geometry(rows, n_out, n_in, sm_count());
-        if (!workspace || workspace_bytes < gemm_partials_bytes(g)) return SD_ERR_OOM;
+        if (!workspace || workspace_bytes < GEMM_COUNTER_BYTES + gemm_partials_bytes(g)) return SD_ERR_OOM;
         TensorMap tw, tx;
         if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
-        CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, (cudaStream_t)stream));
-        RowScale none{nullptr, 0, 0.f, 0.f};
-        CUDA_TRY(launch_reduce_plain((const float*)workspace, g, y, rows, 1, 0, none, (cudaStream_t)stream));
+        Epilogue e;
+        memset(&e, 0, sizeof(e));
+        e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
+        CUDA_TRY(cudaMemsetAsync(workspace, 0, GEMM_COUNTER_BYTES, (cudaStream_t)stream));          // the arrival counters
+        CUDA_TRY(launch_gemm_fused(tw, tx, g, e, nullptr, (float*)((char*)workspace + GEMM_COUNTER_BYTES), (uint32_t*)workspace,
+                                   nullptr, 0, (cudaStream_t)stream));
         return SD_OK;
     }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;
@@ -910,7 +954,8 @@ sd_status sd_op_attention(const void* q, const void* kc, const void* vc, void* o
     if (ws_bytes < sd_op_attention_workspace(rows, H, hd, max_ctx)) return SD_ERR_OOM;
     if (attention_split_supported(dtype, H, Hkv, hd)) {
         if (!ws) return SD_ERR_INVALID_ARG;
-        CUDA_TRY(launch_attention_split(q, kc, vc, out, row_slot, row_pos, rows, 1, H, Hkv, hd, max_ctx, max_ctx, ws, ws_bytes, (cudaStream_t)stream));
+        CUDA_TRY(cudaMemsetAsync(ws, 0, 65536, (cudaStream_t)stream));                               // the arrival counters
+        CUDA_TRY(launch_attention_split(q, kc, vc, out, row_slot, row_pos, rows, 1, H, Hkv, hd, max_ctx, max_ctx, ws, ws_bytes, 0, (cudaStream_t)stream));
         return SD_OK;
     }
     CUDA_TRY(launch_attention(q, kc, vc, out, dtype, row_slot, row_pos, rows, H, Hkv, hd, max_ctx, ws, ws_bytes, (cudaStream_t)stream));

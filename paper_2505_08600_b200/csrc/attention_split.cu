@@ -1,258 +1,363 @@
-// Split-KV attention for the verify / draft rows (bf16 cache, head_dim 64 or 128).
+// Split-KV attention for the verify / draft rows (bf16 cache, head_dim 64 or 128) on the
+// warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 accumulate).
 //
 // A block of consecutive query rows of one sequence (the gamma+1 verify rows) times the query
 // heads that share one KV head is scored against one slice of that head's cache; every slice
 // is streamed from HBM once, whatever the number of rows.  Slices leave unnormalised partial
-// outputs with their running max and sum; a second small kernel merges them.
+// outputs with their running max and sum; the CTA whose slice arrives last (an arrival
+// counter, nothing spins) merges them.
 // Cache layout of one layer: [slot][kv_head][position][head_dim].
+#include "gemm_tc.h"
 #include "kernels.h"
 
 namespace sd {
 
 namespace {
 
-constexpr int ATT_THREADS = 128;
-constexpr int NQ_MAX = 32;          // query vectors per CTA: rows in the block x heads per KV head
-constexpr int QCHUNK = 8;           // query vectors accumulated at once in the value pass
-
-__device__ __forceinline__ void unpack8(const uint4& u, float f[8]) {
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-}
+constexpr int ATT_THREADS = 128;    // four warps; each takes 16 of the 64 keys of a chunk
+constexpr int NQ = 16;              // query vectors per CTA (rows in the block x heads per KV head): one MMA row tile
+constexpr int CK = 64;              // keys per chunk
+constexpr size_t ATTN_COUNTER_BYTES = 65536;     // one arrival counter per (query block, kv head)
 
 struct AttnParams {
     const bf16* q; const bf16* kc; const bf16* vc;
     const int32_t* row_slot; const int32_t* row_pos;
-    float* part_o;      // [rows][H][n_splits][hd]
-    float* part_ml;     // [rows][H][n_splits][2]
-    int n_rows, rows_per_seq, rows_per_block, H, Hkv, max_ctx, split_len, n_splits;
+    float* part_o;      // [rows][H][n_splits][hd] unnormalised partial outputs
+    float* part_ml;     // [rows][H][n_splits][2] running max (log2 domain) and sum
+    uint32_t* counters; // [query block][kv head]: slices that have delivered; zero between launches
+    bf16* out;          // [rows][H][hd]
+    int n_rows, rows_per_seq, rows_per_block, H, Hkv, max_ctx, n_splits;
 };
 
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8 fp32) += A (16x16 bf16, row) * B (16x8 bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One CTA = one slice of one KV head's cache x the query rows of one block (times the query
+// heads that share the KV head), as a 16-row tensor-core tile.  The slice is walked in chunks
+// of 64 keys, double-buffered in shared memory (16-byte asynchronous copies into an
+// XOR-swizzled layout that ldmatrix reads without bank conflicts); each warp owns 16 keys of a
+// chunk and keeps its own running max / sum / output (online softmax, exp2 domain), the four
+// warps are merged at the end, and the slices of a head are merged by whichever CTA arrives last.
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS) k_attn_split(AttnParams P) {
-    extern __shared__ float sm[];
-    constexpr int LPP = 8;                       // lanes that share one key position
-    constexpr int EPL = HD / LPP;                // elements of a key each of them holds (8 or 16)
+__global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
+    extern __shared__ __align__(128) uint8_t sm_raw[];
+    constexpr int ROWB = HD * 2;             // bytes of one key / value row
+    constexpr int CPR = HD / 8;              // 16-byte pieces per row
+    constexpr int KS = HD / 16;              // reduction steps of Q K^T
+    constexpr int NV = HD / 8;               // 8-wide column tiles of the output
+    constexpr int BUF = CK * ROWB;           // one chunk of keys (or values)
+    constexpr int OLD = HD + 8;              // padded row of the cross-warp merge buffer (floats)
+    pdl_launch_dependents();
     const int split = blockIdx.x, kvh = blockIdx.y;
     const int group = P.H / P.Hkv;
     const int bps = (P.rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;     // query blocks per sequence
     const int r0 = (blockIdx.z / bps) * P.rows_per_seq + (blockIdx.z % bps) * P.rows_per_block;
     const int nr = min(P.rows_per_block, P.rows_per_seq - (int)(blockIdx.z % bps) * P.rows_per_block);
     const int nq = nr * group;
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    float* qs = sm;                              // [nq][HD] scaled queries
-    float* sc = qs + NQ_MAX * HD;                // [nq][split_len] scores, then probabilities
-    float* red = sc + NQ_MAX * P.split_len;      // [4][QCHUNK][HD] cross-warp reduction of the value pass
-    __shared__ int pos_sm[NQ_MAX];
-    __shared__ float m_sm[NQ_MAX], l_sm[NQ_MAX];
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, gid = lane >> 2, tig = lane & 3;
+    const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(sm_raw);
+    __shared__ int last_sm;
 
-    int max_pos = -1;
-    for (int j = 0; j < nr; ++j) max_pos = max(max_pos, P.row_pos[r0 + j]);
-    const int p_begin = split * P.split_len;
-    const int p_end = min(p_begin + P.split_len, max_pos + 1);
-    const int np = p_end - p_begin;              // positions of this slice (<= 0: nothing to do)
-    if (np <= 0) {
-        for (int i = t; i < nq; i += ATT_THREADS) {
-            const int r = r0 + i / group, h = kvh * group + i % group;
-            float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
-            ml[0] = -INFINITY; ml[1] = 0.f;
+    pdl_wait();                                  // queries, the appended keys/values and the row plan come from earlier kernels
+    // longest context among the block's rows (every warp works it out for itself), and the sequence slot
+    int mp = lane < nr ? __ldcg(P.row_pos + r0 + lane) : -1;
+    const int slot = __ldcg(P.row_slot + r0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mp = max(mp, __shfl_xor_sync(0xffffffffu, mp, o));
+    // the positions in use are cut evenly into the launched slices, whatever bound the grid was sized for
+    const int len = mp + 1;
+    const int slice = (((len + P.n_splits - 1) / P.n_splits) + 15) & ~15;
+    const int p_begin = split * slice;
+    const int np = min(p_begin + slice, len) - p_begin;          // positions of this slice (<= 0: nothing to do)
+
+    // this thread's two query rows of the tile (gid and gid + 8)
+    const int j_lo = gid, j_hi = gid + 8;
+    const bf16* q_lo = P.q + ((size_t)(r0 + j_lo / group) * P.H + kvh * group + j_lo % group) * HD;
+    const bf16* q_hi = P.q + ((size_t)(r0 + j_hi / group) * P.H + kvh * group + j_hi % group) * HD;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    float O[NV][4];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) { O[i][0] = O[i][1] = O[i][2] = O[i][3] = 0.f; }
+
+    if (np > 0) {
+        const bf16* K = P.kc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
+        const bf16* V = P.vc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
+        const int n_chunks = (np + CK - 1) / CK;
+        auto issue = [&](int c) {                // chunk c -> buffer c & 1: [K][V]
+            const int nk = min(CK, np - c * CK);
+            const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
+            const bf16* ks = K + (size_t)c * CK * HD;
+            const bf16* vs = V + (size_t)c * CK * HD;
+            for (int i = t; i < nk * CPR; i += ATT_THREADS) {
+                const int key = i / CPR, ch = i % CPR;
+                const uint32_t off = (uint32_t)key * ROWB + (uint32_t)((ch ^ (key & 7)) << 4);
+                cp_async16(kb + off, ks + (size_t)i * 8);
+                cp_async16(vb + off, vs + (size_t)i * 8);
+            }
+            // value rows past the end of the slice inside a warp's 16-key group must be finite (their weight is zero)
+            const int nk16 = (nk + 15) & ~15;
+            for (int i = nk * CPR + t; i < nk16 * CPR; i += ATT_THREADS) {
+                const int key = i / CPR, ch = i % CPR;
+                *reinterpret_cast<uint4*>(sm_raw + (size_t)(c & 1) * 2 * BUF + BUF + (size_t)key * ROWB + ((ch ^ (key & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        issue(0);
+        // query fragments (bf16, straight from memory in the MMA's register layout) and the rows' positions
+        uint32_t a[KS][4];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            a[ks][0] = j_lo < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 2 * tig)) : 0u;
+            a[ks][1] = j_hi < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 2 * tig)) : 0u;
+            a[ks][2] = j_lo < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 8 + 2 * tig)) : 0u;
+            a[ks][3] = j_hi < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 8 + 2 * tig)) : 0u;
         }
-        return;
-    }
-    const int slot = P.row_slot[r0];
-    const bf16* K = P.kc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
-    const bf16* V = P.vc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
+        const int pos_lo = j_lo < nq ? __ldcg(P.row_pos + r0 + j_lo / group) : -1;
+        const int pos_hi = j_hi < nq ? __ldcg(P.row_pos + r0 + j_hi / group) : -1;
+        const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;        // softmax scale in the exp2 domain
 
-    const float scale = rsqrtf((float)HD);
+        for (int c = 0; c < n_chunks; ++c) {
+            if (c + 1 < n_chunks) { issue(c + 1); asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+            const int nk = min(CK, np - c * CK);
+            if (16 * warp < nk) {
+                const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
+                float S[2][4];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) { S[i][0] = S[i][1] = S[i][2] = S[i][3] = 0.f; }
+                {
+                    const int mi = lane >> 3, r = lane & 7;
+                    const int key = 16 * warp + 8 * (mi >> 1) + r;
+                    const uint32_t rowaddr = kb + (uint32_t)key * ROWB;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        uint32_t b[4];
+                        ldmatrix_x4(rowaddr + (uint32_t)(((2 * ks + (mi & 1)) ^ (key & 7)) << 4), b);
+                        mma_bf16(S[0], a[ks], b[0], b[1]);
+                        mma_bf16(S[1], a[ks], b[2], b[3]);
+                    }
+                }
+                // scale, mask (past the slice, or after the row's own position), online softmax
+                const int pbase = p_begin + c * CK + 16 * warp + 2 * tig;
+                float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int p = pbase + 8 * nt + (e & 1);
+                        const bool ok = (p - p_begin) < np && p <= ((e < 2) ? pos_lo : pos_hi);
+                        const float v = ok ? S[nt][e] * sl2 : -INFINITY;
+                        S[nt][e] = v;
+                        if (e < 2) mx_lo = fmaxf(mx_lo, v); else mx_hi = fmaxf(mx_hi, v);
+                    }
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1)); mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1)); mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+                const float c_lo = (mn_lo == -INFINITY) ? 1.f : exp2f(m_lo - mn_lo);
+                const float c_hi = (mn_hi == -INFINITY) ? 1.f : exp2f(m_hi - mn_hi);
+                m_lo = mn_lo; m_hi = mn_hi;
+                float s_lo = 0.f, s_hi = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float mn = (e < 2) ? mn_lo : mn_hi;
+                        const float pr = (mn == -INFINITY) ? 0.f : exp2f(S[nt][e] - mn);
+                        S[nt][e] = pr;
+                        if (e < 2) s_lo += pr; else s_hi += pr;
+                    }
+                l_lo = l_lo * c_lo + s_lo; l_hi = l_hi * c_hi + s_hi;
+                uint32_t pa[4];
+                pa[0] = pack_bf16(S[0][0], S[0][1]); pa[1] = pack_bf16(S[0][2], S[0][3]);
+                pa[2] = pack_bf16(S[1][0], S[1][1]); pa[3] = pack_bf16(S[1][2], S[1][3]);
+                {
+                    const int mi = lane >> 3, r = lane & 7;
+                    const int key = 16 * warp + 8 * (mi & 1) + r;
+                    const uint32_t rowaddr = vb + (uint32_t)key * ROWB;
+#pragma unroll
+                    for (int nv = 0; nv < NV; nv += 2) {
+                        O[nv][0] *= c_lo; O[nv][1] *= c_lo; O[nv][2] *= c_hi; O[nv][3] *= c_hi;
+                        O[nv + 1][0] *= c_lo; O[nv + 1][1] *= c_lo; O[nv + 1][2] *= c_hi; O[nv + 1][3] *= c_hi;
+                        uint32_t v[4];
+                        ldmatrix_x4_trans(rowaddr + (uint32_t)(((nv + (mi >> 1)) ^ (key & 7)) << 4), v);
+                        mma_bf16(O[nv], pa, v[0], v[1]);
+                        mma_bf16(O[nv + 1], pa, v[2], v[3]);
+                    }
+                }
+            }
+            __syncthreads();                     // the buffer may be refilled (or reused for the merge) from here on
+        }
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    }
+
+    // ---- merge of the four warps (each saw different keys), then the slice's partial result
+    float* Ow = reinterpret_cast<float*>(sm_raw);                // [4][16][OLD]
+    float* mw = Ow + 4 * NQ * OLD;                               // [4][16]
+    float* lw = mw + 4 * NQ;                                     // [4][16]
+    if (np > 0) {
+#pragma unroll
+        for (int nv = 0; nv < NV; ++nv) {
+            *reinterpret_cast<float2*>(Ow + ((size_t)warp * NQ + gid) * OLD + 8 * nv + 2 * tig) = make_float2(O[nv][0], O[nv][1]);
+            *reinterpret_cast<float2*>(Ow + ((size_t)warp * NQ + gid + 8) * OLD + 8 * nv + 2 * tig) = make_float2(O[nv][2], O[nv][3]);
+        }
+        if (tig == 0) {
+            mw[warp * NQ + gid] = m_lo; mw[warp * NQ + gid + 8] = m_hi;
+            lw[warp * NQ + gid] = l_lo; lw[warp * NQ + gid + 8] = l_hi;
+        }
+    }
+    __syncthreads();
+    {
+        const int j = t >> 3, c0 = (t & 7) * (HD / 8);           // query row of the tile, first of this thread's columns
+        if (j < nq) {
+            const int r = r0 + j / group, h = kvh * group + j % group;
+            float* po = P.part_o + (((size_t)r * P.H + h) * P.n_splits + split) * HD;
+            float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
+            if (np <= 0) {
+                if ((t & 7) == 0) { __stcg(ml, -INFINITY); __stcg(ml + 1, 0.f); }
+            } else {
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) M = fmaxf(M, mw[w * NQ + j]);
+                float wt[4], L = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float m = mw[w * NQ + j];
+                    wt[w] = (m == -INFINITY) ? 0.f : exp2f(m - M);
+                    L += wt[w] * lw[w * NQ + j];
+                }
+#pragma unroll
+                for (int cc = 0; cc < HD / 8; cc += 4) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        if (wt[w] != 0.f) {                   // a warp without keys left nothing behind
+                            const float4 o = *reinterpret_cast<const float4*>(Ow + ((size_t)w * NQ + j) * OLD + c0 + cc);
+                            acc.x = fmaf(wt[w], o.x, acc.x); acc.y = fmaf(wt[w], o.y, acc.y);
+                            acc.z = fmaf(wt[w], o.z, acc.z); acc.w = fmaf(wt[w], o.w, acc.w);
+                        }
+                    }
+                    __stcg(reinterpret_cast<float4*>(po + c0 + cc), acc);
+                }
+                if ((t & 7) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+            }
+        }
+    }
+
+    // ---- the slice that delivers last merges all of them: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
+    //      always in slice order, so the result does not depend on which slice that was
+    __syncthreads();                                 // the block's writes are ordered before thread 0's release below
+    if (t == 0) {
+        uint32_t* ctr = P.counters + (size_t)blockIdx.z * P.Hkv + kvh;
+        uint32_t old;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
+        const int last = old == (uint32_t)P.n_splits - 1u;
+        if (last) *ctr = 0u;
+        last_sm = last;
+    }
+    __syncthreads();
+    if (!last_sm) return;
+    // (1) every slice's max and sum into shared memory, (2) one warp per query turns them into
+    // normalised weights, (3) every thread owns output elements and adds the weighted slices
+    float* m_all = reinterpret_cast<float*>(sm_raw);             // [nq][n_splits]
+    float* l_all = m_all + NQ * 32;                              // [nq][n_splits]
+    const int ns = P.n_splits;
+    for (int i = t; i < nq * ns; i += ATT_THREADS) {
+        const int j = i / ns, s = i % ns;
+        const int r = r0 + j / group, h = kvh * group + j % group;
+        const float* ml = P.part_ml + (((size_t)r * P.H + h) * ns + s) * 2;
+        m_all[i] = __ldcg(ml); l_all[i] = __ldcg(ml + 1);
+    }
+    __syncthreads();
+    for (int j = warp; j < nq; j += ATT_THREADS / 32) {      // n_splits <= 32: one lane per slice
+        const float m = lane < ns ? m_all[j * ns + lane] : -INFINITY;
+        const float M = warp_max(m);
+        const float w = (m == -INFINITY) ? 0.f : exp2f(m - M);
+        const float den = warp_sum(lane < ns ? w * l_all[j * ns + lane] : 0.f);
+        if (lane < ns) m_all[j * ns + lane] = den > 0.f ? w / den : 0.f;
+    }
+    __syncthreads();
     for (int i = t; i < nq * HD; i += ATT_THREADS) {
         const int j = i / HD, e = i % HD;
         const int r = r0 + j / group, h = kvh * group + j % group;
-        qs[j * HD + e] = __bfloat162float(P.q[((size_t)r * P.H + h) * HD + e]) * scale;
+        const float* o = P.part_o + ((size_t)r * P.H + h) * ns * HD + e;
+        float acc = 0.f;
+#pragma unroll 4
+        for (int s = 0; s < ns; ++s) {
+            const float w = m_all[j * ns + s];
+            acc = fmaf(w, w != 0.f ? __ldcg(o + (size_t)s * HD) : 0.f, acc);      // an empty slice left no output behind
+        }
+        P.out[((size_t)r * P.H + h) * HD + e] = __float2bfloat16_rn(acc);
     }
-    if (t < nq) pos_sm[t] = P.row_pos[r0 + t / group];
-    __syncthreads();
-
-    // ---- scores: eight lanes per key position, 16 positions per round
-    const int grp = t / LPP, gl = t % LPP;
-    for (int pb = 0; pb < np; pb += ATT_THREADS / LPP) {
-        const int p = pb + grp;
-        float kf[EPL];
-        if (p < np) {
-#pragma unroll
-            for (int c = 0; c < EPL / 8; ++c) {
-                const uint4 u = *reinterpret_cast<const uint4*>(K + (size_t)p * HD + c * 64 + gl * 8);
-                unpack8(u, kf + 8 * c);
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) kf[e] = 0.f;
-        }
-        for (int j = 0; j < nq; ++j) {
-            float s = 0.f;
-#pragma unroll
-            for (int c = 0; c < EPL / 8; ++c) {
-                const float4 qa = *reinterpret_cast<const float4*>(qs + j * HD + c * 64 + gl * 8);
-                const float4 qb4 = *reinterpret_cast<const float4*>(qs + j * HD + c * 64 + gl * 8 + 4);
-                s = fmaf(kf[8 * c + 0], qa.x, s); s = fmaf(kf[8 * c + 1], qa.y, s);
-                s = fmaf(kf[8 * c + 2], qa.z, s); s = fmaf(kf[8 * c + 3], qa.w, s);
-                s = fmaf(kf[8 * c + 4], qb4.x, s); s = fmaf(kf[8 * c + 5], qb4.y, s);
-                s = fmaf(kf[8 * c + 6], qb4.z, s); s = fmaf(kf[8 * c + 7], qb4.w, s);
-            }
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
-            s += __shfl_xor_sync(0xffffffffu, s, 4);
-            if (gl == 0 && p < np) sc[j * P.split_len + p] = (p_begin + p <= pos_sm[j]) ? s : -INFINITY;
-        }
-    }
-    __syncthreads();
-
-    // ---- per-query max and sum over the slice; scores become probabilities relative to the slice max
-    for (int j = warp; j < nq; j += ATT_THREADS / 32) {
-        float m = -INFINITY;
-        for (int p = lane; p < np; p += 32) m = fmaxf(m, sc[j * P.split_len + p]);
-        m = warp_max(m);
-        float l = 0.f;
-        for (int p = lane; p < np; p += 32) {
-            const float e = (m == -INFINITY) ? 0.f : __expf(sc[j * P.split_len + p] - m);
-            sc[j * P.split_len + p] = e;
-            l += e;
-        }
-        l = warp_sum(l);
-        if (lane == 0) { m_sm[j] = m; l_sm[j] = l; }
-    }
-    __syncthreads();
-
-    // ---- values: 16 (HD 128) or 8 (HD 64) threads span a value row, eight elements each
-    constexpr int TPR = HD / 8;                  // threads per value row
-    constexpr int PGROUPS = ATT_THREADS / TPR;   // positions in flight per step
-    const int vg = t / TPR, ve = (t % TPR) * 8;
-    for (int j0 = 0; j0 < nq; j0 += QCHUNK) {
-        const int nj = min(QCHUNK, nq - j0);
-        float acc[QCHUNK][8];
-#pragma unroll
-        for (int j = 0; j < QCHUNK; ++j)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
-        for (int p = vg; p < np; p += PGROUPS) {
-            float vf[8];
-            unpack8(*reinterpret_cast<const uint4*>(V + (size_t)p * HD + ve), vf);
-#pragma unroll
-            for (int j = 0; j < QCHUNK; ++j) {
-                if (j < nj) {
-                    const float w = sc[(j0 + j) * P.split_len + p];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[j][e] = fmaf(w, vf[e], acc[j][e]);
-                }
-            }
-        }
-        // position groups inside a warp first (TPR 16: two groups, TPR 8: four), then across warps
-#pragma unroll
-        for (int j = 0; j < QCHUNK; ++j)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                float v = acc[j][e];
-                v += __shfl_xor_sync(0xffffffffu, v, 16);
-                if (TPR == 8) v += __shfl_xor_sync(0xffffffffu, v, 8);
-                acc[j][e] = v;
-            }
-        __syncthreads();
-        if (lane < TPR) {
-#pragma unroll
-            for (int j = 0; j < QCHUNK; ++j)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) red[(warp * QCHUNK + j) * HD + lane * 8 + e] = acc[j][e];
-        }
-        __syncthreads();
-        for (int i = t; i < nj * HD; i += ATT_THREADS) {
-            const int j = i / HD, e = i % HD;
-            const float v = red[(0 * QCHUNK + j) * HD + e] + red[(1 * QCHUNK + j) * HD + e] +
-                            red[(2 * QCHUNK + j) * HD + e] + red[(3 * QCHUNK + j) * HD + e];
-            const int jq = j0 + j, r = r0 + jq / group, h = kvh * group + jq % group;
-            P.part_o[(((size_t)r * P.H + h) * P.n_splits + split) * HD + e] = v;
-        }
-    }
-    for (int i = t; i < nq; i += ATT_THREADS) {
-        const int r = r0 + i / group, h = kvh * group + i % group;
-        float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
-        ml[0] = m_sm[i]; ml[1] = l_sm[i];
-    }
-}
-
-// Merge of the slices of one (row, head): out = sum_s e^(m_s - M) O_s / sum_s e^(m_s - M) l_s.
-template <int HD>
-__global__ void k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml, bf16* __restrict__ out,
-                               int H, int n_splits) {
-    const int r = blockIdx.x, h = blockIdx.y, e = threadIdx.x;
-    const float* ml = part_ml + ((size_t)r * H + h) * n_splits * 2;
-    const float* o = part_o + ((size_t)r * H + h) * n_splits * HD;
-    float M = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, ml[2 * s]);
-    float acc = 0.f, den = 0.f;
-    if (M != -INFINITY) {
-        for (int s = 0; s < n_splits; ++s) {
-            const float m = ml[2 * s];
-            if (m == -INFINITY) continue;
-            const float w = __expf(m - M);
-            den = fmaf(w, ml[2 * s + 1], den);
-            acc = fmaf(w, o[(size_t)s * HD + e], acc);
-        }
-    }
-    out[((size_t)r * H + h) * HD + e] = __float2bfloat16_rn(den > 0.f ? acc / den : 0.f);
-}
-
-int pick_split_len(int max_ctx) {
-    int len = 64;
-    while ((max_ctx + len - 1) / len > 32) len += 64;
-    return len;
 }
 
 }  // namespace
 
 bool attention_split_supported(int dtype, int H, int Hkv, int hd) {
-    return dtype == SD_BF16 && (hd == 64 || hd == 128) && H / Hkv <= NQ_MAX;
+    return dtype == SD_BF16 && (hd == 64 || hd == 128) && H / Hkv <= NQ;
 }
 
 size_t attention_split_workspace(int rows, int H, int hd, int max_ctx) {
-    const int n_splits = (max_ctx + pick_split_len(max_ctx) - 1) / pick_split_len(max_ctx);
-    return sizeof(float) * (size_t)rows * H * n_splits * (hd + 2);
+    const int n_splits = std::min(32, (max_ctx + CK - 1) / CK);
+    return ATTN_COUNTER_BYTES + sizeof(float) * (size_t)rows * H * n_splits * (hd + 2);
 }
 
 // Rows come in runs of rows_per_seq consecutive rows of one sequence (n_rows is a multiple of it);
 // ctx_bound: no row sees a position >= ctx_bound (bounds the number of slices launched).
+// The first ATTN_COUNTER_BYTES of the workspace are arrival counters: zero before the first
+// launch, left at zero by every launch.
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
-                                   int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                                   int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
+                                   cudaStream_t st) {
     if (n_rows <= 0) return cudaSuccess;
     ctx_bound = std::max(1, std::min(ctx_bound, max_ctx));
     AttnParams P;
-    P.q = (const bf16*)q; P.kc = (const bf16*)kc; P.vc = (const bf16*)vc;
+    P.q = (const bf16*)q; P.kc = (const bf16*)kc; P.vc = (const bf16*)vc; P.out = (bf16*)out;
     P.row_slot = row_slot; P.row_pos = row_pos;
-    if (rows_per_seq < 1 || n_rows % rows_per_seq) return cudaErrorInvalidValue;
+    if (rows_per_seq < 1 || n_rows % rows_per_seq || H / Hkv > NQ) return cudaErrorInvalidValue;
     P.n_rows = n_rows; P.rows_per_seq = rows_per_seq; P.H = H; P.Hkv = Hkv; P.max_ctx = max_ctx;
-    P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ_MAX / (H / Hkv)));
+    P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ / (H / Hkv)));
     const int bps = (rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;
-    P.split_len = pick_split_len(ctx_bound);
-    P.n_splits = (ctx_bound + P.split_len - 1) / P.split_len;
-    const size_t need = sizeof(float) * (size_t)n_rows * H * P.n_splits * (hd + 2);
-    if (need > workspace_bytes) return cudaErrorInvalidValue;
-    P.part_o = (float*)workspace;
+    const int n_blocks = (n_rows / rows_per_seq) * bps;
+    // enough slices to fill the SMs about three CTAs deep, at least one 64-key chunk each
+    int sm = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
+    P.n_splits = std::max(1, std::min(std::min(32, (ctx_bound + CK - 1) / CK), (3 * sm + Hkv * n_blocks - 1) / (Hkv * n_blocks)));
+    const size_t need = ATTN_COUNTER_BYTES + sizeof(float) * (size_t)n_rows * H * P.n_splits * (hd + 2);
+    if (need > workspace_bytes || (size_t)n_blocks * Hkv * sizeof(uint32_t) > ATTN_COUNTER_BYTES) return cudaErrorInvalidValue;
+    P.counters = (uint32_t*)workspace;
+    P.part_o = (float*)((char*)workspace + ATTN_COUNTER_BYTES);
     P.part_ml = P.part_o + (size_t)n_rows * H * P.n_splits * hd;
-    const size_t smem = sizeof(float) * ((size_t)NQ_MAX * hd + (size_t)NQ_MAX * P.split_len + (size_t)4 * QCHUNK * hd);
-    dim3 grid(P.n_splits, Hkv, (n_rows / rows_per_seq) * bps);
+    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)4 * NQ * (hd + 8) + 8 * NQ));
+    dim3 grid(P.n_splits, Hkv, n_blocks);
     cudaError_t e;
     if (hd == 128) {
-        if ((e = cudaFuncSetAttribute(k_attn_split<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        k_attn_split<128><<<grid, ATT_THREADS, smem, st>>>(P);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        k_attn_combine<128><<<dim3(n_rows, H), 128, 0, st>>>(P.part_o, P.part_ml, (bf16*)out, H, P.n_splits);
-    } else {
-        if ((e = cudaFuncSetAttribute(k_attn_split<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        k_attn_split<64><<<grid, ATT_THREADS, smem, st>>>(P);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        k_attn_combine<64><<<dim3(n_rows, H), 64, 0, st>>>(P.part_o, P.part_ml, (bf16*)out, H, P.n_splits);
+        if ((e = cudaFuncSetAttribute(k_attn_mma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        return launch_pdl(k_attn_mma<128>, grid, dim3(ATT_THREADS), smem, st, dependent, P);
     }
-    return cudaGetLastError();
+    if ((e = cudaFuncSetAttribute(k_attn_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    return launch_pdl(k_attn_mma<64>, grid, dim3(ATT_THREADS), smem, st, dependent, P);
 }
 
 }  // namespace sd

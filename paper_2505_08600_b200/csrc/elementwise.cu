@@ -10,7 +10,9 @@ namespace sd {
 // them for the later kernels of the pass and loads the embedding row as fp32.
 template <typename T>
 __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restrict__ embed, int d, int vocab,
-                        float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos) {
+                        float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos,
+                        const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq) {
+    __shared__ float red[32];
     const int r = blockIdx.x;
     const int i = r / plan.rows_per_seq, j = r % plan.rows_per_seq;
     const int slot = list.ids[i], b = list.out[i];
@@ -34,14 +36,24 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
     if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) atomicOr(S.status, SD_DEV_BAD_TOKEN); tok = 0; }
     if (threadIdx.x == 0) { row_slot[r] = slot; row_pos[r] = pos; }
     const T* e = embed + (size_t)tok * d;
-    for (int k = threadIdx.x; k < d; k += blockDim.x) h[(size_t)r * d + k] = to_f32<T>(e[k]);
+    float ss = 0.f;
+    for (int k = threadIdx.x; k < d; k += blockDim.x) {
+        const float v = to_f32<T>(e[k]);
+        h[(size_t)r * d + k] = v;
+        if (gain) { xn[(size_t)r * d + k] = __float2bfloat16_rn(v * gain[k]); ss += v * v; }
+    }
+    if (gain) {                          // first half of the first layer's RMSNorm: the 1/rms factor follows the GEMM
+        ss = block_sum(ss, red);
+        if (threadIdx.x == 0) ssq[(size_t)r * 64] = ss;
+    }
 }
 
 cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& plan, int n_rows,
                          const void* embed, int dtype, int d, int vocab,
-                         float* h, int32_t* row_slot, int32_t* row_pos, cudaStream_t st) {
-    if (dtype == SD_BF16) k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos);
-    else k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos);
+                         float* h, int32_t* row_slot, int32_t* row_pos, const float* gain, void* xn, float* ssq,
+                         cudaStream_t st) {
+    if (dtype == SD_BF16) k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq);
+    else k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr);
     return cudaGetLastError();
 }
 
@@ -118,17 +130,18 @@ cudaError_t launch_residual_add(float* h, const float* y, size_t n, cudaStream_t
 }
 
 template <typename T>
-__global__ void k_swiglu(const float* __restrict__ gu, T* __restrict__ act, int F) {
+__global__ void k_swiglu(const float* __restrict__ gu, T* __restrict__ act, int F, int interleaved) {
     const int r = blockIdx.y;
     const int f = blockIdx.x * blockDim.x + threadIdx.x;
     if (f >= F) return;
-    float g = gu[(size_t)r * 2 * F + f], u = gu[(size_t)r * 2 * F + F + f];
+    const int ig = interleaved ? (f / 64) * 128 + f % 64 : f, iu = interleaved ? ig + 64 : F + f;
+    float g = gu[(size_t)r * 2 * F + ig], u = gu[(size_t)r * 2 * F + iu];
     act[(size_t)r * F + f] = from_f32<T>(g / (1.f + expf(-g)) * u);
 }
-cudaError_t launch_swiglu(const float* gu, void* act, int dtype, int n_rows, int F, cudaStream_t st) {
+cudaError_t launch_swiglu(const float* gu, void* act, int dtype, int n_rows, int F, int interleaved, cudaStream_t st) {
     dim3 grid((F + 255) / 256, n_rows);
-    if (dtype == SD_BF16) k_swiglu<bf16><<<grid, 256, 0, st>>>(gu, (bf16*)act, F);
-    else k_swiglu<float><<<grid, 256, 0, st>>>(gu, (float*)act, F);
+    if (dtype == SD_BF16) k_swiglu<bf16><<<grid, 256, 0, st>>>(gu, (bf16*)act, F, interleaved);
+    else k_swiglu<float><<<grid, 256, 0, st>>>(gu, (float*)act, F, interleaved);
     return cudaGetLastError();
 }
 

@@ -11,10 +11,20 @@
 //     and split evenly over the grid, so that every SM streams the same number of bytes
 //     whatever the matrix shape; a CTA whose range crosses a tile boundary produces one
 //     partial accumulator ("segment") per tile it touches;
-//   - segments are written to a workspace as fp32 [slot][token][128]; the consumer kernels
-//     add the segments of a tile in a fixed order, which keeps results run-to-run identical.
-// Roles: warp 0 issues TMA, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM.
-// Every wait is bounded; on expiry the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
+//   - segments are written to a workspace as fp32 [slot][token][128]; each tile has an arrival
+//     counter, and the CTA whose segment arrives last adds the segments of the tile in the fixed
+//     order of their CTAs (results are run-to-run identical) and applies, in the same pass, the
+//     step that follows the GEMM in the decoder layer (rotary + KV append, residual + next norm,
+//     SwiGLU, or plain fp32 output); nothing spins: a CTA that is not last just moves on;
+//   - the kernel is written for programmatic dependent launch: it lets its successor start at
+//     once; its weight stream never waits for the predecessor (only the token rows and the
+//     workspace do); at most a few weight tiles per SM are in flight (enough to saturate HBM, a
+//     deeper queue only adds latency), the rest of the ring is run-ahead buffer; and after its
+//     own last tile the producer pulls the head of the next GEMM's weights through the freed
+//     stages so that they wait in L2 and HBM stays busy across the kernel boundary.
+// Roles: warp 0 streams weights, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM and
+// run the fused step, warp 6 loads the token rows.  Every mbarrier wait is bounded; on expiry
+// the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
 #include <cuda.h>
 
 #include "gemm_tc.h"
@@ -26,8 +36,11 @@ namespace {
 constexpr int TILE_N = 128;                 // weight rows per tile (UMMA M)
 constexpr int TILE_K = 64;                  // bf16 elements per k block = one 128-byte swizzle row
 constexpr int A_BYTES = TILE_N * TILE_K * 2;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
+constexpr int GEMM_WINDOW = 5;               // weight tiles in flight per SM: 80 KB x 148 SMs saturates HBM
+constexpr int EPI_MB = 8;                    // token rows the fused step handles at a time
+constexpr int EPI_CB = 8;                    // pieces of a tile whose loads are in flight together
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -101,33 +114,225 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t r[16]) {
         : "r"(taddr) : "memory");
 }
 
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }    // the four epilogue warps
+
 struct Shared {
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t full_w[MAX_STAGES], full_x[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
+    int epi_abort, last_flag;
+    int epi_done;                   // the epilogue warps are through: stop pulling the next GEMM's weights
+    float scale[SD_MAX_ROWS];       // 1/rms factor of each token row
+    int pos[SD_MAX_ROWS];           // cache position and sequence slot of each token row (rotary / KV append)
+    int slot[SD_MAX_ROWS];
+    float val[EPI_MB][TILE_N];      // EPI_MB token rows of the tile, for exchanges between its rows
+    float wsum[EPI_MB][4];          // per-warp sums of squares
 };
 
+// First and last CTA that hold a piece of `tile` (see GemmGeom).
+__device__ __forceinline__ void tile_contributors(const GemmGeom& g, uint32_t tile, uint32_t& i_first, uint32_t& i_last) {
+    const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
+    const uint32_t ua = tile * KB, ub = ua + KB - 1;
+    i_first = (uint32_t)((((uint64_t)ua + 1) * G + T - 1) / T) - 1;
+    i_last = (uint32_t)((((uint64_t)ub + 1) * G + T - 1) / T) - 1;
+}
+
+// What the fused step needs per token row and does not depend on the tile: the 1/rms factors,
+// cache positions and slots.  Loaded once per CTA, while the main loop streams.
+__device__ void epilogue_prologue(const GemmGeom& g, const Epilogue& ep, Shared& sh, int et) {
+    if (ep.rs.ssq) {                       // one warp per token row, one lane per piece of its sum of squares
+        const int w = et >> 5, lane = et & 31;
+        for (int m = w; m < g.m_tok; m += 8) {
+            const int m2 = m + 4;
+            const float* pa = ep.rs.ssq + (size_t)m * SSQ_STRIDE;
+            const float* pb = ep.rs.ssq + (size_t)m2 * SSQ_STRIDE;
+            float a = lane < ep.rs.n_parts ? __ldcg(pa + lane) : 0.f;
+            float a2 = lane + 32 < ep.rs.n_parts ? __ldcg(pa + lane + 32) : 0.f;
+            float b = (m2 < g.m_tok && lane < ep.rs.n_parts) ? __ldcg(pb + lane) : 0.f;
+            float b2 = (m2 < g.m_tok && lane + 32 < ep.rs.n_parts) ? __ldcg(pb + lane + 32) : 0.f;
+            a = warp_sum(a + a2); b = warp_sum(b + b2);
+            if (lane == 0) {
+                sh.scale[m] = rsqrtf(a * ep.rs.inv_d + ep.rs.eps);
+                if (m2 < g.m_tok) sh.scale[m2] = rsqrtf(b * ep.rs.inv_d + ep.rs.eps);
+            }
+        }
+    }
+    if (ep.mode == EPI_QKV_ROPE)
+        for (int m = et; m < g.m_tok; m += 128) { sh.pos[m] = __ldcg(ep.row_pos + m); sh.slot[m] = __ldcg(ep.row_slot + m); }
+    epi_bar();
+}
+
+// The step after the GEMM, on one finished 128-row tile.  Runs on the four epilogue warps
+// (et = 0..127 is the row inside the tile) of the CTA whose piece arrived last; sums the pieces
+// in the fixed order of their CTAs, so the result does not depend on which CTA that was.
+// Token rows are taken EPI_MB at a time so that their loads are in flight together.
+__device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float* __restrict__ partials, uint32_t tile,
+                              Shared& sh, int et) {
+    uint32_t i_first, i_last;
+    tile_contributors(g, tile, i_first, i_last);
+    const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
+    const int n = (int)tile * TILE_N + et;
+    const bool live = n < g.n_out;
+    // v[i] = sum over the pieces of (token rows[i], feature n); rows[i] < 0: skipped.  The loads of
+    // up to EPI_CB pieces x EPI_MB rows are issued together; the additions keep the pieces' order.
+    auto reduce_rows = [&](const int (&rows)[EPI_MB], float (&v)[EPI_MB]) {
+#pragma unroll
+        for (int i = 0; i < EPI_MB; ++i) v[i] = 0.f;
+        if (!live) return;
+        for (uint32_t c0 = i_first; c0 <= i_last; c0 += EPI_CB) {
+            float tmp[EPI_CB][EPI_MB];
+#pragma unroll
+            for (int cc = 0; cc < EPI_CB; ++cc) {
+                const uint32_t c = c0 + cc;
+                const bool ok = c <= i_last;
+                const uint32_t j = ok ? tile - (uint32_t)(((uint64_t)c * T) / G) / KB : 0u;
+                const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
+#pragma unroll
+                for (int i = 0; i < EPI_MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+            }
+#pragma unroll
+            for (int cc = 0; cc < EPI_CB; ++cc)
+#pragma unroll
+                for (int i = 0; i < EPI_MB; ++i) v[i] += tmp[cc][i];
+        }
+    };
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    const float gain = (ep.mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;
+    for (int m0 = 0; m0 < n_rows; m0 += EPI_MB) {
+        int rows[EPI_MB];
+        float v[EPI_MB];
+#pragma unroll
+        for (int i = 0; i < EPI_MB; ++i) {
+            const int r = m0 + i;
+            rows[i] = r < n_rows ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
+        }
+        // loads that do not depend on the sum go out first, so that everything is in flight together
+        float hv[EPI_MB], cs[EPI_MB], sn[EPI_MB];
+        int pos[EPI_MB];
+        if (ep.mode == EPI_RESIDUAL) {
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
+        } else if (ep.mode == EPI_QKV_ROPE) {
+            const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
+            const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) {
+                pos[i] = (lower && rows[i] >= 0) ? sh.pos[rows[i]] : -1;
+                cs[i] = 1.f; sn[i] = 0.f;
+                if (pos[i] >= 0 && rot) { cs[i] = ep.rcos[(size_t)pos[i] * half + e]; sn[i] = ep.rsin[(size_t)pos[i] * half + e]; }
+            }
+        }
+        reduce_rows(rows, v);
+        if (ep.rs.ssq) {
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) if (rows[i] >= 0) v[i] *= sh.scale[rows[i]];
+        }
+        switch (ep.mode) {
+        case EPI_PLAIN: {
+            if (live) {
+#pragma unroll
+                for (int i = 0; i < EPI_MB; ++i) if (rows[i] >= 0) ep.y[(size_t)(m0 + i) * g.n_out + n] = v[i];
+            }
+            break;
+        }
+        case EPI_QKV_ROPE: {
+            const int hd = ep.hd, half = hd >> 1, head = n / hd, e = n % hd;
+            const bool rot = head < ep.H + ep.Hkv;
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) sh.val[i][et] = v[i];
+            epi_bar();
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) {
+                if (pos[i] < 0) continue;
+                const float a = v[i], b = sh.val[i][et + half];
+                const float ra = a * cs[i] - b * sn[i], rb = a * sn[i] + b * cs[i];
+                bf16* dst;
+                if (head < ep.H) dst = ep.q_out + ((size_t)rows[i] * ep.H + head) * hd;
+                else {
+                    const int kvh = (head - ep.H) % ep.Hkv;
+                    bf16* base = rot ? ep.kc : ep.vc;
+                    dst = base + (((size_t)sh.slot[rows[i]] * ep.Hkv + kvh) * ep.max_ctx + pos[i]) * hd;
+                }
+                dst[e] = __float2bfloat16_rn(ra);
+                dst[e + half] = __float2bfloat16_rn(rb);
+            }
+            epi_bar();
+            break;
+        }
+        case EPI_RESIDUAL: {
+            const int d = g.n_out;
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) {
+                hv[i] += v[i];
+                if (live && rows[i] >= 0) {
+                    ep.h[(size_t)rows[i] * d + n] = hv[i];
+                    if (ep.gain_next) ep.xn[(size_t)rows[i] * d + n] = __float2bfloat16_rn(hv[i] * gain);
+                }
+            }
+            if (ep.gain_next) {
+#pragma unroll
+                for (int i = 0; i < EPI_MB; ++i) {
+                    const float ss = warp_sum(hv[i] * hv[i]);
+                    if ((et & 31) == 0) sh.wsum[i][et >> 5] = ss;
+                }
+                epi_bar();
+                if (et < EPI_MB && m0 + et < n_rows) {
+                    const float* w = sh.wsum[et];
+                    ep.ssq_out[(size_t)(m0 + et) * SSQ_STRIDE + tile] = (w[0] + w[1]) + (w[2] + w[3]);
+                }
+                epi_bar();
+            }
+            break;
+        }
+        case EPI_SWIGLU: {
+            const int f = (int)tile * 64 + et;
+#pragma unroll
+            for (int i = 0; i < EPI_MB; ++i) sh.val[i][et] = v[i];
+            epi_bar();
+            if (et < 64 && f < ep.F) {
+#pragma unroll
+                for (int i = 0; i < EPI_MB; ++i) {
+                    if (rows[i] < 0) continue;
+                    const float gt = v[i], up = sh.val[i][et + 64];
+                    ep.act[(size_t)rows[i] * ep.F + f] = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
+                }
+            }
+            epi_bar();
+            break;
+        }
+        default: break;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, GemmGeom g,
-               float* __restrict__ partials, uint32_t* status) {
+k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+             const __grid_constant__ CUtensorMap tm_next, GemmGeom g, Epilogue ep, int nx_tiles, int nx_kb, int nx_grid,
+             int nx_units, int window, float* __restrict__ partials, uint32_t* __restrict__ counters, uint32_t* status) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ Shared sh;
+    pdl_launch_dependents();                 // the next kernel may be scheduled; it waits for this one where it must
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t tiles0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;        // 1024-byte aligned stage ring
-    const uint32_t stage_bytes = A_BYTES + (uint32_t)g.m_pad * 128u;
+    const uint32_t x_bytes = (uint32_t)g.m_pad * 128u, stage_bytes = A_BYTES + x_bytes;
     volatile int* abort_flag = &sh.abort_flag;
 
     // this CTA's share of the (row tile, k block) pairs
     const uint32_t T = (uint32_t)g.n_tiles * (uint32_t)g.kb_per_tile;
     const uint32_t u0 = (uint32_t)(((uint64_t)blockIdx.x * T) / gridDim.x);
     const uint32_t u1 = (uint32_t)(((uint64_t)(blockIdx.x + 1) * T) / gridDim.x);
+    const uint32_t n_units = u1 - u0;
     uint32_t tmem_cols = 32;
     while (tmem_cols < 2u * (uint32_t)g.m_pad) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < g.stages; ++s) { mbar_init(smem_u32(&sh.full[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1); }
+        for (int s = 0; s < g.stages; ++s) {
+            mbar_init(smem_u32(&sh.full_w[s]), 1); mbar_init(smem_u32(&sh.full_x[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
         sh.abort_flag = 0;
+        sh.epi_abort = 0;
+        sh.epi_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -141,21 +346,70 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const uint32_t tmem_base = sh.tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ weight producer
+        // The weights do not depend on the previous kernel, so this thread never waits for it: the
+        // stream starts as soon as the CTA is resident.  At most `window` loads are in flight, the
+        // rest of the ring is run-ahead buffer for the time the consumers wait on the previous kernel.
         if (lane == 0) {
-            uint64_t pol_stream, pol_keep;
+            uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            bool ok = true;
             uint32_t it = 0;
-            for (uint32_t u = u0; u < u1; ++u, ++it) {
+            for (; it < n_units; ++it) {
+                const uint32_t u = u0 + it;
                 const int s = it % g.stages;
-                const uint32_t ph = (it / g.stages) & 1u;
-                if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag)) break;
+                if (it >= (uint32_t)window) {
+                    const uint32_t j = it - window;
+                    if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) { ok = false; break; }
+                }
+                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 const int tile = u / g.kb_per_tile, kb = u % g.kb_per_tile;
-                const uint32_t a = tiles0 + s * stage_bytes, b = a + A_BYTES, bar = smem_u32(&sh.full[s]);
-                mbar_expect_tx(bar, stage_bytes);
-                tma_load_2d(a, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
-                tma_load_2d(b, &tm_x, kb * TILE_K, 0, bar, pol_keep);
+                const uint32_t bar = smem_u32(&sh.full_w[s]);
+                mbar_expect_tx(bar, A_BYTES);
+                tma_load_2d(tiles0 + s * stage_bytes, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
+            }
+            // While the rest of the CTA finishes (drain, reduction, fused step), keep HBM busy: pull the
+            // head of the next GEMM's weight stream through the freed stages, so that it waits in L2.
+            if (ok && nx_units > 0 && (int)blockIdx.x < nx_grid) {
+                const uint32_t Tn = (uint32_t)nx_tiles * (uint32_t)nx_kb;
+                const uint32_t v0 = (uint32_t)(((uint64_t)blockIdx.x * Tn) / nx_grid);
+                const uint32_t v1 = min((uint32_t)(((uint64_t)(blockIdx.x + 1) * Tn) / nx_grid), v0 + (uint32_t)nx_units);
+                const uint32_t first_pull = it;
+                for (uint32_t v = v0; v < v1; ++v, ++it) {
+                    const int s = it % g.stages;
+                    if (it >= (uint32_t)window) {
+                        const uint32_t j = it - window;
+                        if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) { ok = false; break; }
+                    }
+                    if (it >= (uint32_t)g.stages) {              // the stage's previous occupant must be done with it:
+                        const uint32_t j = it - g.stages;        // a real tile is released by the MMAs, a pulled one by its own arrival
+                        const bool was_real = j < n_units;
+                        if (!mbar_wait(smem_u32(was_real ? &sh.empty[s] : &sh.full_w[s]),
+                                       was_real ? (((it / g.stages) & 1u) ^ 1u) : ((j / g.stages) & 1u), abort_flag)) { ok = false; break; }
+                    }
+                    if (*(volatile int*)&sh.epi_done) break;
+                    const uint32_t bar = smem_u32(&sh.full_w[s]);
+                    mbar_expect_tx(bar, A_BYTES);
+                    tma_load_2d(tiles0 + s * stage_bytes, &tm_next, (int)(v % nx_kb) * TILE_K, (int)(v / nx_kb) * TILE_N, bar, pol_stream);
+                }
+                // nothing may still be landing in shared memory when the CTA goes away
+                for (uint32_t j = (it > first_pull + (uint32_t)window) ? it - window : first_pull; j < it && ok; ++j)
+                    if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) ok = false;
+            }
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ token-row producer
+        if (lane == 0) {
+            uint64_t pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            pdl_wait();                                           // the token rows are the previous kernel's output
+            for (uint32_t it = 0; it < n_units; ++it) {
+                const int s = it % g.stages;
+                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) break;
+                const int kb = (u0 + it) % g.kb_per_tile;
+                const uint32_t bar = smem_u32(&sh.full_x[s]);
+                mbar_expect_tx(bar, x_bytes);
+                tma_load_2d(tiles0 + s * stage_bytes + A_BYTES, &tm_x, kb * TILE_K, 0, bar, pol_keep);
             }
         }
     } else if (warp == 1) {
@@ -174,7 +428,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 for (uint32_t j = 0; j < n_kb; ++j, ++it) {
                     const int s = it % g.stages;
                     const uint32_t ph = (it / g.stages) & 1u;
-                    if (!mbar_wait(smem_u32(&sh.full[s]), ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&sh.full_w[s]), ph, abort_flag) || !mbar_wait(smem_u32(&sh.full_x[s]), ph, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a = tiles0 + s * stage_bytes;
                     const uint64_t da = umma_desc(a), db = umma_desc(a + A_BYTES);
@@ -188,15 +442,19 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: TMEM -> partials
+        // ------------------------------------------------------------------ epilogue: TMEM -> partials -> fused step
+        pdl_wait();                                                        // the workspace may still be read by the previous kernel
         const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
-        const int row = quarter * 32 + lane;                               // weight row inside the tile
+        const int et = quarter * 32 + lane;                                // weight row inside the tile
+        epilogue_prologue(g, ep, sh, et);
         uint32_t seg = 0;
         for (uint32_t u = u0; u < u1; ++seg) {
             const uint32_t kb0 = u % g.kb_per_tile;
             const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
             const uint32_t buf = seg & 1u;
-            if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) break;
+            if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) sh.epi_abort = 1;
+            epi_bar();
+            if (sh.epi_abort) break;                                       // all four warps leave together
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
             for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
@@ -205,13 +463,36 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    if (c0 + j < g.m_tok) out[(size_t)(c0 + j) * TILE_N + row] = __uint_as_float(r[j]);
+                    if (c0 + j < g.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+            // who completes the tile runs the step that follows the GEMM on it
+            const uint32_t tile = u / g.kb_per_tile;
+            uint32_t i_first, i_last;
+            tile_contributors(g, tile, i_first, i_last);
+            bool last = true;
+            if (i_last > i_first) {
+                // The barrier orders the four warps' writes before thread 0's release; the acquire
+                // side of the same operation, followed by the second barrier, orders every other
+                // CTA's pieces before the reads below (release/acquire are cumulative).
+                epi_bar();
+                if (et == 0) {
+                    uint32_t old;
+                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile) : "memory");
+                    const int l = old == i_last - i_first;
+                    if (l) counters[tile] = 0u;                            // left at zero for the next launch
+                    sh.last_flag = l;
+                }
+                epi_bar();
+                last = sh.last_flag != 0;
+            }
+            if (last) tile_epilogue(g, ep, partials, tile, sh, et);
+            epi_bar();
             u += n_kb;
         }
+        if (et == 0) *(volatile int*)&sh.epi_done = 1;
     }
 
     // ---------------------------------------------------------------------- wind-down
@@ -276,7 +557,7 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     g.max_seg = (per_cta + g.kb_per_tile - 2) / g.kb_per_tile + 1;
     if (T * g.grid >= (1ll << 32)) g.grid = 0;          // the consumers' 32-bit index arithmetic would overflow
     const int stage_bytes = A_BYTES + g.m_pad * 128;
-    g.stages = std::max(2, std::min(MAX_STAGES, (200 * 1024) / stage_bytes));
+    g.stages = std::max(2, std::min(MAX_STAGES, (198 * 1024) / stage_bytes));
     return g;
 }
 
@@ -286,34 +567,26 @@ bool gemm_tc_supported(int m_tok, int n_out, int K) {
     return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0 && (long long)((n_out + 127) / 128) * ((K + 63) / 64) < (1ll << 24);
 }
 
-cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials,
-                                uint32_t* status, cudaStream_t st) {
+cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
+                              const NextWeights* next, float* partials, uint32_t* counters, uint32_t* status,
+                              int dependent, cudaStream_t st) {
     const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_streamk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 512);
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - (int)sizeof(Shared) - 256);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    k_gemm_streamk<<<g.grid, NUM_THREADS, smem, st>>>(*(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, partials, status);
-    return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------- plain consumer
-// y[i][n] = scale(row) * (sum of the segments of n's tile, in the fixed order of their CTAs).
-__global__ void k_reduce_plain(const float* __restrict__ partials, GemmGeom g, float* __restrict__ y, int row_stride,
-                               int row_offset, RowScale rs) {
-    const int n = blockIdx.x * blockDim.x + threadIdx.x, i = blockIdx.y;
-    if (n >= g.n_out) return;
-    const int m = i * row_stride + row_offset;
-    y[(size_t)i * g.n_out + n] = gemm_reduce(partials, g, m, n) * row_scale(rs, m);
-}
-
-cudaError_t launch_reduce_plain(const float* partials, const GemmGeom& g, float* y, int n_out_rows, int row_stride,
-                                int row_offset, const RowScale& rs, cudaStream_t st) {
-    dim3 grid((g.n_out + 255) / 256, n_out_rows);
-    k_reduce_plain<<<grid, 256, 0, st>>>(partials, g, y, row_stride, row_offset, rs);
-    return cudaGetLastError();
+    if (g.grid < 1 || g.stages < 2 || g.n_tiles > GEMM_MAX_TILES || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
+    if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
+    if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
+    if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
+    const bool pull = next && next->units > 0;
+    const CUtensorMap* tn = (const CUtensorMap*)(pull ? &next->tm : &tm_w);
+    const int window = std::min(GEMM_WINDOW, g.stages - 1);          // a stage's barrier must not be polled two uses later
+    return launch_pdl(k_gemm_fused, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,
+                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, *tn, g, ep, pull ? next->n_tiles : 0,
+                      pull ? next->kb_per_tile : 1, pull ? next->grid : 1, pull ? next->units : 0, window, partials, counters, status);
 }
 
 }  // namespace sd

@@ -1,7 +1,7 @@
-// Interface of the tensor-core weight-streaming GEMM (gemm_tc.cu) and of the fixed-order
-// reduction its consumers use.
+// Interface of the tensor-core weight-streaming GEMM (gemm_tc.cu) with its fused epilogues.
 #pragma once
 #include <algorithm>
+#include <utility>
 
 #include "common.cuh"
 
@@ -18,27 +18,6 @@ struct GemmGeom {
     int grid, max_seg, stages;
 };
 
-bool gemm_tc_supported(int m_tok, int n_out, int K);
-GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm);
-size_t gemm_partials_bytes(const GemmGeom& g);
-bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows);
-cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials,
-                                uint32_t* status, cudaStream_t st);
-struct RowScale;
-// y[i][n] = scale(row) * sum of segments, row = i * row_stride + row_offset, i < n_out_rows
-cudaError_t launch_reduce_plain(const float* partials, const GemmGeom& g, float* y, int n_out_rows, int row_stride,
-                                int row_offset, const RowScale& rs, cudaStream_t st);
-
-// fused.cu: consumers that fold the step after the GEMM into the reduction of its partials
-cudaError_t launch_prep_norm(const float* h, const float* gain, void* xn, float* ssq, int n_rows, int d, cudaStream_t st);
-cudaError_t launch_cons_qkv_rope(const float* partials, const GemmGeom& g, const RowScale& rs, void* q_out, void* kc, void* vc,
-                                 const int32_t* row_slot, const int32_t* row_pos, int n_rows, int H, int Hkv, int hd,
-                                 int max_ctx, const float* rcos, const float* rsin, cudaStream_t st);
-cudaError_t launch_cons_residual(const float* partials, const GemmGeom& g, float* h, const float* gain_next, void* xn,
-                                 float* ssq, int n_rows, cudaStream_t st);
-cudaError_t launch_cons_swiglu(const float* partials, const GemmGeom& g, const RowScale& rs, void* act, int n_rows, int F,
-                               cudaStream_t st);
-
 // RMSNorm folded around a GEMM: the GEMM's input rows are h * gain (no 1/rms factor), the
 // factor rsqrt(mean(h^2) + eps) of each row multiplies the GEMM's output instead.  The sum of
 // squares of a row arrives in n_parts pieces (one per 128-wide tile of the kernel that wrote h).
@@ -49,27 +28,61 @@ struct RowScale {
 };
 constexpr int SSQ_STRIDE = 64;
 
-__device__ __forceinline__ float row_scale(const RowScale& rs, int row) {
-    if (!rs.ssq) return 1.f;
-    float ss = 0.f;
-    for (int i = 0; i < rs.n_parts; ++i) ss += rs.ssq[(size_t)row * SSQ_STRIDE + i];
-    return rsqrtf(ss * rs.inv_d + rs.eps);
+// What the CTA that completes a 128-row output tile does with it (the step that follows the
+// GEMM in the decoder layer), so that no fp32 intermediate matrix goes through memory.
+enum { EPI_PLAIN = 0, EPI_QKV_ROPE = 1, EPI_RESIDUAL = 2, EPI_SWIGLU = 3 };
+struct Epilogue {
+    int mode;
+    RowScale rs;                     // PLAIN, QKV_ROPE, SWIGLU: 1/rms factor of each token row
+    // EPI_PLAIN: y[i][n] = scale * acc[token i*row_stride + row_offset][n], i < n_out_rows
+    float* y; int n_out_rows, row_stride, row_offset;
+    // EPI_QKV_ROPE: rotary embedding, then query buffer / KV-cache append (bf16)
+    bf16* q_out; bf16* kc; bf16* vc; const int32_t* row_slot; const int32_t* row_pos;
+    int H, Hkv, hd, max_ctx; const float* rcos; const float* rsin;
+    // EPI_RESIDUAL: h += acc; xn = bf16(h * gain_next); ssq_out[row][tile] = sum over the tile of h^2
+    float* h; const float* gain_next; bf16* xn; float* ssq_out;
+    // EPI_SWIGLU: rows of the weight matrix interleaved per tile (64 gate rows, then the 64 up
+    // rows of the same features): act[row][tile*64 + f] = silu(gate_f) * up_f
+    bf16* act; int F;
+};
+
+// The weight matrix the NEXT GEMM on the stream will read: while this launch finishes (drain,
+// reduction, fused step), up to `units` of its (tile, k block) boxes per CTA are pulled through
+// the freed pipeline stages so that they wait in L2.  units == 0: nothing.
+struct NextWeights {
+    TensorMap tm;
+    int n_tiles, kb_per_tile, grid, units;
+};
+
+bool gemm_tc_supported(int m_tok, int n_out, int K);
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm);
+size_t gemm_partials_bytes(const GemmGeom& g);
+constexpr int GEMM_MAX_TILES = 4096;                                  // arrival counters, one per output tile
+constexpr size_t GEMM_COUNTER_BYTES = sizeof(uint32_t) * GEMM_MAX_TILES;
+bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows);
+// counters: GEMM_MAX_TILES words, zero before the first launch (every launch leaves them zero).
+// dependent != 0: launched with programmatic stream serialisation (may start while the previous
+// kernel on the stream drains; the kernel itself waits before it touches that kernel's results).
+cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
+                              const NextWeights* next, float* partials, uint32_t* counters, uint32_t* status,
+                              int dependent, cudaStream_t st);
+
+// Launch with the programmatic-dependent-launch attribute (or plainly when dependent == 0).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int dependent, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-// Sum of the partial accumulators that cover output (token m, feature n), always in the
-// order of the CTAs that produced them.  (T * grid < 2^32 is checked by gemm_geometry.)
-__device__ __forceinline__ float gemm_reduce(const float* __restrict__ partials, const GemmGeom& g, int m, int n) {
-    const uint32_t tile = (uint32_t)n >> 7, r = (uint32_t)n & 127u, KB = (uint32_t)g.kb_per_tile;
-    const uint32_t T = (uint32_t)g.n_tiles * KB, G = (uint32_t)g.grid;
-    const uint32_t ua = tile * KB, ub = ua + KB - 1;
-    const uint32_t i_first = ((ua + 1) * G + T - 1) / T - 1;
-    const uint32_t i_last = ((ub + 1) * G + T - 1) / T - 1;
-    float acc = 0.f;
-    for (uint32_t i = i_first; i <= i_last; ++i) {
-        const uint32_t j = tile - (i * T / G) / KB;
-        acc += partials[(((size_t)i * g.max_seg + j) * g.m_pad + m) * 128 + r];
-    }
-    return acc;
-}
+// Device side of the same protocol: let the next kernel on the stream start its prologue, and
+// wait until everything the previous kernel wrote is visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 }  // namespace sd

@@ -8,7 +8,9 @@ namespace sd {
 // ---- elementwise.cu
 cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& plan, int n_rows,
                          const void* embed, int dtype, int d, int vocab,
-                         float* h, int32_t* row_slot, int32_t* row_pos, cudaStream_t st);
+                         float* h, int32_t* row_slot, int32_t* row_pos,
+                         const float* gain /*nullable: also writes xn = bf16(h * gain) and ssq[row][0] = sum h^2*/,
+                         void* xn, float* ssq, cudaStream_t st);
 // xn[i] = rmsnorm(h[src_row(i)]) * gain; src_row(i) = i * row_stride + row_offset
 cudaError_t launch_rmsnorm(const float* h, const float* gain, void* xn, int dtype, int n_rows, int d, float eps,
                            int row_stride, int row_offset, cudaStream_t st);
@@ -17,8 +19,9 @@ cudaError_t launch_rope_kv(const float* qkv, void* q_out, void* kcache_layer, vo
                            int n_heads, int n_kv_heads, int head_dim, int max_ctx,
                            const float* rope_cos, const float* rope_sin, uint32_t* status, cudaStream_t st);
 cudaError_t launch_residual_add(float* h, const float* y, size_t n, cudaStream_t st);
-// act[r][f] = silu(gu[r][f]) * gu[r][F + f]
-cudaError_t launch_swiglu(const float* gu, void* act, int dtype, int n_rows, int F, cudaStream_t st);
+// act[r][f] = silu(gate_f) * up_f; gu[r] holds the gate values then the up values, or, when
+// interleaved, 128-wide groups of 64 gate values followed by the 64 up values of the same features
+cudaError_t launch_swiglu(const float* gu, void* act, int dtype, int n_rows, int F, int interleaved, cudaStream_t st);
 cudaError_t launch_set_state(const SeqState& S, int slot, int len, int tkv, int dkv, uint32_t iter, uint32_t seq_id,
                              int reset_counters, cudaStream_t st);
 cudaError_t launch_rollback(const SeqState& S, const SeqList& list, int gamma, const int32_t* n_acc,
@@ -40,7 +43,8 @@ bool attention_split_supported(int dtype, int H, int Hkv, int hd);
 size_t attention_split_workspace(int rows, int H, int hd, int max_ctx);
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
-                                   int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, cudaStream_t st);
+                                   int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
+                                   cudaStream_t st);
 
 // ---- sampling.cu
 cudaError_t launch_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, cudaStream_t st);
@@ -57,7 +61,7 @@ struct AcceptParams {
     int use_list; SeqList list;
     int32_t* n_acc; int32_t* out_tok;
 };
-cudaError_t launch_accept(const AcceptParams& p, cudaStream_t st);
+cudaError_t launch_accept(const AcceptParams& p, int dependent, cudaStream_t st);
 
 // ---- classifier.cu
 cudaError_t launch_classifier(const SeqState& S, const SeqList& list, const SeqList& forced /*ids[i] >= 0: given task*/,

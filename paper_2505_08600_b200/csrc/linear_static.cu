@@ -11,6 +11,7 @@
 // cudaGetSymbolAddress returns for the device that is current at the time.  The address is
 // looked up once per device, on the first call made with that device current.
 #include <stdio.h>
+#include <string.h>
 
 #include <mutex>
 
@@ -52,20 +53,24 @@ extern "C" sd_status sd_op_linear_static(const void* x, const void* w, float* y,
         return SD_ERR_CUDA;
     const GemmGeom g = gemm_geometry(rows, n_out, n_in, n_sm);
     if (g.grid < 1) return SD_ERR_UNSUPPORTED;
-    if (gemm_partials_bytes(g) > (size_t)SD_STATIC_SCRATCH_BYTES) {
+    if (GEMM_COUNTER_BYTES + gemm_partials_bytes(g) > (size_t)SD_STATIC_SCRATCH_BYTES) {
         fprintf(stderr, "[sd] sd_op_linear_static: %d x %d x %d needs %zu bytes of scratch, the built-in array holds %d\n",
-                rows, n_out, n_in, gemm_partials_bytes(g), (int)SD_STATIC_SCRATCH_BYTES);
+                rows, n_out, n_in, GEMM_COUNTER_BYTES + gemm_partials_bytes(g), (int)SD_STATIC_SCRATCH_BYTES);
         return SD_ERR_CAPACITY;
     }
-    float* scratch = (float*)scratch_on_current_device();
+    char* scratch = (char*)scratch_on_current_device();
     if (!scratch) return SD_ERR_CUDA;
     TensorMap tw, tx;
     if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // Every (slot, token, row) of the scratch that the reduction reads is written by this call's
-    // GEMM first, so nothing left over from an earlier call needs clearing.
-    if (launch_gemm_streamk(tw, tx, g, scratch, nullptr, st) != cudaSuccess) return SD_ERR_CUDA;
-    RowScale none{nullptr, 0, 0.f, 0.f};
-    if (launch_reduce_plain(scratch, g, y, rows, 1, 0, none, st) != cudaSuccess) return SD_ERR_CUDA;
+    // The head of the array holds the tiles' arrival counters, which must start at zero (a call that
+    // was cut short could have left some behind); every accumulator word that is read is written by
+    // this call's own GEMM first, so the rest needs no clearing.
+    if (cudaMemsetAsync(scratch, 0, GEMM_COUNTER_BYTES, st) != cudaSuccess) return SD_ERR_CUDA;
+    Epilogue e;
+    memset(&e, 0, sizeof(e));
+    e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
+    if (launch_gemm_fused(tw, tx, g, e, nullptr, (float*)(scratch + GEMM_COUNTER_BYTES), (uint32_t*)scratch, nullptr, 0, st) != cudaSuccess)
+        return SD_ERR_CUDA;
     return SD_OK;
 }

@@ -1,5 +1,8 @@
 // Vocabulary-wide kernels: softmax with temperature, the exact integer inverse-CDF draw, the
 // draft's per-step sampler and the fused accept / reject / resample kernel.
+#include <cooperative_groups.h>
+
+#include "gemm_tc.h"
 #include "kernels.h"
 
 namespace sd {
@@ -158,15 +161,24 @@ cudaError_t launch_draft_sample(const float* logits, const SeqState& S, const Se
 }
 
 // ---------------------------------------------------------------- accept / reject / resample
-// One block per sequence.  Slot s is accepted iff u_s * q_s(x_s) <= p_s(x_s) with a single
-// rounded fp32 multiply; the first rejected slot n (or gamma) picks the row the next token is
-// drawn from: the residual max(0, p_n - q_n) or, after gamma accepts, p_gamma itself.
-__global__ void __launch_bounds__(1024) k_accept(AcceptParams P) {
+// One thread-block cluster per sequence, one CTA per target row (two when gamma + 1 > 8).
+// Every CTA works out the softmax statistics of its row(s) and, for a draft slot, the accept
+// test u_s * q_s(x_s) <= p_s(x_s) with a single rounded fp32 multiply.  The flags are exchanged
+// through distributed shared memory; the CTA that owns the first rejected row n (or row gamma
+// after gamma accepts) draws the next token from the residual max(0, p_n - q_n), or from
+// p_gamma itself, and writes the result.
+constexpr int ACC_ROWS_PER_CTA = 2;
+
+__global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     __shared__ BlockScratch sh;
-    __shared__ float row_max[SD_MAX_GAMMA + 1], row_sum[SD_MAX_GAMMA + 1];
-    __shared__ int row_arg[SD_MAX_GAMMA + 1];
+    __shared__ float row_max[ACC_ROWS_PER_CTA], row_sum[ACC_ROWS_PER_CTA];
+    __shared__ int row_arg[ACC_ROWS_PER_CTA];
+    __shared__ int flag_sh[ACC_ROWS_PER_CTA];
     __shared__ int n_sh;
-    const int i = blockIdx.x;
+    pdl_launch_dependents();
+    const int i = blockIdx.x / csize, rank = blockIdx.x % csize;
     const int idx = P.use_list ? P.list.ids[i] : i;
     const int b = P.use_list ? P.list.out[i] : i;
     const int V = P.V, gamma = P.gamma;
@@ -175,67 +187,92 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P) {
     const float* q = P.q + (size_t)b * gamma * V;
     const int32_t* x = P.x + (size_t)b * gamma;
     const bool logits = P.target_is_logits != 0;
+    pdl_wait();                                   // target rows, drafts and per-sequence state come from earlier kernels
 
-    if (logits) {
-        for (int j = 0; j <= gamma; ++j) {
+    auto prob = [&](int j, int li, int k) -> float {          // li: index of row j among this CTA's rows
+        const float v = tgt[(size_t)j * V + k];
+        if (!logits) return v;
+        if (T == 0.f) return k == row_arg[li] ? 1.f : 0.f;
+        return expf((v - row_max[li]) / T) / row_sum[li];
+    };
+
+    for (int li = 0; li < ACC_ROWS_PER_CTA; ++li) {
+        const int j = rank + li * csize;
+        if (j > gamma) break;                                   // uniform in the CTA
+        if (logits) {
             const float* l = tgt + (size_t)j * V;
             if (T == 0.f) {
                 int a = block_argmax([&](int k) { return l[k]; }, V, sh, nullptr);
-                if (threadIdx.x == 0) row_arg[j] = a;
+                if (threadIdx.x == 0) row_arg[li] = a;
             } else {
                 float m = -INFINITY;
                 for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, l[k]);
                 m = block_max(m, sh.red);
-                float s = 0.f;
-                for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) / T);
-                s = block_sum(s, sh.red);
-                if (threadIdx.x == 0) { row_max[j] = m; row_sum[j] = s; }
+                float sum = 0.f;
+                for (int k = threadIdx.x; k < V; k += blockDim.x) sum += expf((l[k] - m) / T);
+                sum = block_sum(sum, sh.red);
+                if (threadIdx.x == 0) { row_max[li] = m; row_sum[li] = sum; }
             }
+            __syncthreads();
         }
-        __syncthreads();
+        if (threadIdx.x == 0 && j < gamma) {
+            int ok = 0;
+            const int xs = x[j];
+            if (xs >= 0 && xs < V) {                            // an impossible token counts as rejected
+                const uint32_t ui = uniform24(P.seed, P.iter[idx], (uint32_t)j, P.seq_id[idx], DRAW_ACCEPT);
+                const float u = (float)ui * (1.0f / 16777216.0f);
+                const float lhs = __fmul_rn(u, q[(size_t)j * V + xs]);
+                ok = lhs <= prob(j, li, xs);
+            }
+            flag_sh[li] = ok;
+        }
     }
-    auto prob = [&](int j, int k) -> float {
-        const float v = tgt[(size_t)j * V + k];
-        if (!logits) return v;
-        if (T == 0.f) return k == row_arg[j] ? 1.f : 0.f;
-        return expf((v - row_max[j]) / T) / row_sum[j];
-    };
-
+    cluster.sync();                                             // every CTA's flags are in place
     if (threadIdx.x == 0) {
-        const uint32_t it = P.iter[idx], sid = P.seq_id[idx];
         int n = 0;
         while (n < gamma) {
-            int xs = x[n];
-            if (xs < 0 || xs >= V) break;                        // impossible token: treat as rejected
-            const uint32_t ui = uniform24(P.seed, it, (uint32_t)n, sid, DRAW_ACCEPT);
-            const float u = (float)ui * (1.0f / 16777216.0f);
-            const float lhs = __fmul_rn(u, q[(size_t)n * V + xs]);
-            if (!(lhs <= prob(n, xs))) break;
+            const int* remote = cluster.map_shared_rank(flag_sh, n % csize);
+            if (!remote[n / csize]) break;
             ++n;
         }
         n_sh = n;
     }
     __syncthreads();
     const int n = n_sh;
-    const uint32_t ui = uniform24(P.seed, P.iter[idx], (uint32_t)n, P.seq_id[idx], DRAW_RESAMPLE);
-    int y;
-    if (n < gamma) {
-        const float* qn = q + (size_t)n * V;
-        y = block_icdf([&](int k) { return fmaxf(__fsub_rn(prob(n, k), qn[k]), 0.f); }, V, ui, sh);
-        if (y < 0) y = block_icdf([&](int k) { return prob(n, k); }, V, ui, sh);
-    } else {
-        y = block_icdf([&](int k) { return prob(n, k); }, V, ui, sh);
+    if (n % csize == rank) {                                    // this CTA holds the statistics of row n
+        const int li = n / csize;
+        const uint32_t ui = uniform24(P.seed, P.iter[idx], (uint32_t)n, P.seq_id[idx], DRAW_RESAMPLE);
+        int y;
+        if (n < gamma) {
+            const float* qn = q + (size_t)n * V;
+            y = block_icdf([&](int k) { return fmaxf(__fsub_rn(prob(n, li, k), qn[k]), 0.f); }, V, ui, sh);
+            if (y < 0) y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+        } else {
+            y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+        }
+        if (y < 0) y = block_argmax([&](int k) { return prob(n, li, k); }, V, sh, nullptr);
+        if (threadIdx.x == 0) P.n_acc[b] = n;
+        for (int s = threadIdx.x; s <= gamma; s += blockDim.x)
+            P.out_tok[(size_t)b * (gamma + 1) + s] = s < n ? x[s] : (s == n ? y : -1);
     }
-    if (y < 0) y = block_argmax([&](int k) { return prob(n, k); }, V, sh, nullptr);
-    if (threadIdx.x == 0) P.n_acc[b] = n;
-    for (int s = threadIdx.x; s <= gamma; s += blockDim.x)
-        P.out_tok[(size_t)b * (gamma + 1) + s] = s < n ? x[s] : (s == n ? y : -1);
+    cluster.sync();                                             // no CTA leaves while its flags may still be read
 }
 
-cudaError_t launch_accept(const AcceptParams& p, cudaStream_t st) {
+cudaError_t launch_accept(const AcceptParams& p, int dependent, cudaStream_t st) {
     if (p.B <= 0) return cudaSuccess;
-    k_accept<<<p.B, 1024, 0, st>>>(p);
-    return cudaGetLastError();
+    int csize = 1;
+    while (csize < p.gamma + 1 && csize < 8) csize <<= 1;      // portable cluster sizes only
+    if (csize * ACC_ROWS_PER_CTA < p.gamma + 1) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.B * csize); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, k_accept, p, csize);
 }
 
 }  // namespace sd
