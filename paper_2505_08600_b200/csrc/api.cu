@@ -68,7 +68,6 @@ struct sd_ctx {
     float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
     uint32_t* gemm_counters;                    // arrival counters of the GEMM's output tiles (zero between launches)
-    int pull_units;                             // weight boxes per CTA that a GEMM pulls into L2 for its successor
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
     struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
@@ -302,23 +301,13 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     return SD_OK;
 }
 
-// One weight GEMM with its fused epilogue.  `next` names the matrix the following GEMM on the
-// stream will read (nullptr: none), so that this launch can pull its head into L2 while finishing.
-struct NextMat { const TensorMap* tm; int n_out, K; };
-
-sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep,
-                  const NextMat* next) {
+// One weight GEMM with its fused epilogue.
+sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
     const GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
-    NextWeights nw;
-    nw.units = 0;
-    if (next && next->tm && c->pull_units > 0) {
-        const GemmGeom gn = gemm_geometry(rows, next->n_out, next->K, sm_count());
-        nw.tm = *next->tm; nw.n_tiles = gn.n_tiles; nw.kb_per_tile = gn.kb_per_tile; nw.grid = gn.grid; nw.units = c->pull_units;
-    }
-    LAUNCH(CAT_LINEAR, launch_gemm_fused(tw, tx, g, ep, &nw, c->partials, c->gemm_counters, c->S.status, 1, c->st));
+    LAUNCH(CAT_LINEAR, launch_gemm_fused(tw, tx, g, ep, c->partials, c->gemm_counters, c->S.status, 1, c->st));
     return SD_OK;
 }
 
@@ -342,24 +331,19 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.mode = EPI_QKV_ROPE; e.rs = l == 0 ? first : tiled;
         e.q_out = (bf16*)c->q; e.kc = (bf16*)kc; e.vc = (bf16*)vc; e.row_slot = c->row_slot; e.row_pos = c->row_pos;
         e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = M.rope_cos; e.rsin = M.rope_sin;
-        NextMat nx{&L.tm_wo, d, H * hd};
-        SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e, &nx));
+        SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
                                                      hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st));
         memset(&e, 0, sizeof(e));
         e.mode = EPI_RESIDUAL; e.h = c->h; e.gain_next = L.norm2; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
-        nx = NextMat{&L.tm_gu, 2 * F, d};
-        SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e, &nx));
+        SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e));
         memset(&e, 0, sizeof(e));
         e.mode = EPI_SWIGLU; e.rs = tiled; e.act = (bf16*)c->act; e.F = F;
-        nx = NextMat{&L.tm_wd, d, F};
-        SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, e, &nx));
+        SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, e));
         memset(&e, 0, sizeof(e));
         e.mode = EPI_RESIDUAL; e.h = c->h; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
         e.gain_next = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
-        if (l + 1 < m.n_layers) nx = NextMat{&M.layers[l + 1].tm_qkv, M.n_qkv(), d};
-        else nx = NextMat{mode != LOGITS_NONE ? &M.tm_lm : nullptr, m.vocab, d};
-        SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, e, &nx));
+        SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, e));
     }
     if (mode != LOGITS_NONE) {
         // the lm_head GEMM runs over all rows (they share the one pass over the weights); only the wanted rows are written
@@ -369,7 +353,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.mode = EPI_PLAIN; e.rs = tiled; e.y = logits_out;
         if (mode == LOGITS_ALL) { e.n_out_rows = n_rows; e.row_stride = 1; e.row_offset = 0; }
         else { e.n_out_rows = list.n; e.row_stride = R; e.row_offset = R - 1; }
-        SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, e, nullptr));
+        SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, e));
     }
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
@@ -518,7 +502,6 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
     c->force_plain = false;
-    c->pull_units = 16;
     c->graphs_on = true;
     c->graph_clock = 0;
     for (Model& M : c->models) {
@@ -932,7 +915,7 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
         memset(&e, 0, sizeof(e));
         e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
         CUDA_TRY(cudaMemsetAsync(workspace, 0, GEMM_COUNTER_BYTES, (cudaStream_t)stream));          // the arrival counters
-        CUDA_TRY(launch_gemm_fused(tw, tx, g, e, nullptr, (float*)((char*)workspace + GEMM_COUNTER_BYTES), (uint32_t*)workspace,
+        CUDA_TRY(launch_gemm_fused(tw, tx, g, e, (float*)((char*)workspace + GEMM_COUNTER_BYTES), (uint32_t*)workspace,
                                    nullptr, 0, (cudaStream_t)stream));
         return SD_OK;
     }

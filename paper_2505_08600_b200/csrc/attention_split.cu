@@ -277,37 +277,69 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     }
     __syncthreads();
     if (!last_sm) return;
-    // (1) every slice's max and sum into shared memory, (2) one warp per query turns them into
-    // normalised weights, (3) every thread owns output elements and adds the weighted slices
-    float* m_all = reinterpret_cast<float*>(sm_raw);             // [nq][n_splits]
-    float* l_all = m_all + NQ * 32;                              // [nq][n_splits]
+    // Everything the merge reads (every slice's max, sum and partial output for the block's
+    // queries) is fetched into shared memory in one go, so the merge costs one memory round trip.
     const int ns = P.n_splits;
-    for (int i = t; i < nq * ns; i += ATT_THREADS) {
-        const int j = i / ns, s = i % ns;
-        const int r = r0 + j / group, h = kvh * group + j % group;
-        const float* ml = P.part_ml + (((size_t)r * P.H + h) * ns + s) * 2;
-        m_all[i] = __ldcg(ml); l_all[i] = __ldcg(ml + 1);
+    float* o_all = reinterpret_cast<float*>(sm_raw);             // [nq][ns][HD]
+    __shared__ float wgt[NQ * 32];                               // normalised weight of each (query, slice)
+    const bool staged = (size_t)nq * ns * HD * sizeof(float) <= (size_t)4 * BUF;
+    if (staged) {
+        const int per_q = ns * (HD / 4);                         // 16-byte pieces of one query's partial outputs
+        for (int j = 0; j < nq; ++j) {
+            const int r = r0 + j / group, h = kvh * group + j % group;
+            const float* src = P.part_o + ((size_t)r * P.H + h) * ns * HD;
+            const uint32_t dst = smem0 + (uint32_t)j * (uint32_t)per_q * 16u;
+            for (int c = t; c < per_q; c += ATT_THREADS) cp_async16(dst + (uint32_t)c * 16u, src + (size_t)c * 4);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    __syncthreads();
-    for (int j = warp; j < nq; j += ATT_THREADS / 32) {      // n_splits <= 32: one lane per slice
-        const float m = lane < ns ? m_all[j * ns + lane] : -INFINITY;
+    for (int j = warp; j < nq; j += ATT_THREADS / 32) {          // n_splits <= 32: one lane per slice
+        const int r = r0 + j / group, h = kvh * group + j % group;
+        const float* mlg = P.part_ml + ((size_t)r * P.H + h) * ns * 2;
+        float m = -INFINITY, l = 0.f;
+        if (lane < ns) { const float2 v = __ldcg(reinterpret_cast<const float2*>(mlg) + lane); m = v.x; l = v.y; }
         const float M = warp_max(m);
         const float w = (m == -INFINITY) ? 0.f : exp2f(m - M);
-        const float den = warp_sum(lane < ns ? w * l_all[j * ns + lane] : 0.f);
-        if (lane < ns) m_all[j * ns + lane] = den > 0.f ? w / den : 0.f;
+        const float den = warp_sum(w * l);
+        if (lane < ns) wgt[j * 32 + lane] = den > 0.f ? w / den : 0.f;
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-    for (int i = t; i < nq * HD; i += ATT_THREADS) {
-        const int j = i / HD, e = i % HD;
-        const int r = r0 + j / group, h = kvh * group + j % group;
-        const float* o = P.part_o + ((size_t)r * P.H + h) * ns * HD + e;
-        float acc = 0.f;
-#pragma unroll 4
-        for (int s = 0; s < ns; ++s) {
-            const float w = m_all[j * ns + s];
-            acc = fmaf(w, w != 0.f ? __ldcg(o + (size_t)s * HD) : 0.f, acc);      // an empty slice left no output behind
+    // each thread owns one output column of up to NQ queries: independent sums, slices in order
+    constexpr int TPQ = ATT_THREADS / HD;                        // queries handled side by side (1 or 2)
+    const int e = t % HD, jq0 = t / HD;
+    float acc[NQ / TPQ];
+#pragma unroll
+    for (int i = 0; i < NQ / TPQ; ++i) acc[i] = 0.f;
+    if (staged) {                    // branch-free: rows past nq re-read the last valid row and are dropped below
+        for (int sidx = 0; sidx < ns; ++sidx) {
+#pragma unroll
+            for (int i = 0; i < NQ / TPQ; ++i) {
+                const int j = min(jq0 + i * TPQ, nq - 1);
+                const float w = wgt[j * 32 + sidx];
+                const float o = o_all[((size_t)j * ns + sidx) * HD + e];
+                acc[i] = fmaf(w, w != 0.f ? o : 0.f, acc[i]);    // an empty slice left no output behind
+            }
         }
-        P.out[((size_t)r * P.H + h) * HD + e] = __float2bfloat16_rn(acc);
+    } else {
+        for (int sidx = 0; sidx < ns; ++sidx) {
+#pragma unroll
+            for (int i = 0; i < NQ / TPQ; ++i) {
+                const int j = min(jq0 + i * TPQ, nq - 1);
+                const int r = r0 + j / group, h = kvh * group + j % group;
+                const float w = wgt[j * 32 + sidx];
+                const float o = __ldcg(P.part_o + (((size_t)r * P.H + h) * ns + sidx) * HD + e);
+                acc[i] = fmaf(w, w != 0.f ? o : 0.f, acc[i]);
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NQ / TPQ; ++i) {
+        const int j = jq0 + i * TPQ;
+        if (j < nq) {
+            const int r = r0 + j / group, h = kvh * group + j % group;
+            P.out[((size_t)r * P.H + h) * HD + e] = __float2bfloat16_rn(acc[i]);
+        }
     }
 }
 

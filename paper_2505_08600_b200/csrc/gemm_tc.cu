@@ -18,10 +18,7 @@
 //     SwiGLU, or plain fp32 output); nothing spins: a CTA that is not last just moves on;
 //   - the kernel is written for programmatic dependent launch: it lets its successor start at
 //     once; its weight stream never waits for the predecessor (only the token rows and the
-//     workspace do); at most a few weight tiles per SM are in flight (enough to saturate HBM, a
-//     deeper queue only adds latency), the rest of the ring is run-ahead buffer; and after its
-//     own last tile the producer pulls the head of the next GEMM's weights through the freed
-//     stages so that they wait in L2 and HBM stays busy across the kernel boundary.
+//     workspace do), so the ring is full when the consumers are released.
 // Roles: warp 0 streams weights, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM and
 // run the fused step, warp 6 loads the token rows.  Every mbarrier wait is bounded; on expiry
 // the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
@@ -38,7 +35,6 @@ constexpr int TILE_K = 64;                  // bf16 elements per k block = one 1
 constexpr int A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
-constexpr int GEMM_WINDOW = 5;               // weight tiles in flight per SM: 80 KB x 148 SMs saturates HBM
 constexpr int EPI_MB = 8;                    // token rows the fused step handles at a time
 constexpr int EPI_CB = 8;                    // pieces of a tile whose loads are in flight together
 
@@ -121,7 +117,6 @@ struct Shared {
     uint32_t tmem_base;
     int abort_flag;
     int epi_abort, last_flag;
-    int epi_done;                   // the epilogue warps are through: stop pulling the next GEMM's weights
     float scale[SD_MAX_ROWS];       // 1/rms factor of each token row
     int pos[SD_MAX_ROWS];           // cache position and sequence slot of each token row (rotary / KV append)
     int slot[SD_MAX_ROWS];
@@ -133,8 +128,8 @@ struct Shared {
 __device__ __forceinline__ void tile_contributors(const GemmGeom& g, uint32_t tile, uint32_t& i_first, uint32_t& i_last) {
     const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
     const uint32_t ua = tile * KB, ub = ua + KB - 1;
-    i_first = (uint32_t)((((uint64_t)ua + 1) * G + T - 1) / T) - 1;
-    i_last = (uint32_t)((((uint64_t)ub + 1) * G + T - 1) / T) - 1;
+    i_first = ((ua + 1) * G + T - 1) / T - 1;                    // T * G < 2^32 (checked on the host): 32-bit arithmetic
+    i_last = ((ub + 1) * G + T - 1) / T - 1;
 }
 
 // What the fused step needs per token row and does not depend on the tile: the 1/rms factors,
@@ -185,7 +180,7 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
             for (int cc = 0; cc < EPI_CB; ++cc) {
                 const uint32_t c = c0 + cc;
                 const bool ok = c <= i_last;
-                const uint32_t j = ok ? tile - (uint32_t)(((uint64_t)c * T) / G) / KB : 0u;
+                const uint32_t j = ok ? tile - ((c * T) / G) / KB : 0u;      // c * T < 2^32 (checked on the host)
                 const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
 #pragma unroll
                 for (int i = 0; i < EPI_MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
@@ -307,8 +302,7 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
-             const __grid_constant__ CUtensorMap tm_next, GemmGeom g, Epilogue ep, int nx_tiles, int nx_kb, int nx_grid,
-             int nx_units, int window, float* __restrict__ partials, uint32_t* __restrict__ counters, uint32_t* status) {
+             GemmGeom g, Epilogue ep, float* __restrict__ partials, uint32_t* __restrict__ counters, uint32_t* status) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ Shared sh;
     pdl_launch_dependents();                 // the next kernel may be scheduled; it waits for this one where it must
@@ -319,8 +313,8 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
 
     // this CTA's share of the (row tile, k block) pairs
     const uint32_t T = (uint32_t)g.n_tiles * (uint32_t)g.kb_per_tile;
-    const uint32_t u0 = (uint32_t)(((uint64_t)blockIdx.x * T) / gridDim.x);
-    const uint32_t u1 = (uint32_t)(((uint64_t)(blockIdx.x + 1) * T) / gridDim.x);
+    const uint32_t u0 = (blockIdx.x * T) / gridDim.x;
+    const uint32_t u1 = ((blockIdx.x + 1) * T) / gridDim.x;
     const uint32_t n_units = u1 - u0;
     uint32_t tmem_cols = 32;
     while (tmem_cols < 2u * (uint32_t)g.m_pad) tmem_cols <<= 1;
@@ -332,7 +326,6 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
         sh.abort_flag = 0;
         sh.epi_abort = 0;
-        sh.epi_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -348,53 +341,20 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------------------------ weight producer
         // The weights do not depend on the previous kernel, so this thread never waits for it: the
-        // stream starts as soon as the CTA is resident.  At most `window` loads are in flight, the
-        // rest of the ring is run-ahead buffer for the time the consumers wait on the previous kernel.
+        // stream starts as soon as the CTA is resident and runs ahead by the depth of the ring while
+        // the consumers wait on the previous kernel.  (Capping the loads in flight below the ring
+        // depth was tried: polling for their arrival cost more than the shorter queues gained.)
         if (lane == 0) {
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            bool ok = true;
-            uint32_t it = 0;
-            for (; it < n_units; ++it) {
+            for (uint32_t it = 0; it < n_units; ++it) {
                 const uint32_t u = u0 + it;
                 const int s = it % g.stages;
-                if (it >= (uint32_t)window) {
-                    const uint32_t j = it - window;
-                    if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) { ok = false; break; }
-                }
-                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) break;
                 const int tile = u / g.kb_per_tile, kb = u % g.kb_per_tile;
                 const uint32_t bar = smem_u32(&sh.full_w[s]);
                 mbar_expect_tx(bar, A_BYTES);
                 tma_load_2d(tiles0 + s * stage_bytes, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
-            }
-            // While the rest of the CTA finishes (drain, reduction, fused step), keep HBM busy: pull the
-            // head of the next GEMM's weight stream through the freed stages, so that it waits in L2.
-            if (ok && nx_units > 0 && (int)blockIdx.x < nx_grid) {
-                const uint32_t Tn = (uint32_t)nx_tiles * (uint32_t)nx_kb;
-                const uint32_t v0 = (uint32_t)(((uint64_t)blockIdx.x * Tn) / nx_grid);
-                const uint32_t v1 = min((uint32_t)(((uint64_t)(blockIdx.x + 1) * Tn) / nx_grid), v0 + (uint32_t)nx_units);
-                const uint32_t first_pull = it;
-                for (uint32_t v = v0; v < v1; ++v, ++it) {
-                    const int s = it % g.stages;
-                    if (it >= (uint32_t)window) {
-                        const uint32_t j = it - window;
-                        if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) { ok = false; break; }
-                    }
-                    if (it >= (uint32_t)g.stages) {              // the stage's previous occupant must be done with it:
-                        const uint32_t j = it - g.stages;        // a real tile is released by the MMAs, a pulled one by its own arrival
-                        const bool was_real = j < n_units;
-                        if (!mbar_wait(smem_u32(was_real ? &sh.empty[s] : &sh.full_w[s]),
-                                       was_real ? (((it / g.stages) & 1u) ^ 1u) : ((j / g.stages) & 1u), abort_flag)) { ok = false; break; }
-                    }
-                    if (*(volatile int*)&sh.epi_done) break;
-                    const uint32_t bar = smem_u32(&sh.full_w[s]);
-                    mbar_expect_tx(bar, A_BYTES);
-                    tma_load_2d(tiles0 + s * stage_bytes, &tm_next, (int)(v % nx_kb) * TILE_K, (int)(v / nx_kb) * TILE_N, bar, pol_stream);
-                }
-                // nothing may still be landing in shared memory when the CTA goes away
-                for (uint32_t j = (it > first_pull + (uint32_t)window) ? it - window : first_pull; j < it && ok; ++j)
-                    if (!mbar_wait(smem_u32(&sh.full_w[j % g.stages]), (j / g.stages) & 1u, abort_flag)) ok = false;
             }
         }
     } else if (warp == 6) {
@@ -492,7 +452,6 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
             epi_bar();
             u += n_kb;
         }
-        if (et == 0) *(volatile int*)&sh.epi_done = 1;
     }
 
     // ---------------------------------------------------------------------- wind-down
@@ -555,7 +514,7 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     g.grid = (int)std::min<long long>(n_sm, T);
     const int per_cta = (int)((T + g.grid - 1) / g.grid);
     g.max_seg = (per_cta + g.kb_per_tile - 2) / g.kb_per_tile + 1;
-    if (T * g.grid >= (1ll << 32)) g.grid = 0;          // the consumers' 32-bit index arithmetic would overflow
+    if ((T + 1) * (g.grid + 1) >= (1ll << 32)) g.grid = 0;   // the kernels split the work in 32-bit arithmetic
     const int stage_bytes = A_BYTES + g.m_pad * 128;
     g.stages = std::max(2, std::min(MAX_STAGES, (198 * 1024) / stage_bytes));
     return g;
@@ -568,8 +527,7 @@ bool gemm_tc_supported(int m_tok, int n_out, int K) {
 }
 
 cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
-                              const NextWeights* next, float* partials, uint32_t* counters, uint32_t* status,
-                              int dependent, cudaStream_t st) {
+                              float* partials, uint32_t* counters, uint32_t* status, int dependent, cudaStream_t st) {
     const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
@@ -581,12 +539,8 @@ cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, cons
     if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
-    const bool pull = next && next->units > 0;
-    const CUtensorMap* tn = (const CUtensorMap*)(pull ? &next->tm : &tm_w);
-    const int window = std::min(GEMM_WINDOW, g.stages - 1);          // a stage's barrier must not be polled two uses later
     return launch_pdl(k_gemm_fused, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,
-                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, *tn, g, ep, pull ? next->n_tiles : 0,
-                      pull ? next->kb_per_tile : 1, pull ? next->grid : 1, pull ? next->units : 0, window, partials, counters, status);
+                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, ep, partials, counters, status);
 }
 
 }  // namespace sd

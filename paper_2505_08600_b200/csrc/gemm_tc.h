@@ -46,14 +46,6 @@ struct Epilogue {
     bf16* act; int F;
 };
 
-// The weight matrix the NEXT GEMM on the stream will read: while this launch finishes (drain,
-// reduction, fused step), up to `units` of its (tile, k block) boxes per CTA are pulled through
-// the freed pipeline stages so that they wait in L2.  units == 0: nothing.
-struct NextWeights {
-    TensorMap tm;
-    int n_tiles, kb_per_tile, grid, units;
-};
-
 bool gemm_tc_supported(int m_tok, int n_out, int K);
 GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm);
 size_t gemm_partials_bytes(const GemmGeom& g);
@@ -64,8 +56,7 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
 // dependent != 0: launched with programmatic stream serialisation (may start while the previous
 // kernel on the stream drains; the kernel itself waits before it touches that kernel's results).
 cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
-                              const NextWeights* next, float* partials, uint32_t* counters, uint32_t* status,
-                              int dependent, cudaStream_t st);
+                              float* partials, uint32_t* counters, uint32_t* status, int dependent, cudaStream_t st);
 
 // Launch with the programmatic-dependent-launch attribute (or plainly when dependent == 0).
 template <typename... KArgs, typename... Args>

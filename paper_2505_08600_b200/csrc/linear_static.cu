@@ -70,7 +70,7 @@ extern "C" sd_status sd_op_linear_static(const void* x, const void* w, float* y,
     Epilogue e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
-    if (launch_gemm_fused(tw, tx, g, e, nullptr, (float*)(scratch + GEMM_COUNTER_BYTES), (uint32_t*)scratch, nullptr, 0, st) != cudaSuccess)
+    if (launch_gemm_fused(tw, tx, g, e, (float*)(scratch + GEMM_COUNTER_BYTES), (uint32_t*)scratch, nullptr, 0, st) != cudaSuccess)
         return SD_ERR_CUDA;
     return SD_OK;
 }
