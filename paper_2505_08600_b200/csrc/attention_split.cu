@@ -14,9 +14,11 @@ namespace sd {
 
 namespace {
 
-constexpr int ATT_THREADS = 128;    // four warps; each takes 16 of the 64 keys of a chunk
+constexpr int ATT_WARPS = 8;
+constexpr int ATT_THREADS = 32 * ATT_WARPS;   // each warp takes 16 of the keys of a chunk
 constexpr int NQ = 16;              // query vectors per CTA (rows in the block x heads per KV head): one MMA row tile
-constexpr int CK = 64;              // keys per chunk
+constexpr int CK = 16 * ATT_WARPS;  // keys per chunk
+constexpr int SLICE_KEYS = 1024;    // a slice of the cache per CTA: up to this many positions
 constexpr size_t ATTN_COUNTER_BYTES = 65536;     // one arrival counter per (query block, kv head)
 
 struct AttnParams {
@@ -55,8 +57,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // heads that share the KV head), as a 16-row tensor-core tile.  The slice is walked in chunks
 // of 64 keys, double-buffered in shared memory (16-byte asynchronous copies into an
 // XOR-swizzled layout that ldmatrix reads without bank conflicts); each warp owns 16 keys of a
-// chunk and keeps its own running max / sum / output (online softmax, exp2 domain), the four
-// warps are merged at the end, and the slices of a head are merged by whichever CTA arrives last.
+// chunk and keeps its own running max / sum / output (online softmax, exp2 domain), the warps
+// are merged at the end.  A context of up to SLICE_KEYS positions is one slice: the CTA then
+// writes the attention output itself; longer contexts are cut into slices whose partial results
+// are merged by whichever CTA arrives last.
 template <int HD>
 __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
@@ -211,10 +215,10 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
     }
 
-    // ---- merge of the four warps (each saw different keys), then the slice's partial result
-    float* Ow = reinterpret_cast<float*>(sm_raw);                // [4][16][OLD]
-    float* mw = Ow + 4 * NQ * OLD;                               // [4][16]
-    float* lw = mw + 4 * NQ;                                     // [4][16]
+    // ---- merge of the warps (each saw different keys), then the slice's partial result
+    float* Ow = reinterpret_cast<float*>(sm_raw);                // [warps][16][OLD]
+    float* mw = Ow + ATT_WARPS * NQ * OLD;                       // [warps][16]
+    float* lw = mw + ATT_WARPS * NQ;                             // [warps][16]
     if (np > 0) {
 #pragma unroll
         for (int nv = 0; nv < NV; ++nv) {
@@ -228,41 +232,51 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     }
     __syncthreads();
     {
-        const int j = t >> 3, c0 = (t & 7) * (HD / 8);           // query row of the tile, first of this thread's columns
+        constexpr int CPT = HD / 16;                             // columns per thread: 16 threads span a query row
+        const int j = t >> 4, c0 = (t & 15) * CPT;
         if (j < nq) {
             const int r = r0 + j / group, h = kvh * group + j % group;
             float* po = P.part_o + (((size_t)r * P.H + h) * P.n_splits + split) * HD;
             float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
+            bf16* dst = P.out + ((size_t)r * P.H + h) * HD;
             if (np <= 0) {
-                if ((t & 7) == 0) { __stcg(ml, -INFINITY); __stcg(ml + 1, 0.f); }
+                if (P.n_splits == 1) {
+#pragma unroll
+                    for (int cc = 0; cc < CPT; ++cc) dst[c0 + cc] = __float2bfloat16_rn(0.f);
+                } else if ((t & 15) == 0) { __stcg(ml, -INFINITY); __stcg(ml + 1, 0.f); }
             } else {
                 float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) M = fmaxf(M, mw[w * NQ + j]);
-                float wt[4], L = 0.f;
+                for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, mw[w * NQ + j]);
+                float wt[ATT_WARPS], L = 0.f;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
+                for (int w = 0; w < ATT_WARPS; ++w) {
                     const float m = mw[w * NQ + j];
                     wt[w] = (m == -INFINITY) ? 0.f : exp2f(m - M);
                     L += wt[w] * lw[w * NQ + j];
                 }
+                const float inv = (P.n_splits == 1) ? (L > 0.f ? 1.f / L : 0.f) : 1.f;     // a single slice is final: normalise here
 #pragma unroll
-                for (int cc = 0; cc < HD / 8; cc += 4) {
+                for (int cc = 0; cc < CPT; cc += 4) {
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
+                    for (int w = 0; w < ATT_WARPS; ++w) {
                         if (wt[w] != 0.f) {                   // a warp without keys left nothing behind
                             const float4 o = *reinterpret_cast<const float4*>(Ow + ((size_t)w * NQ + j) * OLD + c0 + cc);
                             acc.x = fmaf(wt[w], o.x, acc.x); acc.y = fmaf(wt[w], o.y, acc.y);
                             acc.z = fmaf(wt[w], o.z, acc.z); acc.w = fmaf(wt[w], o.w, acc.w);
                         }
                     }
-                    __stcg(reinterpret_cast<float4*>(po + c0 + cc), acc);
+                    if (P.n_splits == 1) {
+                        dst[c0 + cc] = __float2bfloat16_rn(acc.x * inv); dst[c0 + cc + 1] = __float2bfloat16_rn(acc.y * inv);
+                        dst[c0 + cc + 2] = __float2bfloat16_rn(acc.z * inv); dst[c0 + cc + 3] = __float2bfloat16_rn(acc.w * inv);
+                    } else __stcg(reinterpret_cast<float4*>(po + c0 + cc), acc);
                 }
-                if ((t & 7) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+                if (P.n_splits > 1 && (t & 15) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
             }
         }
     }
+    if (P.n_splits == 1) return;                     // nothing to merge
 
     // ---- the slice that delivers last merges all of them: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
     //      always in slice order, so the result does not depend on which slice that was
@@ -350,7 +364,7 @@ bool attention_split_supported(int dtype, int H, int Hkv, int hd) {
 }
 
 size_t attention_split_workspace(int rows, int H, int hd, int max_ctx) {
-    const int n_splits = std::min(32, (max_ctx + CK - 1) / CK);
+    const int n_splits = std::min(32, (max_ctx + SLICE_KEYS - 1) / SLICE_KEYS);
     return ATTN_COUNTER_BYTES + sizeof(float) * (size_t)rows * H * n_splits * (hd + 2);
 }
 
@@ -372,16 +386,14 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
     P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ / (H / Hkv)));
     const int bps = (rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;
     const int n_blocks = (n_rows / rows_per_seq) * bps;
-    // enough slices to fill the SMs about three CTAs deep, at least one 64-key chunk each
-    int sm = 148;
-    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
-    P.n_splits = std::max(1, std::min(std::min(32, (ctx_bound + CK - 1) / CK), (3 * sm + Hkv * n_blocks - 1) / (Hkv * n_blocks)));
+    // one slice while the context is short (no cross-CTA merge at all), SLICE_KEYS positions per slice beyond
+    P.n_splits = std::max(1, std::min(32, (ctx_bound + SLICE_KEYS - 1) / SLICE_KEYS));
     const size_t need = ATTN_COUNTER_BYTES + sizeof(float) * (size_t)n_rows * H * P.n_splits * (hd + 2);
     if (need > workspace_bytes || (size_t)n_blocks * Hkv * sizeof(uint32_t) > ATTN_COUNTER_BYTES) return cudaErrorInvalidValue;
     P.counters = (uint32_t*)workspace;
     P.part_o = (float*)((char*)workspace + ATTN_COUNTER_BYTES);
     P.part_ml = P.part_o + (size_t)n_rows * H * P.n_splits * hd;
-    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)4 * NQ * (hd + 8) + 8 * NQ));
+    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)ATT_WARPS * NQ * (hd + 8) + 2 * ATT_WARPS * NQ));
     dim3 grid(P.n_splits, Hkv, n_blocks);
     cudaError_t e;
     if (hd == 128) {

@@ -35,6 +35,7 @@ constexpr int TILE_K = 64;                  // bf16 elements per k block = one 1
 constexpr int A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
+constexpr int GEMM_STEADY_BYTES = 112 * 1024;   // bytes per SM kept in flight once the ring has been filled
 constexpr int EPI_MB = 8;                    // token rows the fused step handles at a time
 constexpr int EPI_CB = 8;                    // pieces of a tile whose loads are in flight together
 
@@ -123,6 +124,17 @@ struct Shared {
     float val[EPI_MB][TILE_N];      // EPI_MB token rows of the tile, for exchanges between its rows
     float wsum[EPI_MB][4];          // per-warp sums of squares
 };
+
+// Ring bookkeeping.  The first `stages` loads of a CTA fill the whole ring (run-ahead while the
+// consumers wait for the previous kernel); after that only the first `steady` stages are reused,
+// which keeps fewer loads in flight: the same bandwidth with a shorter queue, so the last tile
+// arrives sooner after it is requested.  use = how often the stage was used before this load.
+struct RingPos { int stage; uint32_t use; };
+__device__ __forceinline__ RingPos ring_pos(uint32_t it, int stages, int steady) {
+    if (it < (uint32_t)stages) return RingPos{(int)it, 0u};
+    const uint32_t r = it - stages;
+    return RingPos{(int)(r % steady), 1u + r / steady};
+}
 
 // First and last CTA that hold a piece of `tile` (see GemmGeom).
 __device__ __forceinline__ void tile_contributors(const GemmGeom& g, uint32_t tile, uint32_t& i_first, uint32_t& i_last) {
@@ -349,8 +361,9 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             for (uint32_t it = 0; it < n_units; ++it) {
                 const uint32_t u = u0 + it;
-                const int s = it % g.stages;
-                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) break;
+                const RingPos rp = ring_pos(it, g.stages, g.steady);
+                const int s = rp.stage;
+                if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
                 const int tile = u / g.kb_per_tile, kb = u % g.kb_per_tile;
                 const uint32_t bar = smem_u32(&sh.full_w[s]);
                 mbar_expect_tx(bar, A_BYTES);
@@ -364,8 +377,9 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             pdl_wait();                                           // the token rows are the previous kernel's output
             for (uint32_t it = 0; it < n_units; ++it) {
-                const int s = it % g.stages;
-                if (it >= (uint32_t)g.stages && !mbar_wait(smem_u32(&sh.empty[s]), ((it / g.stages) & 1u) ^ 1u, abort_flag)) break;
+                const RingPos rp = ring_pos(it, g.stages, g.steady);
+                const int s = rp.stage;
+                if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
                 const int kb = (u0 + it) % g.kb_per_tile;
                 const uint32_t bar = smem_u32(&sh.full_x[s]);
                 mbar_expect_tx(bar, x_bytes);
@@ -386,8 +400,9 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)g.m_pad;
                 for (uint32_t j = 0; j < n_kb; ++j, ++it) {
-                    const int s = it % g.stages;
-                    const uint32_t ph = (it / g.stages) & 1u;
+                    const RingPos rp = ring_pos(it, g.stages, g.steady);
+                    const int s = rp.stage;
+                    const uint32_t ph = rp.use & 1u;
                     if (!mbar_wait(smem_u32(&sh.full_w[s]), ph, abort_flag) || !mbar_wait(smem_u32(&sh.full_x[s]), ph, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a = tiles0 + s * stage_bytes;
@@ -517,6 +532,7 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     if ((T + 1) * (g.grid + 1) >= (1ll << 32)) g.grid = 0;   // the kernels split the work in 32-bit arithmetic
     const int stage_bytes = A_BYTES + g.m_pad * 128;
     g.stages = std::max(2, std::min(MAX_STAGES, (198 * 1024) / stage_bytes));
+    g.steady = std::min(g.stages, std::max(2, (GEMM_STEADY_BYTES + stage_bytes - 1) / stage_bytes));
     return g;
 }
 
@@ -535,7 +551,7 @@ cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, cons
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    if (g.grid < 1 || g.stages < 2 || g.n_tiles > GEMM_MAX_TILES || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
+    if (g.grid < 1 || g.stages < 2 || g.steady < 1 || g.steady > g.stages || g.n_tiles > GEMM_MAX_TILES || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
     if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;

@@ -16,6 +16,7 @@ struct GemmGeom {
     int m_tok, m_pad, n_out, K;
     int n_tiles, kb_per_tile;
     int grid, max_seg, stages;
+    int steady;             // stages reused once the ring has been filled (<= stages)
 };
 
 // RMSNorm folded around a GEMM: the GEMM's input rows are h * gain (no 1/rms factor), the
