@@ -146,6 +146,14 @@ def test_small_bf16_gqa_teacher_forced(sd, T):
     ctx.close()
 
 
+def test_long_prompt_crosses_the_slice_boundary(sd):
+    # prompt of 1100 tokens: prefill in 256-row passes, verify rows against a cache cut into two slices
+    ctx, om = _build(sd, SMALL_BF16, [SMALL_BF16_DRAFT], "bf16", 1.0, 11, max_ctx=1280)
+    prompt = synth.make_prompt(4096, 1100, seed=12)
+    _replay(sd, ctx, om, 0, prompt, 5, 1.0, 11, 12, "bf16", min_agree=0.5)
+    ctx.close()
+
+
 def test_wide_bf16_head_dim_128_teacher_forced(sd):
     ctx, om = _build(sd, WIDE_BF16, [SMALL_BF16_DRAFT | dict(vocab=8192)], "bf16", 1.0, 7, max_ctx=96)
     prompt = synth.make_prompt(8192, 33, seed=8)

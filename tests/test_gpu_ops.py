@@ -57,6 +57,10 @@ ATTN_CASES = [  # H, Hkv, hd, max_ctx, positions of the rows
     (4, 2, 64, 300, [5, 128, 129, 255, 299]),
     (8, 2, 128, 700, [0, 63, 64, 65, 511, 699]),
     (2, 1, 16, 33, [32, 31, 0]),
+    # long caches: several slices per head merged by the last CTA (odd and even slice counts), rows inside one slice
+    (4, 2, 128, 2600, [0, 1023, 1024, 1025, 2047, 2599]),
+    (4, 4, 64, 4100, [4099, 3000, 17, 1024]),
+    (2, 2, 128, 8192, [8191, 4096, 100]),
 ]
 
 
