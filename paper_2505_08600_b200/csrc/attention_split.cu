@@ -7,6 +7,8 @@
 // outputs with their running max and sum; the CTA whose slice arrives last (an arrival
 // counter, nothing spins) merges them.
 // Cache layout of one layer: [slot][kv_head][position][head_dim].
+#include <cooperative_groups.h>
+
 #include "gemm_tc.h"
 #include "kernels.h"
 
@@ -29,6 +31,7 @@ struct AttnParams {
     uint32_t* counters; // [query block][kv head]: slices that have delivered; zero between launches
     bf16* out;          // [rows][H][hd]
     int n_rows, rows_per_seq, rows_per_block, H, Hkv, max_ctx, n_splits;
+    int csize;          // CTAs of a thread-block cluster that share one slice (1, 2 or 4)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
@@ -58,9 +61,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // of 64 keys, double-buffered in shared memory (16-byte asynchronous copies into an
 // XOR-swizzled layout that ldmatrix reads without bank conflicts); each warp owns 16 keys of a
 // chunk and keeps its own running max / sum / output (online softmax, exp2 domain), the warps
-// are merged at the end.  A context of up to SLICE_KEYS positions is one slice: the CTA then
-// writes the attention output itself; longer contexts are cut into slices whose partial results
-// are merged by whichever CTA arrives last.
+// are merged at the end.  When there are few (head, row block, slice) items, two or four CTAs of
+// a thread-block cluster share a slice and hand their results to the first one through
+// distributed shared memory.  A context of up to SLICE_KEYS positions is one slice, whose output
+// is written directly; longer contexts are cut into slices whose partial results are merged by
+// whichever slice arrives last.
 template <int HD>
 __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
@@ -71,7 +76,8 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     constexpr int BUF = CK * ROWB;           // one chunk of keys (or values)
     constexpr int OLD = HD + 8;              // padded row of the cross-warp merge buffer (floats)
     pdl_launch_dependents();
-    const int split = blockIdx.x, kvh = blockIdx.y;
+    const int CS = P.csize;
+    const int split = blockIdx.x / CS, crank = blockIdx.x % CS, kvh = blockIdx.y;
     const int group = P.H / P.Hkv;
     const int bps = (P.rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;     // query blocks per sequence
     const int r0 = (blockIdx.z / bps) * P.rows_per_seq + (blockIdx.z % bps) * P.rows_per_block;
@@ -90,8 +96,11 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     // the positions in use are cut evenly into the launched slices, whatever bound the grid was sized for
     const int len = mp + 1;
     const int slice = (((len + P.n_splits - 1) / P.n_splits) + 15) & ~15;
-    const int p_begin = split * slice;
-    const int np = min(p_begin + slice, len) - p_begin;          // positions of this slice (<= 0: nothing to do)
+    const int s_begin = split * slice;
+    const int s_np = max(0, min(s_begin + slice, len) - s_begin);    // positions of the slice, shared by the cluster's CTAs
+    const int sub = (((s_np + CS - 1) / CS) + 15) & ~15;
+    const int p_begin = s_begin + crank * sub;
+    const int np = min(p_begin + sub, s_begin + s_np) - p_begin;     // positions of this CTA (<= 0: nothing to do)
 
     // this thread's two query rows of the tile (gid and gid + 8)
     const int j_lo = gid, j_hi = gid + 8;
@@ -231,51 +240,95 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
         }
     }
     __syncthreads();
+    // this CTA's result: per query row the running max, the sum and the unnormalised output
+    constexpr int CPT = HD / 16;                                 // columns per thread: 16 threads span a query row
+    float* Oc = reinterpret_cast<float*>(sm_raw) + ATT_WARPS * NQ * OLD + 2 * ATT_WARPS * NQ;   // [16][HD]
+    float* Mc = Oc + NQ * HD;                                    // [16]
+    float* Lc = Mc + NQ;                                         // [16]
+    const int j = t >> 4, c0 = (t & 15) * CPT;
     {
-        constexpr int CPT = HD / 16;                             // columns per thread: 16 threads span a query row
-        const int j = t >> 4, c0 = (t & 15) * CPT;
-        if (j < nq) {
-            const int r = r0 + j / group, h = kvh * group + j % group;
-            float* po = P.part_o + (((size_t)r * P.H + h) * P.n_splits + split) * HD;
-            float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
-            bf16* dst = P.out + ((size_t)r * P.H + h) * HD;
-            if (np <= 0) {
-                if (P.n_splits == 1) {
+        float M = -INFINITY, L = 0.f;
+        float4 acc[CPT / 4];
 #pragma unroll
-                    for (int cc = 0; cc < CPT; ++cc) dst[c0 + cc] = __float2bfloat16_rn(0.f);
-                } else if ((t & 15) == 0) { __stcg(ml, -INFINITY); __stcg(ml + 1, 0.f); }
-            } else {
-                float M = -INFINITY;
+        for (int cc = 0; cc < CPT / 4; ++cc) acc[cc] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (np > 0) {
 #pragma unroll
-                for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, mw[w * NQ + j]);
-                float wt[ATT_WARPS], L = 0.f;
+            for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, mw[w * NQ + j]);
+            float wt[ATT_WARPS];
+#pragma unroll
+            for (int w = 0; w < ATT_WARPS; ++w) {
+                const float m = mw[w * NQ + j];
+                wt[w] = (m == -INFINITY) ? 0.f : exp2f(m - M);
+                L += wt[w] * lw[w * NQ + j];
+            }
+#pragma unroll
+            for (int cc = 0; cc < CPT / 4; ++cc)
 #pragma unroll
                 for (int w = 0; w < ATT_WARPS; ++w) {
-                    const float m = mw[w * NQ + j];
-                    wt[w] = (m == -INFINITY) ? 0.f : exp2f(m - M);
-                    L += wt[w] * lw[w * NQ + j];
-                }
-                const float inv = (P.n_splits == 1) ? (L > 0.f ? 1.f / L : 0.f) : 1.f;     // a single slice is final: normalise here
-#pragma unroll
-                for (int cc = 0; cc < CPT; cc += 4) {
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                    for (int w = 0; w < ATT_WARPS; ++w) {
-                        if (wt[w] != 0.f) {                   // a warp without keys left nothing behind
-                            const float4 o = *reinterpret_cast<const float4*>(Ow + ((size_t)w * NQ + j) * OLD + c0 + cc);
-                            acc.x = fmaf(wt[w], o.x, acc.x); acc.y = fmaf(wt[w], o.y, acc.y);
-                            acc.z = fmaf(wt[w], o.z, acc.z); acc.w = fmaf(wt[w], o.w, acc.w);
-                        }
+                    if (wt[w] != 0.f) {                       // a warp without keys left nothing behind
+                        const float4 o = *reinterpret_cast<const float4*>(Ow + ((size_t)w * NQ + j) * OLD + c0 + 4 * cc);
+                        acc[cc].x = fmaf(wt[w], o.x, acc[cc].x); acc[cc].y = fmaf(wt[w], o.y, acc[cc].y);
+                        acc[cc].z = fmaf(wt[w], o.z, acc[cc].z); acc[cc].w = fmaf(wt[w], o.w, acc[cc].w);
                     }
-                    if (P.n_splits == 1) {
-                        dst[c0 + cc] = __float2bfloat16_rn(acc.x * inv); dst[c0 + cc + 1] = __float2bfloat16_rn(acc.y * inv);
-                        dst[c0 + cc + 2] = __float2bfloat16_rn(acc.z * inv); dst[c0 + cc + 3] = __float2bfloat16_rn(acc.w * inv);
-                    } else __stcg(reinterpret_cast<float4*>(po + c0 + cc), acc);
                 }
-                if (P.n_splits > 1 && (t & 15) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+        }
+#pragma unroll
+        for (int cc = 0; cc < CPT / 4; ++cc) *reinterpret_cast<float4*>(Oc + (size_t)j * HD + c0 + 4 * cc) = acc[cc];
+        if ((t & 15) == 0) { Mc[j] = M; Lc[j] = L; }
+    }
+    // the CTAs of the cluster hand their results to the first one through distributed shared memory
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    if (CS > 1) cluster.sync(); else __syncthreads();
+    if (crank == 0 && j < nq) {
+        float Mr[4], Lr[4];
+        float M = -INFINITY, L = 0.f;
+#pragma unroll
+        for (int rc = 0; rc < 4; ++rc) {
+            Mr[rc] = -INFINITY; Lr[rc] = 0.f;
+            if (rc < CS) {
+                const float* rm = CS > 1 ? cluster.map_shared_rank(Mc, rc) : Mc;
+                const float* rl = CS > 1 ? cluster.map_shared_rank(Lc, rc) : Lc;
+                Mr[rc] = rm[j]; Lr[rc] = rl[j];
+            }
+            M = fmaxf(M, Mr[rc]);
+        }
+        float4 acc[CPT / 4];
+#pragma unroll
+        for (int cc = 0; cc < CPT / 4; ++cc) acc[cc] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int rc = 0; rc < 4; ++rc) {
+            const float w = (rc < CS && Mr[rc] != -INFINITY) ? exp2f(Mr[rc] - M) : 0.f;
+            L += w * Lr[rc];
+            if (w != 0.f) {
+                const float* ro = CS > 1 ? cluster.map_shared_rank(Oc, rc) : Oc;
+#pragma unroll
+                for (int cc = 0; cc < CPT / 4; ++cc) {
+                    const float4 o = *reinterpret_cast<const float4*>(ro + (size_t)j * HD + c0 + 4 * cc);
+                    acc[cc].x = fmaf(w, o.x, acc[cc].x); acc[cc].y = fmaf(w, o.y, acc[cc].y);
+                    acc[cc].z = fmaf(w, o.z, acc[cc].z); acc[cc].w = fmaf(w, o.w, acc[cc].w);
+                }
             }
         }
+        const int r = r0 + j / group, h = kvh * group + j % group;
+        if (P.n_splits == 1) {                       // a single slice is final: normalise and write the output
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            bf16* dst = P.out + ((size_t)r * P.H + h) * HD + c0;
+#pragma unroll
+            for (int cc = 0; cc < CPT / 4; ++cc) {
+                dst[4 * cc] = __float2bfloat16_rn(acc[cc].x * inv); dst[4 * cc + 1] = __float2bfloat16_rn(acc[cc].y * inv);
+                dst[4 * cc + 2] = __float2bfloat16_rn(acc[cc].z * inv); dst[4 * cc + 3] = __float2bfloat16_rn(acc[cc].w * inv);
+            }
+        } else {
+            float* po = P.part_o + (((size_t)r * P.H + h) * P.n_splits + split) * HD + c0;
+            float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
+#pragma unroll
+            for (int cc = 0; cc < CPT / 4; ++cc) __stcg(reinterpret_cast<float4*>(po + 4 * cc), acc[cc]);
+            if ((t & 15) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+        }
     }
+    if (CS > 1) cluster.sync();                      // nobody leaves while its shared memory may still be read
+    if (crank != 0) return;
     if (P.n_splits == 1) return;                     // nothing to merge
 
     // ---- the slice that delivers last merges all of them: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
@@ -393,15 +446,27 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
     P.counters = (uint32_t*)workspace;
     P.part_o = (float*)((char*)workspace + ATTN_COUNTER_BYTES);
     P.part_ml = P.part_o + (size_t)n_rows * H * P.n_splits * hd;
-    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)ATT_WARPS * NQ * (hd + 8) + 2 * ATT_WARPS * NQ));
-    dim3 grid(P.n_splits, Hkv, n_blocks);
+    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)ATT_WARPS * NQ * (hd + 8) + 2 * ATT_WARPS * NQ + (size_t)NQ * hd + 2 * NQ));
+    // few (head, row block, slice) items: two or four CTAs of a cluster share each of them
+    int sm = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
+    const int items = P.n_splits * Hkv * n_blocks;
+    P.csize = items * 4 <= sm ? 4 : (items * 2 <= sm ? 2 : 1);
+    dim3 grid(P.n_splits * P.csize, Hkv, n_blocks);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(ATT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (P.csize > 1) { attr[na].id = cudaLaunchAttributeClusterDimension; attr[na].val.clusterDim.x = P.csize; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1; ++na; }
+    if (dependent) { attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na; }
+    cfg.attrs = attr; cfg.numAttrs = na;
     cudaError_t e;
     if (hd == 128) {
         if ((e = cudaFuncSetAttribute(k_attn_mma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        return launch_pdl(k_attn_mma<128>, grid, dim3(ATT_THREADS), smem, st, dependent, P);
+        return cudaLaunchKernelEx(&cfg, k_attn_mma<128>, P);
     }
     if ((e = cudaFuncSetAttribute(k_attn_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    return launch_pdl(k_attn_mma<64>, grid, dim3(ATT_THREADS), smem, st, dependent, P);
+    return cudaLaunchKernelEx(&cfg, k_attn_mma<64>, P);
 }
 
 }  // namespace sd
