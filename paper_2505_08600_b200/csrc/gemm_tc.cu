@@ -172,7 +172,10 @@ __device__ void epilogue_prologue(const GemmGeom& g, const Epilogue& ep, Shared&
 // The step after the GEMM, on one finished 128-row tile.  Runs on the four epilogue warps
 // (et = 0..127 is the row inside the tile) of the CTA whose piece arrived last; sums the pieces
 // in the fixed order of their CTAs, so the result does not depend on which CTA that was.
-// Token rows are taken EPI_MB at a time so that their loads are in flight together.
+// Token rows are taken MB at a time and pieces CB at a time so that MB x CB loads are in flight
+// together: (8, 8) for the verify rows, (2, 32) for one or two rows (draft steps), where a tile
+// of a small matrix is cut into many pieces.
+template <int MB, int CB>
 __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float* __restrict__ partials, uint32_t tile,
                               Shared& sh, int et) {
     uint32_t i_first, i_last;
@@ -180,50 +183,51 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
     const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
     const int n = (int)tile * TILE_N + et;
     const bool live = n < g.n_out;
+    const uint32_t j_first = tile - ((i_first * T) / G) / KB;      // which of its pieces the first CTA gave to this tile (c * T < 2^32)
     // v[i] = sum over the pieces of (token rows[i], feature n); rows[i] < 0: skipped.  The loads of
-    // up to EPI_CB pieces x EPI_MB rows are issued together; the additions keep the pieces' order.
-    auto reduce_rows = [&](const int (&rows)[EPI_MB], float (&v)[EPI_MB]) {
+    // up to CB pieces x MB rows are issued together; the additions keep the pieces' order.
+    auto reduce_rows = [&](const int (&rows)[MB], float (&v)[MB]) {
 #pragma unroll
-        for (int i = 0; i < EPI_MB; ++i) v[i] = 0.f;
+        for (int i = 0; i < MB; ++i) v[i] = 0.f;
         if (!live) return;
-        for (uint32_t c0 = i_first; c0 <= i_last; c0 += EPI_CB) {
-            float tmp[EPI_CB][EPI_MB];
+        for (uint32_t c0 = i_first; c0 <= i_last; c0 += CB) {
+            float tmp[CB][MB];
 #pragma unroll
-            for (int cc = 0; cc < EPI_CB; ++cc) {
+            for (int cc = 0; cc < CB; ++cc) {
                 const uint32_t c = c0 + cc;
                 const bool ok = c <= i_last;
-                const uint32_t j = ok ? tile - ((c * T) / G) / KB : 0u;      // c * T < 2^32 (checked on the host)
+                const uint32_t j = c == i_first ? j_first : 0u;              // later CTAs start inside the tile: their first piece
                 const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
 #pragma unroll
-                for (int i = 0; i < EPI_MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+                for (int i = 0; i < MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
             }
 #pragma unroll
-            for (int cc = 0; cc < EPI_CB; ++cc)
+            for (int cc = 0; cc < CB; ++cc)
 #pragma unroll
-                for (int i = 0; i < EPI_MB; ++i) v[i] += tmp[cc][i];
+                for (int i = 0; i < MB; ++i) v[i] += tmp[cc][i];
         }
     };
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
     const float gain = (ep.mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;
-    for (int m0 = 0; m0 < n_rows; m0 += EPI_MB) {
-        int rows[EPI_MB];
-        float v[EPI_MB];
+    for (int m0 = 0; m0 < n_rows; m0 += MB) {
+        int rows[MB];
+        float v[MB];
 #pragma unroll
-        for (int i = 0; i < EPI_MB; ++i) {
+        for (int i = 0; i < MB; ++i) {
             const int r = m0 + i;
             rows[i] = r < n_rows ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
         }
         // loads that do not depend on the sum go out first, so that everything is in flight together
-        float hv[EPI_MB], cs[EPI_MB], sn[EPI_MB];
-        int pos[EPI_MB];
+        float hv[MB], cs[MB], sn[MB];
+        int pos[MB];
         if (ep.mode == EPI_RESIDUAL) {
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
+            for (int i = 0; i < MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
         } else if (ep.mode == EPI_QKV_ROPE) {
             const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
             const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) {
+            for (int i = 0; i < MB; ++i) {
                 pos[i] = (lower && rows[i] >= 0) ? sh.pos[rows[i]] : -1;
                 cs[i] = 1.f; sn[i] = 0.f;
                 if (pos[i] >= 0 && rot) { cs[i] = ep.rcos[(size_t)pos[i] * half + e]; sn[i] = ep.rsin[(size_t)pos[i] * half + e]; }
@@ -232,13 +236,13 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
         reduce_rows(rows, v);
         if (ep.rs.ssq) {
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) if (rows[i] >= 0) v[i] *= sh.scale[rows[i]];
+            for (int i = 0; i < MB; ++i) if (rows[i] >= 0) v[i] *= sh.scale[rows[i]];
         }
         switch (ep.mode) {
         case EPI_PLAIN: {
             if (live) {
 #pragma unroll
-                for (int i = 0; i < EPI_MB; ++i) if (rows[i] >= 0) ep.y[(size_t)(m0 + i) * g.n_out + n] = v[i];
+                for (int i = 0; i < MB; ++i) if (rows[i] >= 0) ep.y[(size_t)(m0 + i) * g.n_out + n] = v[i];
             }
             break;
         }
@@ -246,10 +250,10 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
             const int hd = ep.hd, half = hd >> 1, head = n / hd, e = n % hd;
             const bool rot = head < ep.H + ep.Hkv;
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) sh.val[i][et] = v[i];
+            for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
             epi_bar();
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) {
+            for (int i = 0; i < MB; ++i) {
                 if (pos[i] < 0) continue;
                 const float a = v[i], b = sh.val[i][et + half];
                 const float ra = a * cs[i] - b * sn[i], rb = a * sn[i] + b * cs[i];
@@ -269,7 +273,7 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
         case EPI_RESIDUAL: {
             const int d = g.n_out;
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) {
+            for (int i = 0; i < MB; ++i) {
                 hv[i] += v[i];
                 if (live && rows[i] >= 0) {
                     ep.h[(size_t)rows[i] * d + n] = hv[i];
@@ -278,12 +282,12 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
             }
             if (ep.gain_next) {
 #pragma unroll
-                for (int i = 0; i < EPI_MB; ++i) {
+                for (int i = 0; i < MB; ++i) {
                     const float ss = warp_sum(hv[i] * hv[i]);
                     if ((et & 31) == 0) sh.wsum[i][et >> 5] = ss;
                 }
                 epi_bar();
-                if (et < EPI_MB && m0 + et < n_rows) {
+                if (et < MB && m0 + et < n_rows) {
                     const float* w = sh.wsum[et];
                     ep.ssq_out[(size_t)(m0 + et) * SSQ_STRIDE + tile] = (w[0] + w[1]) + (w[2] + w[3]);
                 }
@@ -294,11 +298,11 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
         case EPI_SWIGLU: {
             const int f = (int)tile * 64 + et;
 #pragma unroll
-            for (int i = 0; i < EPI_MB; ++i) sh.val[i][et] = v[i];
+            for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
             epi_bar();
             if (et < 64 && f < ep.F) {
 #pragma unroll
-                for (int i = 0; i < EPI_MB; ++i) {
+                for (int i = 0; i < MB; ++i) {
                     if (rows[i] < 0) continue;
                     const float gt = v[i], up = sh.val[i][et + 64];
                     ep.act[(size_t)rows[i] * ep.F + f] = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
@@ -463,7 +467,10 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
                 epi_bar();
                 last = sh.last_flag != 0;
             }
-            if (last) tile_epilogue(g, ep, partials, tile, sh, et);
+            if (last) {
+                if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, sh, et);
+                else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, sh, et);
+            }
             epi_bar();
             u += n_kb;
         }
