@@ -177,9 +177,7 @@ __device__ void epilogue_prologue(const GemmGeom& g, const Epilogue& ep, Shared&
 // of a small matrix is cut into many pieces.
 template <int MB, int CB>
 __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float* __restrict__ partials, uint32_t tile,
-                              Shared& sh, int et) {
-    uint32_t i_first, i_last;
-    tile_contributors(g, tile, i_first, i_last);
+                              uint32_t i_first, uint32_t i_last, Shared& sh, int et) {
     const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
     const int n = (int)tile * TILE_N + et;
     const bool live = n < g.n_out;
@@ -468,8 +466,8 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
                 last = sh.last_flag != 0;
             }
             if (last) {
-                if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, sh, et);
-                else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, sh, et);
+                if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, i_first, i_last, sh, et);
+                else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, i_first, i_last, sh, et);
             }
             epi_bar();
             u += n_kb;
