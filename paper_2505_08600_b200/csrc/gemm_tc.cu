@@ -314,6 +314,65 @@ __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float
     }
 }
 
+// The four epilogue warps of a CTA: drain each finished accumulator from TMEM into the workspace,
+// count the arrival at its tile and, when this piece was the last, run the fused step on the tile.
+__device__ void epilogue_warps(const GemmGeom& g, const Epilogue& ep, float* __restrict__ partials, uint32_t* __restrict__ counters,
+                               Shared& sh, uint32_t tmem_base, int warp, int lane, uint32_t u0, uint32_t u1) {
+    volatile int* abort_flag = &sh.abort_flag;
+            pdl_wait();                                                        // the workspace may still be read by the previous kernel
+            const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
+            const int et = quarter * 32 + lane;                                // weight row inside the tile
+            epilogue_prologue(g, ep, sh, et);
+            uint32_t seg = 0;
+            for (uint32_t u = u0; u < u1; ++seg) {
+                const uint32_t kb0 = u % g.kb_per_tile;
+                const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
+                const uint32_t buf = seg & 1u;
+                if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) sh.epi_abort = 1;
+                epi_bar();
+                if (sh.epi_abort) break;                                       // all four warps leave together
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
+                for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    #pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < g.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+                // who completes the tile runs the step that follows the GEMM on it
+                const uint32_t tile = u / g.kb_per_tile;
+                uint32_t i_first, i_last;
+                tile_contributors(g, tile, i_first, i_last);
+                bool last = true;
+                if (i_last > i_first) {
+                    // The barrier orders the four warps' writes before thread 0's release; the acquire
+                    // side of the same operation, followed by the second barrier, orders every other
+                    // CTA's pieces before the reads below (release/acquire are cumulative).
+                    epi_bar();
+                    if (et == 0) {
+                        uint32_t old;
+                        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile) : "memory");
+                        const int l = old == i_last - i_first;
+                        if (l) counters[tile] = 0u;                            // left at zero for the next launch
+                        sh.last_flag = l;
+                    }
+                    epi_bar();
+                    last = sh.last_flag != 0;
+                }
+                if (last) {
+                    if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, i_first, i_last, sh, et);
+                    else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, i_first, i_last, sh, et);
+                }
+                epi_bar();
+                u += n_kb;
+            }
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
              GemmGeom g, Epilogue ep, float* __restrict__ partials, uint32_t* __restrict__ counters, uint32_t* status) {
@@ -420,58 +479,7 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------------ epilogue: TMEM -> partials -> fused step
-        pdl_wait();                                                        // the workspace may still be read by the previous kernel
-        const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
-        const int et = quarter * 32 + lane;                                // weight row inside the tile
-        epilogue_prologue(g, ep, sh, et);
-        uint32_t seg = 0;
-        for (uint32_t u = u0; u < u1; ++seg) {
-            const uint32_t kb0 = u % g.kb_per_tile;
-            const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
-            const uint32_t buf = seg & 1u;
-            if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) sh.epi_abort = 1;
-            epi_bar();
-            if (sh.epi_abort) break;                                       // all four warps leave together
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
-            for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (c0 + j < g.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
-            // who completes the tile runs the step that follows the GEMM on it
-            const uint32_t tile = u / g.kb_per_tile;
-            uint32_t i_first, i_last;
-            tile_contributors(g, tile, i_first, i_last);
-            bool last = true;
-            if (i_last > i_first) {
-                // The barrier orders the four warps' writes before thread 0's release; the acquire
-                // side of the same operation, followed by the second barrier, orders every other
-                // CTA's pieces before the reads below (release/acquire are cumulative).
-                epi_bar();
-                if (et == 0) {
-                    uint32_t old;
-                    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile) : "memory");
-                    const int l = old == i_last - i_first;
-                    if (l) counters[tile] = 0u;                            // left at zero for the next launch
-                    sh.last_flag = l;
-                }
-                epi_bar();
-                last = sh.last_flag != 0;
-            }
-            if (last) {
-                if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, i_first, i_last, sh, et);
-                else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, i_first, i_last, sh, et);
-            }
-            epi_bar();
-            u += n_kb;
-        }
+        epilogue_warps(g, ep, partials, counters, sh, tmem_base, warp, lane, u0, u1);
     }
 
     // ---------------------------------------------------------------------- wind-down
