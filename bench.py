@@ -346,6 +346,49 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_accept_microbench(args):
+    """Accept / reject / resample kernel alone at the 13B configuration's shape (8 sequences, gamma 8, vocab 32000):
+    draft distributions are softmax(target_logits + N(0, sigma^2)) so that sigma sets the acceptance rate."""
+    import torch
+    from paper_2505_08600_b200 import binding as sd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    wl, t = synth.CONFIGS["13b"]["workload"], synth.CONFIGS["13b"]["target"]
+    B, gamma, V, T = wl["batch"], wl["gamma"], t["vocab"], wl["temperature"]
+    g = torch.Generator(device=dev); g.manual_seed(5)
+    logits = torch.randn((B, gamma + 1, V), generator=g, device=dev) * (0.02 * t["d_model"] ** 0.5)   # spread of random-init logits
+    p = torch.softmax(logits.double() / T, dim=-1)
+    n_acc = torch.zeros((B,), dtype=torch.int32, device=dev); out_tok = torch.zeros((B, gamma + 1), dtype=torch.int32, device=dev)
+    seq_id = torch.arange(B, dtype=torch.int32, device=dev)
+    out = []
+    for sigma in (0.5, 1.0, 2.0):
+        q = torch.softmax((logits[:, :gamma] + sigma * torch.randn((B, gamma, V), generator=g, device=dev)).double() / T, dim=-1).float().contiguous()
+        alpha_hat = float(torch.minimum(p[:, :gamma].float(), q).sum(-1).mean())
+        x = torch.multinomial(q.reshape(-1, V), 1, generator=g).reshape(B, gamma).to(torch.int32)
+        hist = [0] * (gamma + 1)
+        its = 200
+        it = torch.zeros((B,), dtype=torch.int32, device=dev)
+        for i in range(3):
+            sd.sd_accept(logits, q, x, T, 5, it, seq_id, n_acc, out_tok, target_is_logits=1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(torch.cuda.current_stream())
+        for i in range(its):
+            sd.sd_accept(logits, q, x, T, 5, it, seq_id, n_acc, out_tok, target_is_logits=1)
+        e1.record(torch.cuda.current_stream()); torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / its * 1e3
+        for i in range(64):                                   # acceptance statistics over fresh uniforms (the iteration is a Philox counter word)
+            it.fill_(i)
+            sd.sd_accept(logits, q, x, T, 5, it, seq_id, n_acc, out_tok, target_is_logits=1)
+            for n in n_acc.cpu().tolist():
+                hist[n] += 1
+        tot = sum(hist)
+        out.append({"sigma": sigma, "alpha_hat": alpha_hat, "kernel_us": us, "mean_accepted": sum(i * h for i, h in enumerate(hist)) / tot,
+                    "n_acc_hist": [h / tot for h in hist]})
+    print(json.dumps({"metric": "accept_kernel_us", "unit": "us per call", "config": {"workload": f"accept microbench: {B} sequences, gamma {gamma}, vocab {V}, T {T}"},
+                      "bytes_touched_upper": B * (2 * gamma + 1) * V * 4, "results": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -356,9 +399,12 @@ def main():
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.accept_microbench:
+        run_accept_microbench(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -68,7 +68,12 @@ __device__ __forceinline__ int block_icdf(F w, int V, uint32_t u_int, BlockScrat
     const int chunk = (V + blockDim.x - 1) / blockDim.x;
     const int k0 = min(V, t * chunk), k1 = min(V, k0 + chunk);
     unsigned long long local = 0;
-    for (int k = k0; k < k1; ++k) local += __float2ull_rz(w(k) * 4294967296.0f);
+    {   // every thread starts its chunk at a different offset, so that a vocabulary row staged in shared
+        // memory is read without bank conflicts (the order inside a sum of integers does not matter)
+        const int n = k1 - k0;
+        int i = n > 0 ? t % n : 0;
+        for (int c = 0; c < n; ++c) { local += __float2ull_rz(w(k0 + i) * 4294967296.0f); i = (i + 1 == n) ? 0 : i + 1; }
+    }
     unsigned long long incl = local;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -106,11 +111,37 @@ __device__ __forceinline__ int block_icdf(F w, int V, uint32_t u_int, BlockScrat
     return sh.tok;
 }
 
+// Copies one vocabulary row into shared memory with every load in flight at once (the later
+// passes over the row - max, sum, probabilities, CDF - then cost no memory round trips).
+__device__ __forceinline__ void stage_row(const float* __restrict__ src, float* __restrict__ dst, int V) {
+    if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+        const float4* s4 = reinterpret_cast<const float4*>(src);
+        float4* d4 = reinterpret_cast<float4*>(dst);
+        const int n4 = V >> 2;
+        for (int k0 = 0; k0 < n4; k0 += 8 * blockDim.x) {
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { const int k = k0 + i * blockDim.x + threadIdx.x; if (k < n4) v[i] = __ldcg(s4 + k); }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { const int k = k0 + i * blockDim.x + threadIdx.x; if (k < n4) d4[k] = v[i]; }
+        }
+    } else {
+        for (int k = threadIdx.x; k < V; k += blockDim.x) dst[k] = __ldcg(src + k);
+    }
+    __syncthreads();
+}
+constexpr int STAGE_MAX_BYTES = 200 * 1024;      // a row of up to 51200 fp32 values fits beside the static shared memory
+
+// Dynamic shared memory for one staged row, or 0 when the vocabulary is too large to stage.
+static size_t row_stage_bytes(int V) { return (size_t)V * 4 <= (size_t)STAGE_MAX_BYTES ? (size_t)V * 4 : 0; }
+
 // ---------------------------------------------------------------- softmax + draw (draft steps)
 // One block per row.  probs = softmax(logits / T) (one-hot argmax when T == 0) is written out,
 // then one token is drawn from the written fp32 values.
-__device__ __forceinline__ int softmax_sample_row(const float* __restrict__ l, int V, float T, uint32_t u_int,
-                                                  float* __restrict__ probs, BlockScratch& sh) {
+__device__ __forceinline__ int softmax_sample_row(const float* __restrict__ l_global, int V, float T, uint32_t u_int,
+                                                  float* __restrict__ probs, BlockScratch& sh, float* rowbuf) {
+    const float* l = l_global;
+    if (rowbuf) { stage_row(l_global, rowbuf, V); l = rowbuf; }
     if (T == 0.f) {
         int a = block_argmax([&](int k) { return l[k]; }, V, sh, nullptr);
         for (int k = threadIdx.x; k < V; k += blockDim.x) probs[k] = (k == a) ? 1.f : 0.f;
@@ -122,41 +153,54 @@ __device__ __forceinline__ int softmax_sample_row(const float* __restrict__ l, i
     float s = 0.f;
     for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) / T);
     s = block_sum(s, sh.red);
-    for (int k = threadIdx.x; k < V; k += blockDim.x) probs[k] = expf((l[k] - m) / T) / s;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) {
+        const float pk = expf((l[k] - m) / T) / s;
+        probs[k] = pk;
+        if (rowbuf) rowbuf[k] = pk;                      // the draw below reads the same fp32 values
+    }
     __syncthreads();
-    int tok = block_icdf([&](int k) { return probs[k]; }, V, u_int, sh);
-    if (tok < 0) tok = block_argmax([&](int k) { return probs[k]; }, V, sh, nullptr);
+    const float* pr = rowbuf ? rowbuf : probs;
+    int tok = block_icdf([&](int k) { return pr[k]; }, V, u_int, sh);
+    if (tok < 0) tok = block_argmax([&](int k) { return pr[k]; }, V, sh, nullptr);
     return tok;
 }
 
 __global__ void __launch_bounds__(1024) k_softmax_sample_explicit(const float* __restrict__ logits, int V, float T,
                                                                   const uint32_t* __restrict__ u_int,
-                                                                  float* __restrict__ probs, int32_t* __restrict__ tok) {
+                                                                  float* __restrict__ probs, int32_t* __restrict__ tok, int staged) {
+    extern __shared__ __align__(16) float rowbuf[];
     __shared__ BlockScratch sh;
     const int r = blockIdx.x;
-    int k = softmax_sample_row(logits + (size_t)r * V, V, T, u_int[r], probs + (size_t)r * V, sh);
+    int k = softmax_sample_row(logits + (size_t)r * V, V, T, u_int[r], probs + (size_t)r * V, sh, staged ? rowbuf : nullptr);
     if (threadIdx.x == 0) tok[r] = k;
 }
 cudaError_t launch_softmax_sample_explicit(const float* logits, int rows, int V, float T, const uint32_t* u_int,
                                            float* probs, int32_t* tok, cudaStream_t st) {
     if (rows <= 0) return cudaSuccess;
-    k_softmax_sample_explicit<<<rows, 1024, 0, st>>>(logits, V, T, u_int, probs, tok);
+    const size_t smem = row_stage_bytes(V);
+    cudaError_t e = cudaFuncSetAttribute(k_softmax_sample_explicit, cudaFuncAttributeMaxDynamicSharedMemorySize, STAGE_MAX_BYTES);
+    if (e != cudaSuccess) return e;
+    k_softmax_sample_explicit<<<rows, 1024, smem, st>>>(logits, V, T, u_int, probs, tok, smem > 0);
     return cudaGetLastError();
 }
 
 __global__ void __launch_bounds__(1024) k_draft_sample(const float* __restrict__ logits, SeqState S, SeqList list, int V, float T,
                                                        uint64_t seed, int step, int gamma, float* __restrict__ q_out,
-                                                       int32_t* __restrict__ x_out) {
+                                                       int32_t* __restrict__ x_out, int staged) {
+    extern __shared__ __align__(16) float rowbuf[];
     __shared__ BlockScratch sh;
     const int i = blockIdx.x, slot = list.ids[i], b = list.out[i];
     const uint32_t u = uniform24(seed, S.iter[slot], (uint32_t)step, S.seq_id[slot], DRAW_DRAFT);
-    int k = softmax_sample_row(logits + (size_t)i * V, V, T, u, q_out + ((size_t)b * gamma + step) * V, sh);
+    int k = softmax_sample_row(logits + (size_t)i * V, V, T, u, q_out + ((size_t)b * gamma + step) * V, sh, staged ? rowbuf : nullptr);
     if (threadIdx.x == 0) x_out[(size_t)b * gamma + step] = k;
 }
 cudaError_t launch_draft_sample(const float* logits, const SeqState& S, const SeqList& list, int V, float T,
                                 uint64_t seed, int step, int gamma, float* q_out, int32_t* x_out, cudaStream_t st) {
     if (list.n <= 0) return cudaSuccess;
-    k_draft_sample<<<list.n, 1024, 0, st>>>(logits, S, list, V, T, seed, step, gamma, q_out, x_out);
+    const size_t smem = row_stage_bytes(V);
+    cudaError_t e = cudaFuncSetAttribute(k_draft_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, STAGE_MAX_BYTES);
+    if (e != cudaSuccess) return e;
+    k_draft_sample<<<list.n, 1024, smem, st>>>(logits, S, list, V, T, seed, step, gamma, q_out, x_out, smem > 0);
     return cudaGetLastError();
 }
 
@@ -169,9 +213,10 @@ cudaError_t launch_draft_sample(const float* logits, const SeqState& S, const Se
 // p_gamma itself, and writes the result.
 constexpr int ACC_ROWS_PER_CTA = 2;
 
-__global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize) {
+__global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int staged) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) float rowbuf[];            // one target row (when it fits): every pass over it reads shared memory
     __shared__ BlockScratch sh;
     __shared__ float row_max[ACC_ROWS_PER_CTA], row_sum[ACC_ROWS_PER_CTA];
     __shared__ int row_arg[ACC_ROWS_PER_CTA];
@@ -189,27 +234,32 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize) {
     const bool logits = P.target_is_logits != 0;
     pdl_wait();                                   // target rows, drafts and per-sequence state come from earlier kernels
 
+    int cur = -1;                                 // which of this CTA's rows the buffer holds
+    auto ensure = [&](int j, int li) {
+        if (staged && cur != li) { __syncthreads(); stage_row(tgt + (size_t)j * V, rowbuf, V); cur = li; }
+    };
+    auto val = [&](int j, int k) -> float { return staged ? rowbuf[k] : tgt[(size_t)j * V + k]; };
     auto prob = [&](int j, int li, int k) -> float {          // li: index of row j among this CTA's rows
-        const float v = tgt[(size_t)j * V + k];
+        if (logits && T == 0.f) return k == row_arg[li] ? 1.f : 0.f;
+        const float v = val(j, k);
         if (!logits) return v;
-        if (T == 0.f) return k == row_arg[li] ? 1.f : 0.f;
         return expf((v - row_max[li]) / T) / row_sum[li];
     };
 
     for (int li = 0; li < ACC_ROWS_PER_CTA; ++li) {
         const int j = rank + li * csize;
         if (j > gamma) break;                                   // uniform in the CTA
+        ensure(j, li);
         if (logits) {
-            const float* l = tgt + (size_t)j * V;
             if (T == 0.f) {
-                int a = block_argmax([&](int k) { return l[k]; }, V, sh, nullptr);
+                int a = block_argmax([&](int k) { return val(j, k); }, V, sh, nullptr);
                 if (threadIdx.x == 0) row_arg[li] = a;
             } else {
                 float m = -INFINITY;
-                for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, l[k]);
+                for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, val(j, k));
                 m = block_max(m, sh.red);
                 float sum = 0.f;
-                for (int k = threadIdx.x; k < V; k += blockDim.x) sum += expf((l[k] - m) / T);
+                for (int k = threadIdx.x; k < V; k += blockDim.x) sum += expf((val(j, k) - m) / T);
                 sum = block_sum(sum, sh.red);
                 if (threadIdx.x == 0) { row_max[li] = m; row_sum[li] = sum; }
             }
@@ -242,15 +292,35 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize) {
     if (n % csize == rank) {                                    // this CTA holds the statistics of row n
         const int li = n / csize;
         const uint32_t ui = uniform24(P.seed, P.iter[idx], (uint32_t)n, P.seq_id[idx], DRAW_RESAMPLE);
+        const float* qn = q + (size_t)(n < gamma ? n : 0) * V;
         int y;
-        if (n < gamma) {
-            const float* qn = q + (size_t)n * V;
-            y = block_icdf([&](int k) { return fmaxf(__fsub_rn(prob(n, li, k), qn[k]), 0.f); }, V, ui, sh);
-            if (y < 0) y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+        if (staged) {
+            // the weights of the draw replace the row in shared memory (one coalesced pass over q), then the
+            // integer CDF runs on them; residual all zero -> the target distribution itself -> its argmax
+            ensure(n, li);
+            for (int k = threadIdx.x; k < V; k += blockDim.x) {
+                const float pk = prob(n, li, k);
+                rowbuf[k] = n < gamma ? fmaxf(__fsub_rn(pk, qn[k]), 0.f) : pk;
+            }
+            __syncthreads();
+            y = block_icdf([&](int k) { return rowbuf[k]; }, V, ui, sh);
+            if (y < 0 && n < gamma) {
+                cur = -1;
+                ensure(n, li);
+                for (int k = threadIdx.x; k < V; k += blockDim.x) rowbuf[k] = prob(n, li, k);
+                __syncthreads();
+                y = block_icdf([&](int k) { return rowbuf[k]; }, V, ui, sh);
+            }
+            if (y < 0) y = block_argmax([&](int k) { return rowbuf[k]; }, V, sh, nullptr);
         } else {
-            y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+            if (n < gamma) {
+                y = block_icdf([&](int k) { return fmaxf(__fsub_rn(prob(n, li, k), qn[k]), 0.f); }, V, ui, sh);
+                if (y < 0) y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+            } else {
+                y = block_icdf([&](int k) { return prob(n, li, k); }, V, ui, sh);
+            }
+            if (y < 0) y = block_argmax([&](int k) { return prob(n, li, k); }, V, sh, nullptr);
         }
-        if (y < 0) y = block_argmax([&](int k) { return prob(n, li, k); }, V, sh, nullptr);
         if (threadIdx.x == 0) P.n_acc[b] = n;
         for (int s = threadIdx.x; s <= gamma; s += blockDim.x)
             P.out_tok[(size_t)b * (gamma + 1) + s] = s < n ? x[s] : (s == n ? y : -1);
@@ -264,7 +334,10 @@ cudaError_t launch_accept(const AcceptParams& p, int dependent, cudaStream_t st)
     while (csize < p.gamma + 1 && csize < 8) csize <<= 1;      // portable cluster sizes only
     if (csize * ACC_ROWS_PER_CTA < p.gamma + 1) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.B * csize); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    const size_t smem = row_stage_bytes(p.V);
+    cudaError_t e = cudaFuncSetAttribute(k_accept, cudaFuncAttributeMaxDynamicSharedMemorySize, STAGE_MAX_BYTES);
+    if (e != cudaSuccess) return e;
+    cfg.gridDim = dim3(p.B * csize); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -272,7 +345,7 @@ cudaError_t launch_accept(const AcceptParams& p, int dependent, cudaStream_t st)
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, k_accept, p, csize);
+    return cudaLaunchKernelEx(&cfg, k_accept, p, csize, (int)(smem > 0));
 }
 
 }  // namespace sd
