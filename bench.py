@@ -23,7 +23,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2505_08600_b200 import synth  # noqa: E402
+from paper_2505_08600_b200 import replicas, synth  # noqa: E402
 
 GEMM_TRAFFIC_PER_WEIGHT_BYTE = 1.0103      # measured: (dram read + write) / weight bytes of k_gemm_fused
 METRIC = "verify_step_tokens_per_s"
@@ -164,9 +164,7 @@ def run_gpu(args):
     import torch.distributed as dist
     from paper_2505_08600_b200 import binding as sd
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local)
@@ -220,11 +218,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(v, world, dev)
 
     stream = torch.cuda.current_stream(dev)
     # ---- phase A: the headline, device-resident inputs
@@ -250,7 +244,7 @@ def run_gpu(args):
     clocks = sampler.stop()
     launches = ctx.sd_launch_count() - l0
     ms_step = ms_total / K
-    value = world * B * (gamma + 1) / (ms_step * 1e-3)
+    value = replicas.whole_job_tokens_per_s(world, B, gamma, ms_step)
     ctx.sd_seq_read(0)
 
     # ---- per-kernel split of the same step (events between launches; separate from the timed run)
@@ -295,7 +289,7 @@ def run_gpu(args):
     ev1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3)) / K
-    e2e = {"value": world * B * (gamma + 1) / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+    e2e = {"value": replicas.whole_job_tokens_per_s(world, B, gamma, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": int(xh.numel() * 4 + qh.numel() * 4), "d2h_bytes_per_step": int(nh.numel() * 4 + oh.numel() * 4)}
     ctx.sd_seq_read(0)
 
