@@ -36,8 +36,7 @@ constexpr int A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
 constexpr int GEMM_STEADY_BYTES = 112 * 1024;   // bytes per SM kept in flight once the ring has been filled
-constexpr int EPI_MB = 8;                    // token rows the fused step handles at a time
-constexpr int EPI_CB = 8;                    // pieces of a tile whose loads are in flight together
+constexpr int EPI_MB = 16;                   // most token rows the fused step handles at a time (sizes its exchange buffers)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -174,7 +173,7 @@ __device__ void epilogue_prologue(const GemmGeom& g, const Epilogue& ep, Shared&
 // in the fixed order of their CTAs, so the result does not depend on which CTA that was.
 // Token rows are taken MB at a time and pieces CB at a time so that MB x CB loads are in flight
 // together: (8, 8) for the verify rows, (2, 32) for one or two rows (draft steps), where a tile
-// of a small matrix is cut into many pieces.
+// of a small matrix is cut into many pieces, (16, 4) for many rows on few pieces.
 template <int MB, int CB>
 __device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float* __restrict__ partials, uint32_t tile,
                               uint32_t i_first, uint32_t i_last, Shared& sh, int et) {
@@ -366,7 +365,8 @@ __device__ void epilogue_warps(const GemmGeom& g, const Epilogue& ep, float* __r
                 }
                 if (last) {
                     if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, i_first, i_last, sh, et);
-                    else tile_epilogue<EPI_MB, EPI_CB>(g, ep, partials, tile, i_first, i_last, sh, et);
+                    else if (g.m_tok > 8 && i_last - i_first < 4) tile_epilogue<16, 4>(g, ep, partials, tile, i_first, i_last, sh, et);
+                    else tile_epilogue<8, 8>(g, ep, partials, tile, i_first, i_last, sh, et);
                 }
                 epi_bar();
                 u += n_kb;
