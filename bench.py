@@ -318,6 +318,7 @@ def run_gpu(args):
     extras = {"draft_step_ms": draft_ms, "target_decode_step_ms": decode_ms, "iteration_ms": iter_ms, "c": c,
               "verify_over_decode": ms_step / decode_ms,
               "eq1_speedup": {f"alpha={a}": eq1_speedup(a, gamma, c) for a in (0.6, 0.8)},
+              "best_gamma": {f"alpha={a}": dict(zip(("gamma", "speedup"), sd.sd_best_gamma(a, c, 15))) for a in (0.6, 0.8)},
               "routed_drafts": [int(r) for r in routed]}
     status = ctx.sd_device_status()
 

@@ -208,6 +208,19 @@ sd_status sd_verify_accept_host(sd_ctx* ctx, const int32_t* seqs_host, int n_seq
                                 const int32_t* x_host, const float* q_host,
                                 int32_t* n_acc_host, int32_t* out_tok_host);
 
+/* ------------------------------------------------------ choice of gamma (host) */
+
+/* Eq. 1: expected speedup over plain autoregressive decoding when the draft agrees with the
+ * target with probability alpha per token, gamma tokens are drafted per iteration and one draft
+ * pass costs c target passes: (1 - alpha^(gamma+1)) / ((1 - alpha) (gamma c + 1)).
+ * alpha in [0, 1], gamma >= 0, c >= 0; alpha = 1 gives (gamma + 1) / (gamma c + 1).  Pure host arithmetic. */
+double sd_eq1_speedup(double alpha, int gamma, double c);
+
+/* The gamma in [1, gamma_max] that maximises Eq. 1 for a measured alpha and c (the paper tunes gamma
+ * per task by sweeping it, Sec. 3.2); ties go to the smaller gamma.  Returns 0 when no gamma beats
+ * plain decoding (speedup <= 1) or on bad arguments.  speedup_out may be NULL. */
+int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
+
 /* -------------------------------------------------------------- observation */
 
 /* Repeated calls replay captured CUDA graphs by default (keyed by sequences, gamma, buffers

@@ -85,6 +85,8 @@ _PROTOS = {
     "sd_op_philox": (_i, [_vp, _i, C.c_uint32, C.c_uint32, _vp, _vp]),
     "sd_op_softmax_sample": (_i, [_vp, _i, _i, C.c_float, _vp, _vp, _vp, _vp]),
     "sd_status_str": (C.c_char_p, [_i]),
+    "sd_eq1_speedup": (C.c_double, [C.c_double, _i, C.c_double]),
+    "sd_best_gamma": (_i, [C.c_double, C.c_double, _i, C.POINTER(C.c_double)]),
 }
 
 
@@ -291,6 +293,17 @@ def sd_accept(target, q, x, temperature, seed, it, seq_id, n_acc, out_tok, targe
                    x.data_ptr() if x is not None else None, B, g1 - 1, V, float(temperature), int(seed),
                    it.data_ptr(), seq_id.data_ptr(), n_acc.data_ptr(), out_tok.data_ptr(), _stream_ptr(stream).value)
     _check(lib().sd_accept(C.byref(a)), "sd_accept")
+
+
+def sd_eq1_speedup(alpha, gamma, c):
+    return float(lib().sd_eq1_speedup(float(alpha), int(gamma), float(c)))
+
+
+def sd_best_gamma(alpha, c, gamma_max):
+    """(gamma, speedup) maximising Eq. 1; gamma 0 when speculative decoding does not pay."""
+    s = C.c_double()
+    g = lib().sd_best_gamma(float(alpha), float(c), int(gamma_max), C.byref(s))
+    return int(g), float(s.value)
 
 
 def sd_op_linear(x, w, y, dtype, impl=0, stream=None):

@@ -852,6 +852,24 @@ sd_status sd_verify_accept_host(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     return SD_OK;
 }
 
+double sd_eq1_speedup(double alpha, int gamma, double c) {
+    if (!(alpha >= 0.0) || alpha > 1.0 || gamma < 0 || !(c >= 0.0)) return 0.0;
+    const double tokens = alpha == 1.0 ? (double)(gamma + 1) : (1.0 - pow(alpha, gamma + 1)) / (1.0 - alpha);
+    return tokens / (gamma * c + 1.0);
+}
+
+int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out) {
+    int best = 0;
+    double best_s = 1.0;
+    if (alpha >= 0.0 && alpha <= 1.0 && c >= 0.0)
+        for (int g = 1; g <= gamma_max; ++g) {
+            const double s = sd_eq1_speedup(alpha, g, c);
+            if (s > best_s) { best_s = s; best = g; }
+        }
+    if (speedup_out) *speedup_out = best_s;
+    return best;
+}
+
 sd_status sd_use_graphs(sd_ctx* c, int on) {
     if (!c) return SD_ERR_INVALID_ARG;
     c->graphs_on = on != 0;

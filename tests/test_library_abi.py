@@ -49,3 +49,22 @@ def test_host_side_validation_needs_no_gpu(sdlib):
     h = C.c_void_p()
     assert L.sd_create(C.byref(cfg), descs, None, None, 0, C.byref(h)) == 1
     assert L.sd_status_str(3) == b"capacity exceeded"
+
+
+def test_eq1_and_gamma_choice_on_the_host(sdlib):
+    # Eq. 1 against its definition as an expected-token count, and the argmax against brute force
+    for alpha in (0.0, 0.3, 0.6, 0.8, 0.95, 1.0):
+        for c in (0.0, 0.02, 0.138, 0.5):
+            best, best_s = 0, 1.0
+            for g in range(0, 16):
+                tokens = sum(alpha ** i for i in range(g + 1))        # 1 + alpha + ... + alpha^gamma
+                want = tokens / (g * c + 1)
+                assert abs(sdlib.sd_eq1_speedup(alpha, g, c) - want) < 1e-12
+                if g >= 1 and want > best_s + 1e-15:
+                    best, best_s = g, want
+            got_g, got_s = sdlib.sd_best_gamma(alpha, c, 15)
+            assert got_g == best and abs(got_s - best_s) < 1e-12
+    assert sdlib.sd_best_gamma(0.1, 0.5, 15) == (0, 1.0)                  # a poor, expensive draft never pays
+    assert sdlib.sd_eq1_speedup(-0.1, 3, 0.1) == 0.0
+    # the paper's Table 1 relation: speedup = tau / (gamma c + 1) with tau = expected tokens per iteration
+    assert abs(sdlib.sd_eq1_speedup(0.8, 5, 0.0) - (1 - 0.8 ** 6) / 0.2) < 1e-12
