@@ -238,8 +238,8 @@ sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);
  * every launch.  sd_profile_read synchronises, adds the time between consecutive events to
  * the category of the launch that followed the first one, and clears the record.
  * Categories: 0 weight GEMMs, 1 attention, 2 norm/rotary/elementwise, 3 sampling and
- * accept, 4 state updates. */
-#define SD_PROF_NCAT 5
+ * accept, 4 state updates, 5 the fused steps that follow the tensor-core GEMMs. */
+#define SD_PROF_NCAT 6
 sd_status sd_profile(sd_ctx* ctx, int enable);
 sd_status sd_profile_read(sd_ctx* ctx, float* ms_by_cat, uint32_t* launches_by_cat);
 

@@ -261,10 +261,10 @@ class Context:
         _check(self.L.sd_profile(self.h, int(enable)), "sd_profile")
 
     def sd_profile_read(self):
-        ms = (C.c_float * 5)()
-        n = (C.c_uint32 * 5)()
+        ms = (C.c_float * 6)()
+        n = (C.c_uint32 * 6)()
         _check(self.L.sd_profile_read(self.h, ms, n), "sd_profile_read")
-        names = ("linear", "attention", "elementwise", "sampling", "state")
+        names = ("linear", "attention", "elementwise", "sampling", "state", "fused_step")
         return {k: dict(ms=float(ms[i]), launches=int(n[i])) for i, k in enumerate(names)}
 
     # ---- observation

@@ -67,7 +67,7 @@ struct sd_ctx {
     void* attn_ws; size_t attn_ws_bytes;
     float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
-    uint32_t* gemm_counters;                    // arrival counters of the GEMM's output tiles (zero between launches)
+    float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
     struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
@@ -198,7 +198,10 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     }
     c->partials = (float*)B.take(c->partials_bytes);
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
-    c->gemm_counters = (uint32_t*)B.take(GEMM_COUNTER_BYTES);
+    size_t half_max = 1;
+    for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
+    c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
+    c->rope_row_sin = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
     const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
@@ -230,7 +233,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     } while (0)
 
 // Categories of the optional per-kernel timing (sd_profile).
-enum { CAT_LINEAR = 0, CAT_ATTENTION = 1, CAT_ELEMENTWISE = 2, CAT_SAMPLING = 3, CAT_STATE = 4, CAT_NONE = 5 };
+enum { CAT_LINEAR = 0, CAT_ATTENTION = 1, CAT_ELEMENTWISE = 2, CAT_SAMPLING = 3, CAT_STATE = 4, CAT_FUSED_STEP = 5, CAT_NONE = 6 };
 
 // When profiling is on, an event is recorded in front of every launch and tagged with the
 // category of that launch; sd_profile_read adds up the gaps between consecutive events.
@@ -270,7 +273,7 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         nullptr, nullptr, nullptr, st));
+                                         nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -301,19 +304,20 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     return SD_OK;
 }
 
-// One weight GEMM with its fused epilogue.
+// One weight GEMM and the step that follows it.
 sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
     const GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
-    LAUNCH(CAT_LINEAR, launch_gemm_fused(tw, tx, g, ep, c->partials, c->gemm_counters, c->S.status, 1, c->st));
+    LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, c->S.status, 1, c->st));
+    LAUNCH(CAT_FUSED_STEP, launch_fused_step(g, ep, c->partials, 1, c->st));
     return SD_OK;
 }
 
-// The same pass on the tensor-core path (bf16 models): five kernels per layer (QKV GEMM,
-// attention, Wo GEMM, gate/up GEMM, down GEMM); each GEMM's finishing CTAs apply the step that
-// follows it, and every kernel is launched as a programmatic dependent of the one before.
+// The same pass on the tensor-core path (bf16 models): per layer the QKV GEMM, attention, the Wo,
+// gate/up and down GEMMs, each GEMM followed by a small kernel that sums its split accumulators
+// and applies the step after it; every kernel is a programmatic dependent of the one before.
 sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
@@ -321,7 +325,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         M.layers[0].norm1, c->xn, c->ssq, st));
+                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -330,7 +334,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         memset(&e, 0, sizeof(e));
         e.mode = EPI_QKV_ROPE; e.rs = l == 0 ? first : tiled;
         e.q_out = (bf16*)c->q; e.kc = (bf16*)kc; e.vc = (bf16*)vc; e.row_slot = c->row_slot; e.row_pos = c->row_pos;
-        e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = M.rope_cos; e.rsin = M.rope_sin;
+        e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = c->rope_row_cos; e.rsin = c->rope_row_sin;
         SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
                                                      hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st));
@@ -497,8 +501,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
             cudaStreamSynchronize(st) != cudaSuccess)
             return fail(SD_ERR_CUDA);
     }
-    if (cudaMemsetAsync(c->gemm_counters, 0, GEMM_COUNTER_BYTES, st) != cudaSuccess ||
-        cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess)
+    if (cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
     c->force_plain = false;
@@ -507,7 +510,6 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     for (Model& M : c->models) {
         const sd_model_desc& m = M.d;
         M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE && m.d_ffn % 64 == 0 &&
-               (m.vocab + 127) / 128 <= GEMM_MAX_TILES && (2 * m.d_ffn + 127) / 128 <= GEMM_MAX_TILES &&
                attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim);
         if (!M.tc) continue;
         const int dq = m.n_heads * m.head_dim;
@@ -915,7 +917,7 @@ sd_status sd_profile_read(sd_ctx* c, float* ms_by_cat, uint32_t* launches_by_cat
 // ------------------------------------------------------------------ single operators
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl) {
     if (impl == 1 || dtype != SD_BF16 || !gemm_tc_supported(rows, n_out, n_in)) return 0;
-    return GEMM_COUNTER_BYTES + gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
+    return gemm_partials_bytes(gemm_geometry(rows, n_out, n_in, sm_count()));
 }
 
 sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype, int impl,
@@ -926,15 +928,14 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
     if (impl == 2 && !tc_ok) return SD_ERR_UNSUPPORTED;
     if (impl == 2 || (impl == 0 && tc_ok)) {
         const GemmGeom g = gemm_geometry(rows, n_out, n_in, sm_count());
-        if (!workspace || workspace_bytes < GEMM_COUNTER_BYTES + gemm_partials_bytes(g)) return SD_ERR_OOM;
+        if (!workspace || workspace_bytes < gemm_partials_bytes(g)) return SD_ERR_OOM;
         TensorMap tw, tx;
         if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
         Epilogue e;
         memset(&e, 0, sizeof(e));
         e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
-        CUDA_TRY(cudaMemsetAsync(workspace, 0, GEMM_COUNTER_BYTES, (cudaStream_t)stream));          // the arrival counters
-        CUDA_TRY(launch_gemm_fused(tw, tx, g, e, (float*)((char*)workspace + GEMM_COUNTER_BYTES), (uint32_t*)workspace,
-                                   nullptr, 0, (cudaStream_t)stream));
+        CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, 0, (cudaStream_t)stream));
+        CUDA_TRY(launch_fused_step(g, e, (const float*)workspace, 1, (cudaStream_t)stream));
         return SD_OK;
     }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;

@@ -11,7 +11,9 @@ namespace sd {
 template <typename T>
 __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restrict__ embed, int d, int vocab,
                         float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos,
-                        const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq) {
+                        const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq,
+                        const float* __restrict__ rcos, const float* __restrict__ rsin, int half,
+                        float* __restrict__ row_cos, float* __restrict__ row_sin) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const int i = r / plan.rows_per_seq, j = r % plan.rows_per_seq;
@@ -35,6 +37,11 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
     if (pos >= S.max_ctx) { if (threadIdx.x == 0) atomicOr(S.status, SD_DEV_BAD_POS); pos = -1; }
     if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) atomicOr(S.status, SD_DEV_BAD_TOKEN); tok = 0; }
     if (threadIdx.x == 0) { row_slot[r] = slot; row_pos[r] = pos; }
+    if (row_cos)                         // the row's rotary factors, so that the step after the QKV GEMM needs no dependent lookup
+        for (int k = threadIdx.x; k < half; k += blockDim.x) {
+            row_cos[(size_t)r * half + k] = pos >= 0 ? rcos[(size_t)pos * half + k] : 1.f;
+            row_sin[(size_t)r * half + k] = pos >= 0 ? rsin[(size_t)pos * half + k] : 0.f;
+        }
     const T* e = embed + (size_t)tok * d;
     float ss = 0.f;
     for (int k = threadIdx.x; k < d; k += blockDim.x) {
@@ -51,9 +58,13 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
 cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& plan, int n_rows,
                          const void* embed, int dtype, int d, int vocab,
                          float* h, int32_t* row_slot, int32_t* row_pos, const float* gain, void* xn, float* ssq,
-                         cudaStream_t st) {
-    if (dtype == SD_BF16) k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq);
-    else k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr);
+                         const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, cudaStream_t st) {
+    if (dtype == SD_BF16)
+        k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq,
+                                              rope_cos, rope_sin, half, row_cos, row_sin);
+    else
+        k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr,
+                                               nullptr, nullptr, 0, nullptr, nullptr);
     return cudaGetLastError();
 }
 

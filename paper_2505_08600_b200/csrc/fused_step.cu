@@ -1,0 +1,211 @@
+// The step that follows each weight GEMM of a decoder layer, fused with the reduction of the
+// GEMM's split accumulators: one small CTA per (128-row output tile, batch of token rows) adds
+// the pieces of the tile in the fixed order of the CTAs that produced them (run-to-run identical
+// results) and applies, in the same pass,
+//   QKV      -> 1/rms factor -> rotary embedding -> query buffer / KV-cache append (bf16),
+//   Wo, down -> residual add -> next norm's operand h * gain in bf16 + the tile's share of sum h^2,
+//   gate/up  -> 1/rms factor -> SwiGLU (gate and up rows of a feature sit in one tile),
+//   lm_head  -> 1/rms factor -> fp32 logits,
+// so that no fp32 intermediate matrix goes through memory.  It runs as a programmatic dependent
+// of the GEMM: its CTAs are resident (and hold only a few KB) while the GEMM streams, the GEMM's
+// CTAs leave their SMs as soon as their pieces are written, and the next GEMM's CTAs take those
+// SMs and start streaming weights while this kernel is still working.  Everything a CTA needs
+// is requested in one round of loads.
+#include "gemm_tc.h"
+
+namespace sd {
+
+namespace {
+
+constexpr int TILE_N = 128;
+
+template <int MB>
+struct StepShared {
+    float scale[MB];                // 1/rms factor of the CTA's token rows
+    float val[MB][TILE_N];          // exchange between the rows of the tile (rotary pairs, gate/up pairs)
+    float wsum[MB][4];              // per-warp sums of squares
+};
+
+// MB token rows x CB pieces are in flight together: (8, 8) for the verify rows, (2, 32) for one or
+// two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) for
+// many rows on few pieces.
+template <int MB, int CB>
+__global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials) {
+    __shared__ StepShared<MB> sh;
+    pdl_launch_dependents();
+    const int et = threadIdx.x, lane = et & 31, warp = et >> 5;
+    const uint32_t tile = blockIdx.x;
+    const int m0 = blockIdx.y * MB;
+    const int n = (int)tile * TILE_N + et;
+    const bool live = n < g.n_out;
+    // first and last CTA of the GEMM that hold a piece of this tile, and which of its pieces the first one gave
+    const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = (uint32_t)g.grid;
+    const uint32_t ua = tile * KB, ub = ua + KB - 1;
+    const uint32_t i_first = ((ua + 1) * G + T - 1) / T - 1;      // T * G < 2^32 (checked on the host)
+    const uint32_t i_last = ((ub + 1) * G + T - 1) / T - 1;
+    const uint32_t j_first = tile - ((i_first * T) / G) / KB;
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    int rows[MB];
+#pragma unroll
+    for (int i = 0; i < MB; ++i) {
+        const int r = m0 + i;
+        rows[i] = r < n_rows ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
+    }
+    const float gain = (ep.mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;   // a weight: needs no wait
+    pdl_wait();                                   // the pieces (and the rows' sums of squares) come from the kernels before
+
+    // ---- one round of loads: sums of squares, residual / row plan / rotary factors, the pieces
+    float ssa[(MB + 3) / 4], ssb[(MB + 3) / 4];
+    if (ep.rs.ssq) {                              // one warp per token row, one lane per piece of its sum of squares
+#pragma unroll
+        for (int ii = 0; ii < (MB + 3) / 4; ++ii) {
+            const int i = warp + 4 * ii, r = m0 + i;
+            const bool ok = i < MB && r < n_rows;
+            const float* ps = ep.rs.ssq + (size_t)(ok ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : 0) * SSQ_STRIDE;
+            ssa[ii] = (ok && lane < ep.rs.n_parts) ? __ldcg(ps + lane) : 0.f;
+            ssb[ii] = (ok && lane + 32 < ep.rs.n_parts) ? __ldcg(ps + lane + 32) : 0.f;
+        }
+    }
+    float hv[MB], cs[MB], sn[MB];
+    int pos[MB], slot[MB];
+    if (ep.mode == EPI_RESIDUAL) {
+#pragma unroll
+        for (int i = 0; i < MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
+    } else if (ep.mode == EPI_QKV_ROPE) {
+        const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
+        const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            const bool ok = lower && rows[i] >= 0;
+            pos[i] = ok ? __ldcg(ep.row_pos + rows[i]) : -1;
+            slot[i] = (ok && head >= ep.H) ? __ldcg(ep.row_slot + rows[i]) : 0;
+            cs[i] = (ok && rot) ? __ldcg(ep.rcos + (size_t)rows[i] * half + e) : 1.f;     // per-row rotary factors (the row's position applied)
+            sn[i] = (ok && rot) ? __ldcg(ep.rsin + (size_t)rows[i] * half + e) : 0.f;
+        }
+    }
+    float v[MB];
+#pragma unroll
+    for (int i = 0; i < MB; ++i) v[i] = 0.f;
+    if (live) {
+        for (uint32_t c0 = i_first; c0 <= i_last; c0 += CB) {
+            float tmp[CB][MB];
+#pragma unroll
+            for (int cc = 0; cc < CB; ++cc) {
+                const uint32_t c = c0 + cc;
+                const bool ok = c <= i_last;
+                const uint32_t j = c == i_first ? j_first : 0u;              // later CTAs start inside the tile: their first piece
+                const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
+#pragma unroll
+                for (int i = 0; i < MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+            }
+#pragma unroll
+            for (int cc = 0; cc < CB; ++cc)                                   // the pieces are added in the order of their CTAs
+#pragma unroll
+                for (int i = 0; i < MB; ++i) v[i] += tmp[cc][i];
+        }
+    }
+    if (ep.rs.ssq) {
+#pragma unroll
+        for (int ii = 0; ii < (MB + 3) / 4; ++ii) {
+            const int i = warp + 4 * ii;
+            const float ss = warp_sum(ssa[ii] + ssb[ii]);
+            if (lane == 0 && i < MB) sh.scale[i] = rsqrtf(ss * ep.rs.inv_d + ep.rs.eps);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < MB; ++i) v[i] *= sh.scale[i];
+    }
+
+    switch (ep.mode) {
+    case EPI_PLAIN: {
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < MB; ++i) if (rows[i] >= 0) ep.y[(size_t)(m0 + i) * g.n_out + n] = v[i];
+        }
+        break;
+    }
+    case EPI_QKV_ROPE: {
+        const int hd = ep.hd, half = hd >> 1, head = n / hd, e = n % hd;
+        const bool rot = head < ep.H + ep.Hkv;
+#pragma unroll
+        for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            if (pos[i] < 0) continue;
+            const float a = v[i], b = sh.val[i][et + half];
+            const float ra = a * cs[i] - b * sn[i], rb = a * sn[i] + b * cs[i];
+            bf16* dst;
+            if (head < ep.H) dst = ep.q_out + ((size_t)rows[i] * ep.H + head) * hd;
+            else {
+                const int kvh = (head - ep.H) % ep.Hkv;
+                bf16* base = rot ? ep.kc : ep.vc;
+                dst = base + (((size_t)slot[i] * ep.Hkv + kvh) * ep.max_ctx + pos[i]) * hd;
+            }
+            dst[e] = __float2bfloat16_rn(ra);
+            dst[e + half] = __float2bfloat16_rn(rb);
+        }
+        break;
+    }
+    case EPI_RESIDUAL: {
+        const int d = g.n_out;
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            hv[i] += v[i];
+            if (live && rows[i] >= 0) {
+                ep.h[(size_t)rows[i] * d + n] = hv[i];
+                if (ep.gain_next) ep.xn[(size_t)rows[i] * d + n] = __float2bfloat16_rn(hv[i] * gain);
+            }
+        }
+        if (ep.gain_next) {
+#pragma unroll
+            for (int i = 0; i < MB; ++i) {
+                const float ss = warp_sum(hv[i] * hv[i]);
+                if (lane == 0) sh.wsum[i][warp] = ss;
+            }
+            __syncthreads();
+            if (et < MB && m0 + et < n_rows) {
+                const float* w = sh.wsum[et];
+                ep.ssq_out[(size_t)(m0 + et) * SSQ_STRIDE + tile] = (w[0] + w[1]) + (w[2] + w[3]);
+            }
+        }
+        break;
+    }
+    case EPI_SWIGLU: {
+        const int f = (int)tile * 64 + et;
+#pragma unroll
+        for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
+        __syncthreads();
+        if (et < 64 && f < ep.F) {
+#pragma unroll
+            for (int i = 0; i < MB; ++i) {
+                if (rows[i] < 0) continue;
+                const float gt = v[i], up = sh.val[i][et + 64];
+                ep.act[(size_t)rows[i] * ep.F + f] = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
+            }
+        }
+        break;
+    }
+    default: break;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, int dependent, cudaStream_t st) {
+    if (g.grid < 1 || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
+    if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
+    if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
+    if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
+    if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    // pieces per tile, at most: a tile's k blocks over the k blocks a CTA owns
+    const long long T = (long long)g.n_tiles * g.kb_per_tile;
+    const int per_cta = (int)std::max<long long>(1, T / g.grid);
+    const int pieces = (g.kb_per_tile + per_cta - 1) / per_cta + 1;
+    if (n_rows <= 2) return launch_pdl(k_fused_step<2, 32>, dim3(g.n_tiles, (n_rows + 1) / 2), dim3(128), 0, st, dependent, g, ep, partials);
+    if (n_rows > 8 && pieces <= 4) return launch_pdl(k_fused_step<16, 4>, dim3(g.n_tiles, (n_rows + 15) / 16), dim3(128), 0, st, dependent, g, ep, partials);
+    return launch_pdl(k_fused_step<8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials);
+}
+
+}  // namespace sd

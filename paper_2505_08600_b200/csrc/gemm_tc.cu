@@ -11,16 +11,15 @@
 //     and split evenly over the grid, so that every SM streams the same number of bytes
 //     whatever the matrix shape; a CTA whose range crosses a tile boundary produces one
 //     partial accumulator ("segment") per tile it touches;
-//   - segments are written to a workspace as fp32 [slot][token][128]; each tile has an arrival
-//     counter, and the CTA whose segment arrives last adds the segments of the tile in the fixed
-//     order of their CTAs (results are run-to-run identical) and applies, in the same pass, the
-//     step that follows the GEMM in the decoder layer (rotary + KV append, residual + next norm,
-//     SwiGLU, or plain fp32 output); nothing spins: a CTA that is not last just moves on;
+//   - segments are written to a workspace as fp32 [slot][token][128] and the CTA is done: the
+//     kernel that follows (fused_step.cu) adds the segments of each tile in the fixed order of
+//     their CTAs and applies the step that follows the GEMM in the decoder layer, while the
+//     next GEMM's CTAs already occupy the SMs this one has left and stream their weights;
 //   - the kernel is written for programmatic dependent launch: it lets its successor start at
 //     once; its weight stream never waits for the predecessor (only the token rows and the
 //     workspace do), so the ring is full when the consumers are released.
-// Roles: warp 0 streams weights, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM and
-// run the fused step, warp 6 loads the token rows.  Every mbarrier wait is bounded; on expiry
+// Roles: warp 0 streams weights, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM
+// into the workspace, warp 6 loads the token rows.  Every mbarrier wait is bounded; on expiry
 // the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
 #include <cuda.h>
 
@@ -35,8 +34,8 @@ constexpr int TILE_K = 64;                  // bf16 elements per k block = one 1
 constexpr int A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
+constexpr int RING_BYTES = 198 * 1024;          // stage ring of a CTA; the rest of the SM's shared memory is left to the fused-step CTAs
 constexpr int GEMM_STEADY_BYTES = 112 * 1024;   // bytes per SM kept in flight once the ring has been filled
-constexpr int EPI_MB = 16;                   // most token rows the fused step handles at a time (sizes its exchange buffers)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -116,12 +115,7 @@ struct Shared {
     uint64_t full_w[MAX_STAGES], full_x[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
-    int epi_abort, last_flag;
-    float scale[SD_MAX_ROWS];       // 1/rms factor of each token row
-    int pos[SD_MAX_ROWS];           // cache position and sequence slot of each token row (rotary / KV append)
-    int slot[SD_MAX_ROWS];
-    float val[EPI_MB][TILE_N];      // EPI_MB token rows of the tile, for exchanges between its rows
-    float wsum[EPI_MB][4];          // per-warp sums of squares
+    int epi_abort;
 };
 
 // Ring bookkeeping.  The first `stages` loads of a CTA fill the whole ring (run-ahead while the
@@ -135,247 +129,41 @@ __device__ __forceinline__ RingPos ring_pos(uint32_t it, int stages, int steady)
     return RingPos{(int)(r % steady), 1u + r / steady};
 }
 
-// First and last CTA that hold a piece of `tile` (see GemmGeom).
-__device__ __forceinline__ void tile_contributors(const GemmGeom& g, uint32_t tile, uint32_t& i_first, uint32_t& i_last) {
-    const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
-    const uint32_t ua = tile * KB, ub = ua + KB - 1;
-    i_first = ((ua + 1) * G + T - 1) / T - 1;                    // T * G < 2^32 (checked on the host): 32-bit arithmetic
-    i_last = ((ub + 1) * G + T - 1) / T - 1;
-}
-
-// What the fused step needs per token row and does not depend on the tile: the 1/rms factors,
-// cache positions and slots.  Loaded once per CTA, while the main loop streams.
-__device__ void epilogue_prologue(const GemmGeom& g, const Epilogue& ep, Shared& sh, int et) {
-    if (ep.rs.ssq) {                       // one warp per token row, one lane per piece of its sum of squares
-        const int w = et >> 5, lane = et & 31;
-        for (int m = w; m < g.m_tok; m += 8) {
-            const int m2 = m + 4;
-            const float* pa = ep.rs.ssq + (size_t)m * SSQ_STRIDE;
-            const float* pb = ep.rs.ssq + (size_t)m2 * SSQ_STRIDE;
-            float a = lane < ep.rs.n_parts ? __ldcg(pa + lane) : 0.f;
-            float a2 = lane + 32 < ep.rs.n_parts ? __ldcg(pa + lane + 32) : 0.f;
-            float b = (m2 < g.m_tok && lane < ep.rs.n_parts) ? __ldcg(pb + lane) : 0.f;
-            float b2 = (m2 < g.m_tok && lane + 32 < ep.rs.n_parts) ? __ldcg(pb + lane + 32) : 0.f;
-            a = warp_sum(a + a2); b = warp_sum(b + b2);
-            if (lane == 0) {
-                sh.scale[m] = rsqrtf(a * ep.rs.inv_d + ep.rs.eps);
-                if (m2 < g.m_tok) sh.scale[m2] = rsqrtf(b * ep.rs.inv_d + ep.rs.eps);
-            }
-        }
-    }
-    if (ep.mode == EPI_QKV_ROPE)
-        for (int m = et; m < g.m_tok; m += 128) { sh.pos[m] = __ldcg(ep.row_pos + m); sh.slot[m] = __ldcg(ep.row_slot + m); }
-    epi_bar();
-}
-
-// The step after the GEMM, on one finished 128-row tile.  Runs on the four epilogue warps
-// (et = 0..127 is the row inside the tile) of the CTA whose piece arrived last; sums the pieces
-// in the fixed order of their CTAs, so the result does not depend on which CTA that was.
-// Token rows are taken MB at a time and pieces CB at a time so that MB x CB loads are in flight
-// together: (8, 8) for the verify rows, (2, 32) for one or two rows (draft steps), where a tile
-// of a small matrix is cut into many pieces, (16, 4) for many rows on few pieces.
-template <int MB, int CB>
-__device__ void tile_epilogue(const GemmGeom& g, const Epilogue& ep, const float* __restrict__ partials, uint32_t tile,
-                              uint32_t i_first, uint32_t i_last, Shared& sh, int et) {
-    const uint32_t KB = (uint32_t)g.kb_per_tile, T = (uint32_t)g.n_tiles * KB, G = gridDim.x;
-    const int n = (int)tile * TILE_N + et;
-    const bool live = n < g.n_out;
-    const uint32_t j_first = tile - ((i_first * T) / G) / KB;      // which of its pieces the first CTA gave to this tile (c * T < 2^32)
-    // v[i] = sum over the pieces of (token rows[i], feature n); rows[i] < 0: skipped.  The loads of
-    // up to CB pieces x MB rows are issued together; the additions keep the pieces' order.
-    auto reduce_rows = [&](const int (&rows)[MB], float (&v)[MB]) {
-#pragma unroll
-        for (int i = 0; i < MB; ++i) v[i] = 0.f;
-        if (!live) return;
-        for (uint32_t c0 = i_first; c0 <= i_last; c0 += CB) {
-            float tmp[CB][MB];
-#pragma unroll
-            for (int cc = 0; cc < CB; ++cc) {
-                const uint32_t c = c0 + cc;
-                const bool ok = c <= i_last;
-                const uint32_t j = c == i_first ? j_first : 0u;              // later CTAs start inside the tile: their first piece
-                const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
-#pragma unroll
-                for (int i = 0; i < MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
-            }
-#pragma unroll
-            for (int cc = 0; cc < CB; ++cc)
-#pragma unroll
-                for (int i = 0; i < MB; ++i) v[i] += tmp[cc][i];
-        }
-    };
-    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
-    const float gain = (ep.mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;
-    for (int m0 = 0; m0 < n_rows; m0 += MB) {
-        int rows[MB];
-        float v[MB];
-#pragma unroll
-        for (int i = 0; i < MB; ++i) {
-            const int r = m0 + i;
-            rows[i] = r < n_rows ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
-        }
-        // loads that do not depend on the sum go out first, so that everything is in flight together
-        float hv[MB], cs[MB], sn[MB];
-        int pos[MB];
-        if (ep.mode == EPI_RESIDUAL) {
-#pragma unroll
-            for (int i = 0; i < MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
-        } else if (ep.mode == EPI_QKV_ROPE) {
-            const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
-            const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
-#pragma unroll
-            for (int i = 0; i < MB; ++i) {
-                pos[i] = (lower && rows[i] >= 0) ? sh.pos[rows[i]] : -1;
-                cs[i] = 1.f; sn[i] = 0.f;
-                if (pos[i] >= 0 && rot) { cs[i] = ep.rcos[(size_t)pos[i] * half + e]; sn[i] = ep.rsin[(size_t)pos[i] * half + e]; }
-            }
-        }
-        reduce_rows(rows, v);
-        if (ep.rs.ssq) {
-#pragma unroll
-            for (int i = 0; i < MB; ++i) if (rows[i] >= 0) v[i] *= sh.scale[rows[i]];
-        }
-        switch (ep.mode) {
-        case EPI_PLAIN: {
-            if (live) {
-#pragma unroll
-                for (int i = 0; i < MB; ++i) if (rows[i] >= 0) ep.y[(size_t)(m0 + i) * g.n_out + n] = v[i];
-            }
-            break;
-        }
-        case EPI_QKV_ROPE: {
-            const int hd = ep.hd, half = hd >> 1, head = n / hd, e = n % hd;
-            const bool rot = head < ep.H + ep.Hkv;
-#pragma unroll
-            for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
-            epi_bar();
-#pragma unroll
-            for (int i = 0; i < MB; ++i) {
-                if (pos[i] < 0) continue;
-                const float a = v[i], b = sh.val[i][et + half];
-                const float ra = a * cs[i] - b * sn[i], rb = a * sn[i] + b * cs[i];
-                bf16* dst;
-                if (head < ep.H) dst = ep.q_out + ((size_t)rows[i] * ep.H + head) * hd;
-                else {
-                    const int kvh = (head - ep.H) % ep.Hkv;
-                    bf16* base = rot ? ep.kc : ep.vc;
-                    dst = base + (((size_t)sh.slot[rows[i]] * ep.Hkv + kvh) * ep.max_ctx + pos[i]) * hd;
-                }
-                dst[e] = __float2bfloat16_rn(ra);
-                dst[e + half] = __float2bfloat16_rn(rb);
-            }
-            epi_bar();
-            break;
-        }
-        case EPI_RESIDUAL: {
-            const int d = g.n_out;
-#pragma unroll
-            for (int i = 0; i < MB; ++i) {
-                hv[i] += v[i];
-                if (live && rows[i] >= 0) {
-                    ep.h[(size_t)rows[i] * d + n] = hv[i];
-                    if (ep.gain_next) ep.xn[(size_t)rows[i] * d + n] = __float2bfloat16_rn(hv[i] * gain);
-                }
-            }
-            if (ep.gain_next) {
-#pragma unroll
-                for (int i = 0; i < MB; ++i) {
-                    const float ss = warp_sum(hv[i] * hv[i]);
-                    if ((et & 31) == 0) sh.wsum[i][et >> 5] = ss;
-                }
-                epi_bar();
-                if (et < MB && m0 + et < n_rows) {
-                    const float* w = sh.wsum[et];
-                    ep.ssq_out[(size_t)(m0 + et) * SSQ_STRIDE + tile] = (w[0] + w[1]) + (w[2] + w[3]);
-                }
-                epi_bar();
-            }
-            break;
-        }
-        case EPI_SWIGLU: {
-            const int f = (int)tile * 64 + et;
-#pragma unroll
-            for (int i = 0; i < MB; ++i) sh.val[i][et] = v[i];
-            epi_bar();
-            if (et < 64 && f < ep.F) {
-#pragma unroll
-                for (int i = 0; i < MB; ++i) {
-                    if (rows[i] < 0) continue;
-                    const float gt = v[i], up = sh.val[i][et + 64];
-                    ep.act[(size_t)rows[i] * ep.F + f] = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
-                }
-            }
-            epi_bar();
-            break;
-        }
-        default: break;
-        }
-    }
-}
-
-// The four epilogue warps of a CTA: drain each finished accumulator from TMEM into the workspace,
-// count the arrival at its tile and, when this piece was the last, run the fused step on the tile.
-__device__ void epilogue_warps(const GemmGeom& g, const Epilogue& ep, float* __restrict__ partials, uint32_t* __restrict__ counters,
-                               Shared& sh, uint32_t tmem_base, int warp, int lane, uint32_t u0, uint32_t u1) {
+// The four epilogue warps of a CTA: drain each finished accumulator from TMEM into the workspace.
+__device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, Shared& sh, uint32_t tmem_base, int warp, int lane,
+                               uint32_t u0, uint32_t u1) {
     volatile int* abort_flag = &sh.abort_flag;
-            pdl_wait();                                                        // the workspace may still be read by the previous kernel
-            const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
-            const int et = quarter * 32 + lane;                                // weight row inside the tile
-            epilogue_prologue(g, ep, sh, et);
-            uint32_t seg = 0;
-            for (uint32_t u = u0; u < u1; ++seg) {
-                const uint32_t kb0 = u % g.kb_per_tile;
-                const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
-                const uint32_t buf = seg & 1u;
-                if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) sh.epi_abort = 1;
-                epi_bar();
-                if (sh.epi_abort) break;                                       // all four warps leave together
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
-                for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-    #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (c0 + j < g.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
-                }
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
-                // who completes the tile runs the step that follows the GEMM on it
-                const uint32_t tile = u / g.kb_per_tile;
-                uint32_t i_first, i_last;
-                tile_contributors(g, tile, i_first, i_last);
-                bool last = true;
-                if (i_last > i_first) {
-                    // The barrier orders the four warps' writes before thread 0's release; the acquire
-                    // side of the same operation, followed by the second barrier, orders every other
-                    // CTA's pieces before the reads below (release/acquire are cumulative).
-                    epi_bar();
-                    if (et == 0) {
-                        uint32_t old;
-                        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile) : "memory");
-                        const int l = old == i_last - i_first;
-                        if (l) counters[tile] = 0u;                            // left at zero for the next launch
-                        sh.last_flag = l;
-                    }
-                    epi_bar();
-                    last = sh.last_flag != 0;
-                }
-                if (last) {
-                    if (g.m_tok <= 2) tile_epilogue<2, 32>(g, ep, partials, tile, i_first, i_last, sh, et);
-                    else if (g.m_tok > 8 && i_last - i_first < 4) tile_epilogue<16, 4>(g, ep, partials, tile, i_first, i_last, sh, et);
-                    else tile_epilogue<8, 8>(g, ep, partials, tile, i_first, i_last, sh, et);
-                }
-                epi_bar();
-                u += n_kb;
-            }
+    pdl_wait();                                                        // the workspace may still be read by the previous kernel
+    const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
+    const int et = quarter * 32 + lane;                                // weight row inside the tile
+    uint32_t seg = 0;
+    for (uint32_t u = u0; u < u1; ++seg) {
+        const uint32_t kb0 = u % g.kb_per_tile;
+        const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
+        const uint32_t buf = seg & 1u;
+        if (!mbar_wait(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) sh.epi_abort = 1;
+        epi_bar();
+        if (sh.epi_abort) break;                                       // all four warps leave together
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
+        for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (c0 + j < g.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+        u += n_kb;
+    }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
-             GemmGeom g, Epilogue ep, float* __restrict__ partials, uint32_t* __restrict__ counters, uint32_t* status) {
+k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+               GemmGeom g, float* __restrict__ partials, uint32_t* status) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ Shared sh;
     pdl_launch_dependents();                 // the next kernel may be scheduled; it waits for this one where it must
@@ -478,8 +266,8 @@ k_gemm_fused(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ C
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: TMEM -> partials -> fused step
-        epilogue_warps(g, ep, partials, counters, sh, tmem_base, warp, lane, u0, u1);
+        // ------------------------------------------------------------------ epilogue: TMEM -> workspace
+        epilogue_warps(g, partials, sh, tmem_base, warp, lane, u0, u1);
     }
 
     // ---------------------------------------------------------------------- wind-down
@@ -544,7 +332,7 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     g.max_seg = (per_cta + g.kb_per_tile - 2) / g.kb_per_tile + 1;
     if ((T + 1) * (g.grid + 1) >= (1ll << 32)) g.grid = 0;   // the kernels split the work in 32-bit arithmetic
     const int stage_bytes = A_BYTES + g.m_pad * 128;
-    g.stages = std::max(2, std::min(MAX_STAGES, (198 * 1024) / stage_bytes));
+    g.stages = std::max(2, std::min(MAX_STAGES, RING_BYTES / stage_bytes));
     g.steady = std::min(g.stages, std::max(2, (GEMM_STEADY_BYTES + stage_bytes - 1) / stage_bytes));
     return g;
 }
@@ -555,21 +343,18 @@ bool gemm_tc_supported(int m_tok, int n_out, int K) {
     return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0 && (long long)((n_out + 127) / 128) * ((K + 63) / 64) < (1ll << 24);
 }
 
-cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
-                              float* partials, uint32_t* counters, uint32_t* status, int dependent, cudaStream_t st) {
+cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* status,
+                                int dependent, cudaStream_t st) {
     const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - (int)sizeof(Shared) - 256);
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_streamk, cudaFuncAttributeMaxDynamicSharedMemorySize, RING_BYTES + 2048);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    if (g.grid < 1 || g.stages < 2 || g.steady < 1 || g.steady > g.stages || g.n_tiles > GEMM_MAX_TILES || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
-    if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
-    if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
-    if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
-    return launch_pdl(k_gemm_fused, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,
-                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, ep, partials, counters, status);
+    if (g.grid < 1 || g.stages < 2 || g.steady < 1 || g.steady > g.stages || g.m_tok > SD_MAX_ROWS || smem > RING_BYTES + 2048) return cudaErrorInvalidValue;
+    return launch_pdl(k_gemm_streamk, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,
+                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, partials, status);
 }
 
 }  // namespace sd

@@ -1,4 +1,4 @@
-// Interface of the tensor-core weight-streaming GEMM (gemm_tc.cu) with its fused epilogues.
+// Interface of the tensor-core weight-streaming GEMM (gemm_tc.cu) and of the fused step that follows it (fused_step.cu).
 #pragma once
 #include <algorithm>
 #include <utility>
@@ -29,7 +29,7 @@ struct RowScale {
 };
 constexpr int SSQ_STRIDE = 64;
 
-// What the CTA that completes a 128-row output tile does with it (the step that follows the
+// What happens to a 128-row output tile once its pieces are summed (the step that follows the
 // GEMM in the decoder layer), so that no fp32 intermediate matrix goes through memory.
 enum { EPI_PLAIN = 0, EPI_QKV_ROPE = 1, EPI_RESIDUAL = 2, EPI_SWIGLU = 3 };
 struct Epilogue {
@@ -39,7 +39,7 @@ struct Epilogue {
     float* y; int n_out_rows, row_stride, row_offset;
     // EPI_QKV_ROPE: rotary embedding, then query buffer / KV-cache append (bf16)
     bf16* q_out; bf16* kc; bf16* vc; const int32_t* row_slot; const int32_t* row_pos;
-    int H, Hkv, hd, max_ctx; const float* rcos; const float* rsin;
+    int H, Hkv, hd, max_ctx; const float* rcos; const float* rsin;     // rcos/rsin: [token row][hd/2], the row's position applied
     // EPI_RESIDUAL: h += acc; xn = bf16(h * gain_next); ssq_out[row][tile] = sum over the tile of h^2
     float* h; const float* gain_next; bf16* xn; float* ssq_out;
     // EPI_SWIGLU: rows of the weight matrix interleaved per tile (64 gate rows, then the 64 up
@@ -50,14 +50,14 @@ struct Epilogue {
 bool gemm_tc_supported(int m_tok, int n_out, int K);
 GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm);
 size_t gemm_partials_bytes(const GemmGeom& g);
-constexpr int GEMM_MAX_TILES = 4096;                                  // arrival counters, one per output tile
-constexpr size_t GEMM_COUNTER_BYTES = sizeof(uint32_t) * GEMM_MAX_TILES;
 bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows);
-// counters: GEMM_MAX_TILES words, zero before the first launch (every launch leaves them zero).
+// The GEMM proper: leaves the split accumulators in `partials` (gemm_partials_bytes()).
 // dependent != 0: launched with programmatic stream serialisation (may start while the previous
 // kernel on the stream drains; the kernel itself waits before it touches that kernel's results).
-cudaError_t launch_gemm_fused(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, const Epilogue& ep,
-                              float* partials, uint32_t* counters, uint32_t* status, int dependent, cudaStream_t st);
+cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* status,
+                                int dependent, cudaStream_t st);
+// The step after the GEMM (fused_step.cu): reduces `partials` and applies `ep`.
+cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, int dependent, cudaStream_t st);
 
 // Launch with the programmatic-dependent-launch attribute (or plainly when dependent == 0).
 template <typename... KArgs, typename... Args>

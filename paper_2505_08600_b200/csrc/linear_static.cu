@@ -53,9 +53,9 @@ extern "C" sd_status sd_op_linear_static(const void* x, const void* w, float* y,
         return SD_ERR_CUDA;
     const GemmGeom g = gemm_geometry(rows, n_out, n_in, n_sm);
     if (g.grid < 1) return SD_ERR_UNSUPPORTED;
-    if (GEMM_COUNTER_BYTES + gemm_partials_bytes(g) > (size_t)SD_STATIC_SCRATCH_BYTES) {
+    if (gemm_partials_bytes(g) > (size_t)SD_STATIC_SCRATCH_BYTES) {
         fprintf(stderr, "[sd] sd_op_linear_static: %d x %d x %d needs %zu bytes of scratch, the built-in array holds %d\n",
-                rows, n_out, n_in, GEMM_COUNTER_BYTES + gemm_partials_bytes(g), (int)SD_STATIC_SCRATCH_BYTES);
+                rows, n_out, n_in, gemm_partials_bytes(g), (int)SD_STATIC_SCRATCH_BYTES);
         return SD_ERR_CAPACITY;
     }
     char* scratch = (char*)scratch_on_current_device();
@@ -63,14 +63,12 @@ extern "C" sd_status sd_op_linear_static(const void* x, const void* w, float* y,
     TensorMap tw, tx;
     if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // The head of the array holds the tiles' arrival counters, which must start at zero (a call that
-    // was cut short could have left some behind); every accumulator word that is read is written by
-    // this call's own GEMM first, so the rest needs no clearing.
-    if (cudaMemsetAsync(scratch, 0, GEMM_COUNTER_BYTES, st) != cudaSuccess) return SD_ERR_CUDA;
+    // Every accumulator word that is read is written by this call's own GEMM first, so the array needs no clearing.
     Epilogue e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
-    if (launch_gemm_fused(tw, tx, g, e, (float*)(scratch + GEMM_COUNTER_BYTES), (uint32_t*)scratch, nullptr, 0, st) != cudaSuccess)
+    if (launch_gemm_streamk(tw, tx, g, (float*)scratch, nullptr, 0, st) != cudaSuccess ||
+        launch_fused_step(g, e, (const float*)scratch, 1, st) != cudaSuccess)
         return SD_ERR_CUDA;
     return SD_OK;
 }
