@@ -112,7 +112,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t r[16]) {
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }    // the four epilogue warps
 
 struct Shared {
-    uint64_t full_w[MAX_STAGES], full_x[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     int epi_abort;
@@ -122,12 +122,15 @@ struct Shared {
 // consumers wait for the previous kernel); after that only the first `steady` stages are reused,
 // which keeps fewer loads in flight: the same bandwidth with a shorter queue, so the last tile
 // arrives sooner after it is requested.  use = how often the stage was used before this load.
-struct RingPos { int stage; uint32_t use; };
-__device__ __forceinline__ RingPos ring_pos(uint32_t it, int stages, int steady) {
-    if (it < (uint32_t)stages) return RingPos{(int)it, 0u};
-    const uint32_t r = it - stages;
-    return RingPos{(int)(r % steady), 1u + r / steady};
-}
+struct RingPos {
+    int stage; uint32_t use; int filled;
+    __device__ __forceinline__ RingPos() : stage(0), use(0u), filled(0) {}
+    __device__ __forceinline__ void next(int stages, int steady) {         // position of the following load (no divisions: the MMA
+        ++stage;                                                           // thread's loop is bound by its own instruction latencies)
+        if (!filled) { if (stage == stages) { stage = 0; use = 1u; filled = 1; } }
+        else if (stage == steady) { stage = 0; ++use; }
+    }
+};
 
 // The four epilogue warps of a CTA: drain each finished accumulator from TMEM into the workspace.
 __device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, Shared& sh, uint32_t tmem_base, int warp, int lane,
@@ -182,7 +185,8 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) {
-            mbar_init(smem_u32(&sh.full_w[s]), 1); mbar_init(smem_u32(&sh.full_x[s]), 1); mbar_init(smem_u32(&sh.empty[s]), 1);
+            mbar_init(smem_u32(&sh.full[s]), 2);           // the weight tile and the token rows arrive from two producers
+            mbar_init(smem_u32(&sh.empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
         sh.abort_flag = 0;
@@ -208,15 +212,15 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         if (lane == 0) {
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            for (uint32_t it = 0; it < n_units; ++it) {
-                const uint32_t u = u0 + it;
-                const RingPos rp = ring_pos(it, g.stages, g.steady);
+            RingPos rp;
+            int tile = u0 / g.kb_per_tile, kb = u0 % g.kb_per_tile;
+            for (uint32_t it = 0; it < n_units; ++it, rp.next(g.stages, g.steady)) {
                 const int s = rp.stage;
                 if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
-                const int tile = u / g.kb_per_tile, kb = u % g.kb_per_tile;
-                const uint32_t bar = smem_u32(&sh.full_w[s]);
+                const uint32_t bar = smem_u32(&sh.full[s]);
                 mbar_expect_tx(bar, A_BYTES);
                 tma_load_2d(tiles0 + s * stage_bytes, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
+                if (++kb == g.kb_per_tile) { kb = 0; ++tile; }
             }
         }
     } else if (warp == 6) {
@@ -225,37 +229,37 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             pdl_wait();                                           // the token rows are the previous kernel's output
-            for (uint32_t it = 0; it < n_units; ++it) {
-                const RingPos rp = ring_pos(it, g.stages, g.steady);
+            RingPos rp;
+            int kb = u0 % g.kb_per_tile;
+            for (uint32_t it = 0; it < n_units; ++it, rp.next(g.stages, g.steady)) {
                 const int s = rp.stage;
                 if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
-                const int kb = (u0 + it) % g.kb_per_tile;
-                const uint32_t bar = smem_u32(&sh.full_x[s]);
+                const uint32_t bar = smem_u32(&sh.full[s]);
                 mbar_expect_tx(bar, x_bytes);
                 tma_load_2d(tiles0 + s * stage_bytes + A_BYTES, &tm_x, kb * TILE_K, 0, bar, pol_keep);
+                if (++kb == g.kb_per_tile) kb = 0;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.m_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-            uint32_t it = 0, seg = 0;
+            uint32_t seg = 0;
             bool ok = true;
-            for (uint32_t u = u0; u < u1 && ok; ++seg) {
-                const uint32_t kb0 = u % g.kb_per_tile;
+            RingPos rp;
+            const uint64_t desc0 = umma_desc(tiles0);
+            uint32_t kb0 = u0 % g.kb_per_tile;
+            for (uint32_t u = u0; u < u1 && ok; ++seg, kb0 = 0) {
                 const uint32_t n_kb = min((uint32_t)g.kb_per_tile - kb0, u1 - u);
                 const uint32_t buf = seg & 1u;
                 if (!mbar_wait(smem_u32(&sh.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, abort_flag)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)g.m_pad;
-                for (uint32_t j = 0; j < n_kb; ++j, ++it) {
-                    const RingPos rp = ring_pos(it, g.stages, g.steady);
+                for (uint32_t j = 0; j < n_kb; ++j, rp.next(g.stages, g.steady)) {
                     const int s = rp.stage;
-                    const uint32_t ph = rp.use & 1u;
-                    if (!mbar_wait(smem_u32(&sh.full_w[s]), ph, abort_flag) || !mbar_wait(smem_u32(&sh.full_x[s]), ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&sh.full[s]), rp.use & 1u, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a = tiles0 + s * stage_bytes;
-                    const uint64_t da = umma_desc(a), db = umma_desc(a + A_BYTES);
+                    const uint64_t da = desc0 + (uint64_t)((uint32_t)s * (stage_bytes >> 4)), db = da + (A_BYTES >> 4);   // start-address field counts 16 bytes
 #pragma unroll
                     for (uint32_t k = 0; k < TILE_K / 16; ++k)     // 16 elements = 32 bytes further along the swizzled row
                         umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (j | k) != 0u);
