@@ -16,10 +16,10 @@ namespace sd {
 
 namespace {
 
-constexpr int ATT_WARPS = 8;
-constexpr int ATT_THREADS = 32 * ATT_WARPS;   // each warp takes 16 of the keys of a chunk
+// Warps per CTA: eight when there are few CTAs (each finishes its slice sooner), four when there are several
+// per SM (three of them fit an SM, and one's set-up and merge overlap the others' streaming).
+constexpr int WARPS_FEW = 8, WARPS_MANY = 4;
 constexpr int NQ = 16;              // query vectors per CTA (rows in the block x heads per KV head): one MMA row tile
-constexpr int CK = 16 * ATT_WARPS;  // keys per chunk
 constexpr int SLICE_KEYS = 1024;    // a slice of the cache per CTA: up to this many positions
 constexpr size_t ATTN_COUNTER_BYTES = 65536;     // one arrival counter per (query block, kv head)
 
@@ -66,8 +66,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // distributed shared memory.  A context of up to SLICE_KEYS positions is one slice, whose output
 // is written directly; longer contexts are cut into slices whose partial results are merged by
 // whichever slice arrives last.
-template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
+template <int HD, int NW>
+__global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
+    constexpr int NT = 32 * NW;              // threads; each warp takes 16 of the keys of a chunk
+    constexpr int CK = 16 * NW;              // keys per chunk
     extern __shared__ __align__(128) uint8_t sm_raw[];
     constexpr int ROWB = HD * 2;             // bytes of one key / value row
     constexpr int CPR = HD / 8;              // 16-byte pieces per row
@@ -120,7 +122,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
             const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
             const bf16* ks = K + (size_t)c * CK * HD;
             const bf16* vs = V + (size_t)c * CK * HD;
-            for (int i = t; i < nk * CPR; i += ATT_THREADS) {
+            for (int i = t; i < nk * CPR; i += NT) {
                 const int key = i / CPR, ch = i % CPR;
                 const uint32_t off = (uint32_t)key * ROWB + (uint32_t)((ch ^ (key & 7)) << 4);
                 cp_async16(kb + off, ks + (size_t)i * 8);
@@ -128,7 +130,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
             }
             // value rows past the end of the slice inside a warp's 16-key group must be finite (their weight is zero)
             const int nk16 = (nk + 15) & ~15;
-            for (int i = nk * CPR + t; i < nk16 * CPR; i += ATT_THREADS) {
+            for (int i = nk * CPR + t; i < nk16 * CPR; i += NT) {
                 const int key = i / CPR, ch = i % CPR;
                 *reinterpret_cast<uint4*>(sm_raw + (size_t)(c & 1) * 2 * BUF + BUF + (size_t)key * ROWB + ((ch ^ (key & 7)) << 4)) = make_uint4(0, 0, 0, 0);
             }
@@ -226,8 +228,8 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
 
     // ---- merge of the warps (each saw different keys), then the slice's partial result
     float* Ow = reinterpret_cast<float*>(sm_raw);                // [warps][16][OLD]
-    float* mw = Ow + ATT_WARPS * NQ * OLD;                       // [warps][16]
-    float* lw = mw + ATT_WARPS * NQ;                             // [warps][16]
+    float* mw = Ow + NW * NQ * OLD;                       // [warps][16]
+    float* lw = mw + NW * NQ;                             // [warps][16]
     if (np > 0) {
 #pragma unroll
         for (int nv = 0; nv < NV; ++nv) {
@@ -241,11 +243,12 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     }
     __syncthreads();
     // this CTA's result: per query row the running max, the sum and the unnormalised output
-    constexpr int CPT = HD / 16;                                 // columns per thread: 16 threads span a query row
-    float* Oc = reinterpret_cast<float*>(sm_raw) + ATT_WARPS * NQ * OLD + 2 * ATT_WARPS * NQ;   // [16][HD]
+    constexpr int TPR = NT / NQ;                                 // threads that span a query row
+    constexpr int CPT = HD / TPR;                                // columns per thread
+    float* Oc = reinterpret_cast<float*>(sm_raw) + NW * NQ * OLD + 2 * NW * NQ;   // [16][HD]
     float* Mc = Oc + NQ * HD;                                    // [16]
     float* Lc = Mc + NQ;                                         // [16]
-    const int j = t >> 4, c0 = (t & 15) * CPT;
+    const int j = t / TPR, c0 = (t % TPR) * CPT;
     {
         float M = -INFINITY, L = 0.f;
         float4 acc[CPT / 4];
@@ -253,10 +256,10 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
         for (int cc = 0; cc < CPT / 4; ++cc) acc[cc] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (np > 0) {
 #pragma unroll
-            for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, mw[w * NQ + j]);
-            float wt[ATT_WARPS];
+            for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w * NQ + j]);
+            float wt[NW];
 #pragma unroll
-            for (int w = 0; w < ATT_WARPS; ++w) {
+            for (int w = 0; w < NW; ++w) {
                 const float m = mw[w * NQ + j];
                 wt[w] = (m == -INFINITY) ? 0.f : exp2f(m - M);
                 L += wt[w] * lw[w * NQ + j];
@@ -264,7 +267,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
 #pragma unroll
             for (int cc = 0; cc < CPT / 4; ++cc)
 #pragma unroll
-                for (int w = 0; w < ATT_WARPS; ++w) {
+                for (int w = 0; w < NW; ++w) {
                     if (wt[w] != 0.f) {                       // a warp without keys left nothing behind
                         const float4 o = *reinterpret_cast<const float4*>(Ow + ((size_t)w * NQ + j) * OLD + c0 + 4 * cc);
                         acc[cc].x = fmaf(wt[w], o.x, acc[cc].x); acc[cc].y = fmaf(wt[w], o.y, acc[cc].y);
@@ -274,7 +277,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
         }
 #pragma unroll
         for (int cc = 0; cc < CPT / 4; ++cc) *reinterpret_cast<float4*>(Oc + (size_t)j * HD + c0 + 4 * cc) = acc[cc];
-        if ((t & 15) == 0) { Mc[j] = M; Lc[j] = L; }
+        if ((t % TPR) == 0) { Mc[j] = M; Lc[j] = L; }
     }
     // the CTAs of the cluster hand their results to the first one through distributed shared memory
     namespace cg = cooperative_groups;
@@ -324,7 +327,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
             float* ml = P.part_ml + (((size_t)r * P.H + h) * P.n_splits + split) * 2;
 #pragma unroll
             for (int cc = 0; cc < CPT / 4; ++cc) __stcg(reinterpret_cast<float4*>(po + 4 * cc), acc[cc]);
-            if ((t & 15) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+            if ((t % TPR) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
         }
     }
     if (CS > 1) cluster.sync();                      // nobody leaves while its shared memory may still be read
@@ -356,11 +359,11 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
             const int r = r0 + j / group, h = kvh * group + j % group;
             const float* src = P.part_o + ((size_t)r * P.H + h) * ns * HD;
             const uint32_t dst = smem0 + (uint32_t)j * (uint32_t)per_q * 16u;
-            for (int c = t; c < per_q; c += ATT_THREADS) cp_async16(dst + (uint32_t)c * 16u, src + (size_t)c * 4);
+            for (int c = t; c < per_q; c += NT) cp_async16(dst + (uint32_t)c * 16u, src + (size_t)c * 4);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    for (int j = warp; j < nq; j += ATT_THREADS / 32) {          // n_splits <= 32: one lane per slice
+    for (int j = warp; j < nq; j += NT / 32) {          // n_splits <= 32: one lane per slice
         const int r = r0 + j / group, h = kvh * group + j % group;
         const float* mlg = P.part_ml + ((size_t)r * P.H + h) * ns * 2;
         float m = -INFINITY, l = 0.f;
@@ -373,7 +376,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_mma(AttnParams P) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     // each thread owns one output column of up to NQ queries: independent sums, slices in order
-    constexpr int TPQ = ATT_THREADS / HD;                        // queries handled side by side (1 or 2)
+    constexpr int TPQ = NT / HD;                        // queries handled side by side (1 or 2)
     const int e = t % HD, jq0 = t / HD;
     float acc[NQ / TPQ];
 #pragma unroll
@@ -446,27 +449,26 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
     P.counters = (uint32_t*)workspace;
     P.part_o = (float*)((char*)workspace + ATTN_COUNTER_BYTES);
     P.part_ml = P.part_o + (size_t)n_rows * H * P.n_splits * hd;
-    const size_t smem = std::max((size_t)4 * CK * hd * 2, sizeof(float) * ((size_t)ATT_WARPS * NQ * (hd + 8) + 2 * ATT_WARPS * NQ + (size_t)NQ * hd + 2 * NQ));
     // few (head, row block, slice) items: two or four CTAs of a cluster share each of them
     int sm = 148;
     { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
     const int items = P.n_splits * Hkv * n_blocks;
     P.csize = items * 4 <= sm ? 4 : (items * 2 <= sm ? 2 : 1);
+    const int nw = items > 2 * sm ? WARPS_MANY : WARPS_FEW;
+    const size_t smem = std::max((size_t)4 * 16 * nw * hd * 2, sizeof(float) * ((size_t)nw * NQ * (hd + 8) + 2 * nw * NQ + (size_t)NQ * hd + 2 * NQ));
     dim3 grid(P.n_splits * P.csize, Hkv, n_blocks);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = dim3(ATT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cfg.gridDim = grid; cfg.blockDim = dim3(32 * nw); cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     int na = 0;
     if (P.csize > 1) { attr[na].id = cudaLaunchAttributeClusterDimension; attr[na].val.clusterDim.x = P.csize; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1; ++na; }
     if (dependent) { attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na; }
     cfg.attrs = attr; cfg.numAttrs = na;
-    cudaError_t e;
-    if (hd == 128) {
-        if ((e = cudaFuncSetAttribute(k_attn_mma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        return cudaLaunchKernelEx(&cfg, k_attn_mma<128>, P);
-    }
-    if ((e = cudaFuncSetAttribute(k_attn_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, k_attn_mma<64>, P);
+    void (*kern)(AttnParams) = hd == 128 ? (nw == WARPS_MANY ? k_attn_mma<128, WARPS_MANY> : k_attn_mma<128, WARPS_FEW>)
+                                         : (nw == WARPS_MANY ? k_attn_mma<64, WARPS_MANY> : k_attn_mma<64, WARPS_FEW>);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, kern, P);
 }
 
 }  // namespace sd

@@ -61,6 +61,9 @@ ATTN_CASES = [  # H, Hkv, hd, max_ctx, positions of the rows
     (4, 2, 128, 2600, [0, 1023, 1024, 1025, 2047, 2599]),
     (4, 4, 64, 4100, [4099, 3000, 17, 1024]),
     (2, 2, 128, 8192, [8191, 4096, 100]),
+    # many (head, row, slice) items: several CTAs per SM, the four-warp form of the kernel (single slice, and merged slices)
+    (32, 32, 128, 700, [0, 63, 64, 127, 128, 300, 511, 640, 698, 699]),
+    (16, 16, 64, 2100, [2099, 1024, 1023, 17, 2048, 700, 1500]),
 ]
 
 
