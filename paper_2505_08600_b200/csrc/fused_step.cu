@@ -27,11 +27,13 @@ struct StepShared {
 };
 
 // MB token rows x CB pieces are in flight together: (8, 8) for the verify rows, (2, 32) for one or
-// two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) for
-// many rows on few pieces.
-template <int MB, int CB>
+// two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) or (16, 2)
+// for many rows on few pieces.  MODE < 0: the step is read from ep.mode; with many row batches one
+// instantiation per step is used instead, whose lower register count lets more CTAs be resident.
+template <int MODE, int MB, int CB>
 __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials) {
     __shared__ StepShared<MB> sh;
+    const int mode = MODE < 0 ? ep.mode : MODE;
     pdl_launch_dependents();
     const int et = threadIdx.x, lane = et & 31, warp = et >> 5;
     const uint32_t tile = blockIdx.x;
@@ -44,14 +46,14 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     const uint32_t i_first = ((ua + 1) * G + T - 1) / T - 1;      // T * G < 2^32 (checked on the host)
     const uint32_t i_last = ((ub + 1) * G + T - 1) / T - 1;
     const uint32_t j_first = tile - ((i_first * T) / G) / KB;
-    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    const int n_rows = mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
     int rows[MB];
 #pragma unroll
     for (int i = 0; i < MB; ++i) {
         const int r = m0 + i;
-        rows[i] = r < n_rows ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
+        rows[i] = r < n_rows ? (mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
     }
-    const float gain = (ep.mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;   // a weight: needs no wait
+    const float gain = (mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;   // a weight: needs no wait
     pdl_wait();                                   // the pieces (and the rows' sums of squares) come from the kernels before
 
     // ---- one round of loads: sums of squares, residual / row plan / rotary factors, the pieces
@@ -61,17 +63,17 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         for (int ii = 0; ii < (MB + 3) / 4; ++ii) {
             const int i = warp + 4 * ii, r = m0 + i;
             const bool ok = i < MB && r < n_rows;
-            const float* ps = ep.rs.ssq + (size_t)(ok ? (ep.mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : 0) * SSQ_STRIDE;
+            const float* ps = ep.rs.ssq + (size_t)(ok ? (mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : 0) * SSQ_STRIDE;
             ssa[ii] = (ok && lane < ep.rs.n_parts) ? __ldcg(ps + lane) : 0.f;
             ssb[ii] = (ok && lane + 32 < ep.rs.n_parts) ? __ldcg(ps + lane + 32) : 0.f;
         }
     }
     float hv[MB], cs[MB], sn[MB];
     int pos[MB], slot[MB];
-    if (ep.mode == EPI_RESIDUAL) {
+    if (mode == EPI_RESIDUAL) {
 #pragma unroll
         for (int i = 0; i < MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
-    } else if (ep.mode == EPI_QKV_ROPE) {
+    } else if (mode == EPI_QKV_ROPE) {
         const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
         const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
 #pragma unroll
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         for (int i = 0; i < MB; ++i) v[i] *= sh.scale[i];
     }
 
-    switch (ep.mode) {
+    switch (mode) {
     case EPI_PLAIN: {
         if (live) {
 #pragma unroll
@@ -190,6 +192,13 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     }
 }
 
+template <int MODE>
+cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float* partials, int n_rows, int pieces, int dependent, cudaStream_t st) {
+    const dim3 grid(g.n_tiles, (n_rows + 15) / 16);
+    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2>, grid, dim3(128), 0, st, dependent, g, ep, partials);
+    return launch_pdl(k_fused_step<MODE, 16, 4>, grid, dim3(128), 0, st, dependent, g, ep, partials);
+}
+
 }  // namespace
 
 cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, int dependent, cudaStream_t st) {
@@ -203,9 +212,17 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     const long long T = (long long)g.n_tiles * g.kb_per_tile;
     const int per_cta = (int)std::max<long long>(1, T / g.grid);
     const int pieces = (g.kb_per_tile + per_cta - 1) / per_cta + 1;
-    if (n_rows <= 2) return launch_pdl(k_fused_step<2, 32>, dim3(g.n_tiles, (n_rows + 1) / 2), dim3(128), 0, st, dependent, g, ep, partials);
-    if (n_rows > 8 && pieces <= 4) return launch_pdl(k_fused_step<16, 4>, dim3(g.n_tiles, (n_rows + 15) / 16), dim3(128), 0, st, dependent, g, ep, partials);
-    return launch_pdl(k_fused_step<8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials);
+    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, (n_rows + 1) / 2), dim3(128), 0, st, dependent, g, ep, partials);
+    if (n_rows > 8 && pieces <= 4) {
+        switch (ep.mode) {
+        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, n_rows, pieces, dependent, st);
+        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, n_rows, pieces, dependent, st);
+        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, n_rows, pieces, dependent, st);
+        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, n_rows, pieces, dependent, st);
+        default: return cudaErrorInvalidValue;
+        }
+    }
+    return launch_pdl(k_fused_step<-1, 8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials);
 }
 
 }  // namespace sd
