@@ -16,8 +16,8 @@
 //     their CTAs and applies the step that follows the GEMM in the decoder layer, while the
 //     next GEMM's CTAs already occupy the SMs this one has left and stream their weights;
 //   - the kernel is written for programmatic dependent launch: it lets its successor start at
-//     once; its weight stream never waits for the predecessor (only the token rows and the
-//     workspace do), so the ring is full when the consumers are released.
+//     once; the first part of its weight stream does not wait for the predecessor (the token rows
+//     and the workspace do), so most of the ring is full when the consumers are released.
 // Roles: warp 0 streams weights, warp 1 allocates TMEM and issues MMAs, warps 2..5 drain TMEM
 // into the workspace, warp 6 loads the token rows.  Every mbarrier wait is bounded; on expiry
 // the kernel flags SD_DEV_WAIT_EXPIRED and winds down.
@@ -35,6 +35,7 @@ constexpr int A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
 constexpr int RING_BYTES = 198 * 1024;          // stage ring of a CTA; the rest of the SM's shared memory is left to the fused-step CTAs
+constexpr int GEMM_PREFILL_BYTES = 120 * 1024;  // bytes per SM requested while the previous kernel is still at work (see the weight producer)
 constexpr int GEMM_STEADY_BYTES = 112 * 1024;   // bytes per SM kept in flight once the ring has been filled
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -205,10 +206,8 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------------ weight producer
-        // The weights do not depend on the previous kernel, so this thread never waits for it: the
-        // stream starts as soon as the CTA is resident and runs ahead by the depth of the ring while
-        // the consumers wait on the previous kernel.  (Capping the loads in flight below the ring
-        // depth was tried: polling for their arrival cost more than the shorter queues gained.)
+        // The first tiles do not wait for the previous kernel (weights do not depend on it): the stream
+        // starts as soon as the CTA is resident, while the consumers wait on the previous kernel.
         if (lane == 0) {
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
@@ -216,6 +215,10 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             int tile = u0 / g.kb_per_tile, kb = u0 % g.kb_per_tile;
             for (uint32_t it = 0; it < n_units; ++it, rp.next(g.stages, g.steady)) {
                 const int s = rp.stage;
+                // A full ring of requests at this point slowed the step down: they compete with the small,
+                // latency-critical reads of the kernel that reduces the previous GEMM.  So the run-ahead stops
+                // short of the ring's depth until that kernel has finished.
+                if (it == (uint32_t)g.prefill) pdl_wait();
                 if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
                 const uint32_t bar = smem_u32(&sh.full[s]);
                 mbar_expect_tx(bar, A_BYTES);
@@ -338,6 +341,8 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     const int stage_bytes = A_BYTES + g.m_pad * 128;
     g.stages = std::max(2, std::min(MAX_STAGES, RING_BYTES / stage_bytes));
     g.steady = std::min(g.stages, std::max(2, (GEMM_STEADY_BYTES + stage_bytes - 1) / stage_bytes));
+    // (measured: with more than 16 token rows the reduction kernel is bound by throughput, not latency, and the full run-ahead wins)
+    g.prefill = g.m_pad > 16 ? g.stages : std::min(g.stages, std::max(2, (GEMM_PREFILL_BYTES + stage_bytes - 1) / stage_bytes));
     return g;
 }
 

@@ -17,6 +17,7 @@ struct GemmGeom {
     int n_tiles, kb_per_tile;
     int grid, max_seg, stages;
     int steady;             // stages reused once the ring has been filled (<= stages)
+    int prefill;            // weight tiles requested before the previous kernel has finished
 };
 
 // RMSNorm folded around a GEMM: the GEMM's input rows are h * gain (no 1/rms factor), the
