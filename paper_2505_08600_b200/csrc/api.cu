@@ -56,6 +56,8 @@ enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
 
 }  // namespace
 
+constexpr size_t ARRIVE_WORDS = 65536;          // arrival words of one pass (the 13B target needs about 17,000)
+
 struct sd_ctx {
     sd_config cfg;
     std::vector<Model> models;
@@ -67,6 +69,8 @@ struct sd_ctx {
     void* attn_ws; size_t attn_ws_bytes;
     float* partials; size_t partials_bytes;     // split accumulators of the tensor-core GEMM
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
+    uint32_t* gemm_arrive;                      // per GEMM of a pass and output tile: pieces that have arrived (zero between passes)
+    size_t arrive_used;                         // words handed out to the GEMMs of the pass being enqueued
     float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
@@ -198,6 +202,8 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     }
     c->partials = (float*)B.take(c->partials_bytes);
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
+    c->gemm_arrive = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
+    c->arrive_used = 0;
     size_t half_max = 1;
     for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
     c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
@@ -310,8 +316,13 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
-    LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, c->S.status, 1, c->st));
-    LAUNCH(CAT_FUSED_STEP, launch_fused_step(g, ep, c->partials, 1, c->st));
+    uint32_t* arrive = nullptr;                 // words of this GEMM alone; when they run out the step waits for the GEMM's grid
+    if (fused_step_polls(g, ep) && c->arrive_used + (size_t)g.n_tiles <= ARRIVE_WORDS) {
+        arrive = c->gemm_arrive + c->arrive_used;
+        c->arrive_used += (size_t)g.n_tiles;
+    }
+    LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, arrive, c->S.status, 1, c->st));
+    LAUNCH(CAT_FUSED_STEP, launch_fused_step(g, ep, c->partials, arrive, c->S.status, 1, c->st));
     return SD_OK;
 }
 
@@ -322,6 +333,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
+    c->arrive_used = 0;                          // the embedding kernel below is an ordinary launch: everything before it has finished
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -501,7 +513,8 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
             cudaStreamSynchronize(st) != cudaSuccess)
             return fail(SD_ERR_CUDA);
     }
-    if (cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess)
+    if (cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess ||
+        cudaMemsetAsync(c->gemm_arrive, 0, sizeof(uint32_t) * ARRIVE_WORDS, st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
     c->force_plain = false;
@@ -934,8 +947,8 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
         Epilogue e;
         memset(&e, 0, sizeof(e));
         e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
-        CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, 0, (cudaStream_t)stream));
-        CUDA_TRY(launch_fused_step(g, e, (const float*)workspace, 1, (cudaStream_t)stream));
+        CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, nullptr, 0, (cudaStream_t)stream));
+        CUDA_TRY(launch_fused_step(g, e, (const float*)workspace, nullptr, nullptr, 1, (cudaStream_t)stream));
         return SD_OK;
     }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;

@@ -19,6 +19,12 @@ namespace {
 
 constexpr int TILE_N = 128;
 
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 template <int MB>
 struct StepShared {
     float scale[MB];                // 1/rms factor of the CTA's token rows
@@ -31,8 +37,10 @@ struct StepShared {
 // for many rows on few pieces.  MODE < 0: the step is read from ep.mode; with many row batches one
 // instantiation per step is used instead, whose lower register count lets more CTAs be resident.
 template <int MODE, int MB, int CB>
-__global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials) {
+__global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials,
+                                                    uint32_t* __restrict__ arrive, uint32_t* status) {
     __shared__ StepShared<MB> sh;
+    __shared__ int tile_seen;
     const int mode = MODE < 0 ? ep.mode : MODE;
     pdl_launch_dependents();
     const int et = threadIdx.x, lane = et & 31, warp = et >> 5;
@@ -54,7 +62,29 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         rows[i] = r < n_rows ? (mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
     }
     const float gain = (mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;   // a weight: needs no wait
-    pdl_wait();                                   // the pieces (and the rows' sums of squares) come from the kernels before
+    // The pieces come from the GEMM before (the rows' sums of squares from kernels further back, long finished).
+    // With arrival words the CTA starts as soon as its own tile is complete; otherwise when the GEMM's grid has retired.
+    if (arrive) {
+        if (et == 0) {
+            const uint32_t need = i_last - i_first + 1u;
+            uint32_t seen = 0;
+            const uint64_t t0 = global_timer_ns();
+            for (uint32_t spin = 0;; ++spin) {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrive + tile) : "memory");
+                if (seen >= need) break;
+                if ((spin & 63u) == 63u && global_timer_ns() - t0 > 200000000ull) break;      // 0.2 s: give up polling
+            }
+            tile_seen = seen >= need;
+        }
+        __syncthreads();
+        if (!tile_seen) {                          // not expected: wait for the whole grid instead, and say so
+            pdl_wait();
+            if (et == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
+        }
+        if (et == 0) arrive[tile] = 0u;            // left at zero for the next GEMM (which starts counting only after this kernel has finished)
+    } else {
+        pdl_wait();
+    }
 
     // ---- one round of loads: sums of squares, residual / row plan / rotary factors, the pieces
     float ssa[(MB + 3) / 4], ssb[(MB + 3) / 4];
@@ -193,15 +223,26 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
 }
 
 template <int MODE>
-cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float* partials, int n_rows, int pieces, int dependent, cudaStream_t st) {
+cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status, int n_rows,
+                             int pieces, int dependent, cudaStream_t st) {
     const dim3 grid(g.n_tiles, (n_rows + 15) / 16);
-    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2>, grid, dim3(128), 0, st, dependent, g, ep, partials);
-    return launch_pdl(k_fused_step<MODE, 16, 4>, grid, dim3(128), 0, st, dependent, g, ep, partials);
+    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    return launch_pdl(k_fused_step<MODE, 16, 4>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
 }  // namespace
 
-cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, int dependent, cudaStream_t st) {
+bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
+    // One batch of rows per tile (several would share a tile's word).  With one or two rows (draft and plain
+    // decoding steps: small matrices, kernels of several GEMMs resident and polling at once) waiting for the
+    // grid measured faster.
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    return n_rows > 2 && n_rows <= 8;
+}
+
+cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status,
+                              int dependent, cudaStream_t st) {
+    if (!fused_step_polls(g, ep)) arrive = nullptr;
     if (g.grid < 1 || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
     if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
@@ -212,17 +253,17 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     const long long T = (long long)g.n_tiles * g.kb_per_tile;
     const int per_cta = (int)std::max<long long>(1, T / g.grid);
     const int pieces = (g.kb_per_tile + per_cta - 1) / per_cta + 1;
-    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, (n_rows + 1) / 2), dim3(128), 0, st, dependent, g, ep, partials);
+    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
     if (n_rows > 8 && pieces <= 4) {
         switch (ep.mode) {
-        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, n_rows, pieces, dependent, st);
-        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, n_rows, pieces, dependent, st);
-        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, n_rows, pieces, dependent, st);
-        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, n_rows, pieces, dependent, st);
+        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
+        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
+        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
+        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
         default: return cudaErrorInvalidValue;
         }
     }
-    return launch_pdl(k_fused_step<-1, 8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials);
+    return launch_pdl(k_fused_step<-1, 8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
 }  // namespace sd

@@ -134,8 +134,8 @@ struct RingPos {
 };
 
 // The four epilogue warps of a CTA: drain each finished accumulator from TMEM into the workspace.
-__device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, Shared& sh, uint32_t tmem_base, int warp, int lane,
-                               uint32_t u0, uint32_t u1) {
+__device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, uint32_t* __restrict__ arrive, Shared& sh,
+                               uint32_t tmem_base, int warp, int lane, uint32_t u0, uint32_t u1) {
     volatile int* abort_flag = &sh.abort_flag;
     pdl_wait();                                                        // the workspace may still be read by the previous kernel
     const uint32_t quarter = (uint32_t)(warp & 3);                    // TMEM lanes this warp may read
@@ -161,13 +161,19 @@ __device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, 
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+        if (arrive) {
+            // The barrier orders the four warps' stores before thread 0's release, which is cumulative: whoever
+            // acquires the tile's word after the last arrival sees every piece of the tile.
+            epi_bar();
+            if (et == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(arrive + u / g.kb_per_tile) : "memory");
+        }
         u += n_kb;
     }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
-               GemmGeom g, float* __restrict__ partials, uint32_t* status) {
+               GemmGeom g, float* __restrict__ partials, uint32_t* __restrict__ arrive, uint32_t* status) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ Shared sh;
     pdl_launch_dependents();                 // the next kernel may be scheduled; it waits for this one where it must
@@ -274,7 +280,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ epilogue: TMEM -> workspace
-        epilogue_warps(g, partials, sh, tmem_base, warp, lane, u0, u1);
+        epilogue_warps(g, partials, arrive, sh, tmem_base, warp, lane, u0, u1);
     }
 
     // ---------------------------------------------------------------------- wind-down
@@ -352,8 +358,8 @@ bool gemm_tc_supported(int m_tok, int n_out, int K) {
     return m_tok >= 1 && m_tok <= 256 && n_out >= 1 && K >= 8 && (K & 7) == 0 && (long long)((n_out + 127) / 128) * ((K + 63) / 64) < (1ll << 24);
 }
 
-cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* status,
-                                int dependent, cudaStream_t st) {
+cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* arrive,
+                                uint32_t* status, int dependent, cudaStream_t st) {
     const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
@@ -363,7 +369,7 @@ cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, co
     }
     if (g.grid < 1 || g.stages < 2 || g.steady < 1 || g.steady > g.stages || g.m_tok > SD_MAX_ROWS || smem > RING_BYTES + 2048) return cudaErrorInvalidValue;
     return launch_pdl(k_gemm_streamk, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,
-                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, partials, status);
+                      *(const CUtensorMap*)&tm_w, *(const CUtensorMap*)&tm_x, g, partials, arrive, status);
 }
 
 }  // namespace sd

@@ -55,10 +55,20 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
 // The GEMM proper: leaves the split accumulators in `partials` (gemm_partials_bytes()).
 // dependent != 0: launched with programmatic stream serialisation (may start while the previous
 // kernel on the stream drains; the kernel itself waits before it touches that kernel's results).
-cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* status,
-                                int dependent, cudaStream_t st);
-// The step after the GEMM (fused_step.cu): reduces `partials` and applies `ep`.
-cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, int dependent, cudaStream_t st);
+// arrive (nullable): one word per output tile, zero before the launch; every CTA adds one to a tile's
+// word when its piece of the tile is in the workspace, so that the step after the GEMM can start on a
+// tile as soon as the tile is complete instead of when the whole grid has retired.  Kernels of several
+// consecutive GEMMs can be resident at once (each only needs its predecessor to have started), so
+// every GEMM between two ordinary (fully ordered) launches needs words of its own.
+cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* arrive,
+                                uint32_t* status, int dependent, cudaStream_t st);
+// The step after the GEMM (fused_step.cu): reduces `partials` and applies `ep`.  With `arrive` (the
+// words the GEMM counts in; left at zero again) and a single batch of rows, a tile's CTA polls its word
+// (bounded; on expiry it falls back to waiting for the GEMM's grid and flags SD_DEV_WAIT_EXPIRED).
+cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status,
+                              int dependent, cudaStream_t st);
+// Whether launch_fused_step polls (and clears) the arrival words for this step; the GEMM must count exactly then.
+bool fused_step_polls(const GemmGeom& g, const Epilogue& ep);
 
 // Launch with the programmatic-dependent-launch attribute (or plainly when dependent == 0).
 template <typename... KArgs, typename... Args>

@@ -67,8 +67,8 @@ extern "C" sd_status sd_op_linear_static(const void* x, const void* w, float* y,
     Epilogue e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0;
-    if (launch_gemm_streamk(tw, tx, g, (float*)scratch, nullptr, 0, st) != cudaSuccess ||
-        launch_fused_step(g, e, (const float*)scratch, 1, st) != cudaSuccess)
+    if (launch_gemm_streamk(tw, tx, g, (float*)scratch, nullptr, nullptr, 0, st) != cudaSuccess ||
+        launch_fused_step(g, e, (const float*)scratch, nullptr, nullptr, 1, st) != cudaSuccess)
         return SD_ERR_CUDA;
     return SD_OK;
 }
