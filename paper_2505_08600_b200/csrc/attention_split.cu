@@ -89,7 +89,9 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(sm_raw);
     __shared__ int last_sm;
 
-    pdl_wait();                                  // queries, the appended keys/values and the row plan come from earlier kernels
+    // The row plan (positions, slots) was written by the pass's first kernel, an ordinary launch that every later
+    // kernel of the pass started after: it may be read before the wait below, and so may the cache positions in
+    // front of the pass's first new one, which earlier passes wrote.
     // longest context among the block's rows (every warp works it out for itself), and the sequence slot
     int mp = lane < nr ? __ldcg(P.row_pos + r0 + lane) : -1;
     const int slot = __ldcg(P.row_slot + r0);
@@ -113,16 +115,25 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
 #pragma unroll
     for (int i = 0; i < NV; ++i) { O[i][0] = O[i][1] = O[i][2] = O[i][3] = 0.f; }
 
-    if (np > 0) {
-        const bf16* K = P.kc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
-        const bf16* V = P.vc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
-        const int n_chunks = (np + CK - 1) / CK;
-        auto issue = [&](int c) {                // chunk c -> buffer c & 1: [K][V]
+    // first position this pass appends for the block's sequence (its rows' positions rise; inactive rows are -1)
+    int new_begin;
+    {
+        const int seq_first = (blockIdx.z / bps) * P.rows_per_seq;
+        const int fp = lane < min(P.rows_per_seq, 32) ? __ldcg(P.row_pos + seq_first + lane) : -1;
+        int nb = fp >= 0 ? fp : 0x7fffffff;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nb = min(nb, __shfl_xor_sync(0xffffffffu, nb, o));
+        new_begin = nb == 0x7fffffff ? 0 : nb;
+    }
+    const bf16* K = P.kc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + max(p_begin, 0)) * HD;
+    const bf16* V = P.vc + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + max(p_begin, 0)) * HD;
+    // keys [k_lo, k_hi) of chunk c -> buffer c & 1: [K][V]; last: also clears the padding rows and closes the chunk
+    auto issue_part = [&](int c, int k_lo, int k_hi, bool last) {
             const int nk = min(CK, np - c * CK);
             const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
             const bf16* ks = K + (size_t)c * CK * HD;
             const bf16* vs = V + (size_t)c * CK * HD;
-            for (int i = t; i < nk * CPR; i += NT) {
+            for (int i = k_lo * CPR + t; i < k_hi * CPR; i += NT) {
                 const int key = i / CPR, ch = i % CPR;
                 const uint32_t off = (uint32_t)key * ROWB + (uint32_t)((ch ^ (key & 7)) << 4);
                 cp_async16(kb + off, ks + (size_t)i * 8);
@@ -130,13 +141,20 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
             }
             // value rows past the end of the slice inside a warp's 16-key group must be finite (their weight is zero)
             const int nk16 = (nk + 15) & ~15;
-            for (int i = nk * CPR + t; i < nk16 * CPR; i += NT) {
+            for (int i = nk * CPR + t; last && i < nk16 * CPR; i += NT) {
                 const int key = i / CPR, ch = i % CPR;
                 *reinterpret_cast<uint4*>(sm_raw + (size_t)(c & 1) * 2 * BUF + BUF + (size_t)key * ROWB + ((ch ^ (key & 7)) << 4)) = make_uint4(0, 0, 0, 0);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-        };
-        issue(0);
+    };
+    auto issue = [&](int c) { issue_part(c, 0, min(CK, np - c * CK), true); };
+    // the part of the first chunk that earlier passes wrote is requested before the wait
+    const int old0 = np > 0 ? max(0, min(min(CK, np), new_begin - p_begin)) : 0;
+    if (np > 0) issue_part(0, 0, old0, false);
+    pdl_wait();                                  // queries and the keys/values appended by this pass come from the kernels before
+    if (np > 0) {
+        const int n_chunks = (np + CK - 1) / CK;
+        issue_part(0, old0, min(CK, np), true);
         // query fragments (bf16, straight from memory in the MMA's register layout) and the rows' positions
         uint32_t a[KS][4];
 #pragma unroll
