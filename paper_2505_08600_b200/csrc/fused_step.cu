@@ -62,6 +62,22 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         rows[i] = r < n_rows ? (mode == EPI_PLAIN ? r * ep.row_stride + ep.row_offset : r) : -1;
     }
     const float gain = (mode == EPI_RESIDUAL && ep.gain_next && live) ? ep.gain_next[n] : 0.f;   // a weight: needs no wait
+    // The row plan and the rows' rotary factors were written by the pass's first kernel, an ordinary launch that every
+    // later kernel of the pass started after: they need no wait either.
+    float cs[MB], sn[MB];
+    int pos[MB], slot[MB];
+    if (mode == EPI_QKV_ROPE) {
+        const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
+        const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            const bool ok = lower && rows[i] >= 0;
+            pos[i] = ok ? __ldcg(ep.row_pos + rows[i]) : -1;
+            slot[i] = (ok && head >= ep.H) ? __ldcg(ep.row_slot + rows[i]) : 0;
+            cs[i] = (ok && rot) ? __ldcg(ep.rcos + (size_t)rows[i] * half + e) : 1.f;     // per-row rotary factors (the row's position applied)
+            sn[i] = (ok && rot) ? __ldcg(ep.rsin + (size_t)rows[i] * half + e) : 0.f;
+        }
+    }
     // The pieces come from the GEMM before (the rows' sums of squares from kernels further back, long finished).
     // With arrival words the CTA starts as soon as its own tile is complete; otherwise when the GEMM's grid has retired.
     if (arrive) {
@@ -98,22 +114,10 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             ssb[ii] = (ok && lane + 32 < ep.rs.n_parts) ? __ldcg(ps + lane + 32) : 0.f;
         }
     }
-    float hv[MB], cs[MB], sn[MB];
-    int pos[MB], slot[MB];
+    float hv[MB];
     if (mode == EPI_RESIDUAL) {
 #pragma unroll
         for (int i = 0; i < MB; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(ep.h + (size_t)rows[i] * g.n_out + n) : 0.f;
-    } else if (mode == EPI_QKV_ROPE) {
-        const int half = ep.hd >> 1, e = n % ep.hd, head = n / ep.hd;
-        const bool lower = live && e < half, rot = head < ep.H + ep.Hkv;
-#pragma unroll
-        for (int i = 0; i < MB; ++i) {
-            const bool ok = lower && rows[i] >= 0;
-            pos[i] = ok ? __ldcg(ep.row_pos + rows[i]) : -1;
-            slot[i] = (ok && head >= ep.H) ? __ldcg(ep.row_slot + rows[i]) : 0;
-            cs[i] = (ok && rot) ? __ldcg(ep.rcos + (size_t)rows[i] * half + e) : 1.f;     // per-row rotary factors (the row's position applied)
-            sn[i] = (ok && rot) ? __ldcg(ep.rsin + (size_t)rows[i] * half + e) : 0.f;
-        }
     }
     float v[MB];
 #pragma unroll
