@@ -36,7 +36,7 @@ constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
 constexpr int RING_BYTES = 198 * 1024;          // stage ring of a CTA; the rest of the SM's shared memory is left to the fused-step CTAs
 constexpr int GEMM_PREFILL_BYTES = 120 * 1024;  // bytes per SM requested while the previous kernel is still at work (see the weight producer)
-constexpr int GEMM_STEADY_BYTES = 112 * 1024;   // bytes per SM kept in flight once the ring has been filled
+constexpr int GEMM_STEADY_BYTES = 160 * 1024;   // bytes per SM kept in flight once the ring has been filled (measured best: 9 of 11 stages at 16 rows)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -121,8 +121,8 @@ struct Shared {
 
 // Ring bookkeeping.  The first `stages` loads of a CTA fill the whole ring (run-ahead while the
 // consumers wait for the previous kernel); after that only the first `steady` stages are reused,
-// which keeps fewer loads in flight: the same bandwidth with a shorter queue, so the last tile
-// arrives sooner after it is requested.  use = how often the stage was used before this load.
+// which keeps somewhat fewer loads in flight: the same bandwidth with a shorter queue, so the last
+// tile arrives sooner after it is requested.  use = how often the stage was used before this load.
 struct RingPos {
     int stage; uint32_t use; int filled;
     __device__ __forceinline__ RingPos() : stage(0), use(0u), filled(0) {}
