@@ -278,7 +278,6 @@ def run_gpu(args):
                 "algorithmic_bytes_per_launch": weight_bytes / n_gemm, "launches_per_step": n_gemm,
                 "algorithmic_bytes_per_step": weight_bytes,
                 "overlapped": {"kernel_share_of_split": gemm_share, "kernel_ms_in_step": in_step_ms,
-                               "gbs": weight_bytes / (in_step_ms * 1e-3) / 1e9, "frac": weight_bytes / (in_step_ms * 1e-3) / 1e9 / peak,
                                # the same bytes over the GEMMs plus the small kernels that sum their pieces and apply the step after them
                                "with_fused_steps": {"ms_in_step": pair_ms, "gbs": weight_bytes / (pair_ms * 1e-3) / 1e9,
                                                     "frac": weight_bytes / (pair_ms * 1e-3) / 1e9 / peak}},
