@@ -235,6 +235,42 @@ def test_batched_ragged_sequences_match_single_sequence_runs(sd):
     ctx.close()
 
 
+def test_batch16_launch_configuration_at_full_width(sd):
+    """The batched benchmark's launch configuration (16 sequences x (gamma + 1) = 96 verify rows in one call: wide-N
+    GEMMs, fused steps in several row batches, the several-CTAs-per-SM form of attention, ragged contexts) at the
+    7B width, with one layer and short prompts so that the oracle finishes in seconds."""
+    cfg = synth.CONFIGS["7b_batch16"]
+    wl = cfg["workload"]
+    t = dict(cfg["target"], n_layers=1)
+    d = dict(cfg["drafts"][0], n_layers=1)
+    gamma, T, seed, B = wl["gamma"], wl["temperature"], wl["seed"], 16
+    ctx, om = _build(sd, t, [d], "bf16", T, seed, max_seqs=B, max_ctx=48, max_gamma=gamma)
+    V = t["vocab"]
+    prompts = [synth.make_prompt(V, 6 + (5 * i) % 15, seed=wl["seed"], seq=i) for i in range(B)]
+    traces = []
+    for i, p in enumerate(prompts):
+        _, _, tr = oracle.spec_decode(om[0], om[1], p, gamma + 1, gamma, T, seed, seq_id=200 + i,
+                                      trace_iters=1, trace_probs=True, trace_logits=True)
+        traces.append(tr)
+        ctx.sd_seq_begin(i, p, 200 + i)
+    seqs = list(range(B))
+    ctx.sd_route_prompt(seqs, forced_task=[0] * B)
+    ctx.sd_prefill(seqs)
+    x = torch.from_numpy(np.stack([traces[s]["x"][0] for s in seqs])).to(DEV)
+    xs = torch.zeros((B, gamma), dtype=torch.int32, device=DEV)
+    q = torch.zeros((B, gamma, V), dtype=torch.float32, device=DEV)
+    logits = torch.zeros((B, gamma + 1, V), dtype=torch.float32, device=DEV)
+    ctx.sd_draft_steps_replay(seqs, gamma, x, xs, q)
+    ctx.sd_verify(seqs, gamma, x, logits)
+    lg, qg = logits.cpu().numpy().astype(np.float64), q.cpu().numpy().astype(np.float64)
+    for b in seqs:
+        scale = max(1.0, float(np.std(traces[b]["logits"][0])))     # as in _replay: bf16 rounding is relative
+        assert np.abs(lg[b] - traces[b]["logits"][0]).max() <= TOL["bf16"]["logits"] * scale, b
+        assert np.abs(qg[b] - traces[b]["q"][0]).max() <= TOL["bf16"]["probs"], b
+    assert ctx.sd_device_status() == 0
+    ctx.close()
+
+
 def test_route_prompt_classifier_matches_oracle(sd):
     cfg = synth.CONFIGS["tiny"]
     t, (d_in, d_h, K) = cfg["target"], cfg["classifier"]
