@@ -236,34 +236,45 @@ cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float*
 
 }  // namespace
 
+namespace {
+
+// Pieces per tile, at most: a tile's k blocks over the k blocks a CTA of the GEMM owns.
+int pieces_bound(const GemmGeom& g) {
+    const long long T = (long long)g.n_tiles * g.kb_per_tile;
+    const int per_cta = (int)std::max<long long>(1, T / g.grid);
+    return (g.kb_per_tile + per_cta - 1) / per_cta + 1;
+}
+
+// Token rows per CTA of the form launch_fused_step picks.
+int rows_per_cta(int n_rows, int pieces) { return n_rows <= 2 ? 2 : (n_rows > 8 && pieces <= 4 ? 16 : 8); }
+
+}  // namespace
+
 bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
     // One batch of rows per tile (several would share a tile's word).  With one or two rows (draft and plain
     // decoding steps: small matrices, kernels of several GEMMs resident and polling at once) waiting for the
     // grid measured faster.
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
-    return n_rows > 2 && n_rows <= 8;
+    return g.grid >= 1 && n_rows > 2 && n_rows <= rows_per_cta(n_rows, pieces_bound(g));
 }
 
 cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status,
                               int dependent, cudaStream_t st) {
-    if (!fused_step_polls(g, ep)) arrive = nullptr;
     if (g.grid < 1 || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
+    if (!fused_step_polls(g, ep)) arrive = nullptr;
     if (ep.mode == EPI_QKV_ROPE && (128 % ep.hd)) return cudaErrorInvalidValue;            // a head must not straddle two tiles
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
     if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
-    // pieces per tile, at most: a tile's k blocks over the k blocks a CTA owns
-    const long long T = (long long)g.n_tiles * g.kb_per_tile;
-    const int per_cta = (int)std::max<long long>(1, T / g.grid);
-    const int pieces = (g.kb_per_tile + per_cta - 1) / per_cta + 1;
+    const int pieces = pieces_bound(g);
     if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
     if (n_rows > 8 && pieces <= 4) {
         switch (ep.mode) {
-        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
-        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
-        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
-        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, nullptr, status, n_rows, pieces, dependent, st);
+        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
         default: return cudaErrorInvalidValue;
         }
     }
