@@ -21,6 +21,7 @@ namespace {
 constexpr int WARPS_FEW = 8, WARPS_MANY = 4;
 constexpr int NQ = 16;              // query vectors per CTA (rows in the block x heads per KV head): one MMA row tile
 constexpr int SLICE_KEYS = 1024;    // a slice of the cache per CTA: up to this many positions
+constexpr int SLICE_KEYS_MANY = 2048; // ... when there are several CTAs per SM anyway (fewer set-ups and merges; 512...8192 swept)
 constexpr size_t ATTN_COUNTER_BYTES = 65536;     // one arrival counter per (query block, kv head)
 
 struct AttnParams {
@@ -462,14 +463,17 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
     const int n_blocks = (n_rows / rows_per_seq) * bps;
     // one slice while the context is short (no cross-CTA merge at all), SLICE_KEYS positions per slice beyond
     P.n_splits = std::max(1, std::min(32, (ctx_bound + SLICE_KEYS - 1) / SLICE_KEYS));
+    int sm = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
+    if (P.n_splits * Hkv * n_blocks > 2 * sm) {
+        P.n_splits = std::max(1, std::min(32, (ctx_bound + SLICE_KEYS_MANY - 1) / SLICE_KEYS_MANY));
+    }
     const size_t need = ATTN_COUNTER_BYTES + sizeof(float) * (size_t)n_rows * H * P.n_splits * (hd + 2);
     if (need > workspace_bytes || (size_t)n_blocks * Hkv * sizeof(uint32_t) > ATTN_COUNTER_BYTES) return cudaErrorInvalidValue;
     P.counters = (uint32_t*)workspace;
     P.part_o = (float*)((char*)workspace + ATTN_COUNTER_BYTES);
     P.part_ml = P.part_o + (size_t)n_rows * H * P.n_splits * hd;
     // few (head, row block, slice) items: two or four CTAs of a cluster share each of them
-    int sm = 148;
-    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev); }
     const int items = P.n_splits * Hkv * n_blocks;
     P.csize = items * 4 <= sm ? 4 : (items * 2 <= sm ? 2 : 1);
     const int nw = items > 2 * sm ? WARPS_MANY : WARPS_FEW;

@@ -64,6 +64,7 @@ ATTN_CASES = [  # H, Hkv, hd, max_ctx, positions of the rows
     # many (head, row, slice) items: several CTAs per SM, the four-warp form of the kernel (single slice, and merged slices)
     (32, 32, 128, 700, [0, 63, 64, 127, 128, 300, 511, 640, 698, 699]),
     (16, 16, 64, 2100, [2099, 1024, 1023, 17, 2048, 700, 1500]),
+    (32, 32, 64, 4200, [4199, 2048, 2047, 17, 4096, 700, 3000, 1]),      # four-warp form with three merged slices
 ]
 
 
