@@ -19,11 +19,6 @@ namespace {
 
 constexpr int TILE_N = 128;
 
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 
 template <int MB>
 struct StepShared {
@@ -84,11 +79,11 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         if (et == 0) {
             const uint32_t need = i_last - i_first + 1u;
             uint32_t seen = 0;
-            const uint64_t t0 = global_timer_ns();
+            const uint64_t t0 = global_ns();
             for (uint32_t spin = 0;; ++spin) {
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrive + tile) : "memory");
                 if (seen >= need) break;
-                if ((spin & 63u) == 63u && global_timer_ns() - t0 > 200000000ull) break;      // 0.2 s: give up polling
+                if ((spin & 63u) == 63u && global_ns() - t0 > 200000000ull) break;      // 0.2 s: give up polling
             }
             tile_seen = seen >= need;
         }
