@@ -231,6 +231,32 @@ sd_status sd_use_graphs(sd_ctx* ctx, int on);
  * plain CUDA-core kernels instead (the two paths check each other in the tests). */
 sd_status sd_force_plain_path(sd_ctx* ctx, int on);
 
+/* Forward passes over few query rows (the verify rows of Fig. 1(b), a decoding row) run by default as ONE launch of a
+ * persistent kernel that streams every weight matrix of every layer through the SMs without stopping at matrix
+ * boundaries; passes with more rows run one kernel per matrix.  target_on / drafts_on switch that kernel on or off
+ * for the target and for the draft models (defaults: on, off); max_rows > 0 sets the largest pass it takes (default
+ * 16, at most 32).  The two paths check each other in the tests. */
+sd_status sd_use_pass_kernel(sd_ctx* ctx, int target_on, int drafts_on, int max_rows);
+
+/* Schedule of that kernel, for measurements: waves[5] = tile waves of the QKV, Wo, gate/up, down and lm_head matrices
+ * (1..8), chunk_major[5] = order of a matrix's (wave, chunk) blocks (0: wave after wave).  NULL waves restores the
+ * defaults.  Drops cached programs and graphs.  Synchronises. */
+sd_status sd_pass_tuning(sd_ctx* ctx, const int32_t* waves, const int32_t* chunk_major);
+
+/* Time stamps of the persistent kernel's passes from now on (NULL: none): stamps_dev is a device buffer of n_words
+ * 64-bit words; CTA b writes, for segment s of iteration it (layers, then the lm_head), the global-timer nanoseconds
+ * at which its MMA thread turned to the segment and at which the segment was committed, at
+ * ((b * n_iterations + it) * max_segments + s) * 2.  Passes whose stamps would not fit write none.  Synchronises. */
+sd_status sd_pass_stamps(sd_ctx* ctx, unsigned long long* stamps_dev, size_t n_words);
+
+/* Builds and replays on the host the schedule of that kernel for a shape (no GPU needed): shape12 = n_layers, d_model,
+ * n_heads, n_kv_heads, head_dim, d_ffn, vocab, rows, rows_per_seq, cache slices, want_logits, CTAs.  info8 receives
+ * words per layer, total words, workspace slots of the two regions, most segments of a CTA per layer, largest CTA
+ * section in bytes, program bytes, 16 KB weight blocks per layer.  SD_ERR_UNSUPPORTED with a message in err when the
+ * shape does not fit or the replay finds a wait that could never be satisfied. */
+sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, int32_t* info8,
+                                 char* err, size_t err_cap);
+
 /* Number of kernels this context has launched since sd_create. */
 sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);
 

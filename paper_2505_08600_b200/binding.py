@@ -69,6 +69,10 @@ _PROTOS = {
     "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_use_graphs": (_i, [_vp, _i]),
+    "sd_use_pass_kernel": (_i, [_vp, _i, _i, _i]),
+    "sd_pass_tuning": (_i, [_vp, _vp, _vp]),
+    "sd_pass_stamps": (_i, [_vp, _vp, _sz]),
+    "sd_pass_schedule_check": (_i, [_vp, _vp, _vp, _vp, C.c_char_p, _sz]),
     "sd_force_plain_path": (_i, [_vp, _i]),
     "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
     "sd_profile": (_i, [_vp, _i]),
@@ -102,6 +106,20 @@ def lib():
             fn.restype, fn.argtypes = res, args
         _lib = L
     return _lib
+
+
+def sd_pass_schedule_check(dims, rows, rows_per_seq, n_splits, want_logits=1, grid=148, waves=None, chunk_major=None):
+    """Builds and replays the persistent kernel's schedule on the host; returns (status, info dict, message)."""
+    shape = np.array([dims["n_layers"], dims["d_model"], dims["n_heads"], dims["n_kv_heads"], dims["head_dim"], dims["d_ffn"],
+                      dims["vocab"], rows, rows_per_seq, n_splits, want_logits, grid], dtype=np.int32)
+    info = np.zeros(8, dtype=np.int32)
+    err = C.create_string_buffer(256)
+    w = np.ascontiguousarray(waves, dtype=np.int32) if waves is not None else None
+    cm = np.ascontiguousarray(chunk_major, dtype=np.int32) if chunk_major is not None else None
+    st = lib().sd_pass_schedule_check(shape.ctypes.data_as(C.c_void_p), w.ctypes.data_as(C.c_void_p) if w is not None else None,
+                                      cm.ctypes.data_as(C.c_void_p) if cm is not None else None, info.ctypes.data_as(C.c_void_p), err, 256)
+    names = ("words_per_layer", "total_words", "slots0", "slots1", "max_seg", "max_section", "program_bytes", "units_per_layer")
+    return st, dict(zip(names, info.tolist())), err.value.decode()
 
 
 def exported_symbols():
@@ -248,6 +266,20 @@ class Context:
 
     def sd_use_graphs(self, on):
         _check(self.L.sd_use_graphs(self.h, int(on)), "sd_use_graphs")
+
+    def sd_use_pass_kernel(self, target_on, drafts_on=0, max_rows=0):
+        _check(self.L.sd_use_pass_kernel(self.h, int(target_on), int(drafts_on), int(max_rows)), "sd_use_pass_kernel")
+
+    def sd_pass_tuning(self, waves=None, chunk_major=None):
+        w = np.ascontiguousarray(waves, dtype=np.int32) if waves is not None else None
+        cm = np.ascontiguousarray(chunk_major, dtype=np.int32) if chunk_major is not None else None
+        _check(self.L.sd_pass_tuning(self.h, w.ctypes.data_as(C.c_void_p) if w is not None else None,
+                                     cm.ctypes.data_as(C.c_void_p) if cm is not None else None), "sd_pass_tuning")
+
+    def sd_pass_stamps(self, stamps):
+        """stamps: int64 device tensor or None."""
+        self._stamps = stamps
+        _check(self.L.sd_pass_stamps(self.h, _dp(stamps), 0 if stamps is None else stamps.numel()), "sd_pass_stamps")
 
     def sd_force_plain_path(self, on):
         _check(self.L.sd_force_plain_path(self.h, int(on)), "sd_force_plain_path")

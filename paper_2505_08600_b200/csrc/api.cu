@@ -9,6 +9,7 @@
 
 #include "gemm_tc.h"
 #include "kernels.h"
+#include "pass_stream.h"
 
 using namespace sd;
 
@@ -49,6 +50,8 @@ struct Model {
     float* rope_sin;
     TensorMap tm_lm;
     bool tc;                        // the tensor-core path applies (bf16, shapes fit)
+    PassMaps pmaps;                 // the layers' matrices as [layer][row][k] tensor maps (persistent streaming kernel)
+    bool pass_ok;                   // ... which applies to this model
     int n_qkv() const { return (d.n_heads + 2 * d.n_kv_heads) * d.head_dim; }
 };
 
@@ -57,6 +60,10 @@ enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
 }  // namespace
 
 constexpr size_t ARRIVE_WORDS = 65536;          // arrival words of one pass (the 13B target needs about 17,000)
+constexpr int PASS_ROWS_CAP = 32;               // most query rows of a pass on the persistent streaming kernel
+constexpr size_t PASS_REGION_BYTES = (size_t)48 << 20;      // each of the two workspace regions of that kernel
+constexpr size_t PASS_PROG_BYTES = (size_t)768 << 10;       // one cached program
+constexpr int PASS_PROG_SLOTS = 8;
 
 struct sd_ctx {
     sd_config cfg;
@@ -72,6 +79,18 @@ struct sd_ctx {
     uint32_t* gemm_arrive;                      // per GEMM of a pass and output tile: pieces that have arrived (zero between passes)
     size_t arrive_used;                         // words handed out to the GEMMs of the pass being enqueued
     float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
+    // persistent streaming kernel (pass_stream.cu): packed input rows, workspace, programs
+    uint8_t* xp_xn; uint8_t* xp_attn; uint8_t* xp_act;
+    float* pass_partials[2];
+    uint8_t* pass_prog;
+    uint32_t* pass_sync;                        // the kernel's arrival / completion words (cleared at the start of every pass)
+    float* pass_part_o; float* pass_part_ml; uint32_t* pass_att_counters;
+    size_t pass_att_counter_words;
+    bool pass_on, pass_drafts; int pass_max_rows;
+    PassTuning pass_tuning; bool pass_tuned;
+    struct CachedProgram { int model, m_tok, rows_per_seq, n_splits, want_logits, slot; PassProgram meta; uint64_t last_use; };
+    std::vector<CachedProgram> programs;
+    unsigned long long* stamps; size_t stamps_words;          // optional time stamps of the next passes (caller's buffer)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
     struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
@@ -208,6 +227,22 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
     c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
     c->rope_row_sin = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
+    {   // persistent streaming kernel: input rows in the packed layout ([k block][row][64], up to PASS_ROWS_CAP rows padded to 16)
+        const size_t rows_pad = (PASS_ROWS_CAP + 15) & ~15;
+        c->xp_xn = (uint8_t*)B.take((size_t)((d_max + 63) / 64) * rows_pad * 128);
+        c->xp_attn = (uint8_t*)B.take((size_t)((dq_max + 63) / 64) * rows_pad * 128);
+        c->xp_act = (uint8_t*)B.take((size_t)((f_max + 63) / 64) * rows_pad * 128);
+        c->pass_partials[0] = (float*)B.take(PASS_REGION_BYTES);
+        c->pass_partials[1] = (float*)B.take(PASS_REGION_BYTES);
+        c->pass_prog = (uint8_t*)B.take(PASS_PROG_BYTES * PASS_PROG_SLOTS);
+        c->pass_sync = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
+        int h_max = 1, hd_max = 8;
+        for (int i = 0; i < nm; ++i) { h_max = std::max(h_max, (int)ms[i].n_heads); hd_max = std::max(hd_max, (int)ms[i].head_dim); }
+        c->pass_part_o = (float*)B.take(sizeof(float) * (size_t)PASS_ROWS_CAP * h_max * 32 * hd_max);
+        c->pass_part_ml = (float*)B.take(sizeof(float) * (size_t)PASS_ROWS_CAP * h_max * 32 * 2);
+        c->pass_att_counter_words = (size_t)PASS_ROWS_CAP * h_max;
+        c->pass_att_counters = (uint32_t*)B.take(sizeof(uint32_t) * c->pass_att_counter_words);
+    }
     const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
@@ -273,13 +308,92 @@ enum LogitsMode { LOGITS_NONE = 0, LOGITS_ALL = 1, LOGITS_LAST = 2 };
 // One pass of a model over n_rows query rows described by `plan`.
 sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out);
 
+sd_ctx::CachedProgram* find_program(sd_ctx* c, int model, int m_tok, int rows_per_seq, int n_splits, int want_logits) {
+    for (auto& p : c->programs)
+        if (p.model == model && p.m_tok == m_tok && p.rows_per_seq == rows_per_seq && p.n_splits == n_splits && p.want_logits == want_logits) return &p;
+    return nullptr;
+}
+
+// Slices of the cache per (query block, kv head) on the persistent kernel: about one attention item per SM, slices
+// of at most 2048 positions.
+int pass_splits(const sd_model_desc& m, int n_rows, int rows_per_seq, int ctx_bound) {
+    const int grp = m.n_heads / m.n_kv_heads;
+    const int rpb = std::max(1, std::min(rows_per_seq, 16 / std::max(1, grp)));
+    const int n_blocks = (n_rows / rows_per_seq) * ((rows_per_seq + rpb - 1) / rpb);
+    int ns = std::max(1, sm_count() / std::max(1, n_blocks * m.n_kv_heads));
+    ns = std::min(ns, std::max(1, ctx_bound / 64));                        // a slice is worth at least one chunk of keys
+    ns = std::max(ns, (ctx_bound + 2047) / 2048);
+    return std::max(1, std::min(32, ns));
+}
+
+bool pass_wanted(sd_ctx* c, const Model& M, const RowPlan& plan, int n_rows) {
+    return c->pass_on && (&M == &c->models[0] || c->pass_drafts) && M.tc && M.pass_ok && !c->force_plain && n_rows <= c->pass_max_rows && n_rows <= PASS_ROWS_CAP &&
+           plan.rows_per_seq >= 1 && n_rows % plan.rows_per_seq == 0;
+}
+
+// Makes sure the program of a pass is built and in device memory.  Called by the entry points before anything is
+// captured into a graph (the upload is an ordinary copy followed by a synchronisation).
+sd_status prepare_pass(sd_ctx* c, int model, const RowPlan& plan, int n_rows, int mode) {
+    Model& M = c->models[model];
+    if (!pass_wanted(c, M, plan, n_rows)) return SD_OK;
+    const sd_model_desc& m = M.d;
+    const int ns = pass_splits(m, n_rows, plan.rows_per_seq, plan.ctx_bound), want = mode != 0 ? 1 : 0;
+    c->graph_clock += 1;
+    if (sd_ctx::CachedProgram* p = find_program(c, model, n_rows, plan.rows_per_seq, ns, want)) { p->last_use = c->graph_clock; return SD_OK; }
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(c->st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return SD_ERR_STATE;
+    PassShape sh{m.n_layers, m.d_model, m.n_heads, m.n_kv_heads, m.head_dim, m.d_ffn, m.vocab, n_rows, plan.rows_per_seq, ns, want, sm_count()};
+    sd_ctx::CachedProgram cp;
+    cp.model = model; cp.m_tok = n_rows; cp.rows_per_seq = plan.rows_per_seq; cp.n_splits = ns; cp.want_logits = want; cp.last_use = c->graph_clock;
+    cp.meta = build_pass_program(sh, c->pass_tuned ? c->pass_tuning : default_pass_tuning(sh));
+    const bool fits = cp.meta.error.empty() && cp.meta.blob.size() <= PASS_PROG_BYTES && cp.meta.max_section <= 8192 &&
+                      (size_t)cp.meta.total_words + 2 <= ARRIVE_WORDS &&
+                      (size_t)std::max(cp.meta.slots[0], cp.meta.slots[1]) * n_rows * 128 * sizeof(float) <= PASS_REGION_BYTES &&
+                      (size_t)cp.meta.n_blocks * m.n_kv_heads <= (size_t)PASS_ROWS_CAP * m.n_heads;
+    if (!fits) {                                      // remembered, so that the pass quietly takes the kernel-per-matrix path
+        cp.slot = -1; cp.meta.blob.clear();
+        c->programs.push_back(cp);
+        return SD_OK;
+    }
+    int slot = -1;
+    std::vector<bool> used(PASS_PROG_SLOTS, false);
+    for (auto& p : c->programs) if (p.slot >= 0) used[p.slot] = true;
+    for (int i = 0; i < PASS_PROG_SLOTS; ++i) if (!used[i]) { slot = i; break; }
+    if (slot < 0) {
+        // every slot is taken: drop the least recently used program, and the graphs that may have captured its address
+        size_t victim = c->programs.size();
+        for (size_t i = 0; i < c->programs.size(); ++i)
+            if (c->programs[i].slot >= 0 && (victim == c->programs.size() || c->programs[i].last_use < c->programs[victim].last_use)) victim = i;
+        CUDA_TRY(cudaStreamSynchronize(c->st));
+        for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
+        c->graphs.clear();
+        slot = c->programs[victim].slot;
+        c->programs.erase(c->programs.begin() + victim);
+    }
+    cp.slot = slot;
+    CUDA_TRY(cudaMemcpyAsync(c->pass_prog + (size_t)slot * PASS_PROG_BYTES, cp.meta.blob.data(), cp.meta.blob.size(), cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    cp.meta.blob.clear(); cp.meta.blob.shrink_to_fit();
+    c->programs.push_back(cp);
+    return SD_OK;
+}
+
+sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, const SeqList& list, const RowPlan& plan, int n_rows, int mode,
+                       float* logits_out);
+
 sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out) {
+    if (pass_wanted(c, M, plan, n_rows)) {
+        const int model = (int)(&M - &c->models[0]);
+        SD_TRY(prepare_pass(c, model, plan, n_rows, mode));
+        const sd_ctx::CachedProgram* cp = find_program(c, model, n_rows, plan.rows_per_seq, pass_splits(M.d, n_rows, plan.rows_per_seq, plan.ctx_bound), mode != 0 ? 1 : 0);
+        if (cp && cp->slot >= 0) return forward_pass(c, M, *cp, list, plan, n_rows, mode, logits_out);
+    }
     if (M.tc && !c->force_plain) return forward_tc(c, M, list, plan, n_rows, mode, logits_out);
     const sd_model_desc& m = M.d;
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, st));
+                                         nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -337,7 +451,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, st));
+                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, 0, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -371,6 +485,47 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         else { e.n_out_rows = list.n; e.row_stride = R; e.row_offset = R - 1; }
         SD_TRY(gemm_tc(c, M.tm_lm, c->xn, n_rows, m.vocab, d, e));
     }
+    CUDA_TRY(prof_mark(c, CAT_NONE));
+    return SD_OK;
+}
+
+// The same pass as one launch of the persistent streaming kernel (few query rows): the embedding kernel writes the first
+// input rows in the packed layout, then every layer and the lm_head run inside k_pass_stream.
+sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, const SeqList& list, const RowPlan& plan, int n_rows, int mode,
+                       float* logits_out) {
+    const sd_model_desc& m = M.d;
+    const int d = m.d_model, hd = m.head_dim;
+    cudaStream_t st = c->st;
+    PassParams P;
+    memset(&P, 0, sizeof(P));
+    P.m_tok = n_rows; P.m_pad = (n_rows + 15) & ~15; P.n_layers = m.n_layers; P.has_tail = mode != LOGITS_NONE ? 1 : 0;
+    P.d = d; P.H = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = hd; P.F = m.d_ffn; P.V = m.vocab; P.max_ctx = c->cfg.max_ctx;
+    P.n_out[MAT_QKV] = M.n_qkv(); P.n_out[MAT_WO] = d; P.n_out[MAT_GU] = 2 * m.d_ffn; P.n_out[MAT_DN] = d; P.n_out[MAT_LM] = m.vocab;
+    (void)pass_stream_smem(P.m_pad, &P.stages);
+    P.words_per_layer = cp.meta.words_per_layer;
+    P.h = c->h; P.xn = c->xp_xn; P.attn = c->xp_attn; P.act = c->xp_act;
+    P.x[MAT_QKV] = c->xp_xn; P.x[MAT_WO] = c->xp_attn; P.x[MAT_GU] = c->xp_xn; P.x[MAT_DN] = c->xp_act; P.x[MAT_LM] = c->xp_xn;
+    P.q = (bf16*)c->q; P.kc = (bf16*)M.kcache; P.vc = (bf16*)M.vcache; P.kv_layer_elems = M.kv_layer_bytes / sizeof(bf16);
+    P.row_slot = c->row_slot; P.row_pos = c->row_pos; P.rcos = c->rope_row_cos; P.rsin = c->rope_row_sin; P.ssq = c->ssq;
+    P.norm1 = M.layers[0].norm1; P.norm2 = M.layers[0].norm2;
+    P.norm_stride = m.n_layers > 1 ? (size_t)(M.layers[1].norm1 - M.layers[0].norm1) : 0;
+    P.final_norm = M.final_norm; P.rms_eps = m.rms_eps;
+    P.logits = logits_out;
+    const int R = plan.rows_per_seq;
+    if (mode == LOGITS_LAST) { P.logits_rows = list.n; P.row_stride = R; P.row_offset = R - 1; }
+    else { P.logits_rows = n_rows; P.row_stride = 1; P.row_offset = 0; }
+    P.partials[0] = c->pass_partials[0]; P.partials[1] = c->pass_partials[1];
+    P.sync = c->pass_sync; P.abort_word = c->pass_sync + cp.meta.total_words; P.status = c->S.status;
+    P.program = c->pass_prog + (size_t)cp.slot * PASS_PROG_BYTES;
+    P.rows_per_seq = R; P.rows_per_block = cp.meta.rows_per_block; P.n_splits = cp.n_splits;
+    P.part_o = c->pass_part_o; P.part_ml = c->pass_part_ml; P.att_counters = c->pass_att_counters;
+    const int n_it = m.n_layers + P.has_tail;
+    if (c->stamps && (size_t)sm_count() * n_it * cp.meta.max_seg * 2 <= c->stamps_words) { P.stamps = c->stamps; P.stamp_segs = cp.meta.max_seg; }
+    CUDA_TRY(prof_mark(c, CAT_STATE));
+    CUDA_TRY(cudaMemsetAsync(c->pass_sync, 0, sizeof(uint32_t) * ((size_t)cp.meta.total_words + 1), st));
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, m.dtype, d, m.vocab, c->h, c->row_slot, c->row_pos,
+                                         M.layers[0].norm1, c->xp_xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, P.m_pad, st));
+    LAUNCH(CAT_LINEAR, launch_pass_stream(M.pmaps, P, sm_count(), 1, st));
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
 }
@@ -517,11 +672,17 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         cudaMemsetAsync(c->gemm_arrive, 0, sizeof(uint32_t) * ARRIVE_WORDS, st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
+    if (cudaMemsetAsync(c->xp_xn, 0, (char*)c->pass_partials[0] - (char*)c->xp_xn, st) != cudaSuccess ||
+        cudaMemsetAsync(c->pass_att_counters, 0, sizeof(uint32_t) * c->pass_att_counter_words, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return fail(SD_ERR_CUDA);
+    c->pass_on = true; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->stamps = nullptr; c->stamps_words = 0;
     c->force_plain = false;
     c->graphs_on = true;
     c->graph_clock = 0;
     for (Model& M : c->models) {
         const sd_model_desc& m = M.d;
+        M.pass_ok = false;
         M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE && m.d_ffn % 64 == 0 &&
                attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim);
         if (!M.tc) continue;
@@ -534,6 +695,17 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
             ok = ok && make_tensor_map_bf16(&L.tm_wd, L.wd, m.d_model, m.d_ffn, 128);
         }
         if (!ok) return fail(SD_ERR_CUDA);
+        // the persistent streaming kernel sees the layers of a matrix as one [layer][row][k] tensor
+        const size_t stride = m.n_layers > 1 ? (size_t)((char*)M.layers[1].wqkv - (char*)M.layers[0].wqkv) : 0;
+        M.pass_ok = m.d_model % 64 == 0 && dq % 64 == 0 && m.d_ffn % 64 == 0 &&
+                    make_tensor_map_layers(&M.pmaps.m[MAT_QKV], M.layers[0].wqkv, M.n_qkv(), m.d_model, m.n_layers, stride) &&
+                    make_tensor_map_layers(&M.pmaps.m[MAT_WO], M.layers[0].wo, m.d_model, dq, m.n_layers, stride) &&
+                    make_tensor_map_layers(&M.pmaps.m[MAT_GU], M.layers[0].wgu, 2 * m.d_ffn, m.d_model, m.n_layers, stride) &&
+                    make_tensor_map_layers(&M.pmaps.m[MAT_DN], M.layers[0].wd, m.d_model, m.d_ffn, m.n_layers, stride) &&
+                    make_tensor_map_layers(&M.pmaps.m[MAT_LM], M.lm_head, m.vocab, m.d_model, 1, 0);
+        for (int l = 1; l < m.n_layers && M.pass_ok; ++l)         // every layer at the same distance from the one before
+            M.pass_ok = (size_t)((char*)M.layers[l].wqkv - (char*)M.layers[l - 1].wqkv) == stride &&
+                        (size_t)((char*)M.layers[l].norm1 - (char*)M.layers[l - 1].norm1) == stride;
     }
     *out = c;
     return SD_OK;
@@ -685,9 +857,18 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     KeyBuilder key;
-    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain);
+    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows);
     for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
     bound = bound_bucket(bound + gamma) - gamma;
+    for (int k = 0; k < c->cfg.n_drafts; ++k) {             // programs of the persistent kernel exist before anything is captured
+        int n = 0;
+        for (int i = 0; i < n_seq; ++i) n += c->draft_id[seqs[i]] == k;
+        if (n == 0) continue;
+        for (int s = 0; s < gamma; ++s) {
+            if (s == 0) { RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_in, bound}; SD_TRY(prepare_pass(c, 1 + k, plan, 2 * n, LOGITS_LAST)); }
+            else { RowPlan plan{PLAN_DRAFT_NEXT, 1, 0, s, gamma, x_in, bound + s}; SD_TRY(prepare_pass(c, 1 + k, plan, n, LOGITS_ALL)); }
+        }
+    }
     return run_graphed(c, key, [&]() -> sd_status {
     for (int k = 0; k < c->cfg.n_drafts; ++k) {             // sequences grouped per routed draft
         SeqList g = all;
@@ -722,7 +903,8 @@ sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const 
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
     RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound_bucket(bound)};
     KeyBuilder key;
-    key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain);
+    key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
+    SD_TRY(prepare_pass(c, 0, plan, n_seq * (gamma + 1), LOGITS_ALL));
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev); });
 }
 
@@ -736,7 +918,8 @@ sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logit
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr, bound_bucket(bound)};
     KeyBuilder key;
-    key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain);
+    key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
+    SD_TRY(prepare_pass(c, 0, plan, n_seq, LOGITS_ALL));
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev); });
 }
 
@@ -819,10 +1002,22 @@ sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma,
     if (!c || !seqs || !logits_dev || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
     const bool saved = c->graphs_on;
     KeyBuilder key;
-    key.add(4).add_list(seqs, n_seq).add(gamma).add(x_dev).add(q_dev).add(logits_dev).add(n_acc_dev).add(out_tok_dev).add(c->force_plain);
+    // argument and capacity checks run on every call, captured or replayed, and before anything reads the lists
+    if (n_seq < 1 || n_seq > SD_MAX_BATCH || gamma < 0 || gamma > c->cfg.max_gamma || n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i];
+        if (s < 0 || s >= c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
+        if (c->phase[s] < PH_READY) return SD_ERR_STATE;
+        if (c->len_ub[s] + gamma + 1 > c->S.tok_stride || c->len_ub[s] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
+    }
+    key.add(4).add_list(seqs, n_seq).add(gamma).add(x_dev).add(q_dev).add(logits_dev).add(n_acc_dev).add(out_tok_dev).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
     int bound = 0;
-    for (int i = 0; i < n_seq && seqs[i] >= 0 && seqs[i] < c->cfg.max_seqs; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
+    for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
     key.add(bound_bucket(bound));
+    {
+        RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound_bucket(bound)};
+        SD_TRY(prepare_pass(c, 0, plan, n_seq * (gamma + 1), LOGITS_ALL));
+    }
     std::vector<int> ub(c->len_ub);
     auto body = [&]() -> sd_status {
         c->graphs_on = false;                    // the three calls below must launch into this capture, not replay their own graphs
@@ -832,14 +1027,6 @@ sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma,
         c->graphs_on = saved;
         return s;
     };
-    // argument and capacity checks must run on every call, captured or replayed
-    if (n_seq < 1 || n_seq > SD_MAX_BATCH || gamma < 0 || gamma > c->cfg.max_gamma || n_seq * (gamma + 1) > SD_MAX_ROWS) return SD_ERR_INVALID_ARG;
-    for (int i = 0; i < n_seq; ++i) {
-        const int s = seqs[i];
-        if (s < 0 || s >= c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
-        if (c->phase[s] < PH_READY) return SD_ERR_STATE;
-        if (c->len_ub[s] + gamma + 1 > c->S.tok_stride || c->len_ub[s] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
-    }
     const bool replay = saved && !c->prof_on;
     bool cached = false;
     if (replay) for (auto& g : c->graphs) cached |= g.key == key.bytes;
@@ -883,6 +1070,50 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out) {
         }
     if (speedup_out) *speedup_out = best_s;
     return best;
+}
+
+sd_status sd_use_pass_kernel(sd_ctx* c, int target_on, int drafts_on, int max_rows) {
+    if (!c || max_rows < 0 || max_rows > PASS_ROWS_CAP) return SD_ERR_INVALID_ARG;
+    c->pass_on = target_on != 0 || drafts_on != 0;
+    c->pass_drafts = drafts_on != 0;
+    if (max_rows > 0) c->pass_max_rows = max_rows;
+    return SD_OK;
+}
+
+sd_status sd_pass_tuning(sd_ctx* c, const int32_t* waves, const int32_t* chunk_major) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);        // programs and the graphs that captured them are rebuilt
+    c->graphs.clear();
+    c->programs.clear();
+    c->pass_tuned = waves != nullptr;
+    for (int m = 0; m < N_MAT && waves; ++m) {
+        if (waves[m] < 1 || waves[m] > PASS_MAX_WAVES) return SD_ERR_INVALID_ARG;
+        c->pass_tuning.waves[m] = waves[m];
+        c->pass_tuning.chunk_major[m] = chunk_major ? (chunk_major[m] != 0) : 0;
+    }
+    return SD_OK;
+}
+
+sd_status sd_pass_stamps(sd_ctx* c, unsigned long long* stamps_dev, size_t n_words) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);        // the buffer's address is a kernel argument
+    c->graphs.clear();
+    c->stamps = stamps_dev; c->stamps_words = stamps_dev ? n_words : 0;
+    return SD_OK;
+}
+
+sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, int32_t* info8, char* err, size_t err_cap) {
+    if (!shape12 || !info8) return SD_ERR_INVALID_ARG;
+    PassShape sh{shape12[0], shape12[1], shape12[2], shape12[3], shape12[4], shape12[5], shape12[6], shape12[7], shape12[8], shape12[9], shape12[10], shape12[11]};
+    PassTuning t = default_pass_tuning(sh);
+    for (int m = 0; m < N_MAT && waves; ++m) { t.waves[m] = waves[m]; t.chunk_major[m] = chunk_major ? chunk_major[m] : 0; }
+    const PassProgram p = build_pass_program(sh, t);
+    info8[0] = p.words_per_layer; info8[1] = p.total_words; info8[2] = p.slots[0]; info8[3] = p.slots[1];
+    info8[4] = p.max_seg; info8[5] = p.max_section; info8[6] = (int32_t)p.blob.size(); info8[7] = (int32_t)p.units_per_layer;
+    if (err && err_cap) { strncpy(err, p.error.c_str(), err_cap - 1); err[err_cap - 1] = 0; }
+    return p.error.empty() ? SD_OK : SD_ERR_UNSUPPORTED;
 }
 
 sd_status sd_use_graphs(sd_ctx* c, int on) {

@@ -1,6 +1,7 @@
 // Small memory-bound kernels around the GEMMs: token embedding + row planning, RMSNorm,
 // rotary embedding + KV append, residual add, SwiGLU, and the per-sequence state updates.
 #include "kernels.h"
+#include "pass_stream.h"
 
 namespace sd {
 
@@ -13,7 +14,7 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
                         float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos,
                         const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq,
                         const float* __restrict__ rcos, const float* __restrict__ rsin, int half,
-                        float* __restrict__ row_cos, float* __restrict__ row_sin) {
+                        float* __restrict__ row_cos, float* __restrict__ row_sin, int packed_m_pad) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const int i = r / plan.rows_per_seq, j = r % plan.rows_per_seq;
@@ -47,7 +48,12 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
     for (int k = threadIdx.x; k < d; k += blockDim.x) {
         const float v = to_f32<T>(e[k]);
         h[(size_t)r * d + k] = v;
-        if (gain) { xn[(size_t)r * d + k] = __float2bfloat16_rn(v * gain[k]); ss += v * v; }
+        if (gain) {
+            const bf16 g = __float2bfloat16_rn(v * gain[k]);
+            if (packed_m_pad) *reinterpret_cast<bf16*>(reinterpret_cast<uint8_t*>(xn) + xpacked_offset(r, k, packed_m_pad)) = g;   // layout of the streaming kernel's input rows
+            else xn[(size_t)r * d + k] = g;
+            ss += v * v;
+        }
     }
     if (gain) {                          // first half of the first layer's RMSNorm: the 1/rms factor follows the GEMM
         ss = block_sum(ss, red);
@@ -58,13 +64,14 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
 cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& plan, int n_rows,
                          const void* embed, int dtype, int d, int vocab,
                          float* h, int32_t* row_slot, int32_t* row_pos, const float* gain, void* xn, float* ssq,
-                         const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, cudaStream_t st) {
+                         const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, int packed_m_pad,
+                         cudaStream_t st) {
     if (dtype == SD_BF16)
         k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq,
-                                              rope_cos, rope_sin, half, row_cos, row_sin);
+                                              rope_cos, rope_sin, half, row_cos, row_sin, packed_m_pad);
     else
         k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr,
-                                               nullptr, nullptr, 0, nullptr, nullptr);
+                                               nullptr, nullptr, 0, nullptr, nullptr, 0);
     return cudaGetLastError();
 }
 

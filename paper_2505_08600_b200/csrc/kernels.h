@@ -12,7 +12,8 @@ cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& 
                          const float* gain /*nullable: also writes xn = bf16(h * gain) and ssq[row][0] = sum h^2*/,
                          void* xn, float* ssq,
                          const float* rope_cos, const float* rope_sin, int half,      // position tables [max_ctx][half]
-                         float* row_cos, float* row_sin /*nullable: [row][half] factors of each row's position*/, cudaStream_t st);
+                         float* row_cos, float* row_sin /*nullable: [row][half] factors of each row's position*/,
+                         int packed_m_pad /*0: xn is [row][d]; else xn is in the streaming kernel's packed layout for m_pad rows*/, cudaStream_t st);
 // xn[i] = rmsnorm(h[src_row(i)]) * gain; src_row(i) = i * row_stride + row_offset
 cudaError_t launch_rmsnorm(const float* h, const float* gain, void* xn, int dtype, int n_rows, int d, float eps,
                            int row_stride, int row_offset, cudaStream_t st);

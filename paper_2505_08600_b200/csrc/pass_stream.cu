@@ -1,0 +1,765 @@
+// Persistent streaming kernel: one launch runs every decoder layer and the lm_head of a forward pass over a
+// handful of query rows (the verify rows of Fig. 1(b), or one decoding row), one CTA per SM.
+//
+// The pass is bound by one read of every weight matrix from HBM, and between two matrices of a layer lies a
+// chain of small dependent steps (sum the split accumulators, normalise / rotate / gate, publish the next
+// matrix's input rows).  With a kernel per matrix that chain is paid at every boundary while HBM idles.  Here
+//   - every CTA streams its share of ALL matrices, layer after layer, through one ring of shared-memory stages
+//     (tcgen05.mma, bf16 in, fp32 accumulators in TMEM; weights by TMA, input rows by bulk copies);
+//   - a matrix is cut into tile waves x K chunks (pass_program.h): four spare warps per CTA sum the pieces of
+//     finished tiles and apply the step after the GEMM while later waves stream, and the next matrix starts on
+//     the chunk of its input that the first wave produced;
+//   - attention over the cache runs on the same spare warps, head by head, as soon as a head's query / key /
+//     value tiles are reduced; its output feeds the Wo GEMM chunk by chunk.
+// Readiness travels through counters in global memory (red.release / ld.acquire at GPU scope).  Every wait
+// is bounded: the first one that gives up raises a flag that winds the whole grid down, and the host sees
+// SD_DEV_WAIT_EXPIRED.
+// Warps: 0 weight producer, 1 MMA issuer, 2 input-row producer, 4..7 TMEM -> workspace, 8..11 tasks.
+#include <cuda.h>
+
+#include "pass_stream.h"
+#include "tc_ptx.cuh"
+
+namespace sd {
+
+namespace {
+
+constexpr int TILE_N = 128, TILE_K = 64, A_BYTES = TILE_N * TILE_K * 2;
+constexpr int NUM_THREADS = 384;
+constexpr int MAX_STAGES = 10;
+constexpr int PROG_BYTES = 8 * 1024;             // the CTA's section of the program
+constexpr int RING_BUDGET = 148 * 1024;
+constexpr int ATTN_BYTES = 64 * 1024;            // key / value chunks and merge buffers of the attention tasks
+constexpr int NQ = 16;                           // query vectors of one attention item (one MMA row tile)
+constexpr int AW = 4;                            // warps of the task group
+constexpr uint64_t WAIT_NS = 500000000ull;       // every wait gives up after half a second
+
+struct PassShared {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    int abort_flag, epi_abort, aux_flag;
+    float scale[8];
+    float val[8][TILE_N];
+    float wsum[8][4];
+    float wgt[NQ * 32];
+};
+
+struct Abort { volatile int* local; volatile uint32_t* global; };
+__device__ __forceinline__ bool aborted(const Abort& a) { return *a.local != 0 || *a.global != 0u; }
+__device__ __forceinline__ void give_up(const Abort& a) { *a.local = 1; *a.global = 1u; }
+
+__device__ __forceinline__ bool mbar_wait_b(uint32_t bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0u) {
+            if (aborted(ab)) return false;
+            if (global_ns() - t0 > WAIT_NS) { give_up(ab); return false; }
+        }
+    }
+}
+// Waits until a counter in global memory has reached `need` (acquire: what the counting threads wrote is visible).
+__device__ __forceinline__ bool word_wait(const uint32_t* w, uint32_t need, const Abort& ab) {
+    const uint64_t t0 = global_ns();
+    for (uint32_t i = 0;; ++i) {
+        uint32_t seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(w) : "memory");
+        if (seen >= need) return true;
+        if ((i & 31u) == 31u) {
+            if (aborted(ab)) return false;
+            if (global_ns() - t0 > WAIT_NS) { give_up(ab); return false; }
+        }
+        __nanosleep(32);
+    }
+}
+__device__ __forceinline__ void word_add(uint32_t* w) { asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(w) : "memory"); }
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }    // warps 4..7
+__device__ __forceinline__ void aux_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }    // warps 8..11
+
+// One value from the task group's first thread to all 128 of them (the flag may be rewritten right after).
+template <class SH> __device__ __forceinline__ int aux_broadcast(SH& sh, int t, int v) {
+    if (t == 0) sh.aux_flag = v;
+    aux_bar();
+    const int r = sh.aux_flag;
+    aux_bar();
+    return r;
+}
+
+__device__ __forceinline__ void ring_next(int& stage, uint32_t& use, int stages) { if (++stage == stages) { stage = 0; ++use; } }
+
+struct Program {
+    const PassSeg* segs[2]; const PassTask* tasks[2]; const uint16_t* pieces;
+    int n_seg[2], n_task[2];
+};
+
+// ------------------------------------------------------------------------------------------ reduce task
+// Sums the pieces of one 128-row output tile in the program's fixed order and applies the step that follows
+// the GEMM in the decoder layer: QKV -> 1/rms, rotary embedding, query buffer / KV append; Wo and down ->
+// residual add, next norm's operand h * gain (bf16, in the packed layout) and the tile's share of sum h^2;
+// gate/up -> 1/rms, SwiGLU; lm_head -> 1/rms, fp32 logits.  128 threads, one per row of the tile.
+__device__ void reduce_task(const PassParams& P, PassShared& sh, const PassTask& tk, const uint16_t* pl, int it, uint32_t* words,
+                            const Abort& ab, int et) {
+    const int mat = tk.mat, tile = (int)tk.item, lane = et & 31, warp = et >> 5;
+    if (!aux_broadcast(sh, et, et == 0 && word_wait(words + tk.wait_word, tk.wait_need, ab) ? 1 : 0)) return;
+    enum { ROPE, RESID, SWIGLU, PLAIN };
+    const int mode = mat == MAT_QKV ? ROPE : mat == MAT_GU ? SWIGLU : mat == MAT_LM ? PLAIN : RESID;
+    const int n_out = P.n_out[mat], n = tile * TILE_N + et;
+    const bool live = n < n_out;
+    const float* __restrict__ partials = P.partials[mat & 1];
+    const size_t piece_elems = (size_t)P.m_tok * TILE_N;
+    const int n_parts = (mat == MAT_QKV && it == 0) ? 1 : (P.d + 127) / 128;
+    const float inv_d = 1.f / (float)P.d;
+    const float* gain_next = nullptr;
+    if (mode == RESID)
+        gain_next = mat == MAT_WO ? P.norm2 + (size_t)it * P.norm_stride
+                                  : (it + 1 < P.n_layers ? P.norm1 + (size_t)(it + 1) * P.norm_stride : (P.has_tail ? P.final_norm : nullptr));
+    const float gain = (gain_next && live) ? gain_next[n] : 0.f;
+    const int n_rows = mode == PLAIN ? P.logits_rows : P.m_tok;
+    const int hd = P.hd, half = hd >> 1, head = n / hd, e = n % hd;
+    const bool rot = head < P.H + P.Hkv;
+    bf16* kc = P.kc + (size_t)it * P.kv_layer_elems;
+    bf16* vc = P.vc + (size_t)it * P.kv_layer_elems;
+    for (int m0 = 0; m0 < n_rows; m0 += 8) {
+        int rows[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = m0 + i;
+            rows[i] = r < n_rows ? (mode == PLAIN ? r * P.row_stride + P.row_offset : r) : -1;
+        }
+        float cs[8], sn[8];
+        int pos[8], slot[8];
+        if (mode == ROPE) {
+            const bool lower = live && e < half;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool ok = lower && rows[i] >= 0;
+                pos[i] = ok ? __ldcg(P.row_pos + rows[i]) : -1;
+                slot[i] = (ok && head >= P.H) ? __ldcg(P.row_slot + rows[i]) : 0;
+                cs[i] = (ok && rot) ? __ldcg(P.rcos + (size_t)rows[i] * half + e) : 1.f;
+                sn[i] = (ok && rot) ? __ldcg(P.rsin + (size_t)rows[i] * half + e) : 0.f;
+            }
+        }
+        float ssa[2] = {0.f, 0.f}, ssb[2] = {0.f, 0.f};
+        if (mode != RESID) {                      // one warp per token row, one lane per piece of its sum of squares
+#pragma unroll
+            for (int ii = 0; ii < 2; ++ii) {
+                const int r = m0 + warp + 4 * ii;
+                const bool ok = r < n_rows;
+                const float* ps = P.ssq + (size_t)(ok ? (mode == PLAIN ? r * P.row_stride + P.row_offset : r) : 0) * SSQ_STRIDE;
+                ssa[ii] = (ok && lane < n_parts) ? __ldcg(ps + lane) : 0.f;
+                ssb[ii] = (ok && lane + 32 < n_parts) ? __ldcg(ps + lane + 32) : 0.f;
+            }
+        }
+        float hv[8];
+        if (mode == RESID) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) hv[i] = (live && rows[i] >= 0) ? __ldcg(P.h + (size_t)rows[i] * n_out + n) : 0.f;
+        }
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        if (live) {
+            for (int c0 = 0; c0 < (int)tk.n_pieces; c0 += 4) {
+                float tmp[4][8];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const bool okc = c0 + cc < (int)tk.n_pieces;
+                    const float* base = partials + (size_t)(okc ? pl[c0 + cc] : 0) * piece_elems + et;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) tmp[cc][i] = (okc && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+                }
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[i] += tmp[cc][i];
+            }
+        }
+        if (mode != RESID) {
+#pragma unroll
+            for (int ii = 0; ii < 2; ++ii) {
+                const float ss = warp_sum(ssa[ii] + ssb[ii]);
+                if (lane == 0) sh.scale[warp + 4 * ii] = rsqrtf(ss * inv_d + P.rms_eps);
+            }
+            aux_bar();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] *= sh.scale[i];
+        }
+        if (mode == PLAIN) {
+            if (live) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) if (rows[i] >= 0) P.logits[(size_t)(m0 + i) * n_out + n] = v[i];
+            }
+        } else if (mode == ROPE) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sh.val[i][et] = v[i];
+            aux_bar();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (pos[i] < 0) continue;
+                const float a = v[i], b = sh.val[i][et + half];
+                const float ra = a * cs[i] - b * sn[i], rb = a * sn[i] + b * cs[i];
+                bf16* dst;
+                if (head < P.H) dst = P.q + ((size_t)rows[i] * P.H + head) * hd;
+                else {
+                    const int kvh = (head - P.H) % P.Hkv;
+                    dst = (rot ? kc : vc) + (((size_t)slot[i] * P.Hkv + kvh) * P.max_ctx + pos[i]) * hd;
+                }
+                dst[e] = __float2bfloat16_rn(ra);
+                dst[e + half] = __float2bfloat16_rn(rb);
+            }
+        } else if (mode == RESID) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                hv[i] += v[i];
+                if (live && rows[i] >= 0) {
+                    P.h[(size_t)rows[i] * n_out + n] = hv[i];
+                    if (gain_next) *reinterpret_cast<bf16*>(P.xn + xpacked_offset(rows[i], n, P.m_pad)) = __float2bfloat16_rn(hv[i] * gain);
+                }
+            }
+            if (gain_next) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float ss = warp_sum(hv[i] * hv[i]);
+                    if (lane == 0) sh.wsum[i][warp] = ss;
+                }
+                aux_bar();
+                if (et < 8 && m0 + et < n_rows) {
+                    const float* w = sh.wsum[et];
+                    P.ssq[(size_t)(m0 + et) * SSQ_STRIDE + tile] = (w[0] + w[1]) + (w[2] + w[3]);
+                }
+            }
+        } else {                                  // SWIGLU: 64 gate rows then the 64 up rows of the same features
+            const int f = tile * 64 + et;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sh.val[i][et] = v[i];
+            aux_bar();
+            if (et < 64 && f < P.F) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (rows[i] < 0) continue;
+                    const float gt = v[i], up = sh.val[i][et + 64];
+                    *reinterpret_cast<bf16*>(P.act + xpacked_offset(rows[i], f, P.m_pad)) = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
+                }
+            }
+        }
+        if (m0 + 8 < n_rows) aux_bar();           // the exchange buffers are reused by the next batch of rows
+    }
+    if (tk.done_word != NO_WORD) {
+        // the rows written above are read by bulk copies (another proxy) on other SMs once the word has counted
+        asm volatile("fence.proxy.async;" ::: "memory");
+        aux_bar();
+        if (et == 0) word_add(words + tk.done_word);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ attention task
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One slice of one KV head's cache x the query rows of one block (times the query heads that share the KV
+// head) as a 16-row tensor-core tile (mma.sync m16n8k16, bf16 in, fp32 accumulate).  The slice is walked in
+// chunks of 64 keys, double-buffered in shared memory (16-byte asynchronous copies into an XOR-swizzled layout
+// that ldmatrix reads without bank conflicts); each warp owns 16 keys of a chunk and keeps its own running
+// max / sum / output (online softmax, exp2 domain).  With one slice the normalised output is written directly
+// (packed layout of the Wo GEMM's input rows); with several, the slice that delivers last merges them all in
+// slice order.  The item's completion word counts once, when the merged output is in memory.
+template <int HD>
+__device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_raw, const PassTask& tk, int it, uint32_t* words,
+                               const Abort& ab, int t) {
+    constexpr int NT = 32 * AW, CK = 16 * AW;
+    constexpr int ROWB = HD * 2, CPR = HD / 8, KS = HD / 16, NV = HD / 8, BUF = CK * ROWB, OLD = HD + 8;
+    if (!aux_broadcast(sh, t, t == 0 && word_wait(words + tk.wait_word, tk.wait_need, ab) ? 1 : 0)) return;
+    const int ns = P.n_splits;
+    const int split = (int)(tk.item % (uint32_t)ns), rest = (int)(tk.item / (uint32_t)ns);
+    const int kvh = rest % P.Hkv, blk = rest / P.Hkv;
+    const int group = P.H / P.Hkv;
+    const int bps = (P.rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;
+    const int r0 = (blk / bps) * P.rows_per_seq + (blk % bps) * P.rows_per_block;
+    const int nr = min(P.rows_per_block, P.rows_per_seq - (blk % bps) * P.rows_per_block);
+    const int nq = nr * group;
+    const int lane = t & 31, warp = t >> 5, gid = lane >> 2, tig = lane & 3;
+    const uint32_t smem0 = smem_u32(sm_raw);
+    const bf16* kcl = P.kc + (size_t)it * P.kv_layer_elems;
+    const bf16* vcl = P.vc + (size_t)it * P.kv_layer_elems;
+
+    int mp = lane < nr ? __ldcg(P.row_pos + r0 + lane) : -1;
+    const int slot = __ldcg(P.row_slot + r0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mp = max(mp, __shfl_xor_sync(0xffffffffu, mp, o));
+    const int len = mp + 1;
+    const int slice = (((len + ns - 1) / ns) + 15) & ~15;
+    const int p_begin = split * slice;
+    const int np = max(0, min(p_begin + slice, len) - p_begin);
+
+    const int j_lo = gid, j_hi = gid + 8;
+    const bf16* q_lo = P.q + ((size_t)(r0 + j_lo / group) * P.H + kvh * group + j_lo % group) * HD;
+    const bf16* q_hi = P.q + ((size_t)(r0 + j_hi / group) * P.H + kvh * group + j_hi % group) * HD;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    float O[NV][4];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) { O[i][0] = O[i][1] = O[i][2] = O[i][3] = 0.f; }
+
+    const bf16* K = kcl + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
+    const bf16* V = vcl + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
+    auto issue = [&](int c) {
+        const int nk = min(CK, np - c * CK);
+        const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
+        const bf16* ks = K + (size_t)c * CK * HD;
+        const bf16* vs = V + (size_t)c * CK * HD;
+        for (int i = t; i < nk * CPR; i += NT) {
+            const int key = i / CPR, ch = i % CPR;
+            const uint32_t off = (uint32_t)key * ROWB + (uint32_t)((ch ^ (key & 7)) << 4);
+            cp_async16(kb + off, ks + (size_t)i * 8);
+            cp_async16(vb + off, vs + (size_t)i * 8);
+        }
+        const int nk16 = (nk + 15) & ~15;         // value rows past the slice inside a warp's 16-key group must be finite
+        for (int i = nk * CPR + t; i < nk16 * CPR; i += NT) {
+            const int key = i / CPR, ch = i % CPR;
+            *reinterpret_cast<uint4*>(sm_raw + (size_t)(c & 1) * 2 * BUF + BUF + (size_t)key * ROWB + ((ch ^ (key & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (np > 0) {
+        const int n_chunks = (np + CK - 1) / CK;
+        issue(0);
+        uint32_t a[KS][4];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            a[ks][0] = j_lo < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 2 * tig)) : 0u;
+            a[ks][1] = j_hi < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 2 * tig)) : 0u;
+            a[ks][2] = j_lo < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 8 + 2 * tig)) : 0u;
+            a[ks][3] = j_hi < nq ? __ldcg(reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 8 + 2 * tig)) : 0u;
+        }
+        const int pos_lo = j_lo < nq ? __ldcg(P.row_pos + r0 + j_lo / group) : -1;
+        const int pos_hi = j_hi < nq ? __ldcg(P.row_pos + r0 + j_hi / group) : -1;
+        const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
+        for (int c = 0; c < n_chunks; ++c) {
+            if (c + 1 < n_chunks) { issue(c + 1); asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            aux_bar();
+            const int nk = min(CK, np - c * CK);
+            if (16 * warp < nk) {
+                const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
+                float S[2][4];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) { S[i][0] = S[i][1] = S[i][2] = S[i][3] = 0.f; }
+                {
+                    const int mi = lane >> 3, r = lane & 7;
+                    const int key = 16 * warp + 8 * (mi >> 1) + r;
+                    const uint32_t rowaddr = kb + (uint32_t)key * ROWB;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        uint32_t b[4];
+                        ldmatrix_x4(rowaddr + (uint32_t)(((2 * ks + (mi & 1)) ^ (key & 7)) << 4), b);
+                        mma_bf16(S[0], a[ks], b[0], b[1]);
+                        mma_bf16(S[1], a[ks], b[2], b[3]);
+                    }
+                }
+                const int pbase = p_begin + c * CK + 16 * warp + 2 * tig;
+                float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int p = pbase + 8 * nt + (e & 1);
+                        const bool ok = (p - p_begin) < np && p <= ((e < 2) ? pos_lo : pos_hi);
+                        const float v = ok ? S[nt][e] * sl2 : -INFINITY;
+                        S[nt][e] = v;
+                        if (e < 2) mx_lo = fmaxf(mx_lo, v); else mx_hi = fmaxf(mx_hi, v);
+                    }
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1)); mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1)); mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+                const float c_lo = (mn_lo == -INFINITY) ? 1.f : exp2f(m_lo - mn_lo);
+                const float c_hi = (mn_hi == -INFINITY) ? 1.f : exp2f(m_hi - mn_hi);
+                m_lo = mn_lo; m_hi = mn_hi;
+                float s_lo = 0.f, s_hi = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float mn = (e < 2) ? mn_lo : mn_hi;
+                        const float pr = (mn == -INFINITY) ? 0.f : exp2f(S[nt][e] - mn);
+                        S[nt][e] = pr;
+                        if (e < 2) s_lo += pr; else s_hi += pr;
+                    }
+                l_lo = l_lo * c_lo + s_lo; l_hi = l_hi * c_hi + s_hi;
+                uint32_t pa[4];
+                pa[0] = pack_bf16(S[0][0], S[0][1]); pa[1] = pack_bf16(S[0][2], S[0][3]);
+                pa[2] = pack_bf16(S[1][0], S[1][1]); pa[3] = pack_bf16(S[1][2], S[1][3]);
+                {
+                    const int mi = lane >> 3, r = lane & 7;
+                    const int key = 16 * warp + 8 * (mi & 1) + r;
+                    const uint32_t rowaddr = vb + (uint32_t)key * ROWB;
+#pragma unroll
+                    for (int nv = 0; nv < NV; nv += 2) {
+                        O[nv][0] *= c_lo; O[nv][1] *= c_lo; O[nv][2] *= c_hi; O[nv][3] *= c_hi;
+                        O[nv + 1][0] *= c_lo; O[nv + 1][1] *= c_lo; O[nv + 1][2] *= c_hi; O[nv + 1][3] *= c_hi;
+                        uint32_t v[4];
+                        ldmatrix_x4_trans(rowaddr + (uint32_t)(((nv + (mi >> 1)) ^ (key & 7)) << 4), v);
+                        mma_bf16(O[nv], pa, v[0], v[1]);
+                        mma_bf16(O[nv + 1], pa, v[2], v[3]);
+                    }
+                }
+            }
+            aux_bar();
+        }
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    }
+
+    // ---- merge of the warps (each saw different keys)
+    float* Ow = reinterpret_cast<float*>(sm_raw);           // [warps][16][OLD]
+    float* mw = Ow + AW * NQ * OLD;                         // [warps][16]
+    float* lw = mw + AW * NQ;
+    if (np > 0) {
+#pragma unroll
+        for (int nv = 0; nv < NV; ++nv) {
+            *reinterpret_cast<float2*>(Ow + ((size_t)warp * NQ + gid) * OLD + 8 * nv + 2 * tig) = make_float2(O[nv][0], O[nv][1]);
+            *reinterpret_cast<float2*>(Ow + ((size_t)warp * NQ + gid + 8) * OLD + 8 * nv + 2 * tig) = make_float2(O[nv][2], O[nv][3]);
+        }
+        if (tig == 0) {
+            mw[warp * NQ + gid] = m_lo; mw[warp * NQ + gid + 8] = m_hi;
+            lw[warp * NQ + gid] = l_lo; lw[warp * NQ + gid + 8] = l_hi;
+        }
+    }
+    aux_bar();
+    constexpr int TPR = NT / NQ, CPT = HD / TPR;            // threads per query row, columns per thread
+    const int j = t / TPR, c0 = (t % TPR) * CPT;
+    {
+        float M = -INFINITY, L = 0.f;
+        float acc[CPT];
+#pragma unroll
+        for (int cc = 0; cc < CPT; ++cc) acc[cc] = 0.f;
+        if (np > 0) {
+#pragma unroll
+            for (int w = 0; w < AW; ++w) M = fmaxf(M, mw[w * NQ + j]);
+#pragma unroll
+            for (int w = 0; w < AW; ++w) {
+                const float m = mw[w * NQ + j];
+                const float wt = (m == -INFINITY) ? 0.f : exp2f(m - M);
+                L += wt * lw[w * NQ + j];
+                if (wt != 0.f) {
+#pragma unroll
+                    for (int cc = 0; cc < CPT; ++cc) acc[cc] = fmaf(wt, Ow[((size_t)w * NQ + j) * OLD + c0 + cc], acc[cc]);
+                }
+            }
+        }
+        if (j < nq) {
+            const int r = r0 + j / group, h = kvh * group + j % group;
+            if (ns == 1) {
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+                for (int cc = 0; cc < CPT; cc += 2)
+                    *reinterpret_cast<__nv_bfloat162*>(P.attn + xpacked_offset(r, h * HD + c0 + cc, P.m_pad)) = __floats2bfloat162_rn(acc[cc] * inv, acc[cc + 1] * inv);
+            } else {
+                float* po = P.part_o + (((size_t)r * P.H + h) * ns + split) * HD + c0;
+                float* ml = P.part_ml + (((size_t)r * P.H + h) * ns + split) * 2;
+#pragma unroll
+                for (int cc = 0; cc < CPT; cc += 4) __stcg(reinterpret_cast<float4*>(po + cc), make_float4(acc[cc], acc[cc + 1], acc[cc + 2], acc[cc + 3]));
+                if ((t % TPR) == 0) { __stcg(ml, M); __stcg(ml + 1, L); }
+            }
+        }
+    }
+    if (ns > 1) {
+        // ---- the slice that delivers last merges all of them, always in slice order
+        aux_bar();                                          // the group's stores are ordered before its first thread's release
+        int last = 0;
+        if (t == 0) {
+            uint32_t* ctr = P.att_counters + (size_t)blk * P.Hkv + kvh;
+            uint32_t old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
+            last = old == (uint32_t)ns - 1u;
+            if (last) *ctr = 0u;
+        }
+        if (!aux_broadcast(sh, t, last)) return;
+        for (int jq = warp; jq < nq; jq += AW) {            // n_splits <= 32: one lane per slice
+            const int r = r0 + jq / group, h = kvh * group + jq % group;
+            const float* mlg = P.part_ml + ((size_t)r * P.H + h) * ns * 2;
+            float m = -INFINITY, l = 0.f;
+            if (lane < ns) { const float2 v = __ldcg(reinterpret_cast<const float2*>(mlg) + lane); m = v.x; l = v.y; }
+            const float M = warp_max(m);
+            const float w = (m == -INFINITY) ? 0.f : exp2f(m - M);
+            const float den = warp_sum(w * l);
+            if (lane < ns) sh.wgt[jq * 32 + lane] = den > 0.f ? w / den : 0.f;
+        }
+        aux_bar();
+        constexpr int TPQ = NT / HD;                        // queries handled side by side (1 or 2)
+        const int e = t % HD, jq0 = t / HD;
+        for (int jq = jq0; jq < nq; jq += TPQ) {
+            const int r = r0 + jq / group, h = kvh * group + jq % group;
+            float acc = 0.f;
+            for (int s = 0; s < ns; ++s) {
+                const float w = sh.wgt[jq * 32 + s];
+                if (w != 0.f) acc = fmaf(w, __ldcg(P.part_o + (((size_t)r * P.H + h) * ns + s) * HD + e), acc);
+            }
+            *reinterpret_cast<bf16*>(P.attn + xpacked_offset(r, h * HD + e, P.m_pad)) = __float2bfloat16_rn(acc);
+        }
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");
+    aux_bar();
+    if (t == 0) word_add(words + tk.done_word);
+}
+
+// ------------------------------------------------------------------------------------------ the kernel
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ PassParams P) {
+    extern __shared__ __align__(1024) uint8_t dyn[];
+    __shared__ PassShared sh;
+    pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_it = P.n_layers + P.has_tail;
+    const uint32_t x_bytes = (uint32_t)P.m_pad * 128u, stage_bytes = A_BYTES + x_bytes;
+    const uint32_t ring0 = (smem_u32(dyn) + PROG_BYTES + 1023u) & ~1023u;
+    uint8_t* attn_smem = dyn + (ring0 - smem_u32(dyn)) + (size_t)P.stages * stage_bytes;
+    const Abort ab{&sh.abort_flag, P.abort_word};
+
+    // the CTA's section of the program (uploaded long before the launch) -> shared memory
+    {
+        const uint32_t* table = reinterpret_cast<const uint32_t*>(P.program);
+        const uint32_t o0 = table[blockIdx.x], o1 = table[blockIdx.x + 1];
+        const uint4* src = reinterpret_cast<const uint4*>(P.program + o0);
+        uint4* dst = reinterpret_cast<uint4*>(dyn);
+        for (uint32_t i = threadIdx.x; i < (o1 - o0) / 16u && i < PROG_BYTES / 16u; i += NUM_THREADS) dst[i] = src[i];
+    }
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * (uint32_t)P.m_pad) tmem_cols <<= 1;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P.stages; ++s) {
+            mbar_init(smem_u32(&sh.full[s]), 2);           // the weight block and the input rows arrive from two producers
+            mbar_init(smem_u32(&sh.empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
+        sh.abort_flag = 0; sh.epi_abort = 0; sh.aux_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sh.tmem_base;
+    Program pg;
+    {
+        const PassCtaHeader* h = reinterpret_cast<const PassCtaHeader*>(dyn);
+        for (int k = 0; k < 2; ++k) {
+            pg.segs[k] = reinterpret_cast<const PassSeg*>(dyn + h->seg_off[k]);
+            pg.tasks[k] = reinterpret_cast<const PassTask*>(dyn + h->task_off[k]);
+            pg.n_seg[k] = (int)h->n_seg[k]; pg.n_task[k] = (int)h->n_task[k];
+        }
+        pg.pieces = reinterpret_cast<const uint16_t*>(dyn + h->piece_off);
+    }
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ weight producer: never waits for anything but a free stage
+        if (lane == 0) {
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            int stage = 0; uint32_t use = 0; bool ok = true;
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int k = it == P.n_layers ? 1 : 0, z = k ? 0 : it;
+                for (int si = 0; si < pg.n_seg[k] && ok; ++si) {
+                    const PassSeg sg = pg.segs[k][si];
+                    const CUtensorMap* map = reinterpret_cast<const CUtensorMap*>(&maps.m[sg.mat]);
+                    for (int j = 0; j < (int)sg.n_kb; ++j) {
+                        if (use > 0u && !mbar_wait_b(smem_u32(&sh.empty[stage]), (use & 1u) ^ 1u, ab)) { ok = false; break; }
+                        const uint32_t bar = smem_u32(&sh.full[stage]);
+                        mbar_expect_tx(bar, A_BYTES);
+                        tma_load_3d(ring0 + stage * stage_bytes, map, ((int)sg.kb0 + j) * TILE_K, (int)sg.tile * TILE_N, z, bar, pol_stream);
+                        ring_next(stage, use, P.stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ input-row producer: waits until the chunk's rows exist
+        if (lane == 0) {
+            pdl_wait();                                       // the first rows come from the kernel before this one
+            int stage = 0; uint32_t use = 0; bool ok = true;
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int k = it == P.n_layers ? 1 : 0;
+                uint32_t* words = P.sync + (size_t)it * P.words_per_layer;
+                for (int si = 0; si < pg.n_seg[k] && ok; ++si) {
+                    const PassSeg sg = pg.segs[k][si];
+                    if ((sg.flags & SEG_DEP) && !((sg.flags & SEG_DEP_PREV) && it == 0)) {
+                        const uint32_t* w = ((sg.flags & SEG_DEP_PREV) ? words - P.words_per_layer : words) + sg.dep;
+                        if (!word_wait(w, sg.dep_need, ab)) { ok = false; break; }
+                        asm volatile("fence.proxy.async;" ::: "memory");      // rows written by ordinary stores, read by bulk copies
+                    }
+                    const uint8_t* src = P.x[sg.mat] + (size_t)sg.kb0 * x_bytes;
+                    for (int j = 0; j < (int)sg.n_kb; ++j) {
+                        if (use > 0u && !mbar_wait_b(smem_u32(&sh.empty[stage]), (use & 1u) ^ 1u, ab)) { ok = false; break; }
+                        const uint32_t bar = smem_u32(&sh.full[stage]);
+                        mbar_expect_tx(bar, x_bytes);
+                        bulk_load_1d(ring0 + stage * stage_bytes + A_BYTES, src + (size_t)j * x_bytes, x_bytes, bar);
+                        ring_next(stage, use, P.stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.m_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+            const uint64_t desc0 = umma_desc(ring0);
+            int stage = 0; uint32_t use = 0, seg = 0; bool ok = true;
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int k = it == P.n_layers ? 1 : 0;
+                for (int si = 0; si < pg.n_seg[k] && ok; ++si, ++seg) {
+                    const int n_kb = (int)pg.segs[k][si].n_kb;
+                    const uint32_t buf = seg & 1u;
+                    unsigned long long* stamp = P.stamps ? P.stamps + (((size_t)blockIdx.x * n_it + it) * P.stamp_segs + si) * 2 : nullptr;
+                    if (!mbar_wait_b(smem_u32(&sh.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, ab)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (stamp) stamp[0] = global_ns();
+                    const uint32_t d_tmem = tmem_base + buf * (uint32_t)P.m_pad;
+                    for (int j = 0; j < n_kb; ++j) {
+                        if (!mbar_wait_b(smem_u32(&sh.full[stage]), use & 1u, ab)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint64_t da = desc0 + (uint64_t)((uint32_t)stage * (stage_bytes >> 4)), db = da + (A_BYTES >> 4);
+#pragma unroll
+                        for (uint32_t kk = 0; kk < TILE_K / 16; ++kk)
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, ((uint32_t)j | kk) != 0u);
+                        umma_commit(smem_u32(&sh.empty[stage]));
+                        ring_next(stage, use, P.stages);
+                    }
+                    if (ok) umma_commit(smem_u32(&sh.tmem_full[buf]));
+                    if (stamp) stamp[1] = global_ns();
+                }
+            }
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------------ TMEM -> workspace, one piece per segment
+        const uint32_t quarter = (uint32_t)(warp & 3);
+        const int et = quarter * 32 + lane;
+        uint32_t seg = 0;
+        bool ok = true;
+        for (int it = 0; it < n_it && ok; ++it) {
+            const int k = it == P.n_layers ? 1 : 0;
+            uint32_t* words = P.sync + (size_t)it * P.words_per_layer;
+            for (int si = 0; si < pg.n_seg[k]; ++si, ++seg) {
+                const PassSeg sg = pg.segs[k][si];
+                const uint32_t buf = seg & 1u;
+                if (!mbar_wait_b(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, ab)) sh.epi_abort = 1;
+                epi_bar();
+                if (sh.epi_abort) { ok = false; break; }      // all four warps leave together
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                float* out = P.partials[sg.mat & 1] + (size_t)sg.slot * P.m_tok * TILE_N;
+                for (int c0 = 0; c0 < P.m_pad; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)P.m_pad + (uint32_t)c0, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < P.m_tok) __stcg(out + (size_t)(c0 + j) * TILE_N + et, __uint_as_float(r[j]));
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+                epi_bar();                                    // the four warps' stores are ordered before the release below
+                if (et == 0) word_add(words + sg.arrive);
+            }
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------------ tasks: reduce finished tiles, attention
+        const int t = threadIdx.x - 256;
+        pdl_wait();
+        for (int it = 0; it < n_it; ++it) {
+            const int k = it == P.n_layers ? 1 : 0;
+            uint32_t* words = P.sync + (size_t)it * P.words_per_layer;
+            for (int ti = 0; ti < pg.n_task[k]; ++ti) {
+                const PassTask tk = pg.tasks[k][ti];
+                // (after a wait has given up, the remaining tasks return at their own wait: every branch here is taken by all 128 threads)
+                if (tk.kind == TASK_REDUCE) reduce_task(P, sh, tk, pg.pieces + tk.piece0, it, words, ab, t);
+                else if (P.hd == 128) attention_task<128>(P, sh, attn_smem, tk, it, words, ab, t);
+                else attention_task<64>(P, sh, attn_smem, tk, it, words, ab, t);
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- wind-down
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0) sh.aux_flag = (sh.abort_flag != 0 || *ab.global != 0u) ? 1 : 0;
+    __syncthreads();
+    if (sh.aux_flag) {
+        if (threadIdx.x == 0 && P.status) atomicOr(P.status, SD_DEV_WAIT_EXPIRED);
+        const uint64_t t0 = global_ns();                       // let copies in flight land before the CTA goes away
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn3() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+// bf16 matrices [n_layers][rows][K], consecutive layers layer_stride_bytes apart, as a 3-D tensor map with
+// boxes of 128 rows x 64 elements, 128-byte swizzle; reads outside a matrix return zeros.
+bool make_tensor_map_layers(TensorMap* out, const void* base, int rows, int K, int n_layers, size_t layer_stride_bytes) {
+    EncodeTiledFn fn = encode_fn3();
+    if (!fn || ((uintptr_t)base & 15) || (K & 7) || n_layers < 1 || (layer_stride_bytes & 15)) return false;
+    if (n_layers == 1) layer_stride_bytes = ((size_t)rows * K * 2 + 15) & ~(size_t)15;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)n_layers};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)layer_stride_bytes};
+    cuuint32_t box[3] = {(cuuint32_t)TILE_K, (cuuint32_t)TILE_N, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t pass_stream_smem(int m_pad, int* stages_out) {
+    const int stage_bytes = A_BYTES + m_pad * 128;
+    const int stages = std::max(2, std::min(MAX_STAGES, RING_BUDGET / stage_bytes));
+    if (stages_out) *stages_out = stages;
+    return (size_t)PROG_BYTES + 1024 + (size_t)stages * stage_bytes + ATTN_BYTES;
+}
+
+cudaError_t launch_pass_stream(const PassMaps& maps, const PassParams& p, int grid, int dependent, cudaStream_t st) {
+    int stages = 0;
+    const size_t smem = pass_stream_smem(p.m_pad, &stages);
+    if (p.stages != stages || p.m_pad < 16 || p.m_pad > 256 || (p.m_pad & 15) || p.m_tok > p.m_pad || grid < 1) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(k_pass_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(k_pass_stream, dim3(grid), dim3(NUM_THREADS), smem, st, dependent, maps, p);
+}
+
+}  // namespace sd
