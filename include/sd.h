@@ -240,13 +240,16 @@ sd_status sd_use_pass_kernel(sd_ctx* ctx, int target_on, int drafts_on, int max_
 
 /* Schedule of that kernel, for measurements: waves[5] = tile waves of the QKV, Wo, gate/up, down and lm_head matrices
  * (1..8), chunk_major[5] = order of a matrix's (wave, chunk) blocks (0: wave after wave).  NULL waves restores the
- * defaults.  Drops cached programs and graphs.  Synchronises. */
-sd_status sd_pass_tuning(sd_ctx* ctx, const int32_t* waves, const int32_t* chunk_major);
+ * defaults.  stages > 0 caps the ring of shared-memory stages (0: as many as fit).  Drops cached programs and graphs.
+ * Synchronises. */
+sd_status sd_pass_tuning(sd_ctx* ctx, const int32_t* waves, const int32_t* chunk_major, int stages);
 
 /* Time stamps of the persistent kernel's passes from now on (NULL: none): stamps_dev is a device buffer of n_words
  * 64-bit words; CTA b writes, for segment s of iteration it (layers, then the lm_head), the global-timer nanoseconds
  * at which its MMA thread turned to the segment and at which the segment was committed, at
- * ((b * n_iterations + it) * max_segments + s) * 2.  Passes whose stamps would not fit write none.  Synchronises. */
+ * ((b * n_iterations + it) * max_segments + s) * 2; after all of those, at ((b * n_iterations + it) * 16 + k) * 2, the
+ * times at which the CTA's task warps turned to their k-th task of the iteration (k < 16) and finished it.  Passes whose
+ * stamps would not fit write none.  Synchronises. */
 sd_status sd_pass_stamps(sd_ctx* ctx, unsigned long long* stamps_dev, size_t n_words);
 
 /* Builds and replays on the host the schedule of that kernel for a shape (no GPU needed): shape12 = n_layers, d_model,
@@ -256,6 +259,12 @@ sd_status sd_pass_stamps(sd_ctx* ctx, unsigned long long* stamps_dev, size_t n_w
  * shape does not fit or the replay finds a wait that could never be satisfied. */
 sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, int32_t* info8,
                                  char* err, size_t err_cap);
+
+/* The program itself (same arguments): copies it to out when cap suffices and returns its size in bytes (0 on failure).
+ * Layout: uint32 offset of each CTA's section (CTAs + 1 entries), then per CTA a header (segments and tasks per layer
+ * and for the lm_head, byte offsets of the four arrays and of the piece list), 16-byte segment records (tile, first k
+ * block, k blocks, matrix, flags, wait word, wait count, arrival word, workspace slot) and 20-byte task records. */
+size_t sd_pass_schedule_blob(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, void* out, size_t cap);
 
 /* Number of kernels this context has launched since sd_create. */
 sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);

@@ -70,9 +70,10 @@ _PROTOS = {
     "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_use_graphs": (_i, [_vp, _i]),
     "sd_use_pass_kernel": (_i, [_vp, _i, _i, _i]),
-    "sd_pass_tuning": (_i, [_vp, _vp, _vp]),
+    "sd_pass_tuning": (_i, [_vp, _vp, _vp, _i]),
     "sd_pass_stamps": (_i, [_vp, _vp, _sz]),
     "sd_pass_schedule_check": (_i, [_vp, _vp, _vp, _vp, C.c_char_p, _sz]),
+    "sd_pass_schedule_blob": (_sz, [_vp, _vp, _vp, _vp, _sz]),
     "sd_force_plain_path": (_i, [_vp, _i]),
     "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
     "sd_profile": (_i, [_vp, _i]),
@@ -120,6 +121,33 @@ def sd_pass_schedule_check(dims, rows, rows_per_seq, n_splits, want_logits=1, gr
                                       cm.ctypes.data_as(C.c_void_p) if cm is not None else None, info.ctypes.data_as(C.c_void_p), err, 256)
     names = ("words_per_layer", "total_words", "slots0", "slots1", "max_seg", "max_section", "program_bytes", "units_per_layer")
     return st, dict(zip(names, info.tolist())), err.value.decode()
+
+
+def sd_pass_schedule(dims, rows, rows_per_seq, n_splits, want_logits=1, grid=148, waves=None, chunk_major=None):
+    """The persistent kernel's schedule as per-CTA lists: [{'segs': [body, tail], 'tasks': [body, tail]}], records as numpy structured arrays."""
+    shape = np.array([dims["n_layers"], dims["d_model"], dims["n_heads"], dims["n_kv_heads"], dims["head_dim"], dims["d_ffn"],
+                      dims["vocab"], rows, rows_per_seq, n_splits, want_logits, grid], dtype=np.int32)
+    w = np.ascontiguousarray(waves, dtype=np.int32) if waves is not None else None
+    cm = np.ascontiguousarray(chunk_major, dtype=np.int32) if chunk_major is not None else None
+    wp = w.ctypes.data_as(C.c_void_p) if w is not None else None
+    cp = cm.ctypes.data_as(C.c_void_p) if cm is not None else None
+    n = lib().sd_pass_schedule_blob(shape.ctypes.data_as(C.c_void_p), wp, cp, None, 0)
+    if n == 0:
+        raise ValueError("no schedule for this shape")
+    blob = np.zeros(n, dtype=np.uint8)
+    lib().sd_pass_schedule_blob(shape.ctypes.data_as(C.c_void_p), wp, cp, blob.ctypes.data_as(C.c_void_p), n)
+    seg_t = np.dtype([("tile", "<u2"), ("kb0", "<u2"), ("n_kb", "<u2"), ("mat", "u1"), ("flags", "u1"), ("dep", "<u2"),
+                      ("dep_need", "<u2"), ("arrive", "<u2"), ("slot", "<u2")])
+    task_t = np.dtype([("item", "<u4"), ("piece0", "<u4"), ("kind", "<u2"), ("mat", "<u2"), ("wait_word", "<u2"),
+                       ("wait_need", "<u2"), ("done_word", "<u2"), ("n_pieces", "<u2")])
+    offs = blob[: 4 * (grid + 1)].view("<u4")
+    out = []
+    for c in range(grid):
+        sec = blob[offs[c]: offs[c + 1]]
+        h = sec[:40].view("<u4")          # n_seg[2], n_task[2], seg_off[2], task_off[2], piece_off, bytes
+        out.append(dict(segs=[sec[h[4 + k]: h[4 + k] + 16 * h[k]].view(seg_t) for k in range(2)],
+                        tasks=[sec[h[6 + k]: h[6 + k] + 20 * h[2 + k]].view(task_t) for k in range(2)]))
+    return out
 
 
 def exported_symbols():
@@ -270,11 +298,11 @@ class Context:
     def sd_use_pass_kernel(self, target_on, drafts_on=0, max_rows=0):
         _check(self.L.sd_use_pass_kernel(self.h, int(target_on), int(drafts_on), int(max_rows)), "sd_use_pass_kernel")
 
-    def sd_pass_tuning(self, waves=None, chunk_major=None):
+    def sd_pass_tuning(self, waves=None, chunk_major=None, stages=0):
         w = np.ascontiguousarray(waves, dtype=np.int32) if waves is not None else None
         cm = np.ascontiguousarray(chunk_major, dtype=np.int32) if chunk_major is not None else None
         _check(self.L.sd_pass_tuning(self.h, w.ctypes.data_as(C.c_void_p) if w is not None else None,
-                                     cm.ctypes.data_as(C.c_void_p) if cm is not None else None), "sd_pass_tuning")
+                                     cm.ctypes.data_as(C.c_void_p) if cm is not None else None, int(stages)), "sd_pass_tuning")
 
     def sd_pass_stamps(self, stamps):
         """stamps: int64 device tensor or None."""

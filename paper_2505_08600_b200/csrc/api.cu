@@ -87,7 +87,7 @@ struct sd_ctx {
     float* pass_part_o; float* pass_part_ml; uint32_t* pass_att_counters;
     size_t pass_att_counter_words;
     bool pass_on, pass_drafts; int pass_max_rows;
-    PassTuning pass_tuning; bool pass_tuned;
+    PassTuning pass_tuning; bool pass_tuned; int pass_stages;
     struct CachedProgram { int model, m_tok, rows_per_seq, n_splits, want_logits, slot; PassProgram meta; uint64_t last_use; };
     std::vector<CachedProgram> programs;
     unsigned long long* stamps; size_t stamps_words;          // optional time stamps of the next passes (caller's buffer)
@@ -502,6 +502,7 @@ sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, con
     P.d = d; P.H = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = hd; P.F = m.d_ffn; P.V = m.vocab; P.max_ctx = c->cfg.max_ctx;
     P.n_out[MAT_QKV] = M.n_qkv(); P.n_out[MAT_WO] = d; P.n_out[MAT_GU] = 2 * m.d_ffn; P.n_out[MAT_DN] = d; P.n_out[MAT_LM] = m.vocab;
     (void)pass_stream_smem(P.m_pad, &P.stages);
+    if (c->pass_stages >= 2 && c->pass_stages < P.stages) P.stages = c->pass_stages;
     P.words_per_layer = cp.meta.words_per_layer;
     P.h = c->h; P.xn = c->xp_xn; P.attn = c->xp_attn; P.act = c->xp_act;
     P.x[MAT_QKV] = c->xp_xn; P.x[MAT_WO] = c->xp_attn; P.x[MAT_GU] = c->xp_xn; P.x[MAT_DN] = c->xp_act; P.x[MAT_LM] = c->xp_xn;
@@ -520,7 +521,11 @@ sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, con
     P.rows_per_seq = R; P.rows_per_block = cp.meta.rows_per_block; P.n_splits = cp.n_splits;
     P.part_o = c->pass_part_o; P.part_ml = c->pass_part_ml; P.att_counters = c->pass_att_counters;
     const int n_it = m.n_layers + P.has_tail;
-    if (c->stamps && (size_t)sm_count() * n_it * cp.meta.max_seg * 2 <= c->stamps_words) { P.stamps = c->stamps; P.stamp_segs = cp.meta.max_seg; }
+    const size_t seg_words = (size_t)sm_count() * n_it * cp.meta.max_seg * 2, task_words = (size_t)sm_count() * n_it * 16 * 2;
+    if (c->stamps && seg_words + task_words <= c->stamps_words) {
+        P.stamps = c->stamps; P.stamp_segs = cp.meta.max_seg;
+        P.task_stamps = c->stamps + seg_words; P.stamp_tasks = 16;
+    }
     CUDA_TRY(prof_mark(c, CAT_STATE));
     CUDA_TRY(cudaMemsetAsync(c->pass_sync, 0, sizeof(uint32_t) * ((size_t)cp.meta.total_words + 1), st));
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, m.dtype, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -676,7 +681,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         cudaMemsetAsync(c->pass_att_counters, 0, sizeof(uint32_t) * c->pass_att_counter_words, st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
-    c->pass_on = true; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->stamps = nullptr; c->stamps_words = 0;
+    c->pass_on = true; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
     c->force_plain = false;
     c->graphs_on = true;
     c->graph_clock = 0;
@@ -1080,8 +1085,9 @@ sd_status sd_use_pass_kernel(sd_ctx* c, int target_on, int drafts_on, int max_ro
     return SD_OK;
 }
 
-sd_status sd_pass_tuning(sd_ctx* c, const int32_t* waves, const int32_t* chunk_major) {
-    if (!c) return SD_ERR_INVALID_ARG;
+sd_status sd_pass_tuning(sd_ctx* c, const int32_t* waves, const int32_t* chunk_major, int stages) {
+    if (!c || stages < 0) return SD_ERR_INVALID_ARG;
+    c->pass_stages = stages;
     CUDA_TRY(cudaStreamSynchronize(c->st));
     for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);        // programs and the graphs that captured them are rebuilt
     c->graphs.clear();
@@ -1114,6 +1120,17 @@ sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, c
     info8[4] = p.max_seg; info8[5] = p.max_section; info8[6] = (int32_t)p.blob.size(); info8[7] = (int32_t)p.units_per_layer;
     if (err && err_cap) { strncpy(err, p.error.c_str(), err_cap - 1); err[err_cap - 1] = 0; }
     return p.error.empty() ? SD_OK : SD_ERR_UNSUPPORTED;
+}
+
+size_t sd_pass_schedule_blob(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, void* out, size_t cap) {
+    if (!shape12) return 0;
+    PassShape sh{shape12[0], shape12[1], shape12[2], shape12[3], shape12[4], shape12[5], shape12[6], shape12[7], shape12[8], shape12[9], shape12[10], shape12[11]};
+    PassTuning t = default_pass_tuning(sh);
+    for (int m = 0; m < N_MAT && waves; ++m) { t.waves[m] = waves[m]; t.chunk_major[m] = chunk_major ? chunk_major[m] : 0; }
+    const PassProgram p = build_pass_program(sh, t);
+    if (!p.error.empty()) return 0;
+    if (out && cap >= p.blob.size()) memcpy(out, p.blob.data(), p.blob.size());
+    return p.blob.size();
 }
 
 sd_status sd_use_graphs(sd_ctx* c, int on) {

@@ -50,6 +50,7 @@ struct Builder {
         pieces.resize(G);
     }
 
+    int S_n_acc() const { const int m_pad = (S.m_tok + 15) & ~15; return std::max(2, std::min(16, 512 / m_pad)); }
     int done_word(int mat, int wave) const { return done_base + mat * PASS_MAX_WAVES + wave; }
 
     void plan() {
@@ -136,8 +137,12 @@ struct Builder {
         MatPlan& P = mp[m];
         const int W = (int)P.wave_tiles.size(), C = (int)P.chunk_kb.size();
         std::vector<std::vector<uint16_t>> tile_pieces(P.n_tiles);
-        std::vector<int> wave_last_block(W, 0);
+        std::vector<int> wave_last_block(W, 0), wave_rot(W, -1);
         int next_slot = 0;
+        std::vector<size_t> seg0(G);
+        for (int c = 0; c < G; ++c) seg0[c] = segs[kind][c].size();
+        // ---- pass 1: the blocks in ring order, each split evenly over the CTAs.  The chunks of a wave are cut at the same
+        //      places, so that a CTA meets the same tiles again in the wave's next chunk and keeps accumulating.
         for (int idx = 0; idx < W * C; ++idx) {
             const int a = P.chunk_major ? idx % W : idx / C, j = P.chunk_major ? idx / W : idx % C;
             const auto& tl = P.wave_tiles[a];
@@ -146,10 +151,11 @@ struct Builder {
             wave_last_block[a] = block_seq;
             ++block_seq;
             if (Tb == 0) continue;
+            if (wave_rot[a] < 0) { wave_rot[a] = rot; rot = (int)((rot + (Tb % G) * C) % G); }
             const long long base = Tb / G;
             const int rem = (int)(Tb % G);
             for (int pos = 0; pos < G; ++pos) {
-                const int cta = (pos + rot) % G;
+                const int cta = (pos + wave_rot[a]) % G;
                 const long long u0 = pos * base + std::min(pos, rem), u1 = u0 + base + (pos < rem ? 1 : 0);
                 for (long long u = u0; u < u1;) {
                     const int ti = (int)(u / nk), k0 = (int)(u % nk);
@@ -160,15 +166,36 @@ struct Builder {
                     sg.flags = (uint8_t)((P.chunk_dep[j] >= 0 ? SEG_DEP : 0) | (P.dep_prev ? SEG_DEP_PREV : 0));
                     sg.dep = (uint16_t)std::max(0, P.chunk_dep[j]); sg.dep_need = (uint16_t)P.chunk_need[j];
                     sg.arrive = (uint16_t)(arrive_base[m] + tl[ti]);
-                    if (next_slot >= 65535) { error = "too many workspace slots"; return; }
-                    sg.slot = (uint16_t)next_slot;
-                    tile_pieces[tl[ti]].push_back((uint16_t)next_slot);
-                    ++next_slot;
                     segs[kind][cta].push_back(sg);
                     u += n;
                 }
             }
-            rot = (rot + rem) % G;
+        }
+        // ---- pass 2: accumulators.  A CTA's segments of one tile share one accumulator in tensor memory from the first
+        //      to the last of them; only the last one leaves a piece in the workspace.
+        for (int c = 0; c < G; ++c) {
+            std::vector<PassSeg>& v = segs[kind][c];
+            std::vector<int> last_of(P.n_tiles, -1), acc_of(P.n_tiles, -1);
+            for (size_t i = seg0[c]; i < v.size(); ++i) last_of[v[i].tile] = (int)i;
+            std::vector<int> free_acc;
+            for (int k = 0; k < S_n_acc(); ++k) free_acc.push_back(k);
+            for (size_t i = seg0[c]; i < v.size(); ++i) {
+                const int t = v[i].tile;
+                if (acc_of[t] < 0) {
+                    if (free_acc.empty()) { error = "a CTA would hold more accumulators than tensor memory has room for"; return; }
+                    acc_of[t] = free_acc.front(); free_acc.erase(free_acc.begin());
+                    v[i].flags |= SEG_FIRST;
+                }
+                v[i].flags |= (uint8_t)(acc_of[t] << 4);
+                if (last_of[t] == (int)i) {
+                    v[i].flags |= SEG_LAST;
+                    if (next_slot >= 65535) { error = "too many workspace slots"; return; }
+                    v[i].slot = (uint16_t)next_slot;
+                    tile_pieces[t].push_back((uint16_t)next_slot);
+                    ++next_slot;
+                    free_acc.push_back(acc_of[t]);        // reused last: the epilogue has long drained it by then
+                }
+            }
         }
         slots[m & 1] = std::max(slots[m & 1], next_slot);
         // the tasks that sum the pieces of a tile and apply the step after the GEMM, wave by wave
@@ -308,7 +335,7 @@ std::string check_pass_program(const PassShape& s, const PassProgram& p) {
             for (uint32_t i = 0; i < ctas[c].h->n_seg[k]; ++i) {
                 if (sg[i].mat != m) continue;
                 if (sg[i].tile >= nt[m] || sg[i].kb0 + sg[i].n_kb > kbpt[m] || sg[i].n_kb == 0) return "segment out of range";
-                if ((int)sg[i].slot >= p.slots[m & 1]) return "slot out of range";
+                if ((sg[i].flags & SEG_LAST) && (int)sg[i].slot >= p.slots[m & 1]) return "slot out of range";
                 for (int j = 0; j < sg[i].n_kb; ++j) {
                     uint8_t& b = seen[(size_t)sg[i].tile * kbpt[m] + sg[i].kb0 + j];
                     if (b) return "a weight block is scheduled twice";
@@ -338,7 +365,7 @@ std::string check_pass_program(const PassShape& s, const PassProgram& p) {
                 const PassSeg& sg = reinterpret_cast<const PassSeg*>(A.base + A.h->seg_off[k])[A.si];
                 const bool prev = sg.flags & SEG_DEP_PREV;
                 if ((sg.flags & SEG_DEP) && !(prev && A.it_s == 0) && words[word_of(A.it_s, sg.dep, prev)] < sg.dep_need) break;
-                words[word_of(A.it_s, sg.arrive, false)] += 1;
+                if (sg.flags & SEG_LAST) words[word_of(A.it_s, sg.arrive, false)] += 1;
                 ++A.si; --remaining; progress = true;
             }
             for (;;) {                                    // the task warps: tasks in order

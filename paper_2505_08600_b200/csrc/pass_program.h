@@ -23,18 +23,21 @@
 namespace sd {
 
 enum { MAT_QKV = 0, MAT_WO = 1, MAT_GU = 2, MAT_DN = 3, MAT_LM = 4, N_MAT = 5, MAT_ATT = 5 };
-enum { SEG_DEP = 1, SEG_DEP_PREV = 2 };          // waits for a word; the word belongs to the previous layer
+// flags of a segment: waits for a word; the word belongs to the previous layer; first / last segment of its accumulator
+// (bits 4..7: which accumulator in tensor memory)
+enum { SEG_DEP = 1, SEG_DEP_PREV = 2, SEG_FIRST = 4, SEG_LAST = 8 };
 enum { TASK_REDUCE = 0, TASK_ATTENTION = 1 };
 constexpr uint16_t NO_WORD = 0xFFFFu;
 constexpr int PASS_MAX_WAVES = 8;
 
-// One run of k blocks of one output tile: the unit of accumulation (one TMEM accumulator, one piece).
+// One run of k blocks of one output tile.  A CTA's segments of the same tile (one per chunk of the wave) accumulate
+// into one TMEM accumulator; the last of them leaves the CTA's piece of the tile in the workspace.
 struct PassSeg {
     uint16_t tile, kb0, n_kb;
     uint8_t mat, flags;
     uint16_t dep, dep_need;      // word (relative to the layer's words) that must reach dep_need before the input rows are loaded
     uint16_t arrive;             // word that counts the pieces of the tile
-    uint16_t slot;               // workspace slot of the piece (per region: matrices alternate between two regions)
+    uint16_t slot;               // SEG_LAST: workspace slot of the piece (per region: matrices alternate between two regions)
 };
 static_assert(sizeof(PassSeg) == 16, "segment record");
 

@@ -27,6 +27,7 @@ namespace {
 constexpr int TILE_N = 128, TILE_K = 64, A_BYTES = TILE_N * TILE_K * 2;
 constexpr int NUM_THREADS = 384;
 constexpr int MAX_STAGES = 10;
+constexpr int MAX_ACC = 16;                      // accumulators in tensor memory (a CTA returns to a tile in the wave's next chunk)
 constexpr int PROG_BYTES = 8 * 1024;             // the CTA's section of the program
 constexpr int RING_BUDGET = 148 * 1024;
 constexpr int ATTN_BYTES = 64 * 1024;            // key / value chunks and merge buffers of the attention tasks
@@ -35,7 +36,7 @@ constexpr int AW = 4;                            // warps of the task group
 constexpr uint64_t WAIT_NS = 500000000ull;       // every wait gives up after half a second
 
 struct PassShared {
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[MAX_ACC], tmem_empty[MAX_ACC];
     uint32_t tmem_base;
     int abort_flag, epi_abort, aux_flag;
     float scale[8];
@@ -161,17 +162,17 @@ __device__ void reduce_task(const PassParams& P, PassShared& sh, const PassTask&
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = 0.f;
         if (live) {
-            for (int c0 = 0; c0 < (int)tk.n_pieces; c0 += 4) {
-                float tmp[4][8];
+            for (int c0 = 0; c0 < (int)tk.n_pieces; c0 += 8) {
+                float tmp[8][8];
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
+                for (int cc = 0; cc < 8; ++cc) {
                     const bool okc = c0 + cc < (int)tk.n_pieces;
                     const float* base = partials + (size_t)(okc ? pl[c0 + cc] : 0) * piece_elems + et;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) tmp[cc][i] = (okc && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
                 }
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
+                for (int cc = 0; cc < 8; ++cc)
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[i] += tmp[cc][i];
             }
@@ -285,7 +286,6 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
                                const Abort& ab, int t) {
     constexpr int NT = 32 * AW, CK = 16 * AW;
     constexpr int ROWB = HD * 2, CPR = HD / 8, KS = HD / 16, NV = HD / 8, BUF = CK * ROWB, OLD = HD + 8;
-    if (!aux_broadcast(sh, t, t == 0 && word_wait(words + tk.wait_word, tk.wait_need, ab) ? 1 : 0)) return;
     const int ns = P.n_splits;
     const int split = (int)(tk.item % (uint32_t)ns), rest = (int)(tk.item / (uint32_t)ns);
     const int kvh = rest % P.Hkv, blk = rest / P.Hkv;
@@ -299,6 +299,8 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
     const bf16* kcl = P.kc + (size_t)it * P.kv_layer_elems;
     const bf16* vcl = P.vc + (size_t)it * P.kv_layer_elems;
 
+    // The row plan (positions, slots) was written by the kernel before this one: it needs no wait, and neither do the
+    // cache positions in front of the pass's first new one, which earlier passes wrote.
     int mp = lane < nr ? __ldcg(P.row_pos + r0 + lane) : -1;
     const int slot = __ldcg(P.row_slot + r0);
 #pragma unroll
@@ -307,6 +309,15 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
     const int slice = (((len + ns - 1) / ns) + 15) & ~15;
     const int p_begin = split * slice;
     const int np = max(0, min(p_begin + slice, len) - p_begin);
+    int new_begin;                                           // first position this pass appends for the block's sequence
+    {
+        const int seq_first = (blk / bps) * P.rows_per_seq;
+        const int fp = lane < min(P.rows_per_seq, 32) ? __ldcg(P.row_pos + seq_first + lane) : -1;
+        int nb = fp >= 0 ? fp : 0x7fffffff;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nb = min(nb, __shfl_xor_sync(0xffffffffu, nb, o));
+        new_begin = nb == 0x7fffffff ? 0 : nb;
+    }
 
     const int j_lo = gid, j_hi = gid + 8;
     const bf16* q_lo = P.q + ((size_t)(r0 + j_lo / group) * P.H + kvh * group + j_lo % group) * HD;
@@ -318,27 +329,42 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
 
     const bf16* K = kcl + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
     const bf16* V = vcl + (((size_t)slot * P.Hkv + kvh) * P.max_ctx + p_begin) * HD;
-    auto issue = [&](int c) {
+    // keys [k_lo, k_hi) of chunk c -> buffer c & 1: [K][V]; last: also clears the padding rows; one copy group per call
+    auto issue_part = [&](int c, int k_lo, int k_hi, bool last) {
         const int nk = min(CK, np - c * CK);
         const uint32_t kb = smem0 + (uint32_t)(c & 1) * 2u * BUF, vb = kb + BUF;
         const bf16* ks = K + (size_t)c * CK * HD;
         const bf16* vs = V + (size_t)c * CK * HD;
-        for (int i = t; i < nk * CPR; i += NT) {
+        for (int i = k_lo * CPR + t; i < k_hi * CPR; i += NT) {
             const int key = i / CPR, ch = i % CPR;
             const uint32_t off = (uint32_t)key * ROWB + (uint32_t)((ch ^ (key & 7)) << 4);
             cp_async16(kb + off, ks + (size_t)i * 8);
             cp_async16(vb + off, vs + (size_t)i * 8);
         }
         const int nk16 = (nk + 15) & ~15;         // value rows past the slice inside a warp's 16-key group must be finite
-        for (int i = nk * CPR + t; i < nk16 * CPR; i += NT) {
+        for (int i = nk * CPR + t; last && i < nk16 * CPR; i += NT) {
             const int key = i / CPR, ch = i % CPR;
             *reinterpret_cast<uint4*>(sm_raw + (size_t)(c & 1) * 2 * BUF + BUF + (size_t)key * ROWB + ((ch ^ (key & 7)) << 4)) = make_uint4(0, 0, 0, 0);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
+    const int n_chunks = (np + CK - 1) / CK;
+    int old[2] = {0, 0};
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+        if (c < n_chunks) {
+            old[c] = max(0, min(min(CK, np - c * CK), new_begin - (p_begin + c * CK)));
+            issue_part(c, 0, old[c], false);
+        }
+    // the queries and the keys / values this pass appends exist once the wave's QKV tiles are reduced
+    if (!aux_broadcast(sh, t, t == 0 && word_wait(words + tk.wait_word, tk.wait_need, ab) ? 1 : 0)) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        return;
+    }
     if (np > 0) {
-        const int n_chunks = (np + CK - 1) / CK;
-        issue(0);
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+            if (c < n_chunks) issue_part(c, old[c], min(CK, np - c * CK), true);
         uint32_t a[KS][4];
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
@@ -351,7 +377,8 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
         const int pos_hi = j_hi < nq ? __ldcg(P.row_pos + r0 + j_hi / group) : -1;
         const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
         for (int c = 0; c < n_chunks; ++c) {
-            if (c + 1 < n_chunks) { issue(c + 1); asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+            // chunks c and c + 1 are in flight (one copy group each after the first two chunks' early parts)
+            if (c + 1 < n_chunks) asm volatile("cp.async.wait_group 1;" ::: "memory");
             else asm volatile("cp.async.wait_group 0;" ::: "memory");
             aux_bar();
             const int nk = min(CK, np - c * CK);
@@ -420,6 +447,7 @@ __device__ void attention_task(const PassParams& P, PassShared& sh, uint8_t* sm_
                 }
             }
             aux_bar();
+            if (c + 2 < n_chunks) issue_part(c + 2, 0, min(CK, np - (c + 2) * CK), true);      // the buffer just read is free again
         }
         l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
@@ -539,14 +567,15 @@ k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ Pas
         uint4* dst = reinterpret_cast<uint4*>(dyn);
         for (uint32_t i = threadIdx.x; i < (o1 - o0) / 16u && i < PROG_BYTES / 16u; i += NUM_THREADS) dst[i] = src[i];
     }
+    const int n_acc = max(2, min(MAX_ACC, 512 / P.m_pad));
     uint32_t tmem_cols = 32;
-    while (tmem_cols < 2u * (uint32_t)P.m_pad) tmem_cols <<= 1;
+    while (tmem_cols < (uint32_t)(n_acc * P.m_pad)) tmem_cols <<= 1;
     if (threadIdx.x == 0) {
         for (int s = 0; s < P.stages; ++s) {
             mbar_init(smem_u32(&sh.full[s]), 2);           // the weight block and the input rows arrive from two producers
             mbar_init(smem_u32(&sh.empty[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
+        for (int b = 0; b < n_acc; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
         sh.abort_flag = 0; sh.epi_abort = 0; sh.aux_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -622,28 +651,32 @@ k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ Pas
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.m_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
             const uint64_t desc0 = umma_desc(ring0);
-            int stage = 0; uint32_t use = 0, seg = 0; bool ok = true;
+            int stage = 0; uint32_t use = 0, acc_phase = 0; bool ok = true;       // acc_phase: bit a = parity of accumulator a's uses so far
             for (int it = 0; it < n_it && ok; ++it) {
                 const int k = it == P.n_layers ? 1 : 0;
-                for (int si = 0; si < pg.n_seg[k] && ok; ++si, ++seg) {
-                    const int n_kb = (int)pg.segs[k][si].n_kb;
-                    const uint32_t buf = seg & 1u;
+                for (int si = 0; si < pg.n_seg[k] && ok; ++si) {
+                    const PassSeg sg = pg.segs[k][si];
+                    const int n_kb = (int)sg.n_kb;
+                    const uint32_t acc = (uint32_t)sg.flags >> 4;
+                    const uint32_t cont = (sg.flags & SEG_FIRST) ? 0u : 1u;           // 0: the segment starts a fresh accumulator
                     unsigned long long* stamp = P.stamps ? P.stamps + (((size_t)blockIdx.x * n_it + it) * P.stamp_segs + si) * 2 : nullptr;
-                    if (!mbar_wait_b(smem_u32(&sh.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, ab)) { ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (!cont) {                                                       // ... once the epilogue has drained its last use
+                        if (!mbar_wait_b(smem_u32(&sh.tmem_empty[acc]), ((acc_phase >> acc) & 1u) ^ 1u, ab)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    }
                     if (stamp) stamp[0] = global_ns();
-                    const uint32_t d_tmem = tmem_base + buf * (uint32_t)P.m_pad;
+                    const uint32_t d_tmem = tmem_base + acc * (uint32_t)P.m_pad;
                     for (int j = 0; j < n_kb; ++j) {
                         if (!mbar_wait_b(smem_u32(&sh.full[stage]), use & 1u, ab)) { ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint64_t da = desc0 + (uint64_t)((uint32_t)stage * (stage_bytes >> 4)), db = da + (A_BYTES >> 4);
 #pragma unroll
                         for (uint32_t kk = 0; kk < TILE_K / 16; ++kk)
-                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, ((uint32_t)j | kk) != 0u);
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, cont | (uint32_t)j | kk);
                         umma_commit(smem_u32(&sh.empty[stage]));
                         ring_next(stage, use, P.stages);
                     }
-                    if (ok) umma_commit(smem_u32(&sh.tmem_full[buf]));
+                    if (ok && (sg.flags & SEG_LAST)) { umma_commit(smem_u32(&sh.tmem_full[acc])); acc_phase ^= 1u << acc; }
                     if (stamp) stamp[1] = global_ns();
                 }
             }
@@ -652,22 +685,24 @@ k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ Pas
         // ------------------------------------------------------------------ TMEM -> workspace, one piece per segment
         const uint32_t quarter = (uint32_t)(warp & 3);
         const int et = quarter * 32 + lane;
-        uint32_t seg = 0;
+        uint32_t acc_phase = 0;
         bool ok = true;
         for (int it = 0; it < n_it && ok; ++it) {
             const int k = it == P.n_layers ? 1 : 0;
             uint32_t* words = P.sync + (size_t)it * P.words_per_layer;
-            for (int si = 0; si < pg.n_seg[k]; ++si, ++seg) {
+            for (int si = 0; si < pg.n_seg[k]; ++si) {
                 const PassSeg sg = pg.segs[k][si];
-                const uint32_t buf = seg & 1u;
-                if (!mbar_wait_b(smem_u32(&sh.tmem_full[buf]), (seg >> 1) & 1u, ab)) sh.epi_abort = 1;
+                if (!(sg.flags & SEG_LAST)) continue;             // the accumulator goes on in a later segment
+                const uint32_t acc = (uint32_t)sg.flags >> 4;
+                if (!mbar_wait_b(smem_u32(&sh.tmem_full[acc]), (acc_phase >> acc) & 1u, ab)) sh.epi_abort = 1;
+                acc_phase ^= 1u << acc;
                 epi_bar();
                 if (sh.epi_abort) { ok = false; break; }      // all four warps leave together
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 float* out = P.partials[sg.mat & 1] + (size_t)sg.slot * P.m_tok * TILE_N;
                 for (int c0 = 0; c0 < P.m_pad; c0 += 16) {
                     uint32_t r[16];
-                    tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)P.m_pad + (uint32_t)c0, r);
+                    tmem_ld16(tmem_base + ((quarter * 32u) << 16) + acc * (uint32_t)P.m_pad + (uint32_t)c0, r);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
@@ -675,7 +710,7 @@ k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ Pas
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[buf]));
+                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[acc]));
                 epi_bar();                                    // the four warps' stores are ordered before the release below
                 if (et == 0) word_add(words + sg.arrive);
             }
@@ -689,10 +724,13 @@ k_pass_stream(const __grid_constant__ PassMaps maps, const __grid_constant__ Pas
             uint32_t* words = P.sync + (size_t)it * P.words_per_layer;
             for (int ti = 0; ti < pg.n_task[k]; ++ti) {
                 const PassTask tk = pg.tasks[k][ti];
+                unsigned long long* ts = (P.task_stamps && ti < P.stamp_tasks) ? P.task_stamps + (((size_t)blockIdx.x * n_it + it) * P.stamp_tasks + ti) * 2 : nullptr;
+                if (ts && t == 0) ts[0] = global_ns();
                 // (after a wait has given up, the remaining tasks return at their own wait: every branch here is taken by all 128 threads)
                 if (tk.kind == TASK_REDUCE) reduce_task(P, sh, tk, pg.pieces + tk.piece0, it, words, ab, t);
                 else if (P.hd == 128) attention_task<128>(P, sh, attn_smem, tk, it, words, ab, t);
                 else attention_task<64>(P, sh, attn_smem, tk, it, words, ab, t);
+                if (ts && t == 0) ts[1] = global_ns();
             }
         }
     }
@@ -756,7 +794,7 @@ size_t pass_stream_smem(int m_pad, int* stages_out) {
 cudaError_t launch_pass_stream(const PassMaps& maps, const PassParams& p, int grid, int dependent, cudaStream_t st) {
     int stages = 0;
     const size_t smem = pass_stream_smem(p.m_pad, &stages);
-    if (p.stages != stages || p.m_pad < 16 || p.m_pad > 256 || (p.m_pad & 15) || p.m_tok > p.m_pad || grid < 1) return cudaErrorInvalidValue;
+    if (p.stages < 2 || p.stages > stages || p.m_pad < 16 || p.m_pad > 256 || (p.m_pad & 15) || p.m_tok > p.m_pad || grid < 1) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(k_pass_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     return launch_pdl(k_pass_stream, dim3(grid), dim3(NUM_THREADS), smem, st, dependent, maps, p);

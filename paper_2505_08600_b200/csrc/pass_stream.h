@@ -43,6 +43,8 @@ struct PassParams {
     float* part_o; float* part_ml; uint32_t* att_counters;
     // optional time stamps: [cta][iteration][segment][2] = (MMA thread starts waiting for the segment, segment committed)
     unsigned long long* stamps; int stamp_segs;
+    // ... and [cta][iteration][task][2] = (the task warps turn to the task, the task is done), for the first stamp_tasks tasks
+    unsigned long long* task_stamps; int stamp_tasks;
 };
 
 bool make_tensor_map_layers(TensorMap* out, const void* base, int rows, int K, int n_layers, size_t layer_stride_bytes);
