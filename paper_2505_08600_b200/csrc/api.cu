@@ -61,7 +61,7 @@ enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
 
 constexpr size_t ARRIVE_WORDS = 65536;          // arrival words of one pass (the 13B target needs about 17,000)
 constexpr int PASS_ROWS_CAP = 32;               // most query rows of a pass on the persistent streaming kernel
-constexpr size_t PASS_REGION_BYTES = (size_t)48 << 20;      // each of the two workspace regions of that kernel
+constexpr size_t PASS_REGION_BYTES = (size_t)64 << 20;      // each of the two workspace regions of that kernel
 constexpr size_t PASS_PROG_BYTES = (size_t)768 << 10;       // one cached program
 constexpr int PASS_PROG_SLOTS = 8;
 
@@ -80,12 +80,15 @@ struct sd_ctx {
     size_t arrive_used;                         // words handed out to the GEMMs of the pass being enqueued
     float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
     // persistent streaming kernel (pass_stream.cu): packed input rows, workspace, programs
-    uint8_t* xp_xn; uint8_t* xp_attn; uint8_t* xp_act;
-    float* pass_partials[2];
+    // (everything CTAs of that kernel hand to one another is tagged 64-bit words; the whole block is cleared when tags are about to repeat)
+    tagged_t* tg_h; tagged_t* tg_xn; tagged_t* tg_attn; tagged_t* tg_act; tagged_t* tg_q; tagged_t* tg_newkv; tagged_t* tg_ssq;
+    tagged_t* tg_partials[2];
+    tagged_t* tg_part_o; tagged_t* tg_part_ml;
+    char* tg_begin; char* tg_end;               // extent of the tagged buffers
+    uint32_t* pass_epoch;                       // device: number of the pass; pass_epoch + 1: the abort word
+    uint64_t pass_count;                        // host: passes enqueued so far (mirrors the device word)
+    bool tags_due_clear;                        // the tagged buffers are to be cleared before the next launch sequence
     uint8_t* pass_prog;
-    uint32_t* pass_sync;                        // the kernel's arrival / completion words (cleared at the start of every pass)
-    float* pass_part_o; float* pass_part_ml; uint32_t* pass_att_counters;
-    size_t pass_att_counter_words;
     bool pass_on, pass_drafts; int pass_max_rows;
     PassTuning pass_tuning; bool pass_tuned; int pass_stages;
     struct CachedProgram { int model, m_tok, rows_per_seq, n_splits, want_logits, slot; PassProgram meta; uint64_t last_use; };
@@ -93,7 +96,7 @@ struct sd_ctx {
     unsigned long long* stamps; size_t stamps_words;          // optional time stamps of the next passes (caller's buffer)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
-    struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; };
+    struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; uint64_t passes; };
     std::vector<CachedGraph> graphs;
     uint64_t graph_clock;
     // classifier
@@ -227,21 +230,28 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
     c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
     c->rope_row_sin = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
-    {   // persistent streaming kernel: input rows in the packed layout ([k block][row][64], up to PASS_ROWS_CAP rows padded to 16)
+    {   // persistent streaming kernel: tagged 64-bit words for up to PASS_ROWS_CAP rows (padded to a multiple of 16)
         const size_t rows_pad = (PASS_ROWS_CAP + 15) & ~15;
-        c->xp_xn = (uint8_t*)B.take((size_t)((d_max + 63) / 64) * rows_pad * 128);
-        c->xp_attn = (uint8_t*)B.take((size_t)((dq_max + 63) / 64) * rows_pad * 128);
-        c->xp_act = (uint8_t*)B.take((size_t)((f_max + 63) / 64) * rows_pad * 128);
-        c->pass_partials[0] = (float*)B.take(PASS_REGION_BYTES);
-        c->pass_partials[1] = (float*)B.take(PASS_REGION_BYTES);
+        int h_max = 1, hd_max = 8, kvd_max = 8;
+        for (int i = 0; i < nm; ++i) {
+            h_max = std::max(h_max, (int)ms[i].n_heads); hd_max = std::max(hd_max, (int)ms[i].head_dim);
+            kvd_max = std::max(kvd_max, (int)(ms[i].n_kv_heads * ms[i].head_dim));
+        }
+        c->tg_begin = (char*)B.take(0);
+        c->tg_h = (tagged_t*)B.take(sizeof(tagged_t) * rows_pad * d_max);
+        c->tg_xn = (tagged_t*)B.take(sizeof(tagged_t) * (size_t)((d_max + 63) / 64) * rows_pad * 32);
+        c->tg_attn = (tagged_t*)B.take(sizeof(tagged_t) * (size_t)((dq_max + 63) / 64) * rows_pad * 32);
+        c->tg_act = (tagged_t*)B.take(sizeof(tagged_t) * (size_t)((f_max + 63) / 64) * rows_pad * 32);
+        c->tg_q = (tagged_t*)B.take(sizeof(tagged_t) * rows_pad * (dq_max / 2));
+        c->tg_newkv = (tagged_t*)B.take(sizeof(tagged_t) * rows_pad * 2 * (kvd_max / 2));
+        c->tg_ssq = (tagged_t*)B.take(sizeof(tagged_t) * rows_pad * SSQ_STRIDE);
+        c->tg_partials[0] = (tagged_t*)B.take(PASS_REGION_BYTES);
+        c->tg_partials[1] = (tagged_t*)B.take(PASS_REGION_BYTES);
+        c->tg_part_o = (tagged_t*)B.take(sizeof(tagged_t) * (size_t)PASS_ROWS_CAP * h_max * 32 * hd_max);
+        c->tg_part_ml = (tagged_t*)B.take(sizeof(tagged_t) * (size_t)PASS_ROWS_CAP * h_max * 32 * 2);
+        c->tg_end = (char*)B.take(0);
+        c->pass_epoch = (uint32_t*)B.take(sizeof(uint32_t) * 2);
         c->pass_prog = (uint8_t*)B.take(PASS_PROG_BYTES * PASS_PROG_SLOTS);
-        c->pass_sync = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
-        int h_max = 1, hd_max = 8;
-        for (int i = 0; i < nm; ++i) { h_max = std::max(h_max, (int)ms[i].n_heads); hd_max = std::max(hd_max, (int)ms[i].head_dim); }
-        c->pass_part_o = (float*)B.take(sizeof(float) * (size_t)PASS_ROWS_CAP * h_max * 32 * hd_max);
-        c->pass_part_ml = (float*)B.take(sizeof(float) * (size_t)PASS_ROWS_CAP * h_max * 32 * 2);
-        c->pass_att_counter_words = (size_t)PASS_ROWS_CAP * h_max;
-        c->pass_att_counters = (uint32_t*)B.take(sizeof(uint32_t) * c->pass_att_counter_words);
     }
     const size_t V0 = ms[0].vocab, g_max = std::max(cfg.max_gamma, 1);
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
@@ -308,6 +318,22 @@ enum LogitsMode { LOGITS_NONE = 0, LOGITS_ALL = 1, LOGITS_LAST = 2 };
 // One pass of a model over n_rows query rows described by `plan`.
 sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan, int n_rows, int mode, float* logits_out);
 
+// The tags of a pass derive from its number (a device word that every pass bumps).  Well before numbers repeat, every tagged
+// word is cleared: note_passes counts, clear_tags_if_due runs between launch sequences (never inside a capture).
+void note_passes(sd_ctx* c, uint64_t n) {
+    const uint64_t period = PASS_EPOCH_WRAP / 2;
+    if ((c->pass_count + n) / period != c->pass_count / period) c->tags_due_clear = true;
+    c->pass_count += n;
+}
+
+cudaError_t clear_tags_if_due(sd_ctx* c) {
+    if (!c->tags_due_clear) return cudaSuccess;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(c->st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return cudaSuccess;
+    c->tags_due_clear = false;
+    return cudaMemsetAsync(c->tg_begin, 0, c->tg_end - c->tg_begin, c->st);
+}
+
 sd_ctx::CachedProgram* find_program(sd_ctx* c, int model, int m_tok, int rows_per_seq, int n_splits, int want_logits) {
     for (auto& p : c->programs)
         if (p.model == model && p.m_tok == m_tok && p.rows_per_seq == rows_per_seq && p.n_splits == n_splits && p.want_logits == want_logits) return &p;
@@ -347,9 +373,8 @@ sd_status prepare_pass(sd_ctx* c, int model, const RowPlan& plan, int n_rows, in
     cp.model = model; cp.m_tok = n_rows; cp.rows_per_seq = plan.rows_per_seq; cp.n_splits = ns; cp.want_logits = want; cp.last_use = c->graph_clock;
     cp.meta = build_pass_program(sh, c->pass_tuned ? c->pass_tuning : default_pass_tuning(sh));
     const bool fits = cp.meta.error.empty() && cp.meta.blob.size() <= PASS_PROG_BYTES && cp.meta.max_section <= 8192 &&
-                      (size_t)cp.meta.total_words + 2 <= ARRIVE_WORDS &&
-                      (size_t)std::max(cp.meta.slots[0], cp.meta.slots[1]) * n_rows * 128 * sizeof(float) <= PASS_REGION_BYTES &&
-                      (size_t)cp.meta.n_blocks * m.n_kv_heads <= (size_t)PASS_ROWS_CAP * m.n_heads;
+                      (size_t)std::max(cp.meta.slots[0], cp.meta.slots[1]) * n_rows * 128 * sizeof(tagged_t) <= PASS_REGION_BYTES &&
+                      m.n_layers < 255;
     if (!fits) {                                      // remembered, so that the pass quietly takes the kernel-per-matrix path
         cp.slot = -1; cp.meta.blob.clear();
         c->programs.push_back(cp);
@@ -393,7 +418,7 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, st));
+                                         nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -451,7 +476,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, 0, st));
+                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, 0, nullptr, st));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
@@ -503,11 +528,12 @@ sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, con
     P.n_out[MAT_QKV] = M.n_qkv(); P.n_out[MAT_WO] = d; P.n_out[MAT_GU] = 2 * m.d_ffn; P.n_out[MAT_DN] = d; P.n_out[MAT_LM] = m.vocab;
     (void)pass_stream_smem(P.m_pad, &P.stages);
     if (c->pass_stages >= 2 && c->pass_stages < P.stages) P.stages = c->pass_stages;
-    P.words_per_layer = cp.meta.words_per_layer;
-    P.h = c->h; P.xn = c->xp_xn; P.attn = c->xp_attn; P.act = c->xp_act;
-    P.x[MAT_QKV] = c->xp_xn; P.x[MAT_WO] = c->xp_attn; P.x[MAT_GU] = c->xp_xn; P.x[MAT_DN] = c->xp_act; P.x[MAT_LM] = c->xp_xn;
-    P.q = (bf16*)c->q; P.kc = (bf16*)M.kcache; P.vc = (bf16*)M.vcache; P.kv_layer_elems = M.kv_layer_bytes / sizeof(bf16);
-    P.row_slot = c->row_slot; P.row_pos = c->row_pos; P.rcos = c->rope_row_cos; P.rsin = c->rope_row_sin; P.ssq = c->ssq;
+    P.epoch = c->pass_epoch;
+    P.h = c->tg_h; P.xn = c->tg_xn; P.attn = c->tg_attn; P.act = c->tg_act;
+    P.x[MAT_QKV] = c->tg_xn; P.x[MAT_WO] = c->tg_attn; P.x[MAT_GU] = c->tg_xn; P.x[MAT_DN] = c->tg_act; P.x[MAT_LM] = c->tg_xn;
+    P.q = c->tg_q; P.newkv = c->tg_newkv;
+    P.kc = (bf16*)M.kcache; P.vc = (bf16*)M.vcache; P.kv_layer_elems = M.kv_layer_bytes / sizeof(bf16);
+    P.row_slot = c->row_slot; P.row_pos = c->row_pos; P.rcos = c->rope_row_cos; P.rsin = c->rope_row_sin; P.ssq = c->tg_ssq;
     P.norm1 = M.layers[0].norm1; P.norm2 = M.layers[0].norm2;
     P.norm_stride = m.n_layers > 1 ? (size_t)(M.layers[1].norm1 - M.layers[0].norm1) : 0;
     P.final_norm = M.final_norm; P.rms_eps = m.rms_eps;
@@ -515,11 +541,11 @@ sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, con
     const int R = plan.rows_per_seq;
     if (mode == LOGITS_LAST) { P.logits_rows = list.n; P.row_stride = R; P.row_offset = R - 1; }
     else { P.logits_rows = n_rows; P.row_stride = 1; P.row_offset = 0; }
-    P.partials[0] = c->pass_partials[0]; P.partials[1] = c->pass_partials[1];
-    P.sync = c->pass_sync; P.abort_word = c->pass_sync + cp.meta.total_words; P.status = c->S.status;
+    P.partials[0] = c->tg_partials[0]; P.partials[1] = c->tg_partials[1];
+    P.abort_word = c->pass_epoch + 1; P.status = c->S.status;
     P.program = c->pass_prog + (size_t)cp.slot * PASS_PROG_BYTES;
     P.rows_per_seq = R; P.rows_per_block = cp.meta.rows_per_block; P.n_splits = cp.n_splits;
-    P.part_o = c->pass_part_o; P.part_ml = c->pass_part_ml; P.att_counters = c->pass_att_counters;
+    P.part_o = c->tg_part_o; P.part_ml = c->tg_part_ml;
     const int n_it = m.n_layers + P.has_tail;
     const size_t seg_words = (size_t)sm_count() * n_it * cp.meta.max_seg * 2, task_words = (size_t)sm_count() * n_it * 16 * 2;
     if (c->stamps && seg_words + task_words <= c->stamps_words) {
@@ -527,9 +553,13 @@ sd_status forward_pass(sd_ctx* c, Model& M, const sd_ctx::CachedProgram& cp, con
         P.task_stamps = c->stamps + seg_words; P.stamp_tasks = 16;
     }
     CUDA_TRY(prof_mark(c, CAT_STATE));
-    CUDA_TRY(cudaMemsetAsync(c->pass_sync, 0, sizeof(uint32_t) * ((size_t)cp.meta.total_words + 1), st));
-    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, m.dtype, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         M.layers[0].norm1, c->xp_xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, P.m_pad, st));
+    // The tags of a pass derive from its number; well before numbers repeat, every tagged word is cleared.
+    CUDA_TRY(clear_tags_if_due(c));
+    note_passes(c, 1);
+    LAUNCH(CAT_STATE, launch_pass_begin(c->pass_epoch, c->pass_epoch + 1, st));
+    LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, m.dtype, d, m.vocab, (float*)c->tg_h, c->row_slot, c->row_pos,
+                                         M.layers[0].norm1, c->tg_xn, (float*)c->tg_ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin,
+                                         P.m_pad, c->pass_epoch, st));
     LAUNCH(CAT_LINEAR, launch_pass_stream(M.pmaps, P, sm_count(), 1, st));
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
@@ -553,16 +583,18 @@ int bound_bucket(int bound) { return (bound + 255) & ~255; }
 
 template <class Body>
 sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
+    CUDA_TRY(clear_tags_if_due(c));
     if (!c->graphs_on || c->prof_on) return body();
     c->graph_clock += 1;
     for (auto& g : c->graphs)
         if (g.key == key.bytes) {
             CUDA_TRY(cudaGraphLaunch(g.exec, c->st));
             c->launches += g.launches;
+            note_passes(c, g.passes);
             g.last_use = c->graph_clock;
             return SD_OK;
         }
-    const uint64_t l0 = c->launches;
+    const uint64_t l0 = c->launches, p0 = c->pass_count;
     if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         (void)cudaGetLastError();                       // e.g. the legacy default stream cannot capture:
         c->graphs_on = false;                           // launch kernel by kernel from now on
@@ -586,7 +618,7 @@ sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
         cudaGraphExecDestroy(c->graphs[victim].exec);
         c->graphs.erase(c->graphs.begin() + victim);
     }
-    c->graphs.push_back({key.bytes, exec, c->launches - l0, c->graph_clock});
+    c->graphs.push_back({key.bytes, exec, c->launches - l0, c->graph_clock, c->pass_count - p0});
     CUDA_TRY(cudaGraphLaunch(exec, c->st));
     return SD_OK;
 }
@@ -677,11 +709,12 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         cudaMemsetAsync(c->gemm_arrive, 0, sizeof(uint32_t) * ARRIVE_WORDS, st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
-    if (cudaMemsetAsync(c->xp_xn, 0, (char*)c->pass_partials[0] - (char*)c->xp_xn, st) != cudaSuccess ||
-        cudaMemsetAsync(c->pass_att_counters, 0, sizeof(uint32_t) * c->pass_att_counter_words, st) != cudaSuccess ||
+    if (cudaMemsetAsync(c->tg_begin, 0, c->tg_end - c->tg_begin, st) != cudaSuccess ||          // no word carries a tag a pass could expect
+        cudaMemsetAsync(c->pass_epoch, 0, 2 * sizeof(uint32_t), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
-    c->pass_on = true; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
+    c->pass_count = 0; c->tags_due_clear = false;
+    c->pass_on = false; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
     c->force_plain = false;
     c->graphs_on = true;
     c->graph_clock = 0;

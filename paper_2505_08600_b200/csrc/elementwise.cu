@@ -14,7 +14,7 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
                         float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos,
                         const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq,
                         const float* __restrict__ rcos, const float* __restrict__ rsin, int half,
-                        float* __restrict__ row_cos, float* __restrict__ row_sin, int packed_m_pad) {
+                        float* __restrict__ row_cos, float* __restrict__ row_sin, int tagged_m_pad, const uint32_t* __restrict__ epoch) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const int i = r / plan.rows_per_seq, j = r % plan.rows_per_seq;
@@ -45,15 +45,28 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
         }
     const T* e = embed + (size_t)tok * d;
     float ss = 0.f;
+    if (tagged_m_pad) {
+        // For the persistent streaming kernel: h, the first norm's operand and the row's sum of squares as tagged 64-bit
+        // words (payload + the pass's tag), the operand as [k block][row][32 words of two bf16].
+        const uint32_t tag = pass_tag(*epoch, 0, 1);
+        tagged_t* th = reinterpret_cast<tagged_t*>(h);
+        tagged_t* txn = reinterpret_cast<tagged_t*>(xn);
+        for (int k = 2 * threadIdx.x; k < d; k += 2 * blockDim.x) {
+            const float v0 = to_f32<T>(e[k]), v1 = to_f32<T>(e[k + 1]);
+            th[(size_t)r * d + k] = ((tagged_t)tag << 32) | __float_as_uint(v0);
+            th[(size_t)r * d + k + 1] = ((tagged_t)tag << 32) | __float_as_uint(v1);
+            const uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(v0 * gain[k])), hi = __bfloat16_as_ushort(__float2bfloat16_rn(v1 * gain[k + 1]));
+            txn[xtagged_index(r, k, tagged_m_pad)] = ((tagged_t)tag << 32) | lo | (hi << 16);
+            ss += v0 * v0 + v1 * v1;
+        }
+        ss = block_sum(ss, red);
+        if (threadIdx.x == 0) reinterpret_cast<tagged_t*>(ssq)[(size_t)r * 64] = ((tagged_t)tag << 32) | __float_as_uint(ss);
+        return;
+    }
     for (int k = threadIdx.x; k < d; k += blockDim.x) {
         const float v = to_f32<T>(e[k]);
         h[(size_t)r * d + k] = v;
-        if (gain) {
-            const bf16 g = __float2bfloat16_rn(v * gain[k]);
-            if (packed_m_pad) *reinterpret_cast<bf16*>(reinterpret_cast<uint8_t*>(xn) + xpacked_offset(r, k, packed_m_pad)) = g;   // layout of the streaming kernel's input rows
-            else xn[(size_t)r * d + k] = g;
-            ss += v * v;
-        }
+        if (gain) { xn[(size_t)r * d + k] = __float2bfloat16_rn(v * gain[k]); ss += v * v; }
     }
     if (gain) {                          // first half of the first layer's RMSNorm: the 1/rms factor follows the GEMM
         ss = block_sum(ss, red);
@@ -64,14 +77,14 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
 cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& plan, int n_rows,
                          const void* embed, int dtype, int d, int vocab,
                          float* h, int32_t* row_slot, int32_t* row_pos, const float* gain, void* xn, float* ssq,
-                         const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, int packed_m_pad,
-                         cudaStream_t st) {
+                         const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, int tagged_m_pad,
+                         const uint32_t* epoch, cudaStream_t st) {
     if (dtype == SD_BF16)
         k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq,
-                                              rope_cos, rope_sin, half, row_cos, row_sin, packed_m_pad);
+                                              rope_cos, rope_sin, half, row_cos, row_sin, tagged_m_pad, epoch);
     else
         k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr,
-                                               nullptr, nullptr, 0, nullptr, nullptr, 0);
+                                               nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr);
     return cudaGetLastError();
 }
 

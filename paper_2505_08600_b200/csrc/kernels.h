@@ -13,7 +13,8 @@ cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& 
                          void* xn, float* ssq,
                          const float* rope_cos, const float* rope_sin, int half,      // position tables [max_ctx][half]
                          float* row_cos, float* row_sin /*nullable: [row][half] factors of each row's position*/,
-                         int packed_m_pad /*0: xn is [row][d]; else xn is in the streaming kernel's packed layout for m_pad rows*/, cudaStream_t st);
+                         int tagged_m_pad /*0: plain h, xn [row][d], ssq; else all three as tagged 64-bit words for the streaming kernel (m_pad rows)*/,
+                         const uint32_t* epoch /*device word the tags derive from (tagged mode)*/, cudaStream_t st);
 // xn[i] = rmsnorm(h[src_row(i)]) * gain; src_row(i) = i * row_stride + row_offset
 cudaError_t launch_rmsnorm(const float* h, const float* gain, void* xn, int dtype, int n_rows, int d, float eps,
                            int row_stride, int row_offset, cudaStream_t st);

@@ -248,7 +248,7 @@ struct Builder {
 PassTuning default_pass_tuning(const PassShape& s) {
     (void)s;
     PassTuning t;
-    const int w[N_MAT] = {2, 2, 4, 2, 2};
+    const int w[N_MAT] = {2, 1, 4, 1, 2};              // measured best on the 7B shape (QKV and gate/up in waves, the thin Wo and down whole)
     for (int m = 0; m < N_MAT; ++m) { t.waves[m] = w[m]; t.chunk_major[m] = 0; }
     return t;
 }
@@ -377,9 +377,12 @@ std::string check_pass_program(const PassShape& s, const PassProgram& p) {
                 if (have < tk.wait_need) break;
                 if (tk.kind == TASK_REDUCE && have != tk.wait_need) return "a tile received more pieces than its task expects";
                 bool counts = tk.done_word != NO_WORD;
-                if (tk.kind == TASK_ATTENTION) {          // an attention item counts once per (query block, kv head): its last slice to deliver
+                if (tk.kind == TASK_ATTENTION) {
+                    // an item's slice 0 merges the others: it finishes (and the item counts) only when they have all delivered
                     if (tk.item / (uint32_t)s.n_splits >= (uint32_t)n_items) return "attention item out of range";
-                    counts = ++slices_in[(size_t)A.it_t * n_items + tk.item / (uint32_t)s.n_splits] == s.n_splits;
+                    int& in = slices_in[(size_t)A.it_t * n_items + tk.item / (uint32_t)s.n_splits];
+                    if (tk.item % (uint32_t)s.n_splits == 0u) { if (in < s.n_splits - 1) break; }
+                    else { ++in; counts = false; }
                 }
                 if (counts) words[word_of(A.it_t, tk.done_word, false)] += 1;
                 ++A.ti; --remaining; progress = true;

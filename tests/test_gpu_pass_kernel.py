@@ -1,0 +1,77 @@
+"""The persistent streaming kernel (one launch per forward pass, tagged-word hand-offs) against the CPU oracle and
+against the kernel-per-matrix path, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_08600_b200 import synth
+from gpu_util import DEV
+from test_gpu_model import SMALL_BF16, SMALL_BF16_DRAFT, WIDE_BF16, FULL_WIDTH, _build, _replay
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sd():
+    from paper_2505_08600_b200 import binding
+    binding.lib()
+    return binding
+
+
+@pytest.mark.parametrize("T,drafts_too", [(0.7, 0), (0.0, 0), (0.0, 1)])
+def test_small_gqa_teacher_forced_on_the_pass_kernel(sd, T, drafts_too):
+    ctx, om = _build(sd, SMALL_BF16, [SMALL_BF16_DRAFT, SMALL_BF16_DRAFT], "bf16", T, 5, max_ctx=128)
+    ctx.sd_use_pass_kernel(1, drafts_too)
+    prompt = synth.make_prompt(4096, 40, seed=6)
+    r = _replay(sd, ctx, om, 1, prompt, 5, T, 5, 24, "bf16", min_agree=0.6)
+    assert r["iters"] >= 4
+    ctx.close()
+
+
+def test_head_dim_128_and_long_context_on_the_pass_kernel(sd):
+    # 1100 positions: the cache is cut into slices whose partial results one task merges
+    ctx, om = _build(sd, WIDE_BF16, [SMALL_BF16_DRAFT | dict(vocab=8192)], "bf16", 1.0, 7, max_ctx=1280)
+    ctx.sd_use_pass_kernel(1, 0)
+    prompt = synth.make_prompt(8192, 1100, seed=8)
+    _replay(sd, ctx, om, 0, prompt, 3, 1.0, 7, 8, "bf16", min_agree=0.5)
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", sorted(FULL_WIDTH))
+def test_benchmark_shapes_at_full_width_on_the_pass_kernel(sd, name):
+    spec = FULL_WIDTH[name]
+    cfg = synth.CONFIGS[spec["cfg"]]
+    wl = cfg["workload"]
+    t = dict(cfg["target"], n_layers=spec["layers"])
+    d = dict(cfg["drafts"][0], n_layers=1)
+    gamma = wl["gamma"]
+    ctx, om = _build(sd, t, [d], "bf16", wl["temperature"], wl["seed"], max_seqs=1, max_ctx=spec["prompt"] + 40, max_gamma=gamma)
+    ctx.sd_use_pass_kernel(1, 0)
+    prompt = synth.make_prompt(t["vocab"], spec["prompt"], seed=wl["seed"])
+    r = _replay(sd, ctx, om, 0, prompt, gamma, wl["temperature"], wl["seed"], 2 * (gamma + 1), "bf16", min_agree=0.0)
+    assert r["iters"] >= 2
+    ctx.close()
+
+
+def test_pass_kernel_is_bit_reproducible_and_agrees_with_the_other_path(sd):
+    """The pieces of a tile are summed in a fixed order: two runs give identical logits; and the two paths, which round
+    at the same places but sum in different orders, agree to within bf16 noise."""
+    dims = dict(SMALL_BF16, n_layers=3)
+    V, gamma, P = dims["vocab"], 5, 70
+    ctx = sd.Context(dims, [], "bf16", 2, 160, gamma, 1.0, 3)
+    ctx.load_weights(0, synth.make_weights(dims, seed=0, model_index=0, dtype="bf16"))
+    x = torch.from_numpy(synth.make_prompt(V, 2 * gamma, seed=9).reshape(2, gamma).astype(np.int32)).to(DEV)
+    outs = []
+    for on in (1, 1, 0):
+        ctx.sd_use_pass_kernel(on, 0)
+        for s in range(2):
+            ctx.sd_seq_begin(s, synth.make_prompt(V, P - 7 * s, seed=4, seq=s), s)
+        ctx.sd_prefill([0, 1])
+        logits = torch.zeros((2, gamma + 1, V), dtype=torch.float32, device=DEV)
+        ctx.sd_verify([0, 1], gamma, x, logits)
+        outs.append(logits.cpu().numpy().copy())
+    assert ctx.sd_device_status() == 0
+    assert (outs[0] == outs[1]).all()
+    assert np.abs(outs[0].astype(np.float64) - outs[2]).max() <= 2e-2
+    ctx.close()
