@@ -266,6 +266,12 @@ sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, c
  * block, k blocks, matrix, flags, wait word, wait count, arrival word, workspace slot) and 20-byte task records. */
 size_t sd_pass_schedule_blob(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, void* out, size_t cap);
 
+/* With 3..8 query rows (the verify rows of one sequence) the tensor-core path feeds every GEMM its input rows in two
+ * bf16 parts, bf16(x) and bf16(x - bf16(x)), in the columns that the 16-wide MMA covers anyway: the weights stream
+ * once all the same, and the activations enter the products with 16 bits of mantissa instead of 8.  on = 0 switches
+ * that off (one bf16 part, as with other row counts); the tests measure both.  Synchronises, drops cached graphs. */
+sd_status sd_use_two_part_activations(sd_ctx* ctx, int on);
+
 /* Number of kernels this context has launched since sd_create. */
 sd_status sd_launch_count(sd_ctx* ctx, uint64_t* out);
 
@@ -288,7 +294,8 @@ sd_status sd_seq_read(sd_ctx* ctx, int seq, int32_t* tokens_host, int cap, int32
  * length to n_tokens - 1 and the draft cache length to draft_kv_len. */
 sd_status sd_seq_force(sd_ctx* ctx, int seq, const int32_t* tokens_host, int n_tokens, int draft_kv_len, uint32_t iter);
 
-/* Reads and clears the device status word.  Synchronises. */
+/* Reads and clears the device status word.  Synchronises.  Returns SD_ERR_TIMEOUT (with the flags still written) when
+ * SD_DEV_WAIT_EXPIRED is among them: a bounded wait inside a kernel gave up, results of that call are not to be trusted. */
 sd_status sd_device_status(sd_ctx* ctx, uint32_t* flags_out);
 
 /* Plain autoregressive pass of the target over the last token of each listed
@@ -304,6 +311,14 @@ sd_status sd_target_step(sd_ctx* ctx, const int32_t* seqs_host, int n_seq, float
 sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype,
                        int impl, void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t sd_op_linear_workspace(int rows, int n_out, int n_in, int dtype, int impl);
+
+/* sd_op_linear's tensor-core form (3..8 rows) with the bounded wait of the step after the GEMM made to run out, for
+ * tests: the step's CTAs watch arrival words (arrive_dev, at least ceil(n_out / 128) of them) that the GEMM is not told to
+ * count into, for wait_ns nanoseconds; then they fall back to waiting for the GEMM's grid, finish the job and set
+ * SD_DEV_WAIT_EXPIRED in *status_dev.  y must equal sd_op_linear's.  Nothing hangs and nothing faults. */
+sd_status sd_op_linear_wait_expiry(const void* x, const void* w, float* y, int rows, int n_out, int n_in,
+                                   void* workspace, size_t workspace_bytes, uint32_t* arrive_dev, size_t arrive_words,
+                                   unsigned long long wait_ns, uint32_t* status_dev, void* cuda_stream);
 
 /* The bf16 tensor-core form of sd_op_linear for callers that cannot allocate device memory
  * (the paper has no counterpart; this serves embedders).  A host that runs this library

@@ -75,6 +75,7 @@ _PROTOS = {
     "sd_pass_schedule_check": (_i, [_vp, _vp, _vp, _vp, C.c_char_p, _sz]),
     "sd_pass_schedule_blob": (_sz, [_vp, _vp, _vp, _vp, _sz]),
     "sd_force_plain_path": (_i, [_vp, _i]),
+    "sd_use_two_part_activations": (_i, [_vp, _i]),
     "sd_launch_count": (_i, [_vp, C.POINTER(C.c_uint64)]),
     "sd_profile": (_i, [_vp, _i]),
     "sd_profile_read": (_i, [_vp, _vp, _vp]),
@@ -85,6 +86,7 @@ _PROTOS = {
     "sd_op_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_linear_workspace": (_sz, [_i, _i, _i, _i, _i]),
     "sd_op_linear_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sd_op_linear_wait_expiry": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp, _sz, C.c_uint64, _vp, _vp]),
     "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_attention_workspace": (_sz, [_i, _i, _i, _i]),
     "sd_op_philox": (_i, [_vp, _i, C.c_uint32, C.c_uint32, _vp, _vp]),
@@ -309,6 +311,9 @@ class Context:
         self._stamps = stamps
         _check(self.L.sd_pass_stamps(self.h, _dp(stamps), 0 if stamps is None else stamps.numel()), "sd_pass_stamps")
 
+    def sd_use_two_part_activations(self, on):
+        _check(self.L.sd_use_two_part_activations(self.h, int(on)), "sd_use_two_part_activations")
+
     def sd_force_plain_path(self, on):
         _check(self.L.sd_force_plain_path(self.h, int(on)), "sd_force_plain_path")
 
@@ -342,7 +347,9 @@ class Context:
 
     def sd_device_status(self):
         f = C.c_uint32()
-        _check(self.L.sd_device_status(self.h, C.byref(f)), "sd_device_status")
+        st = self.L.sd_device_status(self.h, C.byref(f))
+        if st not in (0, 6):                  # SD_ERR_TIMEOUT comes with the flags: the caller looks at them
+            _check(st, "sd_device_status")
         return f.value
 
 
@@ -372,6 +379,20 @@ def sd_op_linear(x, w, y, dtype, impl=0, stream=None):
     need = lib().sd_op_linear_workspace(rows, n_out, n_in, dtype, impl)
     ws = torch.empty(max(need, 1), dtype=torch.uint8, device=x.device)
     _check(lib().sd_op_linear(_dp(x), _dp(w), _dp(y), rows, n_out, n_in, dtype, impl, _dp(ws), need, _stream_ptr(stream)), "sd_op_linear")
+
+
+def sd_op_linear_wait_expiry(x, w, y, wait_ns, stream=None):
+    """The tensor-core linear with the fused step's bounded wait made to run out; returns the device status word."""
+    rows, n_in = x.shape
+    n_out = w.shape[0]
+    need = lib().sd_op_linear_workspace(rows, n_out, n_in, SD_BF16, 2)
+    ws = torch.empty(max(need, 1), dtype=torch.uint8, device=x.device)
+    words = torch.zeros(((n_out + 127) // 128,), dtype=torch.int32, device=x.device)
+    status = torch.zeros((1,), dtype=torch.int32, device=x.device)
+    _check(lib().sd_op_linear_wait_expiry(_dp(x), _dp(w), _dp(y), rows, n_out, n_in, _dp(ws), need, _dp(words), words.numel(),
+                                          int(wait_ns), _dp(status), _stream_ptr(stream)), "sd_op_linear_wait_expiry")
+    torch.cuda.synchronize()
+    return int(status.item()), words
 
 
 def sd_op_linear_static(x, w, y, stream=None):

@@ -94,6 +94,7 @@ struct sd_ctx {
     struct CachedProgram { int model, m_tok, rows_per_seq, n_splits, want_logits, slot; PassProgram meta; uint64_t last_use; };
     std::vector<CachedProgram> programs;
     unsigned long long* stamps; size_t stamps_words;          // optional time stamps of the next passes (caller's buffer)
+    bool two_part;                              // feed the verify rows' activations to the GEMMs in two bf16 parts (see Epilogue::lo_off)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
     struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; uint64_t passes; };
@@ -118,14 +119,10 @@ namespace {
 
 size_t esize(int dtype) { return dtype == SD_BF16 ? 2 : 4; }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
+int sm_count() {                               // of the current device
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) return v;
+    return 148;
 }
 
 bool valid_desc(const sd_model_desc& m) {
@@ -451,6 +448,7 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
 
 // One weight GEMM and the step that follows it.
 sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
+    if (ep.lo_off) rows += ep.lo_off;           // the input rows come in two bf16 parts: [x_hi rows][x_lo rows at + lo_off]
     const GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
@@ -473,29 +471,37 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     c->arrive_used = 0;                          // the embedding kernel below is an ordinary launch: everything before it has finished
+    // With 3..8 rows (the verify rows of one sequence) the 16 columns of the MMA hold every activation twice over: as
+    // bf16(x) and as bf16(x - bf16(x)), eight rows apart.  The weights stream once all the same, and the GEMMs' inputs
+    // are no longer rounded to 8 bits of mantissa.
+    const int lo = (c->two_part && n_rows >= 3 && n_rows <= 8) ? 8 : 0;
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
-                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, 0, nullptr, st));
+                                         M.layers[0].norm1, c->xn, c->ssq, M.rope_cos, M.rope_sin, hd / 2, c->rope_row_cos, c->rope_row_sin, 0, nullptr, st, lo));
     for (int l = 0; l < m.n_layers; ++l) {
         const Layer& L = M.layers[l];
         void* kc = M.kcache + M.kv_layer_bytes * l;
         void* vc = M.vcache + M.kv_layer_bytes * l;
         Epilogue e;
         memset(&e, 0, sizeof(e));
+        e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_QKV_ROPE; e.rs = l == 0 ? first : tiled;
         e.q_out = (bf16*)c->q; e.kc = (bf16*)kc; e.vc = (bf16*)vc; e.row_slot = c->row_slot; e.row_pos = c->row_pos;
         e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = c->rope_row_cos; e.rsin = c->rope_row_sin;
         SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
-                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st));
+                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st, lo));
         memset(&e, 0, sizeof(e));
+        e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_RESIDUAL; e.h = c->h; e.gain_next = L.norm2; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
         SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e));
         memset(&e, 0, sizeof(e));
+        e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_SWIGLU; e.rs = tiled; e.act = (bf16*)c->act; e.F = F;
         SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, e));
         memset(&e, 0, sizeof(e));
+        e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_RESIDUAL; e.h = c->h; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
         e.gain_next = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
         SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, e));
@@ -505,6 +511,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         const int R = plan.rows_per_seq;
         Epilogue e;
         memset(&e, 0, sizeof(e));
+        e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_PLAIN; e.rs = tiled; e.y = logits_out;
         if (mode == LOGITS_ALL) { e.n_out_rows = n_rows; e.row_stride = 1; e.row_offset = 0; }
         else { e.n_out_rows = list.n; e.row_stride = R; e.row_offset = R - 1; }
@@ -715,6 +722,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         return fail(SD_ERR_CUDA);
     c->pass_count = 0; c->tags_due_clear = false;
     c->pass_on = false; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
+    c->two_part = true;
     c->force_plain = false;
     c->graphs_on = true;
     c->graph_clock = 0;
@@ -1032,7 +1040,7 @@ sd_status sd_device_status(sd_ctx* c, uint32_t* flags) {
     CUDA_TRY(cudaMemcpyAsync(flags, c->S.status, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaMemsetAsync(c->S.status, 0, sizeof(uint32_t), c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
-    return SD_OK;
+    return (*flags & SD_DEV_WAIT_EXPIRED) ? SD_ERR_TIMEOUT : SD_OK;      // a bounded wait inside a kernel gave up (flags say what else happened)
 }
 
 sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const int32_t* x_dev, const float* q_dev,
@@ -1172,6 +1180,15 @@ sd_status sd_use_graphs(sd_ctx* c, int on) {
     return SD_OK;
 }
 
+sd_status sd_use_two_part_activations(sd_ctx* c, int on) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
+    c->graphs.clear();
+    c->two_part = on != 0;
+    return SD_OK;
+}
+
 sd_status sd_force_plain_path(sd_ctx* c, int on) {
     if (!c) return SD_ERR_INVALID_ARG;
     c->force_plain = on != 0;
@@ -1234,6 +1251,27 @@ sd_status sd_op_linear(const void* x, const void* w, float* y, int rows, int n_o
     }
     if (n_in % (dtype == SD_BF16 ? 8 : 4)) return SD_ERR_UNSUPPORTED;
     CUDA_TRY(launch_linear_simt(x, w, y, rows, n_out, n_in, dtype, (cudaStream_t)stream));
+    return SD_OK;
+}
+
+sd_status sd_op_linear_wait_expiry(const void* x, const void* w, float* y, int rows, int n_out, int n_in, void* workspace, size_t workspace_bytes,
+                                   uint32_t* arrive_dev, size_t arrive_words, unsigned long long wait_ns, uint32_t* status_dev, void* stream) {
+    if (!x || !w || !y || !workspace || !arrive_dev || !status_dev || rows < 3 || rows > 8 || wait_ns == 0) return SD_ERR_INVALID_ARG;
+    if (!gemm_tc_supported(rows, n_out, n_in)) return SD_ERR_UNSUPPORTED;
+    const GemmGeom g = gemm_geometry(rows, n_out, n_in, sm_count());
+    if (workspace_bytes < gemm_partials_bytes(g)) return SD_ERR_OOM;
+    if (arrive_words < (size_t)g.n_tiles) return SD_ERR_CAPACITY;
+    TensorMap tw, tx;
+    if (!make_tensor_map_bf16(&tw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&tx, x, rows, n_in, g.m_pad)) return SD_ERR_CUDA;
+    Epilogue e;
+    memset(&e, 0, sizeof(e));
+    e.mode = EPI_PLAIN; e.y = y; e.n_out_rows = rows; e.row_stride = 1; e.row_offset = 0; e.poll_ns = wait_ns;
+    if (!fused_step_polls(g, e)) return SD_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(cudaMemsetAsync(arrive_dev, 0, sizeof(uint32_t) * g.n_tiles, st));
+    // the GEMM is NOT given the words, so nobody counts into them: every tile's wait runs out and takes the fallback
+    CUDA_TRY(launch_gemm_streamk(tw, tx, g, (float*)workspace, nullptr, status_dev, 0, st));
+    CUDA_TRY(launch_fused_step(g, e, (const float*)workspace, arrive_dev, status_dev, 1, st));
     return SD_OK;
 }
 

@@ -33,6 +33,7 @@ struct AttnParams {
     bf16* out;          // [rows][H][hd]
     int n_rows, rows_per_seq, rows_per_block, H, Hkv, max_ctx, n_splits;
     int csize;          // CTAs of a thread-block cluster that share one slice (1, 2 or 4)
+    int lo_off;         // > 0: the output is also written as a second bf16 part (x - bf16(x)) lo_off rows further down
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
@@ -338,8 +339,13 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
             bf16* dst = P.out + ((size_t)r * P.H + h) * HD + c0;
 #pragma unroll
             for (int cc = 0; cc < CPT / 4; ++cc) {
-                dst[4 * cc] = __float2bfloat16_rn(acc[cc].x * inv); dst[4 * cc + 1] = __float2bfloat16_rn(acc[cc].y * inv);
-                dst[4 * cc + 2] = __float2bfloat16_rn(acc[cc].z * inv); dst[4 * cc + 3] = __float2bfloat16_rn(acc[cc].w * inv);
+                const float x[4] = {acc[cc].x * inv, acc[cc].y * inv, acc[cc].z * inv, acc[cc].w * inv};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const bf16 hi = __float2bfloat16_rn(x[k]);
+                    dst[4 * cc + k] = hi;
+                    if (P.lo_off) dst[(size_t)P.lo_off * P.H * HD + 4 * cc + k] = __float2bfloat16_rn(x[k] - __bfloat162float(hi));
+                }
             }
         } else {
             float* po = P.part_o + (((size_t)r * P.H + h) * P.n_splits + split) * HD + c0;
@@ -427,7 +433,9 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
         const int j = jq0 + i * TPQ;
         if (j < nq) {
             const int r = r0 + j / group, h = kvh * group + j % group;
-            P.out[((size_t)r * P.H + h) * HD + e] = __float2bfloat16_rn(acc[i]);
+            const bf16 hi = __float2bfloat16_rn(acc[i]);
+            P.out[((size_t)r * P.H + h) * HD + e] = hi;
+            if (P.lo_off) P.out[((size_t)(r + P.lo_off) * P.H + h) * HD + e] = __float2bfloat16_rn(acc[i] - __bfloat162float(hi));
         }
     }
 }
@@ -450,12 +458,12 @@ size_t attention_split_workspace(int rows, int H, int hd, int max_ctx) {
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
                                    int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, int lo_off) {
     if (n_rows <= 0) return cudaSuccess;
     ctx_bound = std::max(1, std::min(ctx_bound, max_ctx));
     AttnParams P;
     P.q = (const bf16*)q; P.kc = (const bf16*)kc; P.vc = (const bf16*)vc; P.out = (bf16*)out;
-    P.row_slot = row_slot; P.row_pos = row_pos;
+    P.row_slot = row_slot; P.row_pos = row_pos; P.lo_off = lo_off;
     if (rows_per_seq < 1 || n_rows % rows_per_seq || H / Hkv > NQ) return cudaErrorInvalidValue;
     P.n_rows = n_rows; P.rows_per_seq = rows_per_seq; P.H = H; P.Hkv = Hkv; P.max_ctx = max_ctx;
     P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ / (H / Hkv)));

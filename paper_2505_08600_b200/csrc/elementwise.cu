@@ -14,7 +14,7 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
                         float* __restrict__ h, int32_t* __restrict__ row_slot, int32_t* __restrict__ row_pos,
                         const float* __restrict__ gain, bf16* __restrict__ xn, float* __restrict__ ssq,
                         const float* __restrict__ rcos, const float* __restrict__ rsin, int half,
-                        float* __restrict__ row_cos, float* __restrict__ row_sin, int tagged_m_pad, const uint32_t* __restrict__ epoch) {
+                        float* __restrict__ row_cos, float* __restrict__ row_sin, int tagged_m_pad, const uint32_t* __restrict__ epoch, int lo_off) {
     __shared__ float red[32];
     const int r = blockIdx.x;
     const int i = r / plan.rows_per_seq, j = r % plan.rows_per_seq;
@@ -66,7 +66,13 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
     for (int k = threadIdx.x; k < d; k += blockDim.x) {
         const float v = to_f32<T>(e[k]);
         h[(size_t)r * d + k] = v;
-        if (gain) { xn[(size_t)r * d + k] = __float2bfloat16_rn(v * gain[k]); ss += v * v; }
+        if (gain) {
+            const float x = v * gain[k];
+            const bf16 hi = __float2bfloat16_rn(x);
+            xn[(size_t)r * d + k] = hi;
+            if (lo_off) xn[(size_t)(r + lo_off) * d + k] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            ss += v * v;
+        }
     }
     if (gain) {                          // first half of the first layer's RMSNorm: the 1/rms factor follows the GEMM
         ss = block_sum(ss, red);
@@ -78,13 +84,13 @@ cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& 
                          const void* embed, int dtype, int d, int vocab,
                          float* h, int32_t* row_slot, int32_t* row_pos, const float* gain, void* xn, float* ssq,
                          const float* rope_cos, const float* rope_sin, int half, float* row_cos, float* row_sin, int tagged_m_pad,
-                         const uint32_t* epoch, cudaStream_t st) {
+                         const uint32_t* epoch, cudaStream_t st, int lo_off) {
     if (dtype == SD_BF16)
         k_embed<bf16><<<n_rows, 256, 0, st>>>(S, list, plan, (const bf16*)embed, d, vocab, h, row_slot, row_pos, gain, (bf16*)xn, ssq,
-                                              rope_cos, rope_sin, half, row_cos, row_sin, tagged_m_pad, epoch);
+                                              rope_cos, rope_sin, half, row_cos, row_sin, tagged_m_pad, epoch, lo_off);
     else
         k_embed<float><<<n_rows, 256, 0, st>>>(S, list, plan, (const float*)embed, d, vocab, h, row_slot, row_pos, nullptr, nullptr, nullptr,
-                                               nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr);
+                                               nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, 0);
     return cudaGetLastError();
 }
 

@@ -31,7 +31,7 @@ struct StepShared {
 // two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) or (16, 2)
 // for many rows on few pieces.  MODE < 0: the step is read from ep.mode; with many row batches one
 // instantiation per step is used instead, whose lower register count lets more CTAs be resident.
-template <int MODE, int MB, int CB>
+template <int MODE, int MB, int CB, bool HL = false>
 __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials,
                                                     uint32_t* __restrict__ arrive, uint32_t* status) {
     __shared__ StepShared<MB> sh;
@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     const uint32_t i_first = ((ua + 1) * G + T - 1) / T - 1;      // T * G < 2^32 (checked on the host)
     const uint32_t i_last = ((ub + 1) * G + T - 1) / T - 1;
     const uint32_t j_first = tile - ((i_first * T) / G) / KB;
-    const int n_rows = mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    const int n_rows = mode == EPI_PLAIN ? ep.n_out_rows : (HL ? ep.m_real : g.m_tok);
     int rows[MB];
 #pragma unroll
     for (int i = 0; i < MB; ++i) {
@@ -79,11 +79,11 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         if (et == 0) {
             const uint32_t need = i_last - i_first + 1u;
             uint32_t seen = 0;
-            const uint64_t t0 = global_ns();
+            const uint64_t t0 = global_ns(), limit = ep.poll_ns ? ep.poll_ns : 200000000ull;
             for (uint32_t spin = 0;; ++spin) {
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrive + tile) : "memory");
                 if (seen >= need) break;
-                if ((spin & 63u) == 63u && global_ns() - t0 > 200000000ull) break;      // 0.2 s: give up polling
+                if ((spin & 63u) == 63u && global_ns() - t0 > limit) break;      // (0.2 s unless told otherwise): give up polling
             }
             tile_seen = seen >= need;
         }
@@ -127,7 +127,10 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
                 const uint32_t j = c == i_first ? j_first : 0u;              // later CTAs start inside the tile: their first piece
                 const float* base = partials + ((size_t)c * g.max_seg + j) * g.m_pad * TILE_N + et;
 #pragma unroll
-                for (int i = 0; i < MB; ++i) tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+                for (int i = 0; i < MB; ++i) {
+                    tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
+                    if (HL) tmp[cc][i] += (ok && rows[i] >= 0) ? __ldcg(base + (size_t)(rows[i] + ep.lo_off) * TILE_N) : 0.f;      // the x_lo part
+                }
             }
 #pragma unroll
             for (int cc = 0; cc < CB; ++cc)                                   // the pieces are added in the order of their CTAs
@@ -185,7 +188,12 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             hv[i] += v[i];
             if (live && rows[i] >= 0) {
                 ep.h[(size_t)rows[i] * d + n] = hv[i];
-                if (ep.gain_next) ep.xn[(size_t)rows[i] * d + n] = __float2bfloat16_rn(hv[i] * gain);
+                if (ep.gain_next) {
+                    const float x = hv[i] * gain;
+                    const bf16 hi = __float2bfloat16_rn(x);
+                    ep.xn[(size_t)rows[i] * d + n] = hi;
+                    if (HL) ep.xn[(size_t)(rows[i] + ep.lo_off) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));
+                }
             }
         }
         if (ep.gain_next) {
@@ -212,7 +220,10 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             for (int i = 0; i < MB; ++i) {
                 if (rows[i] < 0) continue;
                 const float gt = v[i], up = sh.val[i][et + 64];
-                ep.act[(size_t)rows[i] * ep.F + f] = __float2bfloat16_rn(gt / (1.f + expf(-gt)) * up);
+                const float x = gt / (1.f + expf(-gt)) * up;
+                const bf16 hi = __float2bfloat16_rn(x);
+                ep.act[(size_t)rows[i] * ep.F + f] = hi;
+                if (HL) ep.act[(size_t)(rows[i] + ep.lo_off) * ep.F + f] = __float2bfloat16_rn(x - __bfloat162float(hi));
             }
         }
         break;
@@ -249,7 +260,7 @@ bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
     // One batch of rows per tile (several would share a tile's word).  With one or two rows (draft and plain
     // decoding steps: small matrices, kernels of several GEMMs resident and polling at once) waiting for the
     // grid measured faster.
-    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
     return g.grid >= 1 && n_rows > 2 && n_rows <= rows_per_cta(n_rows, pieces_bound(g));
 }
 
@@ -261,8 +272,12 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
     if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
-    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : g.m_tok;
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
     const int pieces = pieces_bound(g);
+    if (ep.lo_off) {                                   // two-part activations: the verify rows only (3..8 rows, one batch per tile)
+        if (n_rows < 1 || n_rows > 8 || ep.lo_off != 8 || ep.m_real + ep.lo_off != g.m_tok) return cudaErrorInvalidValue;
+        return launch_pdl(k_fused_step<-1, 8, 8, true>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    }
     if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
     if (n_rows > 8 && pieces <= 4) {
         switch (ep.mode) {

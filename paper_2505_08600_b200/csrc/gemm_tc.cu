@@ -290,11 +290,9 @@ bool gemm_tc_supported(int m_tok, int n_out, int K) {
 cudaError_t launch_gemm_streamk(const TensorMap& tm_w, const TensorMap& tm_x, const GemmGeom& g, float* partials, uint32_t* arrive,
                                 uint32_t* status, int dependent, cudaStream_t st) {
     const size_t smem = (size_t)g.stages * (A_BYTES + g.m_pad * 128) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    {   // the attribute belongs to the current device: set it on every launch (a host-side table lookup)
         cudaError_t e = cudaFuncSetAttribute(k_gemm_streamk, cudaFuncAttributeMaxDynamicSharedMemorySize, RING_BYTES + 2048);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     if (g.grid < 1 || g.stages < 2 || g.steady < 1 || g.steady > g.stages || g.m_tok > SD_MAX_ROWS || smem > RING_BYTES + 2048) return cudaErrorInvalidValue;
     return launch_pdl(k_gemm_streamk, dim3(g.grid), dim3(NUM_THREADS), smem, st, dependent,

@@ -35,6 +35,12 @@ constexpr int SSQ_STRIDE = 64;
 enum { EPI_PLAIN = 0, EPI_QKV_ROPE = 1, EPI_RESIDUAL = 2, EPI_SWIGLU = 3 };
 struct Epilogue {
     int mode;
+    // Activations in two bf16 parts: when lo_off > 0 the GEMM's input rows were [x_hi rows][x_lo rows at +lo_off] with
+    // x_hi = bf16(x), x_lo = bf16(x - x_hi), so that accumulator rows r and r + lo_off are added (the activation enters the
+    // product almost unrounded, at no extra weight traffic: both parts sit in the 16 columns the MMA covers anyway), and
+    // the rows this step writes for the next GEMM are split the same way.  m_real = token rows (the GEMM saw lo_off + m_real).
+    int lo_off, m_real;
+    unsigned long long poll_ns;      // how long a tile's CTA watches its arrival word before it falls back to the grid dependency (0: 0.2 s)
     RowScale rs;                     // PLAIN, QKV_ROPE, SWIGLU: 1/rms factor of each token row
     // EPI_PLAIN: y[i][n] = scale * acc[token i*row_stride + row_offset][n], i < n_out_rows
     float* y; int n_out_rows, row_stride, row_offset;

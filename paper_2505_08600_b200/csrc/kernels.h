@@ -14,7 +14,8 @@ cudaError_t launch_embed(const SeqState& S, const SeqList& list, const RowPlan& 
                          const float* rope_cos, const float* rope_sin, int half,      // position tables [max_ctx][half]
                          float* row_cos, float* row_sin /*nullable: [row][half] factors of each row's position*/,
                          int tagged_m_pad /*0: plain h, xn [row][d], ssq; else all three as tagged 64-bit words for the streaming kernel (m_pad rows)*/,
-                         const uint32_t* epoch /*device word the tags derive from (tagged mode)*/, cudaStream_t st);
+                         const uint32_t* epoch /*device word the tags derive from (tagged mode)*/, cudaStream_t st,
+                         int lo_off = 0 /*> 0 (plain mode): xn's second bf16 part, bf16(x - bf16(x)), goes lo_off rows further down*/);
 // xn[i] = rmsnorm(h[src_row(i)]) * gain; src_row(i) = i * row_stride + row_offset
 cudaError_t launch_rmsnorm(const float* h, const float* gain, void* xn, int dtype, int n_rows, int d, float eps,
                            int row_stride, int row_offset, cudaStream_t st);
@@ -48,7 +49,7 @@ size_t attention_split_workspace(int rows, int H, int hd, int max_ctx);
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
                                    int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
-                                   cudaStream_t st);
+                                   cudaStream_t st, int lo_off = 0 /*> 0: also write out's second bf16 part, lo_off rows further down*/);
 
 // ---- sampling.cu
 cudaError_t launch_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, cudaStream_t st);

@@ -87,10 +87,7 @@ def _replay(sd, ctx, omodels, draft_k, prompt, gamma, T, seed, max_new, dtype, s
         L = int(tr["len_before"][it]) + int(tr["n_acc"][it]) + 1
         assert len(got) == L
         assert got.tolist() == toks_ref_full(tr, prompt, it)
-    # bf16 rounding is relative: the stated absolute bound is for logits of about unit scale, and is
-    # widened in proportion where random-init logits are larger (0.02 * sqrt(d) > 1 from d = 4096 on)
-    logit_scale = max(1.0, float(np.std(tr["logits"][0])))
-    assert worst_logit <= tol["logits"] * logit_scale, (worst_logit, logit_scale)
+    assert worst_logit <= tol["logits"], worst_logit
     assert worst_q <= tol["probs"], worst_q
     assert worst_p <= tol["probs"], worst_p
     assert ctx.sd_device_status() == 0
@@ -184,6 +181,64 @@ def test_benchmark_shapes_at_full_width_teacher_forced(sd, name):
     ctx.close()
 
 
+def _one_verify_step_error(sd, t, d, prompt_len, wl, two_part=1):
+    """max |logit - oracle| and max |p - oracle| of one verify step (gamma + 1 rows after a prompt)."""
+    gamma, T, seed, V = wl["gamma"], wl["temperature"], wl["seed"], t["vocab"]
+    wt = synth.make_weights(t, seed=0, model_index=0, dtype="bf16")
+    wd = synth.make_weights(d, seed=0, model_index=1, dtype="bf16")
+    om = [oracle.OracleModel(t, wt), oracle.OracleModel(d, wd)]
+    prompt = synth.make_prompt(V, prompt_len, seed=seed)
+    _, _, tr = oracle.spec_decode(om[0], om[1], prompt, gamma + 1, gamma, T, seed, seq_id=0, trace_iters=1, trace_probs=True, trace_logits=True)
+    ctx = sd.Context(t, [d], "bf16", 1, prompt_len + 40, gamma, T, seed)
+    ctx.load_weights(0, wt); ctx.load_weights(1, wd)
+    del wt, wd, om
+    ctx.sd_use_two_part_activations(two_part)
+    ctx.sd_seq_begin(0, prompt, 0); ctx.sd_route_prompt([0], forced_task=[0]); ctx.sd_prefill([0])
+    x = torch.from_numpy(tr["x"][0:1].copy()).to(DEV)
+    logits = torch.zeros((1, gamma + 1, V), dtype=torch.float32, device=DEV)
+    ctx.sd_verify([0], gamma, x, logits)
+    lg = logits.cpu().numpy()[0].astype(np.float64)
+    p = torch.softmax(logits[0].double() / T, dim=-1).cpu().numpy()
+    assert ctx.sd_device_status() == 0
+    ctx.close()
+    return float(np.abs(lg - tr["logits"][0]).max()), float(np.abs(p - tr["p"][0]).max())
+
+
+# How the error of the verify step's logits grows with depth at the 7B width (bf16 KV cache, queries, keys, values and
+# attention weights against the fp64 oracle; the GEMMs' inputs in two bf16 parts).  Measured on a B200: 0.031, 0.041, 0.061
+# for 1, 2 and 4 layers (one bf16 part: 0.037, 0.049, 0.068) - about the square root of the depth.  The stated 5e-2 holds to
+# two layers; deeper, the bound asserted here is the measured value with a margin, and the probabilities (what the
+# accept rule consumes) stay inside their 1e-3 by an order of magnitude.
+DEPTH_SERIES_7B = [(1, 5e-2), (2, 5e-2), (4, 8e-2)]
+
+
+@pytest.mark.parametrize("layers,bound", DEPTH_SERIES_7B)
+def test_logit_error_against_depth_at_7b_width(sd, layers, bound):
+    cfg = synth.CONFIGS["7b"]
+    t = dict(cfg["target"], n_layers=layers)
+    d = dict(cfg["drafts"][0], n_layers=1)
+    dl, dp = _one_verify_step_error(sd, t, d, 24, cfg["workload"])
+    print(f"7B width, {layers} layer(s): max |logit - oracle| = {dl:.4f}, max |p - oracle| = {dp:.2e}")
+    assert dl <= bound, dl
+    assert dp <= TOL["bf16"]["probs"], dp
+    if layers == 1:                               # the two-part activations are what keeps one layer inside the stated bound with room
+        dl1, _ = _one_verify_step_error(sd, t, d, 24, cfg["workload"], two_part=0)
+        assert dl < dl1, (dl, dl1)
+
+
+def test_full_depth_7b_verify_step_against_the_oracle(sd):
+    """All 32 layers of the 7B configuration, one verify step after a 24-token prompt (the oracle needs about ten seconds,
+    generating the 13 GB of weights on the host a minute or two).  bf16 noise grows with about the square root of the depth:
+    measured max |logit - oracle| at full depth is recorded here and bounded; the probabilities stay inside the stated 1e-3."""
+    cfg = synth.CONFIGS["7b"]
+    t = dict(cfg["target"])
+    d = dict(cfg["drafts"][0], n_layers=1)
+    dl, dp = _one_verify_step_error(sd, t, d, 24, cfg["workload"])
+    print(f"7B, all {t['n_layers']} layers: max |logit - oracle| = {dl:.4f}, max |p - oracle| = {dp:.2e}")
+    assert dl <= 0.30, dl
+    assert dp <= TOL["bf16"]["probs"], dp
+
+
 def test_wide_bf16_head_dim_128_teacher_forced(sd):
     ctx, om = _build(sd, WIDE_BF16, [SMALL_BF16_DRAFT | dict(vocab=8192)], "bf16", 1.0, 7, max_ctx=96)
     prompt = synth.make_prompt(8192, 33, seed=8)
@@ -263,9 +318,10 @@ def test_batch16_launch_configuration_at_full_width(sd):
     ctx.sd_draft_steps_replay(seqs, gamma, x, xs, q)
     ctx.sd_verify(seqs, gamma, x, logits)
     lg, qg = logits.cpu().numpy().astype(np.float64), q.cpu().numpy().astype(np.float64)
+    worst = max(float(np.abs(lg[b] - traces[b]["logits"][0]).max()) for b in seqs)
+    print(f"batch-16 launch, one layer at 7B width: max |logit - oracle| = {worst:.4f}")
+    assert worst <= TOL["bf16"]["logits"], worst
     for b in seqs:
-        scale = max(1.0, float(np.std(traces[b]["logits"][0])))     # as in _replay: bf16 rounding is relative
-        assert np.abs(lg[b] - traces[b]["logits"][0]).max() <= TOL["bf16"]["logits"] * scale, b
         assert np.abs(qg[b] - traces[b]["q"][0]).max() <= TOL["bf16"]["probs"], b
     assert ctx.sd_device_status() == 0
     ctx.close()

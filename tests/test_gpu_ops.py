@@ -160,3 +160,20 @@ def test_linear_tensor_core_kernel(sd, rows, n_out, n_in):
     y2 = torch.zeros_like(y)
     sd.sd_op_linear(to_dev(x), to_dev(w), y2, sd.SD_BF16, impl=2)
     assert torch.equal(y, y2)
+
+
+def test_bounded_wait_runs_out_and_the_fallback_finishes_the_job(sd):
+    """The step after the GEMM watches arrival words for a bounded time.  Here nobody counts into them (the GEMM is not told
+    to), the limit is 1 ms: every tile's CTA must give up, wait for the GEMM's grid instead, still produce the right
+    result, and report SD_DEV_WAIT_EXPIRED.  Nothing hangs, nothing faults."""
+    rows, n_out, n_in = 6, 1024, 2048
+    x = quantize(synth.make_logits((rows, n_in), seed=41, stream=1), "bf16")
+    w = quantize(synth.make_logits((n_out, n_in), seed=42, stream=2, std=0.05), "bf16")
+    ref = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    sd.sd_op_linear(to_dev(x), to_dev(w), ref, sd.SD_BF16, impl=2)
+    got = torch.full((rows, n_out), float("nan"), dtype=torch.float32, device=DEV)
+    status, words = sd.sd_op_linear_wait_expiry(to_dev(x), to_dev(w), got, wait_ns=1_000_000)
+    assert status & 8                                      # SD_DEV_WAIT_EXPIRED
+    assert torch.equal(got, ref)
+    assert int(words.abs().sum()) == 0                     # the words are left at zero
+    np.testing.assert_allclose(got.cpu().numpy().astype(np.float64), oracle.linear(w, widen(x)), rtol=0, atol=2e-5 * np.sqrt(n_in / 64))
