@@ -102,8 +102,10 @@ def lib():
         L.orc_spec_decode.argtypes = [C.POINTER(Model), C.POINTER(Model), C.POINTER(Cache),
                                       C.POINTER(Cache), C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_double, C.c_uint64, C.c_uint32, C.c_void_p,
-                                      C.POINTER(Counters), C.POINTER(Trace)]
+                                      C.POINTER(Counters), C.POINTER(Trace), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.orc_spec_decode.restype = C.c_int
+        L.orc_alpha_terms.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+        L.orc_alpha_terms.restype = None
         L.orc_mc_fixed.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_uint64,
                                    C.c_void_p, C.c_void_p]
         L.orc_mc_fixed.restype = C.c_int64
@@ -159,6 +161,16 @@ def accept(p, q, x, seed, it, seq):
     lib().orc_accept(_ptr(p), _ptr(q), _ptr(x), gamma, V, int(seed), int(it), int(seq), _ptr(n), _ptr(out))
     out[int(n[0]) + 1:] = -1
     return int(n[0]), out
+
+
+def alpha_terms(p, q):
+    """p [gamma+1, V] (or [gamma, V]), q [gamma, V] fp32 -> sum_k min(p_s(k), q_s(k)) for every slot s (float64 [gamma])."""
+    p = np.ascontiguousarray(p, dtype=np.float32)
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    gamma, V = q.shape
+    out = np.zeros(gamma, dtype=np.float64)
+    lib().orc_alpha_terms(_ptr(p), _ptr(q), gamma, V, _ptr(out))
+    return out
 
 
 class OracleModel:
@@ -266,6 +278,7 @@ def spec_decode(target: OracleModel, draft: OracleModel | None, prompt, max_new,
     dc = draft.new_cache(max_ctx) if draft is not None else None
     V = target.dims["vocab"]
     cnt = Counters()
+    alpha_sum, judged = C.c_double(0.0), C.c_int64(0)
     ln = np.zeros(1, dtype=np.int32)
     tr = None
     keep = {}
@@ -288,7 +301,8 @@ def spec_decode(target: OracleModel, draft: OracleModel | None, prompt, max_new,
     rc = lib().orc_spec_decode(C.byref(target.c), C.byref(draft.c) if draft is not None else None,
                                C.byref(tc.c), C.byref(dc.c) if dc is not None else None,
                                _ptr(toks), n_prompt, int(max_new), int(gamma), float(T), int(seed),
-                               int(seq_id), _ptr(ln), C.byref(cnt), C.byref(tr) if tr is not None else None)
+                               int(seq_id), _ptr(ln), C.byref(cnt), C.byref(tr) if tr is not None else None,
+                               C.byref(alpha_sum), C.byref(judged))
     if rc != 0:
         raise RuntimeError("oracle spec_decode failed (cache capacity?)")
     counters = dict(iterations=cnt.iterations, drafted=cnt.drafted, accepted=cnt.accepted, emitted=cnt.emitted)
@@ -296,6 +310,7 @@ def spec_decode(target: OracleModel, draft: OracleModel | None, prompt, max_new,
     if tr is not None:
         n = tr.n_iters
         trace = {k: v[:n] for k, v in keep.items()}
+        trace["alpha_sum"], trace["judged"] = float(alpha_sum.value), int(judged.value)      # estimate of Eq. 1's alpha: their ratio
     return toks[: int(ln[0])].copy(), counters, trace
 
 

@@ -171,6 +171,24 @@ void orc_accept(const float* p, const float* q, const int32_t* x, int gamma, int
     *n_out = n;
 }
 
+/* alpha of Eq. 1 is the probability that the target agrees with one draft token.  For the
+ * stochastic rule that probability, given the two distributions of a slot, is
+ * sum_k min(p_s(k), q_s(k)) (the draft is drawn from q_s and kept with probability
+ * min(1, p_s/q_s)).  terms[s] receives that sum, in double, for every slot s < gamma;
+ * the estimate of alpha over a run is their mean over the slots that were judged
+ * (slot s is judged iff all slots before it were accepted: s <= min(n, gamma - 1)). */
+void orc_alpha_terms(const float* p, const float* q, int gamma, int V, double* terms)
+{
+    for (int s = 0; s < gamma; ++s) {
+        double a = 0.0;
+        for (int k = 0; k < V; ++k) {
+            double pk = (double)p[(size_t)s * V + k], qk = (double)q[(size_t)s * V + k];
+            a += pk < qk ? pk : qk;
+        }
+        terms[s] = a;
+    }
+}
+
 /* ------------------------------------------------------------------------ */
 /* Decoder-only transformer (RMSNorm, rotary embedding, SwiGLU, no biases)   */
 /* ------------------------------------------------------------------------ */
@@ -491,7 +509,8 @@ int orc_spec_decode(const orc_model* target, const orc_model* draft,
                     orc_cache* tcache, orc_cache* dcache,
                     int32_t* tokens, int n_prompt, int max_new, int gamma, double T,
                     uint64_t seed, uint32_t seq_id,
-                    int32_t* len_out, orc_counters* cnt, orc_trace* tr)
+                    int32_t* len_out, orc_counters* cnt, orc_trace* tr,
+                    double* alpha_sum_out, int64_t* judged_out)
 {
     const int V = target->vocab;
     int L = n_prompt, tkv = 0, dkv = 0;
@@ -508,6 +527,9 @@ int orc_spec_decode(const orc_model* target, const orc_model* draft,
     int32_t* x = malloc(sizeof(int32_t) * (size_t)(gamma + 1));
     int32_t* out = malloc(sizeof(int32_t) * (size_t)(gamma + 1));
     int32_t* rows = malloc(sizeof(int32_t) * (size_t)(gamma + 1));
+    double* terms = malloc(sizeof(double) * (size_t)(gamma > 0 ? gamma : 1));
+    double alpha_sum = 0.0;
+    int64_t judged = 0;
     int rc = 0;
 
     /* prefill: everything but the last prompt token */
@@ -550,6 +572,8 @@ int orc_spec_decode(const orc_model* target, const orc_model* draft,
         /* (3) accept / reject */
         int32_t n;
         orc_accept(p, q, x, gamma, V, seed, iter, seq_id, &n, out);
+        orc_alpha_terms(p, q, gamma, V, terms);
+        for (int s = 0; s < gamma && s <= n; ++s) { alpha_sum += terms[s]; judged += 1; }     /* the judged slots */
         if (tr && tr->n_iters < tr->cap_iters) {
             int it = tr->n_iters++;
             tr->len_before[it] = L;
@@ -574,7 +598,9 @@ int orc_spec_decode(const orc_model* target, const orc_model* draft,
     }
     if (L > L_end) L = L_end;       /* the last iteration may overshoot; truncate */
     *len_out = L;
-    free(tl); free(dl); free(p); free(q); free(x); free(out); free(rows);
+    if (alpha_sum_out) *alpha_sum_out = alpha_sum;
+    if (judged_out) *judged_out = judged;
+    free(tl); free(dl); free(p); free(q); free(x); free(out); free(rows); free(terms);
     return rc;
 }
 

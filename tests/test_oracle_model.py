@@ -164,6 +164,15 @@ def test_counters_identity_and_trace_consistency():
         np.testing.assert_allclose(tr["logits"][it], full, rtol=1e-8, atol=1e-9)
         seq += out[: n + 1].tolist()
     assert seq[: len(toks)] == toks.tolist()
+    # the run's estimate of Eq. 1's alpha: sum over judged slots (s <= min(n, gamma - 1)) of sum_k min(p_s, q_s)
+    a_sum, judged = 0.0, 0
+    for it in range(len(tr["n_acc"])):
+        n = int(tr["n_acc"][it])
+        terms = np.minimum(tr["p"][it][:gamma].astype(np.float64), tr["q"][it].astype(np.float64)).sum(axis=1)
+        a_sum += float(terms[: min(n + 1, gamma)].sum())
+        judged += min(n + 1, gamma)
+    assert tr["judged"] == judged
+    assert abs(tr["alpha_sum"] - a_sum) < 1e-9
 
 
 def test_route_prompt_mlp_and_forced_task():

@@ -115,6 +115,35 @@ def test_alpha_of_fixtures():
     assert abs(float(np.minimum(P08, QU).sum()) - 0.8) < 1e-6
 
 
+def test_alpha_terms_closed_forms():
+    """Eq. 1's alpha for one slot, sum_k min(p(k), q(k)): exact values on the fixtures, 1 for q == p, 0 for disjoint supports,
+    symmetric in its arguments, one value per slot."""
+    p = np.stack([P06, P08, QU, P06])
+    q = np.stack([QU, QU, QU])
+    np.testing.assert_allclose(oracle.alpha_terms(p, q), [0.6, 0.8, 1.0], atol=1e-7)
+    a = np.array([[0.5, 0.5, 0, 0, 0, 0, 0, 0]], dtype=np.float32)
+    b = np.array([[0, 0, 0.25, 0.75, 0, 0, 0, 0]], dtype=np.float32)
+    assert oracle.alpha_terms(a, b).tolist() == [0.0]
+    np.testing.assert_allclose(oracle.alpha_terms(P06[None], P08[None]), oracle.alpha_terms(P08[None], P06[None]), atol=0)
+    # 1 - total variation distance
+    np.testing.assert_allclose(oracle.alpha_terms(P06[None], P08[None]), [1.0 - 0.5 * np.abs(P06.astype(np.float64) - P08).sum()], atol=1e-7)
+
+
+@pytest.mark.parametrize("alpha,p", [(0.6, P06), (0.8, P08)])
+def test_alpha_is_the_acceptance_frequency_of_judged_slots(alpha, p):
+    """What the sum of minima estimates is the frequency with which a judged slot is accepted: slot s is judged iff all
+    slots before it were accepted, so an iteration with n accepts judges min(n + 1, gamma) slots."""
+    gamma, iters = 4, 400_000
+    emitted, accepted, _ = oracle.mc_fixed(p, QU, gamma, iters, seed=99)
+    # judged = sum over iterations of min(n + 1, gamma) = emitted - (iterations that accepted everything)
+    # P(n = gamma) = alpha^gamma, so E[judged] = E[n + 1] - alpha^gamma
+    judged_expect = iters * ((1 - alpha ** (gamma + 1)) / (1 - alpha) - alpha ** gamma)
+    freq = accepted / judged_expect
+    se = math.sqrt(alpha * (1 - alpha) / judged_expect) * 2     # judged is itself random: generous
+    assert abs(freq - alpha) < 4 * se + 2e-3, (freq, alpha)
+    assert abs(float(oracle.alpha_terms(p[None], QU[None])[0]) - alpha) < 1e-6
+
+
 @pytest.mark.parametrize("alpha,p", [(0.6, P06), (0.8, P08)])
 @pytest.mark.parametrize("gamma", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_eq1_expected_tokens_monte_carlo(alpha, p, gamma):
