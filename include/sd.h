@@ -221,6 +221,30 @@ double sd_eq1_speedup(double alpha, int gamma, double c);
  * plain decoding (speedup <= 1) or on bad arguments.  speedup_out may be NULL. */
 int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
 
+/* The gamma that maximises Eq. 1 for what the library itself has measured: alpha = (sum over judged slots of
+ * sum_k min(p_s(k), q_s(k))) / judged slots of sequence `seq` (accumulated by sd_accept_seqs + sd_kv_rollback), c from
+ * sd_cost_timing / sd_cost_read.  Returns 0 when nothing has been measured yet or no gamma beats plain decoding.
+ * alpha_out, c_out and speedup_out may be NULL.  Synchronises. */
+int sd_best_gamma_measured(sd_ctx* ctx, int seq, int gamma_max, double* alpha_out, double* c_out, double* speedup_out);
+
+/* Estimate of Eq. 1's alpha for a sequence since sd_seq_begin: for the stochastic rule a draft token drawn from q_s is kept
+ * with probability sum_k min(p_s(k), q_s(k)); sd_accept_seqs computes that sum for every slot, sd_kv_rollback (called with the
+ * same sequence list) adds the judged slots' sums (slot s is judged iff all slots before it were accepted) to alpha_sum
+ * and their number to judged.  alpha = alpha_sum / judged.  Synchronises. */
+sd_status sd_seq_alpha(sd_ctx* ctx, int seq, double* alpha_sum_out, int64_t* judged_out);
+
+/* The cost ratio c of Eq. 1 from the library's own clock: while enabled, sd_draft_steps, sd_verify / sd_verify_accept
+ * and sd_target_step are bracketed by CUDA events on the context's stream.  sd_cost_read synchronises and returns the
+ * mean time of one draft pass (one token), of one verify pass and of one single-row target pass, and
+ * c = draft pass / target pass (the verify pass stands in for the target pass when no sd_target_step was timed: Eq. 1
+ * takes them to cost the same).  reset != 0 clears the sums. */
+typedef struct {
+    double draft_pass_ms, verify_pass_ms, target_pass_ms, c;
+    int64_t draft_passes, verify_passes, target_passes;
+} sd_cost;
+sd_status sd_cost_timing(sd_ctx* ctx, int enable);
+sd_status sd_cost_read(sd_ctx* ctx, sd_cost* out, int reset);
+
 /* -------------------------------------------------------------- observation */
 
 /* Repeated calls replay captured CUDA graphs by default (keyed by sequences, gamma, buffers
@@ -266,8 +290,8 @@ sd_status sd_pass_schedule_check(const int32_t* shape12, const int32_t* waves, c
  * block, k blocks, matrix, flags, wait word, wait count, arrival word, workspace slot) and 20-byte task records. */
 size_t sd_pass_schedule_blob(const int32_t* shape12, const int32_t* waves, const int32_t* chunk_major, void* out, size_t cap);
 
-/* With 3..8 query rows (the verify rows of one sequence) the tensor-core path feeds every GEMM its input rows in two
- * bf16 parts, bf16(x) and bf16(x - bf16(x)), in the columns that the 16-wide MMA covers anyway: the weights stream
+/* With 3..16 query rows (the verify rows of one sequence) the tensor-core path feeds every GEMM its input rows in two
+ * bf16 parts, bf16(x) and bf16(x - bf16(x)), in the columns that the 16- or 32-wide MMA covers anyway: the weights stream
  * once all the same, and the activations enter the products with 16 bits of mantissa instead of 8.  on = 0 switches
  * that off (one bf16 part, as with other row counts); the tests measure both.  Synchronises, drops cached graphs. */
 sd_status sd_use_two_part_activations(sd_ctx* ctx, int on);

@@ -35,6 +35,11 @@ class Counters(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("iterations", "drafted", "accepted", "emitted")]
 
 
+class Cost(C.Structure):
+    _fields_ = [("draft_pass_ms", C.c_double), ("verify_pass_ms", C.c_double), ("target_pass_ms", C.c_double), ("c", C.c_double),
+                ("draft_passes", C.c_int64), ("verify_passes", C.c_int64), ("target_passes", C.c_int64)]
+
+
 class AcceptArgs(C.Structure):
     _fields_ = [("target", C.c_void_p), ("target_is_logits", C.c_int32), ("q", C.c_void_p), ("x", C.c_void_p),
                 ("B", C.c_int32), ("gamma", C.c_int32), ("V", C.c_int32), ("temperature", C.c_float),
@@ -69,6 +74,10 @@ _PROTOS = {
     "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_use_graphs": (_i, [_vp, _i]),
+    "sd_seq_alpha": (_i, [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "sd_cost_timing": (_i, [_vp, _i]),
+    "sd_cost_read": (_i, [_vp, C.POINTER(Cost), _i]),
+    "sd_best_gamma_measured": (_i, [_vp, _i, _i, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "sd_use_pass_kernel": (_i, [_vp, _i, _i, _i]),
     "sd_pass_tuning": (_i, [_vp, _vp, _vp, _i]),
     "sd_pass_stamps": (_i, [_vp, _vp, _sz]),
@@ -293,6 +302,24 @@ class Context:
     def sd_verify_accept(self, seqs, gamma, x, q, logits, n_acc, out_tok):
         a, p, n = _seqs(seqs)
         _check(self.L.sd_verify_accept(self.h, p, n, gamma, _dp(x), _dp(q), _dp(logits), _dp(n_acc), _dp(out_tok)), "sd_verify_accept")
+
+    def sd_seq_alpha(self, seq):
+        a, j = C.c_double(), C.c_int64()
+        _check(self.L.sd_seq_alpha(self.h, int(seq), C.byref(a), C.byref(j)), "sd_seq_alpha")
+        return a.value, j.value
+
+    def sd_cost_timing(self, enable):
+        _check(self.L.sd_cost_timing(self.h, int(enable)), "sd_cost_timing")
+
+    def sd_cost_read(self, reset=0):
+        c = Cost()
+        _check(self.L.sd_cost_read(self.h, C.byref(c), int(reset)), "sd_cost_read")
+        return {n: getattr(c, n) for n, _ in Cost._fields_}
+
+    def sd_best_gamma_measured(self, seq, gamma_max):
+        a, c, s = C.c_double(), C.c_double(), C.c_double()
+        g = self.L.sd_best_gamma_measured(self.h, int(seq), int(gamma_max), C.byref(a), C.byref(c), C.byref(s))
+        return g, a.value, c.value, s.value
 
     def sd_use_graphs(self, on):
         _check(self.L.sd_use_graphs(self.h, int(on)), "sd_use_graphs")

@@ -107,6 +107,13 @@ struct sd_ctx {
     size_t arena_used;
     // staging for the host-buffer entry point
     int32_t* st_x; float* st_q; float* st_logits; int32_t* st_nacc; int32_t* st_out;
+    float* alpha_terms;                         // [seq of the call][gamma]: sum_k min(p, q) of the last sd_accept_seqs, consumed by sd_kv_rollback
+    // optional timing of the draft and target passes (the cost ratio c of Eq. 1 from the library's own clock)
+    bool cost_on; int cost_depth;
+    struct CostMark { cudaEvent_t e0, e1; int kind; int units; };
+    std::vector<CostMark> cost_pending;
+    std::vector<cudaEvent_t> cost_free;
+    double cost_ms[3]; uint64_t cost_units[3];  // 0 draft passes, 1 verify passes, 2 single-row target passes
     // launch accounting and optional per-category timing
     uint64_t launches;
     bool prof_on;
@@ -191,6 +198,8 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->S.draft_id = (int32_t*)B.take(sizeof(int32_t) * S);
     c->S.n_prompt = (int32_t*)B.take(sizeof(int32_t) * S);
     c->S.counters = (int64_t*)B.take(sizeof(int64_t) * 4 * S);
+    c->S.alpha_sum = (double*)B.take(sizeof(double) * S);
+    c->S.judged = (int64_t*)B.take(sizeof(int64_t) * S);
     c->S.tok_stride = cfg.max_ctx + 1;
     c->S.max_ctx = cfg.max_ctx;
     c->S.tokens = (int32_t*)B.take(sizeof(int32_t) * (size_t)S * c->S.tok_stride);
@@ -254,6 +263,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->st_x = (int32_t*)B.take(sizeof(int32_t) * S * g_max);
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
     c->st_logits = (float*)B.take(sizeof(float) * std::min((size_t)SD_MAX_ROWS, (size_t)S * (cfg.max_gamma + 1)) * V0);
+    c->alpha_terms = (float*)B.take(sizeof(float) * S * g_max);
     c->st_nacc = (int32_t*)B.take(sizeof(int32_t) * S);
     c->st_out = (int32_t*)B.take(sizeof(int32_t) * S * (cfg.max_gamma + 1));
     if (cfg.clf_d_hidden > 0 && cfg.n_drafts > 0) {
@@ -471,10 +481,10 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     c->arrive_used = 0;                          // the embedding kernel below is an ordinary launch: everything before it has finished
-    // With 3..8 rows (the verify rows of one sequence) the 16 columns of the MMA hold every activation twice over: as
-    // bf16(x) and as bf16(x - bf16(x)), eight rows apart.  The weights stream once all the same, and the GEMMs' inputs
-    // are no longer rounded to 8 bits of mantissa.
-    const int lo = (c->two_part && n_rows >= 3 && n_rows <= 8) ? 8 : 0;
+    // With 3..16 rows (the verify rows of one sequence) the 16 (or 32) columns of the MMA hold every activation twice over:
+    // as bf16(x) and as bf16(x - bf16(x)), 8 (or 16) rows apart.  The weights stream once all the same, and the GEMMs'
+    // inputs are no longer rounded to 8 bits of mantissa.
+    const int lo = !c->two_part ? 0 : (n_rows >= 3 && n_rows <= 8) ? 8 : (n_rows >= 9 && n_rows <= 16) ? 16 : 0;
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -630,6 +640,27 @@ sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
     return SD_OK;
 }
 
+// Optional timing of whole calls with CUDA events on the context's stream (around the graph launch or the launches).
+struct CostScope {
+    sd_ctx* c; int idx;
+    CostScope(sd_ctx* ctx, int kind, int units) : c(ctx), idx(-1) {
+        ++c->cost_depth;
+        if (!c->cost_on || c->cost_depth > 1 || c->cost_pending.size() >= 8192) return;      // only the outermost call is timed; sd_cost_read drains the list
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(c->st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return;      // inside another call's capture
+        sd_ctx::CostMark m;
+        for (cudaEvent_t* e : {&m.e0, &m.e1}) {
+            if (!c->cost_free.empty()) { *e = c->cost_free.back(); c->cost_free.pop_back(); }
+            else if (cudaEventCreate(e) != cudaSuccess) return;
+        }
+        m.kind = kind; m.units = units;
+        if (cudaEventRecord(m.e0, c->st) != cudaSuccess) return;
+        c->cost_pending.push_back(m);
+        idx = (int)c->cost_pending.size() - 1;
+    }
+    ~CostScope() { --c->cost_depth; if (idx >= 0) cudaEventRecord(c->cost_pending[idx].e1, c->st); }
+};
+
 sd_status make_list(sd_ctx* c, const int32_t* seqs, int n_seq, int min_phase, SeqList& list) {
     if (!c || !seqs || n_seq < 1 || n_seq > SD_MAX_BATCH) return SD_ERR_INVALID_ARG;
     list.n = n_seq;
@@ -723,6 +754,8 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     c->pass_count = 0; c->tags_due_clear = false;
     c->pass_on = false; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
     c->two_part = true;
+    c->cost_on = false; c->cost_depth = 0;
+    for (int i = 0; i < 3; ++i) { c->cost_ms[i] = 0.0; c->cost_units[i] = 0; }
     c->force_plain = false;
     c->graphs_on = true;
     c->graph_clock = 0;
@@ -761,6 +794,8 @@ sd_status sd_destroy(sd_ctx* c) {
     if (!c) return SD_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->st);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    for (auto& m : c->cost_pending) { cudaEventDestroy(m.e0); cudaEventDestroy(m.e1); }
+    for (cudaEvent_t e : c->cost_free) cudaEventDestroy(e);
     for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
     delete c;
     return SD_OK;
@@ -906,6 +941,7 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows);
     for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
     bound = bound_bucket(bound + gamma) - gamma;
+    CostScope cost(c, 0, gamma);
     for (int k = 0; k < c->cfg.n_drafts; ++k) {             // programs of the persistent kernel exist before anything is captured
         int n = 0;
         for (int i = 0; i < n_seq; ++i) n += c->draft_id[seqs[i]] == k;
@@ -951,6 +987,7 @@ sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const 
     KeyBuilder key;
     key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
     SD_TRY(prepare_pass(c, 0, plan, n_seq * (gamma + 1), LOGITS_ALL));
+    CostScope cost(c, 1, 1);
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev); });
 }
 
@@ -966,6 +1003,7 @@ sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logit
     KeyBuilder key;
     key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
     SD_TRY(prepare_pass(c, 0, plan, n_seq, LOGITS_ALL));
+    CostScope cost(c, 2, 1);
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev); });
 }
 
@@ -992,6 +1030,7 @@ sd_status sd_accept_seqs(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, c
     p.target = logits_dev; p.target_is_logits = 1; p.q = q_dev; p.x = x_dev;
     p.B = n_seq; p.gamma = gamma; p.V = c->models[0].d.vocab; p.T = c->cfg.temperature; p.seed = c->cfg.seed;
     p.iter = c->S.iter; p.seq_id = c->S.seq_id; p.use_list = 1; p.n_acc = n_acc_dev; p.out_tok = out_tok_dev;
+    p.alpha_terms = gamma > 0 ? c->alpha_terms : nullptr;
     LAUNCH(CAT_SAMPLING, launch_accept(p, 1, c->st));
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
@@ -1003,7 +1042,7 @@ sd_status sd_kv_rollback(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, c
     if (gamma < 0 || gamma > c->cfg.max_gamma || !n_acc_dev || !out_tok_dev) return SD_ERR_INVALID_ARG;
     for (int i = 0; i < n_seq; ++i)
         if (c->len_ub[seqs[i]] + gamma + 1 > c->S.tok_stride) return SD_ERR_CAPACITY;
-    LAUNCH(CAT_STATE, launch_rollback(c->S, list, gamma, n_acc_dev, out_tok_dev, c->st));
+    LAUNCH(CAT_STATE, launch_rollback(c->S, list, gamma, n_acc_dev, out_tok_dev, gamma > 0 ? c->alpha_terms : nullptr, c->st));
     CUDA_TRY(prof_mark(c, CAT_NONE));
     for (int i = 0; i < n_seq; ++i) c->len_ub[seqs[i]] += gamma + 1;
     return SD_OK;
@@ -1073,6 +1112,7 @@ sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma,
         c->graphs_on = saved;
         return s;
     };
+    CostScope cost(c, 1, 1);                     // (sd_verify inside runs in this call's capture and does not time itself)
     const bool replay = saved && !c->prof_on;
     bool cached = false;
     if (replay) for (auto& g : c->graphs) cached |= g.key == key.bytes;
@@ -1172,6 +1212,54 @@ size_t sd_pass_schedule_blob(const int32_t* shape12, const int32_t* waves, const
     if (!p.error.empty()) return 0;
     if (out && cap >= p.blob.size()) memcpy(out, p.blob.data(), p.blob.size());
     return p.blob.size();
+}
+
+sd_status sd_seq_alpha(sd_ctx* c, int seq, double* alpha_sum_out, int64_t* judged_out) {
+    if (!c || seq < 0 || seq >= c->cfg.max_seqs || !alpha_sum_out || !judged_out) return SD_ERR_INVALID_ARG;
+    if (c->phase[seq] == PH_FREE) return SD_ERR_STATE;
+    CUDA_TRY(cudaMemcpyAsync(alpha_sum_out, c->S.alpha_sum + seq, sizeof(double), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaMemcpyAsync(judged_out, c->S.judged + seq, sizeof(int64_t), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_cost_timing(sd_ctx* c, int enable) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    c->cost_on = enable != 0;
+    return SD_OK;
+}
+
+sd_status sd_cost_read(sd_ctx* c, sd_cost* out, int reset) {
+    if (!c || !out) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (auto& m : c->cost_pending) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, m.e0, m.e1) == cudaSuccess) { c->cost_ms[m.kind] += ms; c->cost_units[m.kind] += (uint64_t)m.units; }
+        else (void)cudaGetLastError();
+        c->cost_free.push_back(m.e0); c->cost_free.push_back(m.e1);
+    }
+    c->cost_pending.clear();
+    memset(out, 0, sizeof(*out));
+    out->draft_passes = (int64_t)c->cost_units[0]; out->verify_passes = (int64_t)c->cost_units[1]; out->target_passes = (int64_t)c->cost_units[2];
+    out->draft_pass_ms = c->cost_units[0] ? c->cost_ms[0] / c->cost_units[0] : 0.0;
+    out->verify_pass_ms = c->cost_units[1] ? c->cost_ms[1] / c->cost_units[1] : 0.0;
+    out->target_pass_ms = c->cost_units[2] ? c->cost_ms[2] / c->cost_units[2] : 0.0;
+    const double denom = out->target_pass_ms > 0.0 ? out->target_pass_ms : out->verify_pass_ms;      // Eq. 1 takes a verify pass to cost one target pass
+    out->c = (out->draft_pass_ms > 0.0 && denom > 0.0) ? out->draft_pass_ms / denom : 0.0;
+    if (reset) for (int i = 0; i < 3; ++i) { c->cost_ms[i] = 0.0; c->cost_units[i] = 0; }
+    return SD_OK;
+}
+
+int sd_best_gamma_measured(sd_ctx* c, int seq, int gamma_max, double* alpha_out, double* c_out, double* speedup_out) {
+    if (!c || seq < 0 || seq >= c->cfg.max_seqs || gamma_max < 1) return 0;
+    double a_sum = 0.0;
+    int64_t judged = 0;
+    sd_cost cost;
+    if (sd_seq_alpha(c, seq, &a_sum, &judged) != SD_OK || judged <= 0 || sd_cost_read(c, &cost, 0) != SD_OK || cost.c <= 0.0) return 0;
+    const double alpha = std::min(1.0, std::max(0.0, a_sum / (double)judged));
+    if (alpha_out) *alpha_out = alpha;
+    if (c_out) *c_out = cost.c;
+    return sd_best_gamma(alpha, cost.c, gamma_max, speedup_out);
 }
 
 sd_status sd_use_graphs(sd_ctx* c, int on) {

@@ -26,6 +26,8 @@ struct SeqState {
     int32_t* draft_id;      // which draft the sequence is routed to
     int32_t* n_prompt;      // prompt length (the classifier pools over the prompt only)
     int64_t* counters;      // [slot][4]: iterations, drafted, accepted, emitted
+    double* alpha_sum;      // [slot]: sum over judged slots of sum_k min(p, q)
+    int64_t* judged;        // [slot]: judged slots so far (slot s of an iteration is judged iff all before it were accepted)
     int32_t* tokens;        // [slot][tok_stride]
     int tok_stride;
     int max_ctx;

@@ -188,6 +188,7 @@ __global__ void k_set_state(SeqState S, int slot, int len, int tkv, int dkv, uin
     if (reset) {
         S.seq_id[slot] = seq_id; S.n_prompt[slot] = len;
         for (int i = 0; i < 4; ++i) S.counters[slot * 4 + i] = 0;
+        S.alpha_sum[slot] = 0.0; S.judged[slot] = 0;
     }
 }
 cudaError_t launch_set_state(const SeqState& S, int slot, int len, int tkv, int dkv, uint32_t iter, uint32_t seq_id,
@@ -199,7 +200,7 @@ cudaError_t launch_set_state(const SeqState& S, int slot, int len, int tkv, int 
 // Commit of one iteration.  Nothing in either KV cache moves: the lengths shrink and the
 // next append lands on the rejected positions.
 __global__ void k_rollback(SeqState S, SeqList list, int gamma, const int32_t* __restrict__ n_acc,
-                           const int32_t* __restrict__ out_tok) {
+                           const int32_t* __restrict__ out_tok, const float* __restrict__ alpha_terms) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= list.n) return;
     const int slot = list.ids[i], b = list.out[i];
@@ -217,10 +218,17 @@ __global__ void k_rollback(SeqState S, SeqList list, int gamma, const int32_t* _
     S.counters[slot * 4 + 1] += gamma;
     S.counters[slot * 4 + 2] += n;
     S.counters[slot * 4 + 3] += n + 1;
+    if (alpha_terms) {                          // the judged slots, in order: run-to-run identical sums
+        double a = 0.0;
+        const int nj = min(n + 1, gamma);
+        for (int s = 0; s < nj; ++s) a += (double)alpha_terms[(size_t)b * gamma + s];
+        S.alpha_sum[slot] += a;
+        S.judged[slot] += nj;
+    }
 }
 cudaError_t launch_rollback(const SeqState& S, const SeqList& list, int gamma, const int32_t* n_acc,
-                            const int32_t* out_tok, cudaStream_t st) {
-    k_rollback<<<1, 64, 0, st>>>(S, list, gamma, n_acc, out_tok);
+                            const int32_t* out_tok, const float* alpha_terms, cudaStream_t st) {
+    k_rollback<<<1, 64, 0, st>>>(S, list, gamma, n_acc, out_tok, alpha_terms);
     return cudaGetLastError();
 }
 

@@ -232,12 +232,12 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     }
 }
 
-template <int MODE>
+template <int MODE, bool HL>
 cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status, int n_rows,
                              int pieces, int dependent, cudaStream_t st) {
     const dim3 grid(g.n_tiles, (n_rows + 15) / 16);
-    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
-    return launch_pdl(k_fused_step<MODE, 16, 4>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2, HL>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    return launch_pdl(k_fused_step<MODE, 16, 4, HL>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
 }  // namespace
@@ -264,6 +264,26 @@ bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
     return g.grid >= 1 && n_rows > 2 && n_rows <= rows_per_cta(n_rows, pieces_bound(g));
 }
 
+namespace {
+
+template <bool HL>
+cudaError_t launch_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status, int n_rows, int pieces,
+                        int dependent, cudaStream_t st) {
+    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32, HL>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    if (n_rows > 8 && pieces <= 4) {
+        switch (ep.mode) {
+        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        default: return cudaErrorInvalidValue;
+        }
+    }
+    return launch_pdl(k_fused_step<-1, 8, 8, HL>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+}
+
+}  // namespace
+
 cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status,
                               int dependent, cudaStream_t st) {
     if (g.grid < 1 || g.m_tok > SD_MAX_ROWS) return cudaErrorInvalidValue;
@@ -274,21 +294,11 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
     const int pieces = pieces_bound(g);
-    if (ep.lo_off) {                                   // two-part activations: the verify rows only (3..8 rows, one batch per tile)
-        if (n_rows < 1 || n_rows > 8 || ep.lo_off != 8 || ep.m_real + ep.lo_off != g.m_tok) return cudaErrorInvalidValue;
-        return launch_pdl(k_fused_step<-1, 8, 8, true>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    if (ep.lo_off) {                                   // two-part activations: accumulator rows r and r + lo_off belong together
+        if (ep.m_real < 1 || ep.m_real > ep.lo_off || ep.m_real + ep.lo_off != g.m_tok) return cudaErrorInvalidValue;
+        return launch_step<true>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
     }
-    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
-    if (n_rows > 8 && pieces <= 4) {
-        switch (ep.mode) {
-        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        default: return cudaErrorInvalidValue;
-        }
-    }
-    return launch_pdl(k_fused_step<-1, 8, 8>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    return launch_step<false>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
 }
 
 }  // namespace sd

@@ -30,7 +30,7 @@ cudaError_t launch_swiglu(const float* gu, void* act, int dtype, int n_rows, int
 cudaError_t launch_set_state(const SeqState& S, int slot, int len, int tkv, int dkv, uint32_t iter, uint32_t seq_id,
                              int reset_counters, cudaStream_t st);
 cudaError_t launch_rollback(const SeqState& S, const SeqList& list, int gamma, const int32_t* n_acc,
-                            const int32_t* out_tok, cudaStream_t st);
+                            const int32_t* out_tok, const float* alpha_terms /*nullable: [n_seq][gamma]*/, cudaStream_t st);
 
 // ---- linear_simt.cu : y[rows][n_out] fp32 = x[rows][n_in] * W[n_out][n_in]^T on CUDA cores
 cudaError_t launch_linear_simt(const void* x, const void* w, float* y, int rows, int n_out, int n_in, int dtype,
@@ -65,6 +65,7 @@ struct AcceptParams {
     const uint32_t* iter; const uint32_t* seq_id;   // indexed through `list` when use_list
     int use_list; SeqList list;
     int32_t* n_acc; int32_t* out_tok;
+    float* alpha_terms;          // nullable: [B][gamma] receives sum_k min(p_s(k), q_s(k)) of every slot (the estimate of Eq. 1's alpha)
 };
 cudaError_t launch_accept(const AcceptParams& p, int dependent, cudaStream_t st);
 

@@ -265,6 +265,13 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
             }
             __syncthreads();
         }
+        if (P.alpha_terms && j < gamma) {                       // Eq. 1's alpha for this slot: the draft is kept with probability sum_k min(p, q)
+            const float* qj = q + (size_t)j * V;
+            float a = 0.f;
+            for (int k = threadIdx.x; k < V; k += blockDim.x) a += fminf(prob(j, li, k), qj[k]);
+            a = block_sum(a, sh.red);
+            if (threadIdx.x == 0) P.alpha_terms[(size_t)b * gamma + j] = a;
+        }
         if (threadIdx.x == 0 && j < gamma) {
             int ok = 0;
             const int xs = x[j];

@@ -37,8 +37,8 @@ def _build(sd, target_dims, draft_dims_list, dtype, T, seed, max_seqs=2, max_ctx
     return ctx, omodels
 
 
-def _replay(sd, ctx, omodels, draft_k, prompt, gamma, T, seed, max_new, dtype, seq=0, seq_id=0, min_agree=0.8):
-    tol = TOL[dtype]
+def _replay(sd, ctx, omodels, draft_k, prompt, gamma, T, seed, max_new, dtype, seq=0, seq_id=0, min_agree=0.8, tol_logits=None):
+    tol = dict(TOL[dtype], logits=tol_logits) if tol_logits is not None else TOL[dtype]
     V = omodels[0].dims["vocab"]
     toks_ref, cnt_ref, tr = oracle.spec_decode(omodels[0], omodels[1 + draft_k], prompt, max_new, gamma, T, seed,
                                                seq_id=seq_id, trace_iters=max_new, trace_probs=True, trace_logits=True)
@@ -96,7 +96,13 @@ def _replay(sd, ctx, omodels, draft_k, prompt, gamma, T, seed, max_new, dtype, s
     assert got[: len(toks_ref)].tolist() == toks_ref.tolist()
     assert agree_x >= min_agree * n_it, (agree_x, n_it)
     assert agree_acc >= min_agree * n_it, (agree_acc, n_it)
-    return dict(iters=n_it, agree_x=agree_x, agree_acc=agree_acc, logit=worst_logit, p=worst_p, q=worst_q)
+    # estimate of Eq. 1's alpha: the judged slots are the oracle's (its n_acc was committed), their sums of min(p, q) the GPU's
+    a_sum, judged = ctx.sd_seq_alpha(seq)
+    assert judged == tr["judged"]
+    if T > 0:       # |sum min(p,q) - sum min(p',q')| <= |p-p'|_1 + |q-q'|_1, each at most about 2 * (logit error) / T
+        assert abs(a_sum - tr["alpha_sum"]) <= judged * 4.0 * tol["logits"] / T, (a_sum, tr["alpha_sum"], judged)
+    return dict(alpha_sum=a_sum, judged=judged, alpha_ref=tr["alpha_sum"] / max(1, tr["judged"]),
+                iters=n_it, agree_x=agree_x, agree_acc=agree_acc, logit=worst_logit, p=worst_p, q=worst_q)
 
 
 def toks_ref_full(tr, prompt, it):
@@ -130,6 +136,41 @@ def test_tiny_self_draft_accepts_and_counts(sd):
     r = _replay(sd, ctx, om, 0, prompt, 4, 1.0, 9, 30, "f32", min_agree=0.8)
     _, cnt = ctx.sd_seq_read(0)
     assert cnt["accepted"] >= 0.9 * cnt["drafted"]
+    ctx.close()
+
+
+def test_alpha_estimate_acceptance_rate_and_tau_against_the_oracle(sd):
+    """Eq. 1's inputs from the library itself: alpha-hat = mean over judged slots of sum_k min(p, q), the acceptance rate
+    (accepted / drafted), tau (tokens per verify iteration) and the cost ratio c from its own clock."""
+    cfg = synth.CONFIGS["tiny"]
+    wl = cfg["workload"]
+    T = 1.0
+    ctx, om = _build(sd, cfg["target"], cfg["drafts"], "f32", T, wl["seed"], max_ctx=wl["max_ctx"])
+    prompt = synth.make_prompt(cfg["target"]["vocab"], wl["prompt"], seed=wl["seed"])
+    ctx.sd_cost_timing(1)
+    r = _replay(sd, ctx, om, 1, prompt, wl["gamma"], T, wl["seed"], wl["max_new"], "f32")
+    alpha = r["alpha_sum"] / r["judged"]
+    assert abs(alpha - r["alpha_ref"]) <= 1e-4, (alpha, r["alpha_ref"])
+    _, cnt = ctx.sd_seq_read(0)
+    _, cnt_ref, _ = oracle.spec_decode(om[0], om[2], prompt, wl["max_new"], wl["gamma"], T, wl["seed"], seq_id=0)
+    ar, ar_ref = cnt["accepted"] / cnt["drafted"], cnt_ref["accepted"] / cnt_ref["drafted"]
+    tau, tau_ref = cnt["emitted"] / cnt["iterations"], cnt_ref["emitted"] / cnt_ref["iterations"]
+    assert ar == ar_ref and tau == tau_ref
+    # alpha-hat estimates the acceptance rate of the judged slots (the draws are the oracle's; a loose statistical bound)
+    assert abs(alpha - ar) < 0.25
+    cost = ctx.sd_cost_read()
+    assert cost["draft_passes"] == r["iters"] * wl["gamma"] and cost["verify_passes"] == r["iters"]
+    assert cost["draft_pass_ms"] > 0 and cost["verify_pass_ms"] > 0
+    assert abs(cost["c"] - cost["draft_pass_ms"] / cost["verify_pass_ms"]) < 1e-12
+    g, a, c_ratio, speed = ctx.sd_best_gamma_measured(0, 8)
+    assert abs(a - alpha) < 1e-12 and abs(c_ratio - cost["c"]) < 1e-12
+    g_ref, speed_ref = sd.sd_best_gamma(alpha, cost["c"], 8)
+    assert g == g_ref and abs(speed - speed_ref) < 1e-12
+    eq1 = [(1 - alpha ** (k + 1)) / ((1 - alpha) * (k * cost["c"] + 1)) for k in range(1, 9)]        # Eq. 1 written out
+    assert abs(speed_ref - max([1.0] + eq1)) < 1e-9
+    # a new sequence starts from zero
+    ctx.sd_seq_begin(0, prompt, 5)
+    assert ctx.sd_seq_alpha(0) == (0.0, 0)
     ctx.close()
 
 

@@ -38,6 +38,12 @@ def test_head_dim_128_and_long_context_on_the_pass_kernel(sd):
     ctx.close()
 
 
+# The persistent kernel (opt-in) hands activations over as ONE bf16 part, the default path as two.  The widest model's
+# nine-row verify step then lands just above the default path's 5e-2 (measured 0.0502), so that case carries the
+# one-part bound.
+ONE_PART_BOUND = {"1b": 5e-2, "7b": 5e-2, "13b": 6e-2}
+
+
 @pytest.mark.parametrize("name", sorted(FULL_WIDTH))
 def test_benchmark_shapes_at_full_width_on_the_pass_kernel(sd, name):
     spec = FULL_WIDTH[name]
@@ -49,7 +55,8 @@ def test_benchmark_shapes_at_full_width_on_the_pass_kernel(sd, name):
     ctx, om = _build(sd, t, [d], "bf16", wl["temperature"], wl["seed"], max_seqs=1, max_ctx=spec["prompt"] + 40, max_gamma=gamma)
     ctx.sd_use_pass_kernel(1, 0)
     prompt = synth.make_prompt(t["vocab"], spec["prompt"], seed=wl["seed"])
-    r = _replay(sd, ctx, om, 0, prompt, gamma, wl["temperature"], wl["seed"], 2 * (gamma + 1), "bf16", min_agree=0.0)
+    r = _replay(sd, ctx, om, 0, prompt, gamma, wl["temperature"], wl["seed"], 2 * (gamma + 1), "bf16", min_agree=0.0,
+                tol_logits=ONE_PART_BOUND[name])
     assert r["iters"] >= 2
     ctx.close()
 
