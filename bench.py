@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the verify step (target pass over gamma+1 rows + accept/reject + KV rollback).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 7b] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 7b|all] [--impl reference] [--gamma-sweep 1..10]
 
 One JSON line on stdout.  `value` is verify-step tokens/s: B * (gamma + 1) query positions per
 sd_verify + sd_accept_seqs + sd_kv_rollback, timed with CUDA events on the library's stream with
@@ -159,7 +159,9 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def run_gpu(args):
+def setup(args, gamma_max, steps_per_phase):
+    """Context with the config's models (random-init, generated on the device), its sequences begun, routed and prefilled.
+    Prompts are shortened where the config's cache could not hold `steps_per_phase` verify steps after them."""
     import torch
     import torch.distributed as dist
     from paper_2505_08600_b200 import binding as sd
@@ -167,6 +169,8 @@ def run_gpu(args):
     rank, world, local = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} wants cuda:{local}, the node has {torch.cuda.device_count()} GPU(s)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     torch.cuda.set_stream(torch.cuda.Stream(dev))           # a capturable (non-default) stream for everything below
@@ -174,18 +178,17 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)      # only for the barrier and the max over ranks
     cfg = synth.CONFIGS[args.config]
     wl, tdims = cfg["workload"], cfg["target"]
-    gamma = args.gamma if args.gamma is not None else wl["gamma"]
     B, V, T, seed = wl["batch"], tdims["vocab"], wl["temperature"], wl["seed"]
-    K, W = args.steps, args.warmup
-    n_iter_phase = min(10, K)
-    total_steps = 2 * (K + W) + args.profile_steps + n_iter_phase + 8
+    need = (gamma_max + 1) * steps_per_phase + gamma_max + 8
     if isinstance(wl["prompt"], int):
         lens = [wl["prompt"]] * B
     else:
         lens = synth.make_prompt_lengths(B, wl["prompt"][0], wl["prompt"][1], seed=seed).tolist()
-    max_ctx = max(wl["max_ctx"], max(lens) + (gamma + 1) * total_steps + 8)
+    if max(lens) + need > wl["max_ctx"] and wl["max_ctx"] - need >= max(lens) // 2:
+        lens = [min(n, wl["max_ctx"] - need) for n in lens]          # the timed steps end at the config's cache size
+    max_ctx = max(wl["max_ctx"], max(lens) + need)
 
-    ctx = sd.Context(tdims, cfg["drafts"], cfg["dtype"], B, max_ctx, max(gamma, 1), T, seed, clf_d_hidden=cfg["classifier"][1], device=dev)
+    ctx = sd.Context(tdims, cfg["drafts"], cfg["dtype"], B, max_ctx, max(gamma_max, 1), T, seed, clf_d_hidden=cfg["classifier"][1], device=dev)
     for mid, dims in enumerate([tdims] + list(cfg["drafts"])):
         for name, l, tensor in device_weights(torch, dims, cfg["dtype"], 0, mid, dev):
             ctx.sd_load_tensor(mid, sd.TENSOR_KIND[name], l, tensor)
@@ -194,11 +197,31 @@ def run_gpu(args):
     torch.cuda.synchronize()
 
     seqs = list(range(B))
+    prompts = [synth.make_prompt(V, lens[s], seed=seed, seq=s) for s in seqs]
     for s in seqs:
-        ctx.sd_seq_begin(s, synth.make_prompt(V, lens[s], seed=seed, seq=s), s)
+        ctx.sd_seq_begin(s, prompts[s], s)
     n_drafts = len(cfg["drafts"])
     routed = ctx.sd_route_prompt(seqs) if B == 1 else ctx.sd_route_prompt(seqs, forced_task=[s % n_drafts for s in seqs])
     ctx.sd_prefill(seqs)
+
+    def rewind():        # back to the prompts (the caches keep their prefix), so that every phase sees the same contexts
+        for s in seqs:
+            ctx.sd_seq_force(s, prompts[s], lens[s] - 1, 0)
+
+    return dict(torch=torch, dist=dist, sd=sd, rank=rank, world=world, local=local, dev=dev, cfg=cfg, ctx=ctx, seqs=seqs, lens=lens,
+                routed=routed, rewind=rewind, max_ctx=max_ctx)
+
+
+def run_gpu(args):
+    K, W = args.steps, args.warmup
+    n_iter_phase = min(10, K)
+    cfg0 = synth.CONFIGS[args.config]
+    gamma = args.gamma if args.gamma is not None else cfg0["workload"]["gamma"]
+    env = setup(args, gamma, K + W + args.profile_steps + 4)
+    torch, dist, sd, ctx = env["torch"], env["dist"], env["sd"], env["ctx"]
+    rank, world, local, dev, cfg, seqs, lens, routed, rewind = (env[k] for k in ("rank", "world", "local", "dev", "cfg", "seqs", "lens", "routed", "rewind"))
+    wl, tdims = cfg["workload"], cfg["target"]
+    B, V, T, seed = wl["batch"], tdims["vocab"], wl["temperature"], wl["seed"]
 
     x = torch.zeros((B, gamma), dtype=torch.int32, device=dev)
     q = torch.zeros((B, gamma, V), dtype=torch.float32, device=dev)
@@ -207,6 +230,7 @@ def run_gpu(args):
     out_tok = torch.zeros((B, gamma + 1), dtype=torch.int32, device=dev)
     ctx.sd_draft_steps(seqs, gamma, x, q)          # the drafts every timed verify step scores (values do not change its cost)
     torch.cuda.synchronize()
+    rewind()
 
     def verify_step():          # sd_verify + sd_accept_seqs + sd_kv_rollback as one captured launch sequence
         ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
@@ -222,15 +246,15 @@ def run_gpu(args):
 
     stream = torch.cuda.current_stream(dev)
     # ---- phase A: the headline, device-resident inputs
-    for _ in range(W):
-        verify_step()
-    l0 = ctx.sd_launch_count()
     try:
         gpu_id = str(torch.cuda.get_device_properties(dev).uuid)
         gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
     except Exception:
         gpu_id = str(local)
-    sampler = ClockSampler(gpu_id)
+    sampler = ClockSampler(gpu_id)                 # samples cover the warm-up steps (the same launches) and the timed steps
+    for _ in range(W):
+        verify_step()
+    l0 = ctx.sd_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.profiler.start()                 # a profiler told to wait for this range sees the timed steps only
@@ -246,6 +270,7 @@ def run_gpu(args):
     ms_step = ms_total / K
     value = replicas.whole_job_tokens_per_s(world, B, gamma, ms_step)
     ctx.sd_seq_read(0)
+    n_ctx = [int(ctx.sd_seq_read(s)[0].shape[0]) for s in seqs]          # context lengths at the end of the timed steps
 
     # ---- per-kernel split of the same step (events between launches; separate from the timed run)
     ctx.sd_profile(1)
@@ -253,7 +278,7 @@ def run_gpu(args):
         verify_step()
     prof = ctx.sd_profile_read()
     ctx.sd_profile(0)
-    n_ctx = [int(ctx.sd_seq_read(s)[0].shape[0]) for s in seqs]
+    rewind()
     esz = 2 if cfg["dtype"] == "bf16" else 4
     weight_bytes = synth.param_count(tdims, streamed_only=True) * esz
     kv_bytes = sum(n_ctx) * 2 * tdims["n_layers"] * tdims["n_kv_heads"] * tdims["head_dim"] * esz
@@ -302,6 +327,7 @@ def run_gpu(args):
     e2e = {"value": replicas.whole_job_tokens_per_s(world, B, gamma, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": int(xh.numel() * 4 + qh.numel() * 4), "d2h_bytes_per_step": int(nh.numel() * 4 + oh.numel() * 4)}
     ctx.sd_seq_read(0)
+    rewind()
 
     # ---- whole iterations and the cost ratio c of Eq. 1
     def timed(fn, n):
@@ -342,6 +368,7 @@ def run_gpu(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
             "config": {"workload": f"{args.config}: batch {B}, gamma {gamma}, prompt {lens if B > 1 else lens[0]}, "
                                    f"target {tdims['n_layers']}x{tdims['d_model']}, verify step = sd_verify + sd_accept_seqs + sd_kv_rollback",
+                       "context_at_end_of_timed_steps": n_ctx if B > 1 else n_ctx[0],
                        "l2": "weights (>= 2 GB per step) far exceed the 126 MB L2; no flush", "replicas": world,
                        "device_status": status},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras,
@@ -349,6 +376,72 @@ def run_gpu(args):
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_gamma_sweep(args):
+    """Verify step, draft step and Eq. 1 against gamma at one configuration (one GPU): for every gamma of the range the
+    verify step is timed like the headline (device-resident inputs, CUDA events), the cost ratio c comes from the
+    library's own clock (sd_cost_read) and alpha-hat from its accumulator (sd_seq_alpha)."""
+    lo, hi = (int(v) for v in args.gamma_sweep.split(".."))
+    K, W = args.steps, args.warmup
+    env = setup(args, hi, K + W + 8)
+    torch, sd, ctx, dev, cfg, seqs, rewind = (env[k] for k in ("torch", "sd", "ctx", "dev", "cfg", "seqs", "rewind"))
+    wl, tdims = cfg["workload"], cfg["target"]
+    B, V = wl["batch"], tdims["vocab"]
+    stream = torch.cuda.current_stream(dev)
+    l1 = torch.zeros((B, 1, V), dtype=torch.float32, device=dev)
+    rows = []
+    for gamma in range(lo, hi + 1):
+        x = torch.zeros((B, gamma), dtype=torch.int32, device=dev)
+        q = torch.zeros((B, gamma, V), dtype=torch.float32, device=dev)
+        logits = torch.zeros((B, gamma + 1, V), dtype=torch.float32, device=dev)
+        n_acc = torch.zeros((B,), dtype=torch.int32, device=dev)
+        out_tok = torch.zeros((B, gamma + 1), dtype=torch.int32, device=dev)
+        rewind()
+        for _ in range(3):                          # graphs captured, caches warm
+            ctx.sd_draft_steps(seqs, gamma, x, q)
+            ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
+            ctx.sd_target_step(seqs, l1)
+        rewind()
+        ctx.sd_cost_timing(1)
+        ctx.sd_cost_read(reset=1)
+        for _ in range(5):                          # whole iterations on the library's clock: c, and alpha-hat of these drafts
+            ctx.sd_draft_steps(seqs, gamma, x, q)
+            ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
+        for _ in range(5):
+            ctx.sd_target_step(seqs, l1)
+        cost = ctx.sd_cost_read(reset=1)
+        ctx.sd_cost_timing(0)
+        a_sum, judged = ctx.sd_seq_alpha(0)
+        rewind()
+        ctx.sd_draft_steps(seqs, gamma, x, q)
+        rewind()
+        for _ in range(W):
+            ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            ctx.sd_verify_accept(seqs, gamma, x, q, logits, n_acc, out_tok)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / K
+        c = cost["c"]
+        rows.append({"gamma": gamma, "verify_step_ms": ms, "verify_step_tokens_per_s": B * (gamma + 1) / (ms * 1e-3),
+                     "draft_pass_ms": cost["draft_pass_ms"], "target_pass_ms": cost["target_pass_ms"], "verify_pass_ms_library_clock": cost["verify_pass_ms"],
+                     "c": c, "verify_over_decode": ms / cost["target_pass_ms"] if cost["target_pass_ms"] else None,
+                     "alpha_hat_random_init": a_sum / judged if judged else None,
+                     "eq1_speedup": {f"alpha={a}": eq1_speedup(a, gamma, c) for a in (0.6, 0.8)},
+                     # Eq. 1 takes the verify pass to cost one decode pass; with the measured verify pass instead:
+                     "speedup_with_measured_verify": {f"alpha={a}": (1 - a ** (gamma + 1)) / (1 - a) * cost["target_pass_ms"] /
+                                                      (gamma * cost["draft_pass_ms"] + ms) for a in (0.6, 0.8)} if cost["target_pass_ms"] else None})
+    c_mean = sum(r["c"] for r in rows) / len(rows)
+    status = ctx.sd_device_status()
+    print(json.dumps({"metric": "gamma_sweep", "unit": "per gamma", "n_gpus": 1, "steps": K, "warmup": W, "dtype": cfg["dtype"], "data": "synthetic",
+                      "config": {"workload": f"{args.config}: batch {B}, gamma {lo}..{hi}, prompt {env['lens'] if B > 1 else env['lens'][0]}", "device_status": status},
+                      "best_gamma": {f"alpha={a}": dict(zip(("gamma", "speedup"), sd.sd_best_gamma(a, c_mean, hi))) for a in (0.6, 0.8)},
+                      "c_mean": c_mean, "sweep": rows}))
+    ctx.close()
 
 
 def run_accept_microbench(args):
@@ -397,18 +490,37 @@ def run_accept_microbench(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=150)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="7b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--config", default="7b", choices=sorted(synth.CONFIGS) + ["all"], help="'all': one JSON line per configuration, each in its own process")
+    ap.add_argument("--gamma-sweep", default=None, metavar="LO..HI", help="time the verify and draft steps for every gamma of the range and exit")
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    launched = "WORLD_SIZE" in os.environ
+    if args.config == "all":
+        if launched and int(os.environ["WORLD_SIZE"]) > 1:
+            raise SystemExit("--config all runs one process per configuration; start it without a launcher")
+        rc = 0
+        for name in synth.CONFIGS:
+            argv = [sys.executable, os.path.abspath(__file__)] + [a for a in sys.argv[1:]]
+            i = argv.index("--config")
+            argv[i + 1] = name
+            rc = rc or subprocess.run(argv).returncode
+        sys.exit(rc)
+    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep:
+        # no launcher: this process starts the N replicas itself (one per GPU) and passes rank 0's line through
+        rc, out = replicas.spawn_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+        sys.stdout.write(out)
+        sys.exit(rc)
     if args.accept_microbench:
         run_accept_microbench(args)
+    elif args.gamma_sweep:
+        run_gamma_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

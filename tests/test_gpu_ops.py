@@ -91,6 +91,38 @@ def test_attention_over_cache(sd, dtype, H, Hkv, hd, max_ctx, positions):
             np.testing.assert_allclose(got[r, h], ref, rtol=0, atol=tol)
 
 
+def test_attention_launch_of_the_eight_sequence_long_cache_configuration(sd):
+    """The attention launch of the 13B-class workload as the verify step issues it: 8 sequences x 9 rows, 40 heads of
+    128, caches of 8192 positions, the rows at the last nine positions.  The oracle scores sampled (row, head) pairs."""
+    B, g1, H, hd, max_ctx = 8, 9, 40, 128, 8192
+    rows = B * g1
+    q = quantize(synth.make_logits((rows, H, hd), seed=41, stream=hd), "bf16")
+    base_k = quantize(synth.make_logits((H, max_ctx, hd), seed=42, stream=hd), "bf16")
+    base_v = quantize(synth.make_logits((H, max_ctx, hd), seed=43, stream=hd), "bf16")
+    # sequence b's cache is the base block rolled by 97 * b positions (eight distinct caches from one generated block)
+    kc = torch.empty((B, H, max_ctx, hd), dtype=torch.bfloat16, device=DEV)
+    vc = torch.empty((B, H, max_ctx, hd), dtype=torch.bfloat16, device=DEV)
+    bk, bv = to_dev(base_k), to_dev(base_v)
+    for b in range(B):
+        kc[b] = torch.roll(bk, 97 * b, dims=1)
+        vc[b] = torch.roll(bv, 97 * b, dims=1)
+    row_slot = np.repeat(np.arange(B, dtype=np.int32), g1)
+    row_pos = np.tile(np.arange(max_ctx - g1, max_ctx, dtype=np.int32), B)
+    out = torch.zeros((rows, H, hd), dtype=torch.bfloat16, device=DEV)
+    sd.sd_op_attention(to_dev(q), kc, vc, out, to_dev(row_slot), to_dev(row_pos), H, H, hd, max_ctx, sd.SD_BF16)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    qf, kf, vf = widen(q), widen(base_k), widen(base_v)
+    rng = np.random.default_rng(7)
+    picks = {(0, 0), (rows - 1, H - 1), (g1 - 1, 17), (g1, 3)} | {(int(rng.integers(rows)), int(rng.integers(H))) for _ in range(28)}
+    for r, h in sorted(picks):
+        b, n_ctx = int(row_slot[r]), int(row_pos[r]) + 1
+        ref = oracle.attention_head(qf[r, h], np.roll(kf[h], 97 * b, axis=0)[:n_ctx], np.roll(vf[h], 97 * b, axis=0)[:n_ctx])
+        np.testing.assert_allclose(got[r, h], ref, rtol=0, atol=2e-2)
+    # rows of one sequence differ only by the causal bound: the last row sees eight more keys than the first
+    assert np.abs(got[0] - got[g1 - 1]).max() > 0
+
+
 def test_attention_inactive_row_gives_zeros(sd):
     H, hd, max_ctx = 2, 64, 16
     q = synth.make_logits((2, H, hd), seed=1)

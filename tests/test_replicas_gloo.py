@@ -49,3 +49,32 @@ def test_two_replicas_report_the_slowest_rank_and_the_whole_job():
 def test_single_process_passthrough():
     assert replicas.max_over_ranks(2.5, 1) == 2.5
     assert replicas.whole_job_tokens_per_s(1, 16, 5, 10.0) == 9600.0
+
+
+_CHILD = """
+import torch.distributed as dist
+from paper_2505_08600_b200 import replicas
+rank, world, local = replicas.rank_env()
+dist.init_process_group('gloo')
+ms = replicas.max_over_ranks(2.0 + 3.0 * rank, world)
+if rank == 0:
+    print('slowest', ms, replicas.whole_job_tokens_per_s(world, 1, 5, ms))
+else:
+    print('not rank 0')
+dist.barrier()
+dist.destroy_process_group()
+"""
+
+
+def test_spawn_local_launches_the_ranks_and_returns_rank_zero_output():
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    rc, out = replicas.spawn_local(2, [sys.executable, "-c", f"import sys; sys.path.insert(0, {root!r})\n" + _CHILD], timeout=180)
+    assert rc == 0
+    assert out.split() == ["slowest", "5.0", str(2 * 6 / 5.0e-3)]
+
+
+def test_spawn_local_reports_a_failing_rank():
+    import sys
+    rc, out = replicas.spawn_local(2, [sys.executable, "-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"], timeout=60)
+    assert rc == 3 and out == ""
