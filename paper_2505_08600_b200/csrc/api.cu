@@ -459,7 +459,8 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
 // One weight GEMM and the step that follows it.
 sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
     if (ep.lo_off) rows += ep.lo_off;           // the input rows come in two bf16 parts: [x_hi rows][x_lo rows at + lo_off]
-    const GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
+    GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
+    if (ep.lo_off) { g.lo_off = ep.lo_off; g.m_real = ep.m_real; }
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;

@@ -129,7 +129,6 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
 #pragma unroll
                 for (int i = 0; i < MB; ++i) {
                     tmp[cc][i] = (ok && rows[i] >= 0) ? __ldcg(base + (size_t)rows[i] * TILE_N) : 0.f;
-                    if (HL) tmp[cc][i] += (ok && rows[i] >= 0) ? __ldcg(base + (size_t)(rows[i] + ep.lo_off) * TILE_N) : 0.f;      // the x_lo part
                 }
             }
 #pragma unroll
@@ -295,7 +294,9 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
     const int pieces = pieces_bound(g);
     if (ep.lo_off) {                                   // two-part activations: accumulator rows r and r + lo_off belong together
-        if (ep.m_real < 1 || ep.m_real > ep.lo_off || ep.m_real + ep.lo_off != g.m_tok) return cudaErrorInvalidValue;
+        // (the GEMM's epilogue has already added the two columns of a row: the pieces hold m_real merged rows)
+        if (ep.m_real < 1 || ep.m_real > ep.lo_off || ep.m_real + ep.lo_off != g.m_tok || g.lo_off != ep.lo_off || g.m_real != ep.m_real) return cudaErrorInvalidValue;
+        if (ep.lo_off != 8 && ep.lo_off != 16) return cudaErrorInvalidValue;
         return launch_step<true>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
     }
     return launch_step<false>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);

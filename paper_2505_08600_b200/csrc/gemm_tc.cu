@@ -79,6 +79,18 @@ __device__ void epilogue_warps(const GemmGeom& g, float* __restrict__ partials, 
         if (sh.epi_abort) break;                                       // all four warps leave together
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         float* out = partials + ((size_t)blockIdx.x * g.max_seg + seg) * (size_t)g.m_pad * TILE_N;
+        if (g.lo_off) {                                                // columns r (x_hi) and r + lo_off (x_lo) are one token row
+            const uint32_t t0 = tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad;
+            uint32_t r[16], r2[16];
+            tmem_ld16(t0, r);
+            if (g.lo_off == 16) tmem_ld16(t0 + 16u, r2);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float lo = g.lo_off == 16 ? __uint_as_float(r2[j]) : __uint_as_float(r[(j + 8) & 15]);
+                if (j < g.m_real) __stcg(out + (size_t)j * TILE_N + et, __uint_as_float(r[j]) + lo);
+            }
+        } else
         for (int c0 = 0; c0 < g.m_pad; c0 += 16) {
             uint32_t r[16];
             tmem_ld16(tmem_base + ((quarter * 32u) << 16) + buf * (uint32_t)g.m_pad + (uint32_t)c0, r);
@@ -262,6 +274,7 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
 
 GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     GemmGeom g;
+    g.lo_off = 0; g.m_real = m_tok;
     g.m_tok = m_tok;
     g.m_pad = (m_tok + 15) & ~15;
     g.n_out = n_out;

@@ -18,6 +18,8 @@ struct GemmGeom {
     int grid, max_seg, stages;
     int steady;             // stages reused once the ring has been filled (<= stages)
     int prefill;            // weight tiles requested before the previous kernel has finished
+    int lo_off, m_real;     // two-part input rows (see Epilogue::lo_off): the epilogue adds accumulator columns r and r + lo_off
+                            // and leaves m_real merged rows in each piece; 0: every column is a row of its own
 };
 
 // RMSNorm folded around a GEMM: the GEMM's input rows are h * gain (no 1/rms factor), the
