@@ -221,6 +221,41 @@ double sd_eq1_speedup(double alpha, int gamma, double c);
  * plain decoding (speedup <= 1) or on bad arguments.  speedup_out may be NULL. */
 int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
 
+/* Time stamps of the launches of a forward pass, taken inside the kernels (the device's nanosecond timer) while the
+ * pass runs the way it always runs (captured graph, programmatic dependent launches): what a profiler's serialised
+ * per-kernel times cannot show.  While enabled, every weight GEMM, the step kernel after it and every attention launch
+ * of the most recent forward pass on the kernel-per-matrix path (bf16 models) fill one record of SD_STAMP_WORDS 64-bit
+ * words; sd_launch_stamps_read synchronises and copies the first `cap` records (launch order) to the host:
+ *   [0] first CTA began                    [1],[2] first / last CTA saw what it waits for (the kernel before it; its
+ *   tile's pieces)                         [3],[4] GEMM only: first / last CTA had its first stage complete
+ *   [5],[6] first / last CTA finished      [7] 0.            A word is 0 when nothing reported it.
+ * kinds_host[i] = SD_STAMP_GEMM / _STEP / _ATTENTION | (step after the GEMM: 0 plain, 1 QKV+rotary, 2 residual,
+ * 3 SwiGLU) << 8; *n_out = records of the pass (may exceed cap).  Enabling changes the captured graphs' keys: the
+ * first call afterwards captures anew.  A few atomics per CTA: for measurement, off by default. */
+/* Measurement knobs of the kernel-per-matrix path (0 = the library's own choice).  Setting one drops the captured graphs.
+ *   SD_TUNE_WO_STAGES       cap on the stage ring of the Wo GEMM (16 KB weight block + token rows per stage): with a
+ *                           smaller ring its CTAs fit beside the attention kernel's and stream weights while it runs
+ *   SD_TUNE_WO_PREFILL_ALL  1: the Wo GEMM requests its whole ring before attention has finished
+ *   SD_TUNE_ATTN_WARPS      4 or 8 warps per attention CTA (64 or 128 KB of shared memory at head_dim 128)
+ *   SD_TUNE_PREFILL_STAGES  stages a weight GEMM requests at once before the kernel before it has finished
+ *   SD_TUNE_PACE_NS         > 0: after those, one more stage every so many nanoseconds until that kernel has finished
+ *   SD_TUNE_ATTN_CLUSTER    1 or 2: at most this many CTAs of a cluster share one slice of a head's cache (default up to 4) */
+#define SD_TUNE_WO_STAGES 0
+#define SD_TUNE_WO_PREFILL_ALL 1
+#define SD_TUNE_ATTN_WARPS 2
+#define SD_TUNE_ATTN_CLUSTER 3
+#define SD_TUNE_PACE_NS 4
+#define SD_TUNE_PREFILL_STAGES 5
+#define SD_TUNE_COUNT 6
+sd_status sd_tuning(sd_ctx* ctx, int knob, int value);
+
+#define SD_STAMP_WORDS 8
+#define SD_STAMP_GEMM 0
+#define SD_STAMP_STEP 1
+#define SD_STAMP_ATTENTION 2
+sd_status sd_launch_stamps(sd_ctx* ctx, int enable);
+sd_status sd_launch_stamps_read(sd_ctx* ctx, uint64_t* stamps_host, int32_t* kinds_host, int cap, int32_t* n_out);
+
 /* The gamma that maximises Eq. 1 for what the library itself has measured: alpha = (sum over judged slots of
  * sum_k min(p_s(k), q_s(k))) / judged slots of sequence `seq` (accumulated by sd_accept_seqs + sd_kv_rollback), c from
  * sd_cost_timing / sd_cost_read.  Returns 0 when nothing has been measured yet or no gamma beats plain decoding.

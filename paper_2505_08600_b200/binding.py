@@ -74,6 +74,9 @@ _PROTOS = {
     "sd_verify_accept_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp]),
     "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_use_graphs": (_i, [_vp, _i]),
+    "sd_tuning": (_i, [_vp, _i, _i]),
+    "sd_launch_stamps": (_i, [_vp, _i]),
+    "sd_launch_stamps_read": (_i, [_vp, _vp, _vp, _i, C.POINTER(C.c_int32)]),
     "sd_seq_alpha": (_i, [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "sd_cost_timing": (_i, [_vp, _i]),
     "sd_cost_read": (_i, [_vp, C.POINTER(Cost), _i]),
@@ -302,6 +305,21 @@ class Context:
     def sd_verify_accept(self, seqs, gamma, x, q, logits, n_acc, out_tok):
         a, p, n = _seqs(seqs)
         _check(self.L.sd_verify_accept(self.h, p, n, gamma, _dp(x), _dp(q), _dp(logits), _dp(n_acc), _dp(out_tok)), "sd_verify_accept")
+
+    def sd_tuning(self, knob, value):
+        _check(self.L.sd_tuning(self.h, int(knob), int(value)), "sd_tuning")
+
+    def sd_launch_stamps(self, enable):
+        _check(self.L.sd_launch_stamps(self.h, int(enable)), "sd_launch_stamps")
+
+    def sd_launch_stamps_read(self, cap=1024):
+        """(stamps [n][8] uint64 nanoseconds, kinds [n] int32) of the most recent forward pass."""
+        st = np.zeros((cap, 8), dtype=np.uint64)
+        kinds = np.zeros(cap, dtype=np.int32)
+        n = C.c_int32()
+        _check(self.L.sd_launch_stamps_read(self.h, st.ctypes.data_as(C.c_void_p), kinds.ctypes.data_as(C.c_void_p), cap, C.byref(n)), "sd_launch_stamps_read")
+        k = min(cap, n.value)
+        return st[:k], kinds[:k]
 
     def sd_seq_alpha(self, seq):
         a, j = C.c_double(), C.c_int64()

@@ -59,6 +59,7 @@ enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
 
 }  // namespace
 
+constexpr int STAMP_CAP = 1024;                 // launches of one pass whose time stamps can be kept
 constexpr size_t ARRIVE_WORDS = 65536;          // arrival words of one pass (the 13B target needs about 17,000)
 constexpr int PASS_ROWS_CAP = 32;               // most query rows of a pass on the persistent streaming kernel
 constexpr size_t PASS_REGION_BYTES = (size_t)64 << 20;      // each of the two workspace regions of that kernel
@@ -97,7 +98,7 @@ struct sd_ctx {
     bool two_part;                              // feed the verify rows' activations to the GEMMs in two bf16 parts (see Epilogue::lo_off)
     bool force_plain;                           // run the CUDA-core kernels even where the tensor-core path applies
     bool graphs_on;                             // replay captured CUDA graphs for repeated calls
-    struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; uint64_t passes; };
+    struct CachedGraph { std::vector<uint8_t> key; cudaGraphExec_t exec; uint64_t launches; uint64_t last_use; uint64_t passes; std::vector<int32_t> stamp_kinds; };
     std::vector<CachedGraph> graphs;
     uint64_t graph_clock;
     // classifier
@@ -110,6 +111,9 @@ struct sd_ctx {
     float* alpha_terms;                         // [seq of the call][gamma]: sum_k min(p, q) of the last sd_accept_seqs, consumed by sd_kv_rollback
     // optional timing of the draft and target passes (the cost ratio c of Eq. 1 from the library's own clock)
     bool cost_on; int cost_depth;
+    // optional time stamps of the launches of a forward pass on the kernel-per-matrix path
+    int tune[SD_TUNE_COUNT];                    // measurement knobs (sd_tuning)
+    bool stamps_on; unsigned long long* stamp_buf; std::vector<int32_t> stamp_kinds;
     struct CostMark { cudaEvent_t e0, e1; int kind; int units; };
     std::vector<CostMark> cost_pending;
     std::vector<cudaEvent_t> cost_free;
@@ -264,6 +268,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->st_q = (float*)B.take(sizeof(float) * S * g_max * V0);
     c->st_logits = (float*)B.take(sizeof(float) * std::min((size_t)SD_MAX_ROWS, (size_t)S * (cfg.max_gamma + 1)) * V0);
     c->alpha_terms = (float*)B.take(sizeof(float) * S * g_max);
+    c->stamp_buf = (unsigned long long*)B.take(sizeof(unsigned long long) * ST_WORDS * STAMP_CAP);
     c->st_nacc = (int32_t*)B.take(sizeof(int32_t) * S);
     c->st_out = (int32_t*)B.take(sizeof(int32_t) * S * (cfg.max_gamma + 1));
     if (cfg.clf_d_hidden > 0 && cfg.n_drafts > 0) {
@@ -456,11 +461,23 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     return SD_OK;
 }
 
+// The next record of the stamp buffer (nullptr when stamps are off or the buffer is full); kind: SD_STAMP_* | detail << 8.
+unsigned long long* next_stamp(sd_ctx* c, int kind) {
+    if (!c->stamps_on || (int)c->stamp_kinds.size() >= STAMP_CAP) return nullptr;
+    c->stamp_kinds.push_back(kind);
+    return c->stamp_buf + (size_t)ST_WORDS * (c->stamp_kinds.size() - 1);
+}
+
 // One weight GEMM and the step that follows it.
 sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
     if (ep.lo_off) rows += ep.lo_off;           // the input rows come in two bf16 parts: [x_hi rows][x_lo rows at + lo_off]
-    GemmGeom g = gemm_geometry(rows, n_out, K, sm_count());
+    GemmGeom g = gemm_geometry(rows, n_out, K, sm_count(), ep.ring_stages, ep.prefill_all != 0);
     if (ep.lo_off) { g.lo_off = ep.lo_off; g.m_real = ep.m_real; }
+    g.pace_ns = c->tune[SD_TUNE_PACE_NS];
+    if (c->tune[SD_TUNE_PREFILL_STAGES] >= 2) g.prefill = std::min(g.stages, c->tune[SD_TUNE_PREFILL_STAGES]);
+    Epilogue eps = ep;
+    g.stamp = next_stamp(c, SD_STAMP_GEMM | (ep.mode << 8));
+    eps.stamp = next_stamp(c, SD_STAMP_STEP | (ep.mode << 8));
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
@@ -470,7 +487,7 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
         c->arrive_used += (size_t)g.n_tiles;
     }
     LAUNCH(CAT_LINEAR, launch_gemm_streamk(tw, tx, g, c->partials, arrive, c->S.status, 1, c->st));
-    LAUNCH(CAT_FUSED_STEP, launch_fused_step(g, ep, c->partials, arrive, c->S.status, 1, c->st));
+    LAUNCH(CAT_FUSED_STEP, launch_fused_step(g, eps, c->partials, arrive, c->S.status, 1, c->st));
     return SD_OK;
 }
 
@@ -486,6 +503,10 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     // as bf16(x) and as bf16(x - bf16(x)), 8 (or 16) rows apart.  The weights stream once all the same, and the GEMMs'
     // inputs are no longer rounded to 8 bits of mantissa.
     const int lo = !c->two_part ? 0 : (n_rows >= 3 && n_rows <= 8) ? 8 : (n_rows >= 9 && n_rows <= 16) ? 16 : 0;
+    if (c->stamps_on) {                                                     // the stamps of this pass replace the previous pass's
+        c->stamp_kinds.clear();
+        CUDA_TRY(cudaMemsetAsync(c->stamp_buf, 0xFF, sizeof(unsigned long long) * ST_WORDS * STAMP_CAP, st));
+    }
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -502,9 +523,11 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = c->rope_row_cos; e.rsin = c->rope_row_sin;
         SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
-                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st, lo));
+                                                     hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st, lo,
+                                                     next_stamp(c, SD_STAMP_ATTENTION), c->tune[SD_TUNE_ATTN_WARPS], c->tune[SD_TUNE_ATTN_CLUSTER]));
         memset(&e, 0, sizeof(e));
         e.lo_off = lo; e.m_real = n_rows;
+        e.ring_stages = c->tune[SD_TUNE_WO_STAGES]; e.prefill_all = c->tune[SD_TUNE_WO_PREFILL_ALL];
         e.mode = EPI_RESIDUAL; e.h = c->h; e.gain_next = L.norm2; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
         SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e));
         memset(&e, 0, sizeof(e));
@@ -609,6 +632,7 @@ sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
             CUDA_TRY(cudaGraphLaunch(g.exec, c->st));
             c->launches += g.launches;
             note_passes(c, g.passes);
+            if (c->stamps_on) c->stamp_kinds = g.stamp_kinds;       // the records this graph's launches fill
             g.last_use = c->graph_clock;
             return SD_OK;
         }
@@ -636,7 +660,7 @@ sd_status run_graphed(sd_ctx* c, const KeyBuilder& key, Body body) {
         cudaGraphExecDestroy(c->graphs[victim].exec);
         c->graphs.erase(c->graphs.begin() + victim);
     }
-    c->graphs.push_back({key.bytes, exec, c->launches - l0, c->graph_clock, c->pass_count - p0});
+    c->graphs.push_back({key.bytes, exec, c->launches - l0, c->graph_clock, c->pass_count - p0, c->stamp_kinds});
     CUDA_TRY(cudaGraphLaunch(exec, c->st));
     return SD_OK;
 }
@@ -756,6 +780,8 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     c->pass_on = false; c->pass_drafts = false; c->pass_max_rows = 16; c->pass_tuned = false; c->pass_stages = 0; c->stamps = nullptr; c->stamps_words = 0;
     c->two_part = true;
     c->cost_on = false; c->cost_depth = 0;
+    c->stamps_on = false;
+    for (int i = 0; i < SD_TUNE_COUNT; ++i) c->tune[i] = 0;
     for (int i = 0; i < 3; ++i) { c->cost_ms[i] = 0.0; c->cost_units[i] = 0; }
     c->force_plain = false;
     c->graphs_on = true;
@@ -939,7 +965,7 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     KeyBuilder key;
-    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows);
+    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows);
     for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
     bound = bound_bucket(bound + gamma) - gamma;
     CostScope cost(c, 0, gamma);
@@ -986,7 +1012,7 @@ sd_status sd_verify(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma, const 
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
     RowPlan plan{PLAN_VERIFY, gamma + 1, 0, 0, gamma, x_dev, bound_bucket(bound)};
     KeyBuilder key;
-    key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
+    key.add(2).add_list(seqs, n_seq).add(gamma).add(x_dev).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_max_rows);
     SD_TRY(prepare_pass(c, 0, plan, n_seq * (gamma + 1), LOGITS_ALL));
     CostScope cost(c, 1, 1);
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq * (gamma + 1), LOGITS_ALL, logits_dev); });
@@ -1002,7 +1028,7 @@ sd_status sd_target_step(sd_ctx* c, const int32_t* seqs, int n_seq, float* logit
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     RowPlan plan{PLAN_TARGET_STEP, 1, 0, 0, 0, nullptr, bound_bucket(bound)};
     KeyBuilder key;
-    key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
+    key.add(3).add_list(seqs, n_seq).add(logits_dev).add(plan.ctx_bound).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_max_rows);
     SD_TRY(prepare_pass(c, 0, plan, n_seq, LOGITS_ALL));
     CostScope cost(c, 2, 1);
     return run_graphed(c, key, [&]() { return forward(c, c->models[0], list, plan, n_seq, LOGITS_ALL, logits_dev); });
@@ -1096,7 +1122,7 @@ sd_status sd_verify_accept(sd_ctx* c, const int32_t* seqs, int n_seq, int gamma,
         if (c->phase[s] < PH_READY) return SD_ERR_STATE;
         if (c->len_ub[s] + gamma + 1 > c->S.tok_stride || c->len_ub[s] + gamma > c->cfg.max_ctx) return SD_ERR_CAPACITY;
     }
-    key.add(4).add_list(seqs, n_seq).add(gamma).add(x_dev).add(q_dev).add(logits_dev).add(n_acc_dev).add(out_tok_dev).add(c->force_plain).add(c->pass_on).add(c->pass_max_rows);
+    key.add(4).add_list(seqs, n_seq).add(gamma).add(x_dev).add(q_dev).add(logits_dev).add(n_acc_dev).add(out_tok_dev).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_max_rows);
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]] + gamma);
     key.add(bound_bucket(bound));
@@ -1221,6 +1247,39 @@ sd_status sd_seq_alpha(sd_ctx* c, int seq, double* alpha_sum_out, int64_t* judge
     CUDA_TRY(cudaMemcpyAsync(alpha_sum_out, c->S.alpha_sum + seq, sizeof(double), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaMemcpyAsync(judged_out, c->S.judged + seq, sizeof(int64_t), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_tuning(sd_ctx* c, int knob, int value) {
+    if (!c || knob < 0 || knob >= SD_TUNE_COUNT || value < 0) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);        // the captured launches were shaped by the old value
+    c->graphs.clear();
+    c->tune[knob] = value;
+    return SD_OK;
+}
+
+sd_status sd_launch_stamps(sd_ctx* c, int enable) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    c->stamps_on = enable != 0;
+    c->stamp_kinds.clear();
+    return SD_OK;
+}
+
+sd_status sd_launch_stamps_read(sd_ctx* c, uint64_t* stamps_host, int32_t* kinds_host, int cap, int32_t* n_out) {
+    if (!c || !stamps_host || !kinds_host || !n_out || cap < 0) return SD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    const int n = std::min<int>(cap, (int)c->stamp_kinds.size());
+    *n_out = (int32_t)c->stamp_kinds.size();
+    if (n == 0) return SD_OK;
+    CUDA_TRY(cudaMemcpy(stamps_host, c->stamp_buf, sizeof(uint64_t) * ST_WORDS * n, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < n; ++i) {
+        kinds_host[i] = c->stamp_kinds[i];
+        uint64_t* r = stamps_host + (size_t)ST_WORDS * i;
+        for (int w : {ST_DEP_LAST, ST_DATA_LAST, ST_DONE_LAST}) r[w] = r[w] == ~0ull ? 0ull : ~r[w];        // "last" words hold complements
+        for (int w : {ST_START, ST_DEP_FIRST, ST_DATA_FIRST, ST_DONE_FIRST}) if (r[w] == ~0ull) r[w] = 0ull;   // never reported
+        r[7] = 0;
+    }
     return SD_OK;
 }
 

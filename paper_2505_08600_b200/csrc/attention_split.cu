@@ -34,6 +34,7 @@ struct AttnParams {
     int n_rows, rows_per_seq, rows_per_block, H, Hkv, max_ctx, n_splits;
     int csize;          // CTAs of a thread-block cluster that share one slice (1, 2 or 4)
     int lo_off;         // > 0: the output is also written as a second bf16 part (x - bf16(x)) lo_off rows further down
+    unsigned long long* stamp;   // optional time stamps of the launch (see LaunchStamp)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
@@ -80,6 +81,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     constexpr int BUF = CK * ROWB;           // one chunk of keys (or values)
     constexpr int OLD = HD + 8;              // padded row of the cross-warp merge buffer (floats)
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_first(P.stamp, ST_START);
     const int CS = P.csize;
     const int split = blockIdx.x / CS, crank = blockIdx.x % CS, kvh = blockIdx.y;
     const int group = P.H / P.Hkv;
@@ -154,6 +156,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     const int old0 = np > 0 ? max(0, min(min(CK, np), new_begin - p_begin)) : 0;
     if (np > 0) issue_part(0, 0, old0, false);
     pdl_wait();                                  // queries and the keys/values appended by this pass come from the kernels before
+    if (threadIdx.x == 0) stamp_pair(P.stamp, ST_DEP_FIRST);
     if (np > 0) {
         const int n_chunks = (np + CK - 1) / CK;
         issue_part(0, old0, min(CK, np), true);
@@ -357,7 +360,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     }
     if (CS > 1) cluster.sync();                      // nobody leaves while its shared memory may still be read
     if (crank != 0) return;
-    if (P.n_splits == 1) return;                     // nothing to merge
+    if (P.n_splits == 1) { if (t == 0) stamp_pair(P.stamp, ST_DONE_FIRST); return; }      // nothing to merge
 
     // ---- the slice that delivers last merges all of them: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
     //      always in slice order, so the result does not depend on which slice that was
@@ -371,7 +374,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
         last_sm = last;
     }
     __syncthreads();
-    if (!last_sm) return;
+    if (!last_sm) { if (t == 0) stamp_pair(P.stamp, ST_DONE_FIRST); return; }
     // Everything the merge reads (every slice's max, sum and partial output for the block's
     // queries) is fetched into shared memory in one go, so the merge costs one memory round trip.
     const int ns = P.n_splits;
@@ -438,6 +441,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
             if (P.lo_off) P.out[((size_t)(r + P.lo_off) * P.H + h) * HD + e] = __float2bfloat16_rn(acc[i] - __bfloat162float(hi));
         }
     }
+    if (t == 0) stamp_pair(P.stamp, ST_DONE_FIRST);
 }
 
 }  // namespace
@@ -458,12 +462,12 @@ size_t attention_split_workspace(int rows, int H, int hd, int max_ctx) {
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
                                    int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
-                                   cudaStream_t st, int lo_off) {
+                                   cudaStream_t st, int lo_off, unsigned long long* stamp, int force_warps, int max_cluster) {
     if (n_rows <= 0) return cudaSuccess;
     ctx_bound = std::max(1, std::min(ctx_bound, max_ctx));
     AttnParams P;
     P.q = (const bf16*)q; P.kc = (const bf16*)kc; P.vc = (const bf16*)vc; P.out = (bf16*)out;
-    P.row_slot = row_slot; P.row_pos = row_pos; P.lo_off = lo_off;
+    P.row_slot = row_slot; P.row_pos = row_pos; P.lo_off = lo_off; P.stamp = stamp;
     if (rows_per_seq < 1 || n_rows % rows_per_seq || H / Hkv > NQ) return cudaErrorInvalidValue;
     P.n_rows = n_rows; P.rows_per_seq = rows_per_seq; P.H = H; P.Hkv = Hkv; P.max_ctx = max_ctx;
     P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ / (H / Hkv)));
@@ -484,7 +488,8 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
     // few (head, row block, slice) items: two or four CTAs of a cluster share each of them
     const int items = P.n_splits * Hkv * n_blocks;
     P.csize = items * 4 <= sm ? 4 : (items * 2 <= sm ? 2 : 1);
-    const int nw = items > 2 * sm ? WARPS_MANY : WARPS_FEW;
+    if (max_cluster == 1 || max_cluster == 2) P.csize = std::min(P.csize, max_cluster);
+    const int nw = force_warps == WARPS_MANY || force_warps == WARPS_FEW ? force_warps : (items > 2 * sm ? WARPS_MANY : WARPS_FEW);
     const size_t smem = std::max((size_t)4 * 16 * nw * hd * 2, sizeof(float) * ((size_t)nw * NQ * (hd + 8) + 2 * nw * NQ + (size_t)NQ * hd + 2 * NQ));
     dim3 grid(P.n_splits * P.csize, Hkv, n_blocks);
     cudaLaunchConfig_t cfg = {};

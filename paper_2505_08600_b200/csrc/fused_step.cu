@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     const int mode = MODE < 0 ? ep.mode : MODE;
     pdl_launch_dependents();
     const int et = threadIdx.x, lane = et & 31, warp = et >> 5;
+    if (et == 0) stamp_first(ep.stamp, ST_START);
     const uint32_t tile = blockIdx.x;
     const int m0 = blockIdx.y * MB;
     const int n = (int)tile * TILE_N + et;
@@ -96,6 +97,8 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     } else {
         pdl_wait();
     }
+
+    if (et == 0) stamp_pair(ep.stamp, ST_DEP_FIRST);
 
     // ---- one round of loads: sums of squares, residual / row plan / rotary factors, the pieces
     float ssa[(MB + 3) / 4], ssb[(MB + 3) / 4];
@@ -229,6 +232,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     }
     default: break;
     }
+    if (et == 0) stamp_pair(ep.stamp, ST_DONE_FIRST);
 }
 
 template <int MODE, bool HL>

@@ -46,6 +46,7 @@ struct Shared {
     uint32_t tmem_base;
     int abort_flag;
     int epi_abort;
+    int dep_seen;            // the token-row producer is past its wait for the kernel before
 };
 
 // Ring bookkeeping.  The first `stages` loads of a CTA fill the whole ring (run-ahead while the
@@ -118,6 +119,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     extern __shared__ uint8_t dyn_smem[];
     __shared__ Shared sh;
     pdl_launch_dependents();                 // the next kernel may be scheduled; it waits for this one where it must
+    if (threadIdx.x == 0) stamp_first(g.stamp, ST_START);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t tiles0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;        // 1024-byte aligned stage ring
     const uint32_t x_bytes = (uint32_t)g.m_pad * 128u, stage_bytes = A_BYTES + x_bytes;
@@ -139,6 +141,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh.tmem_full[b]), 1); mbar_init(smem_u32(&sh.tmem_empty[b]), 4); }
         sh.abort_flag = 0;
         sh.epi_abort = 0;
+        sh.dep_seen = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -159,17 +162,27 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             RingPos rp;
+            bool dep_ok = false;
+            uint64_t t_last = 0;
+            volatile int* dep_seen = &sh.dep_seen;
             int tile = u0 / g.kb_per_tile, kb = u0 % g.kb_per_tile;
             for (uint32_t it = 0; it < n_units; ++it, rp.next(g.stages, g.steady)) {
                 const int s = rp.stage;
                 // A full ring of requests at this point slowed the step down: they compete with the small,
                 // latency-critical reads of the kernel that reduces the previous GEMM.  So the run-ahead stops
                 // short of the ring's depth until that kernel has finished.
-                if (it == (uint32_t)g.prefill) pdl_wait();
+                if (it >= (uint32_t)g.prefill && !dep_ok) {
+                    if (g.pace_ns <= 0) { pdl_wait(); dep_ok = true; }
+                    else {          // paced: one more stage every pace_ns, so that requests stay in flight until the kernel before is done
+                        const uint64_t t_next = t_last + (uint64_t)g.pace_ns;
+                        while (!(dep_ok = *dep_seen != 0) && global_ns() < t_next) {}
+                    }
+                }
                 if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) break;
                 const uint32_t bar = smem_u32(&sh.full[s]);
                 mbar_expect_tx(bar, A_BYTES);
                 tma_load_2d(tiles0 + s * stage_bytes, &tm_w, kb * TILE_K, tile * TILE_N, bar, pol_stream);
+                if (g.pace_ns > 0 && !dep_ok) t_last = global_ns();
                 if (++kb == g.kb_per_tile) { kb = 0; ++tile; }
             }
         }
@@ -179,6 +192,8 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             pdl_wait();                                           // the token rows are the previous kernel's output
+            *(volatile int*)&sh.dep_seen = 1;
+            stamp_pair(g.stamp, ST_DEP_FIRST);
             RingPos rp;
             int kb = u0 % g.kb_per_tile;
             for (uint32_t it = 0; it < n_units; ++it, rp.next(g.stages, g.steady)) {
@@ -208,6 +223,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 for (uint32_t j = 0; j < n_kb; ++j, rp.next(g.stages, g.steady)) {
                     const int s = rp.stage;
                     if (!mbar_wait(smem_u32(&sh.full[s]), rp.use & 1u, abort_flag)) { ok = false; break; }
+                    if (u == u0 && j == 0) stamp_pair(g.stamp, ST_DATA_FIRST);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t da = desc0 + (uint64_t)((uint32_t)s * (stage_bytes >> 4)), db = da + (A_BYTES >> 4);   // start-address field counts 16 bytes
 #pragma unroll
@@ -228,6 +244,7 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (threadIdx.x == 0) stamp_pair(g.stamp, ST_DONE_FIRST);
     if (sh.abort_flag) {
         if (threadIdx.x == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
         const uint64_t t0 = global_ns();                   // let copies in flight land before the CTA goes away
@@ -272,9 +289,9 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages, bool prefill_all) {
     GemmGeom g;
-    g.lo_off = 0; g.m_real = m_tok;
+    g.lo_off = 0; g.m_real = m_tok; g.stamp = nullptr; g.pace_ns = 0;
     g.m_tok = m_tok;
     g.m_pad = (m_tok + 15) & ~15;
     g.n_out = n_out;
@@ -288,9 +305,11 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm) {
     if ((T + 1) * (g.grid + 1) >= (1ll << 32)) g.grid = 0;   // the kernels split the work in 32-bit arithmetic
     const int stage_bytes = A_BYTES + g.m_pad * 128;
     g.stages = std::max(2, std::min(MAX_STAGES, RING_BYTES / stage_bytes));
+    if (max_stages >= 2) g.stages = std::min(g.stages, max_stages);
     g.steady = std::min(g.stages, std::max(2, (GEMM_STEADY_BYTES + stage_bytes - 1) / stage_bytes));
     // (measured: with more than 16 token rows the reduction kernel is bound by throughput, not latency, and the full run-ahead wins)
     g.prefill = g.m_pad > 16 ? g.stages : std::min(g.stages, std::max(2, (GEMM_PREFILL_BYTES + stage_bytes - 1) / stage_bytes));
+    if (prefill_all) g.prefill = g.stages;
     return g;
 }
 

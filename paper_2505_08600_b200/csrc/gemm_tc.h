@@ -18,6 +18,8 @@ struct GemmGeom {
     int grid, max_seg, stages;
     int steady;             // stages reused once the ring has been filled (<= stages)
     int prefill;            // weight tiles requested before the previous kernel has finished
+    unsigned long long* stamp;   // optional time stamps of this launch (see LaunchStamp); nullptr: none
+    int pace_ns;            // > 0: past `prefill`, one more stage is requested every pace_ns until the kernel before has finished
     int lo_off, m_real;     // two-part input rows (see Epilogue::lo_off): the epilogue adds accumulator columns r and r + lo_off
                             // and leaves m_real merged rows in each piece; 0: every column is a row of its own
 };
@@ -42,6 +44,8 @@ struct Epilogue {
     // product almost unrounded, at no extra weight traffic: both parts sit in the 16 columns the MMA covers anyway), and
     // the rows this step writes for the next GEMM are split the same way.  m_real = token rows (the GEMM saw lo_off + m_real).
     int lo_off, m_real;
+    unsigned long long* stamp;       // optional time stamps of the step's launch (see LaunchStamp)
+    int ring_stages, prefill_all;    // GEMM before this step: cap on its stage ring (0: none) / request the whole ring before the dependency
     unsigned long long poll_ns;      // how long a tile's CTA watches its arrival word before it falls back to the grid dependency (0: 0.2 s)
     RowScale rs;                     // PLAIN, QKV_ROPE, SWIGLU: 1/rms factor of each token row
     // EPI_PLAIN: y[i][n] = scale * acc[token i*row_stride + row_offset][n], i < n_out_rows
@@ -57,7 +61,9 @@ struct Epilogue {
 };
 
 bool gemm_tc_supported(int m_tok, int n_out, int K);
-GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm);
+// max_stages > 0 caps the ring (a smaller ring leaves shared memory for CTAs of the kernel before, e.g. attention, so that
+// this GEMM's CTAs are resident and streaming while that kernel still runs); prefill_all: request the whole ring early.
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages = 0, bool prefill_all = false);
 size_t gemm_partials_bytes(const GemmGeom& g);
 bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows);
 // The GEMM proper: leaves the split accumulators in `partials` (gemm_partials_bytes()).
@@ -102,5 +108,18 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+
+// Optional time stamps of one launch: eight 64-bit words that start as all ones and are kept with atomicMin, so a word
+// named "first" holds the earliest time any CTA reported and a word named "last" the bitwise complement of the latest.
+enum LaunchStamp { ST_START = 0,        // a CTA began
+                   ST_DEP_FIRST = 1, ST_DEP_LAST = 2,       // what the CTA waits for (the kernel before it, its tile's pieces) was there
+                   ST_DATA_FIRST = 3, ST_DATA_LAST = 4,     // GEMM: the first stage of a CTA was complete and its first MMA issued
+                   ST_DONE_FIRST = 5, ST_DONE_LAST = 6,     // a CTA had written its results
+                   ST_WORDS = 8 };
+__device__ __forceinline__ void stamp_first(unsigned long long* rec, int i) { if (rec) atomicMin(rec + i, (unsigned long long)global_ns()); }
+__device__ __forceinline__ void stamp_pair(unsigned long long* rec, int i_first) {
+    if (rec) { const unsigned long long t = global_ns(); atomicMin(rec + i_first, t); atomicMin(rec + i_first + 1, ~t); }
+}
+
 
 }  // namespace sd
