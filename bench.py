@@ -212,6 +212,45 @@ def setup(args, gamma_max, steps_per_phase):
                 routed=routed, rewind=rewind, max_ctx=max_ctx)
 
 
+STEP_AFTER = {0: "lm_head", 1: "qkv", 2: "residual", 3: "swiglu"}
+LAYER_LAUNCHES = ["gemm qkv", "step qkv", "attention", "gemm wo", "step wo", "gemm gate_up", "step gate_up", "gemm down", "step down"]
+
+
+def in_graph_timeline(ctx, cfg, step_fn, esz):
+    """Time stamps taken inside the kernels while the step runs as it always runs (captured graph, overlapping
+    dependent launches): per launch of a layer, averaged over the inner layers, in microseconds after the layer's QKV
+    GEMM issued its first MMA.  A GEMM's in-graph duration is counted from the moment its token rows exist (the kernel
+    before it has finished) to its last CTA finishing; weights requested before that moment are part of the overlap."""
+    t = cfg["target"]
+    nl, per = t["n_layers"], len(LAYER_LAUNCHES)
+    ctx.sd_launch_stamps(1)
+    for _ in range(3):
+        step_fn()
+    st, kinds = ctx.sd_launch_stamps_read()
+    ctx.sd_launch_stamps(0)
+    if len(kinds) < nl * per + 2 or nl < 4:
+        return None
+    st = st.astype(np.int64)
+    cols = ["start", "dep_first", "dep_last", "data_first", "data_last", "done_first", "done_last"]
+    inner = range(1, nl - 1)
+    rows = np.array([[[(st[l * per + j][k] - st[l * per][3]) / 1e3 if st[l * per + j][k] else np.nan for k in range(7)]
+                      for j in range(per)] for l in inner])
+    avg = np.nanmean(rows, axis=0)
+    period = float(np.mean([(st[(l + 1) * per][3] - st[l * per][3]) / 1e3 for l in inner]))
+    table = {name: {c: (None if np.isnan(avg[j][k]) else round(float(avg[j][k]), 2)) for k, c in enumerate(cols)} for j, name in enumerate(LAYER_LAUNCHES)}
+    gemm_us = 0.0
+    for j, name in enumerate(LAYER_LAUNCHES):
+        if name.startswith("gemm"):
+            gemm_us += float(avg[j][6] - avg[j][1])
+    # the lm_head GEMM: the last GEMM record of the pass
+    lm = st[nl * per]
+    lm_us = (lm[6] - lm[1]) / 1e3
+    return {"layer_period_us": round(period, 2), "gemm_us_per_layer": round(gemm_us, 2), "lm_head_gemm_us": round(float(lm_us), 2),
+            "columns": "us after the layer's QKV GEMM had its first stage: first CTA start; first/last CTA saw its dependency; "
+                       "first/last CTA had its first stage (GEMM); first/last CTA done",
+            "launches": table}
+
+
 def run_gpu(args):
     K, W = args.steps, args.warmup
     n_iter_phase = min(10, K)
@@ -279,6 +318,9 @@ def run_gpu(args):
     prof = ctx.sd_profile_read()
     ctx.sd_profile(0)
     rewind()
+    esz0 = 2 if cfg["dtype"] == "bf16" else 4
+    tl = in_graph_timeline(ctx, cfg, verify_step, esz0) if cfg["dtype"] == "bf16" else None
+    rewind()
     esz = 2 if cfg["dtype"] == "bf16" else 4
     weight_bytes = synth.param_count(tdims, streamed_only=True) * esz
     kv_bytes = sum(n_ctx) * 2 * tdims["n_layers"] * tdims["n_kv_heads"] * tdims["head_dim"] * esz
@@ -310,6 +352,16 @@ def run_gpu(args):
                                "frac_of_peak": (weight_bytes + kv_bytes) / (ms_step * 1e-3) / 1e9 / peak,
                                "frac_of_nominal_8tbs": (weight_bytes + kv_bytes) / (ms_step * 1e-3) / 1e9 / 8000.0},
                 "split_ms_per_step_serialised": split}
+    if tl:
+        # in-graph: the GEMM launches' own time from "token rows exist" to "last CTA done", summed over the step
+        lm_bytes = tdims["vocab"] * tdims["d_model"] * esz
+        layer_bytes = (weight_bytes - lm_bytes) / tdims["n_layers"]
+        g_ms = (tl["gemm_us_per_layer"] * tdims["n_layers"] + tl["lm_head_gemm_us"]) * 1e-3
+        roofline["in_graph"] = {"gemm_ms_in_step": g_ms, "gbs": weight_bytes / (g_ms * 1e-3) / 1e9, "frac": weight_bytes / (g_ms * 1e-3) / 1e9 / peak,
+                                "layer_period_us": tl["layer_period_us"], "layer_bytes": layer_bytes,
+                                "layer_us_at_peak": layer_bytes / (peak * 1e9) * 1e6,
+                                "timing": "time stamps inside the kernels of the captured step (sd_launch_stamps), inner layers averaged",
+                                "timeline": tl["launches"], "columns": tl["columns"]}
 
     # ---- e2e: drafts and results in pinned host memory, copies inside the timed region
     xh = x.cpu().pin_memory(); qh = q.cpu().pin_memory()

@@ -406,6 +406,14 @@ sd_status sd_op_attention(const void* q, const void* k_cache, const void* v_cach
                           const int32_t* row_slot, const int32_t* row_pos, int rows,
                           int n_heads, int n_kv_heads, int head_dim, int max_ctx, int dtype,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* The same with the rows in runs of rows_per_seq consecutive rows of one sequence at consecutive positions (the
+ * gamma + 1 rows of a verify step): the rows of a run share one pass over their sequence's cache, which is how the
+ * verify step launches attention.  rows must be a multiple of rows_per_seq; the caller guarantees that the rows of a
+ * run have one slot and positions p, p + 1, ... */
+sd_status sd_op_attention_runs(const void* q, const void* k_cache, const void* v_cache, void* out,
+                               const int32_t* row_slot, const int32_t* row_pos, int rows, int rows_per_seq,
+                               int n_heads, int n_kv_heads, int head_dim, int max_ctx, int dtype,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx);
 
 /* Philox4x32-10 on the device: out[i][0..3] for ctr[i][0..3], one key.  For tests. */

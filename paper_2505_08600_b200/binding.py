@@ -100,6 +100,7 @@ _PROTOS = {
     "sd_op_linear_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "sd_op_linear_wait_expiry": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp, _sz, C.c_uint64, _vp, _vp]),
     "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "sd_op_attention_runs": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_attention_workspace": (_sz, [_i, _i, _i, _i]),
     "sd_op_philox": (_i, [_vp, _i, C.c_uint32, C.c_uint32, _vp, _vp]),
     "sd_op_softmax_sample": (_i, [_vp, _i, _i, C.c_float, _vp, _vp, _vp, _vp]),
@@ -446,12 +447,12 @@ def sd_op_linear_static(x, w, y, stream=None):
     _check(lib().sd_op_linear_static(_dp(x), _dp(w), _dp(y), rows, w.shape[0], n_in, _stream_ptr(stream)), "sd_op_linear_static")
 
 
-def sd_op_attention(q, kc, vc, out, row_slot, row_pos, n_heads, n_kv_heads, head_dim, max_ctx, dtype, stream=None):
+def sd_op_attention(q, kc, vc, out, row_slot, row_pos, n_heads, n_kv_heads, head_dim, max_ctx, dtype, stream=None, rows_per_seq=1):
     rows = q.shape[0]
     need = lib().sd_op_attention_workspace(rows, n_heads, head_dim, max_ctx)
     ws = torch.empty(max(need, 1), dtype=torch.uint8, device=q.device)
-    _check(lib().sd_op_attention(_dp(q), _dp(kc), _dp(vc), _dp(out), _dp(row_slot), _dp(row_pos), rows, n_heads,
-                                 n_kv_heads, head_dim, max_ctx, dtype, _dp(ws), need, _stream_ptr(stream)), "sd_op_attention")
+    _check(lib().sd_op_attention_runs(_dp(q), _dp(kc), _dp(vc), _dp(out), _dp(row_slot), _dp(row_pos), rows, int(rows_per_seq), n_heads,
+                                      n_kv_heads, head_dim, max_ctx, dtype, _dp(ws), need, _stream_ptr(stream)), "sd_op_attention_runs")
 
 
 def sd_op_philox(ctr, key0, key1, out, stream=None):

@@ -1431,13 +1431,20 @@ size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ct
 sd_status sd_op_attention(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                           const int32_t* row_pos, int rows, int H, int Hkv, int hd, int max_ctx, int dtype,
                           void* ws, size_t ws_bytes, void* stream) {
+    return sd_op_attention_runs(q, kc, vc, out, row_slot, row_pos, rows, 1, H, Hkv, hd, max_ctx, dtype, ws, ws_bytes, stream);
+}
+
+sd_status sd_op_attention_runs(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
+                               const int32_t* row_pos, int rows, int rows_per_seq, int H, int Hkv, int hd, int max_ctx, int dtype,
+                               void* ws, size_t ws_bytes, void* stream) {
+    if (rows_per_seq < 1 || rows % rows_per_seq) return SD_ERR_INVALID_ARG;
     if (!q || !kc || !vc || !out || !row_slot || !row_pos || rows < 1 || H < 1 || Hkv < 1 || H % Hkv) return SD_ERR_INVALID_ARG;
     if (hd < 8 || hd > 256 || (hd & 7) || max_ctx < 1 || (dtype != SD_F32 && dtype != SD_BF16)) return SD_ERR_INVALID_ARG;
     if (ws_bytes < sd_op_attention_workspace(rows, H, hd, max_ctx)) return SD_ERR_OOM;
     if (attention_split_supported(dtype, H, Hkv, hd)) {
         if (!ws) return SD_ERR_INVALID_ARG;
         CUDA_TRY(cudaMemsetAsync(ws, 0, 65536, (cudaStream_t)stream));                               // the arrival counters
-        CUDA_TRY(launch_attention_split(q, kc, vc, out, row_slot, row_pos, rows, 1, H, Hkv, hd, max_ctx, max_ctx, ws, ws_bytes, 0, (cudaStream_t)stream));
+        CUDA_TRY(launch_attention_split(q, kc, vc, out, row_slot, row_pos, rows, rows_per_seq, H, Hkv, hd, max_ctx, max_ctx, ws, ws_bytes, 0, (cudaStream_t)stream));
         return SD_OK;
     }
     CUDA_TRY(launch_attention(q, kc, vc, out, dtype, row_slot, row_pos, rows, H, Hkv, hd, max_ctx, ws, ws_bytes, (cudaStream_t)stream));

@@ -109,9 +109,13 @@ def test_attention_launch_of_the_eight_sequence_long_cache_configuration(sd):
     row_slot = np.repeat(np.arange(B, dtype=np.int32), g1)
     row_pos = np.tile(np.arange(max_ctx - g1, max_ctx, dtype=np.int32), B)
     out = torch.zeros((rows, H, hd), dtype=torch.bfloat16, device=DEV)
-    sd.sd_op_attention(to_dev(q), kc, vc, out, to_dev(row_slot), to_dev(row_pos), H, H, hd, max_ctx, sd.SD_BF16)
+    sd.sd_op_attention(to_dev(q), kc, vc, out, to_dev(row_slot), to_dev(row_pos), H, H, hd, max_ctx, sd.SD_BF16, rows_per_seq=g1)
     got = out.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
+    # the same rows one by one (every row its own pass over the cache) give the same numbers up to the output's rounding
+    out1 = torch.zeros_like(out)
+    sd.sd_op_attention(to_dev(q), kc, vc, out1, to_dev(row_slot), to_dev(row_pos), H, H, hd, max_ctx, sd.SD_BF16)
+    assert (out.float() - out1.float()).abs().max().item() <= 2e-2
     qf, kf, vf = widen(q), widen(base_k), widen(base_v)
     rng = np.random.default_rng(7)
     picks = {(0, 0), (rows - 1, H - 1), (g1 - 1, 17), (g1, 3)} | {(int(rng.integers(rows)), int(rng.integers(H))) for _ in range(28)}
