@@ -235,7 +235,11 @@ def in_graph_timeline(ctx, cfg, step_fn, esz):
     inner = range(1, nl - 1)
     rows = np.array([[[(st[l * per + j][k] - st[l * per][3]) / 1e3 if st[l * per + j][k] else np.nan for k in range(7)]
                       for j in range(per)] for l in inner])
-    avg = np.nanmean(rows, axis=0)
+    with np.errstate(all="ignore"):
+        import warnings
+        with warnings.catch_warnings():
+            warnings.simplefilter("ignore", RuntimeWarning)
+            avg = np.nanmean(rows, axis=0)           # (columns a kind of launch never reports stay NaN)
     period = float(np.mean([(st[(l + 1) * per][3] - st[l * per][3]) / 1e3 for l in inner]))
     table = {name: {c: (None if np.isnan(avg[j][k]) else round(float(avg[j][k]), 2)) for k, c in enumerate(cols)} for j, name in enumerate(LAYER_LAUNCHES)}
     gemm_us = 0.0
@@ -496,6 +500,49 @@ def run_gamma_sweep(args):
     ctx.close()
 
 
+def run_kmeans_bench(args):
+    """One Lloyd iteration over synthetic sentence vectors (offline task partitioning): 2,097,152 x 384 fp32 points
+    (3.2 GB, far beyond L2), 4 clusters; bound by the one pass over the points."""
+    import torch
+    from paper_2505_08600_b200 import binding as sd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    n, dim, k = 2 * 1024 * 1024, 384, 4
+    g = torch.Generator(device=dev); g.manual_seed(6)
+    centers = torch.nn.functional.normalize(torch.randn((k, dim), generator=g, device=dev), dim=1)
+    task = torch.randint(0, k, (n,), generator=g, device=dev)
+    x = torch.nn.functional.normalize(centers[task] + torch.randn((n, dim), generator=g, device=dev) * (0.6 / dim ** 0.5), dim=1).contiguous()
+    c = x[:k].clone()
+    labels = torch.zeros((n,), dtype=torch.int32, device=dev)
+    c_out = torch.zeros_like(c); counts = torch.zeros((k,), dtype=torch.int64, device=dev); inertia = torch.zeros((1,), dtype=torch.float64, device=dev)
+    for _ in range(max(3, args.warmup)):
+        sd.sd_kmeans_step(x, c, labels, c_out, counts, inertia)
+    torch.cuda.synchronize()
+    K = max(5, min(args.steps, 50))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(torch.cuda.current_stream())
+    for _ in range(K):
+        sd.sd_kmeans_step(x, c, labels, c_out, counts, inertia)
+    e1.record(torch.cuda.current_stream()); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K
+    peak, kind = _peaks()
+    bytes_ = n * dim * 4 + n * 4
+    # the oracle on a bounded sample of the same points
+    from oracle import partition
+    xs = x[: 200000].cpu().numpy(); cs = c.cpu().numpy()
+    t0 = time.perf_counter(); reps = 0
+    while time.perf_counter() - t0 < 10.0:
+        partition.kmeans_step(xs, cs); reps += 1
+    cpu_pts = reps * xs.shape[0] / (time.perf_counter() - t0)
+    print(json.dumps({"metric": "kmeans_points_per_s", "unit": "points/s", "value": n / (ms * 1e-3), "ms_per_step": ms, "n_gpus": 1, "steps": K,
+                      "dtype": "f32", "data": "synthetic", "config": {"workload": f"K-means step: {n} x {dim} fp32 points, {k} clusters (labels + new centroids + inertia)"},
+                      "roofline": {"bound": "hbm", "achieved": bytes_ / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s", "frac": bytes_ / (ms * 1e-3) / 1e9 / peak,
+                                   "peak_kind": f"of {kind}", "algorithmic_bytes_per_launch": bytes_, "traffic": None},
+                      "counts": counts.cpu().tolist(), "inertia": float(inertia.item()),
+                      "cpu_baseline": {"value": cpu_pts, "unit": "points/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                                       "sample": f"{xs.shape[0]} of the points, {reps} repeats"}}))
+
+
 def run_accept_microbench(args):
     """Accept / reject / resample kernel alone at the 13B configuration's shape (8 sequences, gamma 8, vocab 32000):
     draft distributions are softmax(target_logits + N(0, sigma^2)) so that sigma sets the acceptance rate."""
@@ -551,6 +598,7 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
+    ap.add_argument("--kmeans", action="store_true", help="time one K-means step over synthetic sentence vectors and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     launched = "WORLD_SIZE" in os.environ
@@ -564,13 +612,15 @@ def main():
             argv[i + 1] = name
             rc = rc or subprocess.run(argv).returncode
         sys.exit(rc)
-    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep:
+    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep and not args.kmeans:
         # no launcher: this process starts the N replicas itself (one per GPU) and passes rank 0's line through
         rc, out = replicas.spawn_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
         sys.stdout.write(out)
         sys.exit(rc)
     if args.accept_microbench:
         run_accept_microbench(args)
+    elif args.kmeans:
+        run_kmeans_bench(args)
     elif args.gamma_sweep:
         run_gamma_sweep(args)
     elif args.impl == "reference":

@@ -416,6 +416,21 @@ sd_status sd_op_attention_runs(const void* q, const void* k_cache, const void* v
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx);
 
+/* One iteration of the K-means algorithm (Lloyd) over dense fp32 vectors: the offline task-partitioning step of
+ * Section 3.2, which clusters 384-dimensional sentence vectors into one subset per task.
+ *   labels[i]       = argmin_k sum_d (points[i][d] - centroids[k][d])^2, distances summed in fp32, lowest k on ties
+ *   centroids_out   = mean of the points of each cluster (a cluster without points keeps its centroid); nullable
+ *   counts_out[k]   = points per cluster (int64); nullable      inertia_out = sum of the chosen squared distances
+ *                     under the INPUT centroids (double); nullable
+ * points [n][dim] and centroids [k][dim] are device pointers, row-major, 16-byte aligned; dim a multiple of 128 up
+ * to 512, 1 <= k <= 8 (else SD_ERR_UNSUPPORTED); labels int32 [n] on the device.  The caller owns every buffer; the
+ * workspace (device, sd_kmeans_workspace bytes) holds per-block partial sums.  Sums are formed in a fixed order:
+ * results are identical from run to run.  Asynchronous on cuda_stream.  Bound by the one pass over the points. */
+sd_status sd_kmeans_step(const float* points_dev, int64_t n, int dim, const float* centroids_dev, int k,
+                         int32_t* labels_dev, float* centroids_out_dev, int64_t* counts_out_dev, double* inertia_out_dev,
+                         void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+size_t sd_kmeans_workspace(int dim, int k);
+
 /* Philox4x32-10 on the device: out[i][0..3] for ctr[i][0..3], one key.  For tests. */
 sd_status sd_op_philox(const uint32_t* ctr_dev, int n, uint32_t key0, uint32_t key1, uint32_t* out_dev, void* cuda_stream);
 

@@ -99,6 +99,8 @@ _PROTOS = {
     "sd_op_linear_workspace": (_sz, [_i, _i, _i, _i, _i]),
     "sd_op_linear_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "sd_op_linear_wait_expiry": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp, _sz, C.c_uint64, _vp, _vp]),
+    "sd_kmeans_step": (_i, [_vp, C.c_int64, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "sd_kmeans_workspace": (_sz, [_i, _i]),
     "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_attention_runs": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "sd_op_attention_workspace": (_sz, [_i, _i, _i, _i]),
@@ -453,6 +455,18 @@ def sd_op_attention(q, kc, vc, out, row_slot, row_pos, n_heads, n_kv_heads, head
     ws = torch.empty(max(need, 1), dtype=torch.uint8, device=q.device)
     _check(lib().sd_op_attention_runs(_dp(q), _dp(kc), _dp(vc), _dp(out), _dp(row_slot), _dp(row_pos), rows, int(rows_per_seq), n_heads,
                                       n_kv_heads, head_dim, max_ctx, dtype, _dp(ws), need, _stream_ptr(stream)), "sd_op_attention_runs")
+
+
+def sd_kmeans_step(points, centroids, labels, centroids_out=None, counts_out=None, inertia_out=None, stream=None):
+    """One Lloyd iteration on the device (all arguments CUDA tensors: fp32 points [n][dim], centroids [k][dim], int32 labels [n],
+    optional fp32 centroids_out [k][dim], int64 counts_out [k], float64 inertia_out [1])."""
+    n, dim = points.shape
+    k = centroids.shape[0]
+    need = lib().sd_kmeans_workspace(dim, k)
+    ws = torch.empty(max(need, 1), dtype=torch.uint8, device=points.device)
+    opt = lambda t: _dp(t) if t is not None else None
+    _check(lib().sd_kmeans_step(_dp(points), n, dim, _dp(centroids), k, _dp(labels), opt(centroids_out), opt(counts_out), opt(inertia_out),
+                                _dp(ws), need, _stream_ptr(stream)), "sd_kmeans_step")
 
 
 def sd_op_philox(ctr, key0, key1, out, stream=None):

@@ -135,3 +135,40 @@ def make_prompt_lengths(batch, lo, hi, seed=4):
 
 def make_logits(shape, seed, stream=0, std=1.0):
     return _rng(seed, 9000 + stream).standard_normal(shape, dtype=np.float32) * np.float32(std)
+
+
+def make_sentence_vectors(n, dim=384, n_tasks=4, seed=6, spread=0.6):
+    """Stand-in for the sentence vectors of the offline partitioning step: n unit-length fp32 vectors of `dim`
+    components in n_tasks groups (a random unit direction per task plus isotropic noise of relative size `spread`,
+    renormalised), and the group of every vector.  Groups overlap a little, like the paper's 90-99 % clusterable tasks."""
+    g = _rng(seed, 8800)
+    centers = g.standard_normal((n_tasks, dim), dtype=np.float32)
+    centers /= np.linalg.norm(centers, axis=1, keepdims=True)
+    task = g.integers(0, n_tasks, size=n, dtype=np.int64).astype(np.int32)
+    x = centers[task] + g.standard_normal((n, dim), dtype=np.float32) * np.float32(spread / np.sqrt(dim))
+    x /= np.linalg.norm(x, axis=1, keepdims=True)
+    return np.ascontiguousarray(x, dtype=np.float32), task
+
+
+def make_mamba_classifier(vocab, d_model=128, d_state=16, d_conv=4, expand=2, n_classes=4, seed=0):
+    """fp32 weights of the Mamba-based prompt classifier (embedding, one selective state-space layer, pooled output,
+    fully connected layer), initialised the way the Mamba paper initialises its layer: A = -(1..N) per channel, step
+    sizes softplus(b_dt) log-uniform in [1e-3, 1e-1], D = 1, projections N(0, 1/fan_in); embedding N(0, 1)."""
+    g = _rng(seed, 7100)
+    Di, R = expand * d_model, (d_model + 15) // 16
+
+    def n(shape, std):
+        return (g.standard_normal(shape, dtype=np.float32) * np.float32(std)).astype(np.float32)
+
+    dt = np.exp(g.random(Di) * (np.log(0.1) - np.log(1e-3)) + np.log(1e-3))
+    return dict(
+        embed=n((vocab, d_model), 1.0),
+        w_in=n((2 * Di, d_model), d_model ** -0.5),
+        w_conv=n((Di, d_conv), d_conv ** -0.5), b_conv=n((Di,), 0.02),
+        w_x=n((R + 2 * d_state, Di), Di ** -0.5),
+        w_dt=n((Di, R), R ** -0.5), b_dt=(dt + np.log(-np.expm1(-dt))).astype(np.float32),      # inverse softplus
+        a_log=np.log(np.tile(np.arange(1, d_state + 1, dtype=np.float32), (Di, 1))).astype(np.float32),
+        d_skip=np.ones(Di, dtype=np.float32),
+        w_out=n((d_model, Di), Di ** -0.5),
+        w_fc=n((n_classes, d_model), 1.0), b_fc=n((n_classes,), 0.01),
+    )
