@@ -416,6 +416,38 @@ sd_status sd_op_attention_runs(const void* q, const void* k_cache, const void* v
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 size_t sd_op_attention_workspace(int rows, int n_heads, int head_dim, int max_ctx);
 
+/* The Mamba-based prompt classifier of Section 2.4 / Section 3.3.3: embedding layer -> one Mamba (selective state-space)
+ * layer -> average pooling over the prompt -> fully connected layer -> argmax.  The paper names the parts and cites the
+ * Mamba paper for the layer; the layer is that paper's block: input projection to (u, z), causal depthwise convolution
+ * (d_conv taps, zeros before the prompt) + SiLU, input-dependent (dt, B, C) with dt = softplus(W_dt r + b_dt),
+ * h_t = exp(dt_t A) h_{t-1} + dt_t v_t B_t with A = -exp(a_log), y_t = h_t C_t + d_skip v_t, gate silu(z_t), output
+ * projection; no residual connection, no normalisation.  All weights fp32, row-major, DEVICE pointers owned by the
+ * caller (read during the call only):
+ *   embed [vocab][d_model]   w_in [2*Di][d_model] (u rows first, then z), Di = expand * d_model
+ *   w_conv [Di][d_conv]  b_conv [Di]   w_x [dt_rank + 2*d_state][Di] (r, B, C rows)   w_dt [Di][dt_rank]  b_dt [Di]
+ *   a_log [Di][d_state]  d_skip [Di]   w_out [d_model][Di]   w_fc [n_classes][d_model]  b_fc [n_classes]
+ * sd_mamba_classify scores n_prompts prompts in one go: prompt i is tokens_dev[starts_host[i] .. + lens_host[i]) (device
+ * tokens, host offsets and lengths >= 1; token ids are clamped to the vocabulary); scores_dev [n_prompts][n_classes]
+ * fp32 and labels_dev [n_prompts] int32 (argmax, lowest index on ties) are device buffers, either may be NULL.
+ * workspace_dev: sd_mamba_workspace(desc, sum of lengths, n_prompts) bytes of device memory.  Long prompts are scanned
+ * in chunks side by side.  Limits: d_state <= 16, d_conv <= 8, d_model <= 512, Di <= 1024 (else SD_ERR_UNSUPPORTED).
+ * Copies small host tables to the device and synchronises the stream once before launching; the launches are
+ * asynchronous on cuda_stream. */
+typedef struct { int32_t vocab, d_model, d_state, d_conv, expand, n_classes, dt_rank; } sd_mamba_desc;
+typedef struct {
+    const float *embed, *w_in, *w_conv, *b_conv, *w_x, *w_dt, *b_dt, *a_log, *d_skip, *w_out, *w_fc, *b_fc;
+} sd_mamba_weights;
+size_t sd_mamba_workspace(const sd_mamba_desc* desc, int64_t total_tokens, int n_prompts);
+sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba_weights* weights_dev, const int32_t* tokens_dev,
+                            const int64_t* starts_host, const int32_t* lens_host, int n_prompts, float* scores_dev,
+                            int32_t* labels_dev, void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+/* Routes sequences with that classifier instead of the MLP: classifies the prompts of `seqs` (begun with sd_seq_begin)
+ * and records class k as draft k, exactly as sd_route_prompt does with forced tasks.  n_classes must equal the
+ * context's number of drafts.  draft_id_out (host, nullable) receives the ids.  Synchronises. */
+sd_status sd_route_prompt_mamba(sd_ctx* ctx, const sd_mamba_desc* desc, const sd_mamba_weights* weights_dev,
+                                const int32_t* seqs, int n_seq, void* workspace_dev, size_t workspace_bytes,
+                                int32_t* draft_id_out);
+
 /* One iteration of the K-means algorithm (Lloyd) over dense fp32 vectors: the offline task-partitioning step of
  * Section 3.2, which clusters 384-dimensional sentence vectors into one subset per task.
  *   labels[i]       = argmin_k sum_d (points[i][d] - centroids[k][d])^2, distances summed in fp32, lowest k on ties

@@ -40,6 +40,44 @@ class Cost(C.Structure):
                 ("draft_passes", C.c_int64), ("verify_passes", C.c_int64), ("target_passes", C.c_int64)]
 
 
+class MambaDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("vocab", "d_model", "d_state", "d_conv", "expand", "n_classes", "dt_rank")]
+
+
+MAMBA_WEIGHT_NAMES = ("embed", "w_in", "w_conv", "b_conv", "w_x", "w_dt", "b_dt", "a_log", "d_skip", "w_out", "w_fc", "b_fc")
+
+
+class MambaWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in MAMBA_WEIGHT_NAMES]
+
+
+class MambaClassifier:
+    """Device copy of the classifier's weights (fp32 numpy arrays in, CUDA tensors kept here) and its descriptor."""
+
+    def __init__(self, weights, device="cuda:0"):
+        self.t = {n: torch.from_numpy(np.ascontiguousarray(weights[n], dtype=np.float32)).to(device) for n in MAMBA_WEIGHT_NAMES}
+        Di, R = weights["w_dt"].shape
+        V, D = weights["embed"].shape
+        self.desc = MambaDesc(V, D, weights["a_log"].shape[1], weights["w_conv"].shape[1], Di // D, weights["w_fc"].shape[0], R)
+        self.w = MambaWeights(*[self.t[n].data_ptr() for n in MAMBA_WEIGHT_NAMES])
+        self.device = self.t["embed"].device
+
+    def workspace(self, total_tokens, n_prompts):
+        need = lib().sd_mamba_workspace(C.byref(self.desc), int(total_tokens), int(n_prompts))
+        return torch.empty(max(need, 1), dtype=torch.uint8, device=self.device), need
+
+    def classify(self, tokens_dev, starts, lens, stream=None):
+        """(scores [n][K] fp32 tensor, labels [n] int32 tensor) for prompts tokens_dev[starts[i] : starts[i] + lens[i]]."""
+        n = len(lens)
+        starts = np.ascontiguousarray(starts, dtype=np.int64); lens = np.ascontiguousarray(lens, dtype=np.int32)
+        scores = torch.zeros((n, self.desc.n_classes), dtype=torch.float32, device=self.device)
+        labels = torch.full((n,), -1, dtype=torch.int32, device=self.device)
+        ws, need = self.workspace(int(lens.sum()), n)
+        _check(lib().sd_mamba_classify(C.byref(self.desc), C.byref(self.w), _dp(tokens_dev), starts.ctypes.data_as(C.c_void_p),
+                                       lens.ctypes.data_as(C.c_void_p), n, _dp(scores), _dp(labels), _dp(ws), need, _stream_ptr(stream)), "sd_mamba_classify")
+        return scores, labels
+
+
 class AcceptArgs(C.Structure):
     _fields_ = [("target", C.c_void_p), ("target_is_logits", C.c_int32), ("q", C.c_void_p), ("x", C.c_void_p),
                 ("B", C.c_int32), ("gamma", C.c_int32), ("V", C.c_int32), ("temperature", C.c_float),
@@ -99,6 +137,9 @@ _PROTOS = {
     "sd_op_linear_workspace": (_sz, [_i, _i, _i, _i, _i]),
     "sd_op_linear_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "sd_op_linear_wait_expiry": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp, _sz, C.c_uint64, _vp, _vp]),
+    "sd_mamba_workspace": (_sz, [_vp, C.c_int64, _i]),
+    "sd_mamba_classify": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _sz, _vp]),
+    "sd_route_prompt_mamba": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "sd_kmeans_step": (_i, [_vp, C.c_int64, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "sd_kmeans_workspace": (_sz, [_i, _i]),
     "sd_op_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
@@ -308,6 +349,15 @@ class Context:
     def sd_verify_accept(self, seqs, gamma, x, q, logits, n_acc, out_tok):
         a, p, n = _seqs(seqs)
         _check(self.L.sd_verify_accept(self.h, p, n, gamma, _dp(x), _dp(q), _dp(logits), _dp(n_acc), _dp(out_tok)), "sd_verify_accept")
+
+    def sd_route_prompt_mamba(self, clf, seqs):
+        seqs_a = np.ascontiguousarray(seqs, dtype=np.int32)
+        lens_total = int(self.cfg.max_ctx) * len(seqs)
+        ws, need = clf.workspace(lens_total, len(seqs))
+        out = np.zeros(len(seqs), dtype=np.int32)
+        _check(self.L.sd_route_prompt_mamba(self.h, C.byref(clf.desc), C.byref(clf.w), seqs_a.ctypes.data_as(C.c_void_p), len(seqs),
+                                            _dp(ws), need, out.ctypes.data_as(C.c_void_p)), "sd_route_prompt_mamba")
+        return out
 
     def sd_tuning(self, knob, value):
         _check(self.L.sd_tuning(self.h, int(knob), int(value)), "sd_tuning")

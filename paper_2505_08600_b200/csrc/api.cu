@@ -927,6 +927,27 @@ sd_status sd_route_prompt(sd_ctx* c, const int32_t* seqs, int n_seq, const int32
     return SD_OK;
 }
 
+sd_status sd_route_prompt_mamba(sd_ctx* c, const sd_mamba_desc* desc, const sd_mamba_weights* w, const int32_t* seqs, int n_seq,
+                                void* ws, size_t ws_bytes, int32_t* draft_out) {
+    if (!c || !desc || !w || !seqs || n_seq < 1 || n_seq > c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
+    if (desc->n_classes != c->cfg.n_drafts) return SD_ERR_INVALID_ARG;
+    std::vector<int64_t> starts(n_seq);
+    std::vector<int32_t> lens(n_seq), labels(n_seq);
+    for (int i = 0; i < n_seq; ++i) {
+        const int s = seqs[i];
+        if (s < 0 || s >= c->cfg.max_seqs) return SD_ERR_INVALID_ARG;
+        if (c->phase[s] < PH_BEGUN) return SD_ERR_STATE;
+        starts[i] = (int64_t)s * c->S.tok_stride;
+        lens[i] = c->n_prompt[s];
+    }
+    // labels land in the scratch words the accept path uses for its counts (n_seq <= max_seqs of them)
+    SD_TRY(sd_mamba_classify(desc, w, c->S.tokens, starts.data(), lens.data(), n_seq, nullptr, c->st_nacc, ws, ws_bytes, c->st));
+    c->launches += 5;
+    CUDA_TRY(cudaMemcpyAsync(labels.data(), c->st_nacc, sizeof(int32_t) * n_seq, cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    return sd_route_prompt(c, seqs, n_seq, labels.data(), draft_out);
+}
+
 sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
     SeqList all;
     SD_TRY(make_list(c, seqs, n_seq, c->cfg.n_drafts > 0 ? PH_ROUTED : PH_BEGUN, all));
