@@ -543,6 +543,50 @@ def run_kmeans_bench(args):
                                        "sample": f"{xs.shape[0]} of the points, {reps} repeats"}}))
 
 
+def run_mamba_bench(args):
+    """The Mamba-based prompt classifier on a batch the size of the paper's test set: 400 prompts of 32..512 tokens
+    (uniform), vocabulary 21128, d_model 128, 16 states, 4 classes; all 400 scored by one call."""
+    import torch
+    from paper_2505_08600_b200 import binding as sd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    vocab, n_prompts = 21128, 400
+    w = synth.make_mamba_classifier(vocab, d_model=128, d_state=16, d_conv=4, expand=2, n_classes=4, seed=0)
+    clf = sd.MambaClassifier(w)
+    lens = synth.make_prompt_lengths(n_prompts, 32, 512, seed=8)
+    starts = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
+    tokens_h = np.concatenate([synth.make_prompt(vocab, int(n), seed=8, seq=i) for i, n in enumerate(lens)])
+    tokens = torch.from_numpy(tokens_h).to(dev)
+    for _ in range(max(3, args.warmup)):
+        scores, labels = clf.classify(tokens, starts, lens)
+    torch.cuda.synchronize()
+    K = max(5, min(args.steps, 50))
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(torch.cuda.current_stream())
+    for _ in range(K):
+        scores, labels = clf.classify(tokens, starts, lens)
+    e1.record(torch.cuda.current_stream()); torch.cuda.synchronize()
+    ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / K          # the call uploads small host tables: wall time counts
+    T = int(lens.sum())
+    D, Di, N, R, Kc = 128, 256, 16, 8, 4
+    flop = T * 2.0 * (2 * Di * D + Kc * Di + (R + 2 * N) * Di + R * Di + 2 * 3 * Di * N) + n_prompts * 2.0 * (D * Di + 4 * D)
+    alu_peak = 148 * 128 * 2 * 1.965e9                                           # fp32 lanes x 2 flop x clock
+    from oracle import classifier_mamba as om
+    t0 = time.perf_counter(); done = 0
+    while time.perf_counter() - t0 < 10.0 and done < n_prompts:
+        om.classify(w, tokens_h[starts[done]: starts[done] + lens[done]]); done += 1
+    cpu_s = (time.perf_counter() - t0) / done
+    agree = sum(int(om.classify(w, tokens_h[starts[i]: starts[i] + lens[i]])[0] == int(labels[i])) for i in range(min(done, 25)))
+    print(json.dumps({"metric": "mamba_classifier_prompts_per_s", "unit": "prompts/s", "value": n_prompts / (ms * 1e-3), "ms_per_step": ms,
+                      "ms_per_prompt": ms / n_prompts, "n_gpus": 1, "steps": K, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": f"{n_prompts} prompts, {T} tokens (32..512 each), vocab {vocab}, d_model 128, 16 states, 4 classes, one call"},
+                      "roofline": {"bound": "alu", "achieved": flop / (ms * 1e-3) / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
+                                   "frac": flop / (ms * 1e-3) / alu_peak, "peak_kind": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz", "traffic": None},
+                      "labels_agree_with_oracle": f"{agree} of {min(done, 25)}",
+                      "cpu_baseline": {"value": 1.0 / cpu_s, "unit": "prompts/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle", "sample": f"the first {done} prompts"}}))
+
+
 def run_accept_microbench(args):
     """Accept / reject / resample kernel alone at the 13B configuration's shape (8 sequences, gamma 8, vocab 32000):
     draft distributions are softmax(target_logits + N(0, sigma^2)) so that sigma sets the acceptance rate."""
@@ -598,6 +642,7 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
+    ap.add_argument("--mamba", action="store_true", help="time the Mamba-based prompt classifier on 400 synthetic prompts and exit")
     ap.add_argument("--kmeans", action="store_true", help="time one K-means step over synthetic sentence vectors and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -612,7 +657,7 @@ def main():
             argv[i + 1] = name
             rc = rc or subprocess.run(argv).returncode
         sys.exit(rc)
-    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep and not args.kmeans:
+    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep and not args.kmeans and not args.mamba:
         # no launcher: this process starts the N replicas itself (one per GPU) and passes rank 0's line through
         rc, out = replicas.spawn_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
         sys.stdout.write(out)
@@ -621,6 +666,8 @@ def main():
         run_accept_microbench(args)
     elif args.kmeans:
         run_kmeans_bench(args)
+    elif args.mamba:
+        run_mamba_bench(args)
     elif args.gamma_sweep:
         run_gamma_sweep(args)
     elif args.impl == "reference":

@@ -92,10 +92,10 @@ k_kmeans_assign(const float* __restrict__ pts, long long n, int k, const float* 
 #pragma unroll
         for (int v = 0; v < NV; ++v) x[v] = *reinterpret_cast<const ulonglong2*>(ring + slot * DIM + v * 128);
         slot = slot + 1 == KM_DEPTH ? 0 : slot + 1;
-        float best = INFINITY;
-        int label = 0;
+        float dk[KM];                                                             // this lane's share of every squared distance
 #pragma unroll
         for (int kk = 0; kk < KM; ++kk) {
+            dk[kk] = 0.f;
             if (kk < k) {                                                         // uniform
                 f32x2 d2 = 0ull;
 #pragma unroll
@@ -104,12 +104,38 @@ k_kmeans_assign(const float* __restrict__ pts, long long n, int k, const float* 
                     const f32x2 a = f2_sub(x[v].x, c.x), b = f2_sub(x[v].y, c.y);
                     d2 = f2_fma(a, a, d2); d2 = f2_fma(b, b, d2);
                 }
-                float d = f2_hsum(d2);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);      // every lane ends with the same sum
-                if (d < best) { best = d; label = kk; }                           // a later centroid must be strictly closer
+                dk[kk] = f2_hsum(d2);
             }
         }
+        if (KM == 4) {
+            // Four sums over the warp with ten shuffles instead of twenty: halves of the warp trade two of the four
+            // values, quarters one of the two, three more steps finish one value per lane group, and the four totals
+            // are read back from lanes 0, 8, 16 and 24 (every lane ends with the same four numbers).
+            const bool hi16 = lane & 16, hi8 = lane & 8;
+            float a = hi16 ? dk[KM == 4 ? 2 : 0] : dk[0], sa = hi16 ? dk[0] : dk[KM == 4 ? 2 : 0];
+            float b = hi16 ? dk[KM == 4 ? 3 : 0] : dk[KM == 4 ? 1 : 0], sb = hi16 ? dk[KM == 4 ? 1 : 0] : dk[KM == 4 ? 3 : 0];
+            a += __shfl_xor_sync(0xffffffffu, sa, 16);
+            b += __shfl_xor_sync(0xffffffffu, sb, 16);
+            float e = hi8 ? b : a;
+            const float se = hi8 ? a : b;
+            e += __shfl_xor_sync(0xffffffffu, se, 8);
+            e += __shfl_xor_sync(0xffffffffu, e, 4);
+            e += __shfl_xor_sync(0xffffffffu, e, 2);
+            e += __shfl_xor_sync(0xffffffffu, e, 1);
+            // lane group (bit 4, bit 3) holds cluster 2 * bit4 + bit3
+            dk[0] = __shfl_sync(0xffffffffu, e, 0);
+            if (KM == 4) { dk[KM == 4 ? 1 : 0] = __shfl_sync(0xffffffffu, e, 8); dk[KM == 4 ? 2 : 0] = __shfl_sync(0xffffffffu, e, 16); dk[KM == 4 ? 3 : 0] = __shfl_sync(0xffffffffu, e, 24); }
+        } else {
+#pragma unroll
+            for (int kk = 0; kk < KM; ++kk)
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dk[kk] += __shfl_xor_sync(0xffffffffu, dk[kk], o);      // every lane ends with the same sums
+        }
+        float best = INFINITY;
+        int label = 0;
+#pragma unroll
+        for (int kk = 0; kk < KM; ++kk)
+            if (kk < k && dk[kk] < best) { best = dk[kk]; label = kk; }            // a later centroid must be strictly closer
         if (lane == 0) labels[i] = label;
         inertia += (double)best;
 #pragma unroll
@@ -166,11 +192,13 @@ k_kmeans_reduce(const float* __restrict__ part_sums, const long long* __restrict
         for (int b = b0; b < b1; ++b) s += (double)__ldcg(part_sums + ((size_t)b * k + kk) * dim + d);
     }
     run_sum[run][threadIdx.x & 31] = s;
-    if ((threadIdx.x & 31) == 0) {
+    {   // the run's counts and inertia: a lane per block, then a fixed tree over the lanes
         long long c = 0;
         double in = 0.0;
-        for (int b = b0; b < b1; ++b) { c += part_counts[(size_t)b * k + kk]; in += part_inertia[b]; }
-        run_cnt[run] = c; run_in[run] = in;
+        for (int b = b0 + (int)(threadIdx.x & 31); b < b1; b += 32) { c += part_counts[(size_t)b * k + kk]; in += part_inertia[b]; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { c += __shfl_xor_sync(0xffffffffu, c, o); in += __shfl_xor_sync(0xffffffffu, in, o); }
+        if ((threadIdx.x & 31) == 0) { run_cnt[run] = c; run_in[run] = in; }
     }
     __syncthreads();
     if (run != 0) return;
