@@ -77,7 +77,11 @@ typedef struct {
     float temperature;       /* same for draft and target; 0 = greedy */
     uint64_t seed;           /* Philox4x32-10 key */
     int32_t clf_d_hidden;    /* prompt classifier d_model(target) -> clf_d_hidden -> n_drafts; 0 = none */
-    int32_t reserved;
+    int32_t lora_adapters;   /* 0: models[1..K] are K separate drafts.  K (= n_drafts): the drafts are ONE base model,
+                                models[1], plus one low-rank adapter per task (Section 2.3: every draft is the same base
+                                draft fine-tuned with LoRA); sequences of different tasks then share each draft pass */
+    int32_t lora_rank;       /* r: a multiple of 8, lora_adapters * r <= 128 */
+    float lora_scale;        /* alpha / r of the LoRA paper: W' = W + lora_scale * B A */
 } sd_config;
 
 typedef struct {
@@ -90,6 +94,9 @@ enum {
     SD_T_WQ = 3, SD_T_WK = 4, SD_T_WV = 5, SD_T_WO = 6, SD_T_WG = 7, SD_T_WU = 8, SD_T_WD = 9,
     SD_T_NORM1 = 10, SD_T_NORM2 = 11
 };
+
+/* matrices of a layer that carry an adapter (sd_load_lora) */
+enum { SD_LORA_QKV = 0, SD_LORA_WO = 1, SD_LORA_GU = 2, SD_LORA_WD = 3 };
 
 /* ---------------------------------------------------------------- lifecycle */
 
@@ -110,6 +117,16 @@ sd_status sd_destroy(sd_ctx* ctx);
  * Matrices are in the model's dtype (bf16 as raw 16-bit patterns), norm gains
  * are fp32.  src may be host (src_on_device = 0) or device memory. */
 sd_status sd_load_tensor(sd_ctx* ctx, int model_id, int kind, int layer, const void* src, int src_on_device);
+
+/* One low-rank adapter of the shared base draft (contexts created with lora_adapters > 0): for matrix `mat` of `layer`,
+ * task `adapter` uses W' = W + lora_scale * B A (the LoRA paper's definition; Section 2.3 fine-tunes every draft this
+ * way).  a: [lora_rank][in_features], b: [out_features][lora_rank], both bf16 bit patterns, row-major, host or device.
+ * out_features follow the fused matrices: SD_LORA_QKV (H + 2 Hkv) * head_dim rows (query, key, value rows in that
+ * order), SD_LORA_GU 2 * d_ffn rows (gate rows, then up rows), SD_LORA_WO / SD_LORA_WD d_model rows.  Adapters that
+ * were never loaded are zero: the task runs the base draft.  The embedding and the lm_head carry no adapter.
+ * The product x A^T rides along in the matrix's own GEMM (A's rows are appended to W as one more output tile) and
+ * B is applied by the step kernel after the GEMM: no extra launch, no extra pass over the weights. */
+sd_status sd_load_lora(sd_ctx* ctx, int adapter, int layer, int mat, const void* a, const void* b, int src_on_device);
 
 /* Prompt classifier, MLP variant of Sec. 3.3.3: fp32 w1 [h][d], b1 [h], w2 [K][h], b2 [K]. */
 sd_status sd_load_classifier(sd_ctx* ctx, const float* w1, const float* b1, const float* w2, const float* b2,

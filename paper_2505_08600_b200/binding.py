@@ -28,7 +28,8 @@ class ModelDesc(C.Structure):
 
 class Config(C.Structure):
     _fields_ = [("max_seqs", C.c_int32), ("max_ctx", C.c_int32), ("max_gamma", C.c_int32), ("n_drafts", C.c_int32),
-                ("temperature", C.c_float), ("seed", C.c_uint64), ("clf_d_hidden", C.c_int32), ("reserved", C.c_int32)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("clf_d_hidden", C.c_int32), ("lora_adapters", C.c_int32),
+                ("lora_rank", C.c_int32), ("lora_scale", C.c_float)]
 
 
 class Counters(C.Structure):
@@ -99,6 +100,7 @@ _PROTOS = {
     "sd_create": (_i, [C.POINTER(Config), C.POINTER(ModelDesc), _vp, _vp, _sz, C.POINTER(_vp)]),
     "sd_destroy": (_i, [_vp]),
     "sd_load_tensor": (_i, [_vp, _i, _i, _i, _vp, _i]),
+    "sd_load_lora": (_i, [_vp, _i, _i, _i, _vp, _vp, _i]),
     "sd_load_classifier": (_i, [_vp, _vp, _vp, _vp, _vp, _i]),
     "sd_seq_begin": (_i, [_vp, _i, _vp, _i, C.c_uint32]),
     "sd_prefill": (_i, [_vp, _vp, _i]),
@@ -241,7 +243,8 @@ class Context:
     the C calls and do nothing but marshal their arguments."""
 
     def __init__(self, target_dims, draft_dims, dtype, max_seqs, max_ctx, max_gamma, temperature, seed,
-                 clf_d_hidden=0, device="cuda:0", stream=None):
+                 clf_d_hidden=0, device="cuda:0", stream=None, lora_adapters=0, lora_rank=0, lora_scale=0.0):
+        """lora_adapters > 0: draft_dims holds ONE base draft shared by lora_adapters tasks (one low-rank adapter each)."""
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self.device = torch.device(device)
@@ -252,7 +255,9 @@ class Context:
         self.vocab = target_dims["vocab"]
         n = len(self.dims)
         self._descs = (ModelDesc * n)(*[_desc(d, dtype) for d in self.dims])
-        self.cfg = Config(max_seqs, max_ctx, max_gamma, n - 1, float(temperature), int(seed), int(clf_d_hidden), 0)
+        n_tasks = int(lora_adapters) if lora_adapters else n - 1
+        self.cfg = Config(max_seqs, max_ctx, max_gamma, n_tasks, float(temperature), int(seed), int(clf_d_hidden),
+                          int(lora_adapters), int(lora_rank), float(lora_scale))
         need = self.L.sd_arena_bytes(C.byref(self.cfg), self._descs)
         if need == 0:
             raise SdError(1, "sd_arena_bytes")
@@ -275,6 +280,11 @@ class Context:
             pass
 
     # ---- loading
+    def sd_load_lora(self, adapter, layer, mat, a, b):
+        """a [r][in], b [out][r]: numpy uint16 arrays of bf16 bit patterns."""
+        a = np.ascontiguousarray(a, dtype=np.uint16); b = np.ascontiguousarray(b, dtype=np.uint16)
+        _check(self.L.sd_load_lora(self.h, int(adapter), int(layer), int(mat), a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p), 0), "sd_load_lora")
+
     def sd_load_tensor(self, model_id, kind, layer, src):
         """src: numpy array (host) or torch CUDA tensor, already in the model's dtype
         (bf16 as uint16 bit patterns or torch.bfloat16)."""

@@ -34,6 +34,7 @@ struct Layer {
     float* norm1;
     float* norm2;
     TensorMap tm_qkv, tm_wo, tm_gu, tm_wd;   // TMA descriptors of the four matrices (bf16 models)
+    bf16* lora_b[4];                // low-rank adapters: [adapter][out feature][r] per matrix (QKV, Wo, gate/up, down); nullptr: none
 };
 
 struct Model {
@@ -52,6 +53,7 @@ struct Model {
     bool tc;                        // the tensor-core path applies (bf16, shapes fit)
     PassMaps pmaps;                 // the layers' matrices as [layer][row][k] tensor maps (persistent streaming kernel)
     bool pass_ok;                   // ... which applies to this model
+    bool lora;                      // the matrices carry one more 128-row tile: the adapters' A rows
     int n_qkv() const { return (d.n_heads + 2 * d.n_kv_heads) * d.head_dim; }
 };
 
@@ -145,13 +147,28 @@ bool valid_desc(const sd_model_desc& m) {
     return true;
 }
 
+// Contexts with low-rank adapters hold ONE draft model (models[1]) shared by all tasks.
+int n_models(const sd_config& cfg) { return 1 + (cfg.lora_adapters > 0 ? 1 : cfg.n_drafts); }
+int draft_model_index(const sd_config& cfg, int task) { return cfg.lora_adapters > 0 ? 1 : 1 + task; }
+size_t tile_rows(size_t n) { return (n + 127) / 128 * 128; }
+
 bool valid_cfg(const sd_config* c, const sd_model_desc* ms) {
     if (!c || !ms) return false;
     if (c->max_seqs < 1 || c->max_seqs > SD_MAX_BATCH || c->max_ctx < 4 || c->max_gamma < 0 || c->max_gamma > SD_MAX_GAMMA) return false;
     if (c->n_drafts < 0 || c->n_drafts > 16 || !(c->temperature >= 0.f) || c->clf_d_hidden < 0) return false;
-    for (int i = 0; i <= c->n_drafts; ++i) {
+    if (c->lora_adapters < 0) return false;
+    if (c->lora_adapters > 0) {
+        if (c->lora_adapters != c->n_drafts || c->lora_rank < 8 || c->lora_rank > 32 || (c->lora_rank & 7) ||
+            c->lora_adapters * c->lora_rank > 128 || !(c->lora_scale == c->lora_scale))
+            return false;
+    }
+    for (int i = 0; i < n_models(*c); ++i) {
         if (!valid_desc(ms[i])) return false;
         if (ms[i].vocab != ms[0].vocab) return false;        // draft and target share the vocabulary
+    }
+    if (c->lora_adapters > 0) {                              // adapters ride on the tensor-core path: whole tiles of bf16
+        const sd_model_desc& m = ms[1];
+        if (m.dtype != SD_BF16 || ((m.n_heads + 2 * m.n_kv_heads) * m.head_dim) % 128 || m.d_model % 128 || (2 * m.d_ffn) % 128) return false;
     }
     return true;
 }
@@ -160,7 +177,7 @@ bool valid_cfg(const sd_config* c, const sd_model_desc* ms) {
 // the arena, once more with the real base to place the pointers.
 void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     const sd_config& cfg = c->cfg;
-    const int S = cfg.max_seqs, nm = 1 + cfg.n_drafts;
+    const int S = cfg.max_seqs, nm = n_models(cfg);
     c->models.resize(nm);
     int d_max = 0, f_max = 0, qkv_max = 0, dq_max = 0, lin_max = 0;
     for (int i = 0; i < nm; ++i) {
@@ -173,14 +190,19 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
         M.lm_head = B.take((size_t)m.vocab * m.d_model * M.esz);
         M.final_norm = (float*)B.take(sizeof(float) * m.d_model);
         M.layers.resize(m.n_layers);
+        M.lora = cfg.lora_adapters > 0 && i == 1;
+        const size_t extra = M.lora ? 128 : 0;               // one more tile of rows per matrix: A of every adapter
+        const size_t n_lb = M.lora ? (size_t)cfg.lora_adapters * cfg.lora_rank : 0;
         for (int l = 0; l < m.n_layers; ++l) {
             Layer& L = M.layers[l];
-            L.wqkv = B.take((dq + 2 * dkv) * m.d_model * M.esz);
-            L.wo = B.take((size_t)m.d_model * dq * M.esz);
-            L.wgu = B.take((size_t)2 * m.d_ffn * m.d_model * M.esz);
-            L.wd = B.take((size_t)m.d_model * m.d_ffn * M.esz);
+            L.wqkv = B.take((dq + 2 * dkv + extra) * m.d_model * M.esz);
+            L.wo = B.take(((size_t)m.d_model + extra) * dq * M.esz);
+            L.wgu = B.take(((size_t)2 * m.d_ffn + extra) * m.d_model * M.esz);
+            L.wd = B.take(((size_t)m.d_model + extra) * m.d_ffn * M.esz);
             L.norm1 = (float*)B.take(sizeof(float) * m.d_model);
             L.norm2 = (float*)B.take(sizeof(float) * m.d_model);
+            const size_t outs[4] = {dq + 2 * dkv, (size_t)m.d_model, (size_t)2 * m.d_ffn, (size_t)m.d_model};
+            for (int k = 0; k < 4; ++k) L.lora_b[k] = M.lora ? (bf16*)B.take(n_lb * outs[k] * sizeof(bf16)) : nullptr;
         }
         M.kv_layer_bytes = (size_t)S * dkv * cfg.max_ctx * M.esz;
         M.kcache = (char*)B.take(M.kv_layer_bytes * m.n_layers);
@@ -230,7 +252,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
         const int shapes[5][2] = {{(m.n_heads + 2 * m.n_kv_heads) * m.head_dim, m.d_model}, {m.d_model, m.n_heads * m.head_dim},
                                   {2 * m.d_ffn, m.d_model}, {m.d_model, m.d_ffn}, {m.vocab, m.d_model}};
         for (auto& s : shapes)
-            c->partials_bytes = std::max(c->partials_bytes, gemm_partials_bytes(gemm_geometry(SD_MAX_ROWS, s[0], s[1], sm_count())));
+            c->partials_bytes = std::max(c->partials_bytes, gemm_partials_bytes(gemm_geometry(SD_MAX_ROWS, s[0], s[1], sm_count(), 0, false, 1)));
     }
     c->partials = (float*)B.take(c->partials_bytes);
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
@@ -471,7 +493,7 @@ unsigned long long* next_stamp(sd_ctx* c, int kind) {
 // One weight GEMM and the step that follows it.
 sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n_out, int K, const Epilogue& ep) {
     if (ep.lo_off) rows += ep.lo_off;           // the input rows come in two bf16 parts: [x_hi rows][x_lo rows at + lo_off]
-    GemmGeom g = gemm_geometry(rows, n_out, K, sm_count(), ep.ring_stages, ep.prefill_all != 0);
+    GemmGeom g = gemm_geometry(rows, n_out, K, sm_count(), ep.ring_stages, ep.prefill_all != 0, ep.lora_b ? 1 : 0);
     if (ep.lo_off) { g.lo_off = ep.lo_off; g.m_real = ep.m_real; }
     g.pace_ns = c->tune[SD_TUNE_PACE_NS];
     if (c->tune[SD_TUNE_PREFILL_STAGES] >= 2) g.prefill = std::min(g.stages, c->tune[SD_TUNE_PREFILL_STAGES]);
@@ -482,7 +504,7 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     TensorMap tx;
     if (!make_tensor_map_bf16(&tx, x, rows, K, g.m_pad)) return SD_ERR_CUDA;
     uint32_t* arrive = nullptr;                 // words of this GEMM alone; when they run out the step waits for the GEMM's grid
-    if (fused_step_polls(g, ep) && c->arrive_used + (size_t)g.n_tiles <= ARRIVE_WORDS) {
+    if (!ep.lora_b && fused_step_polls(g, ep) && c->arrive_used + (size_t)g.n_tiles <= ARRIVE_WORDS) {
         arrive = c->gemm_arrive + c->arrive_used;
         c->arrive_used += (size_t)g.n_tiles;
     }
@@ -507,6 +529,11 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         c->stamp_kinds.clear();
         CUDA_TRY(cudaMemsetAsync(c->stamp_buf, 0xFF, sizeof(unsigned long long) * ST_WORDS * STAMP_CAP, st));
     }
+    auto with_lora = [&](Epilogue& e, const Layer& L, int mat) {            // the adapters of this matrix, if the model has any
+        if (!M.lora) return;
+        e.lora_b = L.lora_b[mat]; e.lora_task = c->S.draft_id; e.lora_r = c->cfg.lora_rank; e.lora_n = c->cfg.lora_adapters;
+        e.lora_scale = c->cfg.lora_scale; e.row_slot = c->row_slot;
+    };
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -521,6 +548,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.mode = EPI_QKV_ROPE; e.rs = l == 0 ? first : tiled;
         e.q_out = (bf16*)c->q; e.kc = (bf16*)kc; e.vc = (bf16*)vc; e.row_slot = c->row_slot; e.row_pos = c->row_pos;
         e.H = H; e.Hkv = Hkv; e.hd = hd; e.max_ctx = c->cfg.max_ctx; e.rcos = c->rope_row_cos; e.rsin = c->rope_row_sin;
+        with_lora(e, L, SD_LORA_QKV);
         SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
                                                      hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st, lo,
@@ -529,15 +557,18 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.lo_off = lo; e.m_real = n_rows;
         e.ring_stages = c->tune[SD_TUNE_WO_STAGES]; e.prefill_all = c->tune[SD_TUNE_WO_PREFILL_ALL];
         e.mode = EPI_RESIDUAL; e.h = c->h; e.gain_next = L.norm2; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
+        with_lora(e, L, SD_LORA_WO);
         SD_TRY(gemm_tc(c, L.tm_wo, c->attn, n_rows, d, H * hd, e));
         memset(&e, 0, sizeof(e));
         e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_SWIGLU; e.rs = tiled; e.act = (bf16*)c->act; e.F = F;
+        with_lora(e, L, SD_LORA_GU);
         SD_TRY(gemm_tc(c, L.tm_gu, c->xn, n_rows, 2 * F, d, e));
         memset(&e, 0, sizeof(e));
         e.lo_off = lo; e.m_real = n_rows;
         e.mode = EPI_RESIDUAL; e.h = c->h; e.xn = (bf16*)c->xn; e.ssq_out = c->ssq;
         e.gain_next = l + 1 < m.n_layers ? M.layers[l + 1].norm1 : (mode != LOGITS_NONE ? M.final_norm : nullptr);
+        with_lora(e, L, SD_LORA_WD);
         SD_TRY(gemm_tc(c, L.tm_wd, c->act, n_rows, d, F, e));
     }
     if (mode != LOGITS_NONE) {
@@ -791,19 +822,31 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
         M.pass_ok = false;
         M.tc = m.dtype == SD_BF16 && (m.head_dim == 64 || m.head_dim == 128) && m.d_model <= 128 * SSQ_STRIDE && m.d_ffn % 64 == 0 &&
                attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim);
+        if (!M.tc && M.lora) return fail(SD_ERR_UNSUPPORTED);
         if (!M.tc) continue;
         const int dq = m.n_heads * m.head_dim;
+        const int extra = M.lora ? 128 : 0;
         bool ok = make_tensor_map_bf16(&M.tm_lm, M.lm_head, m.vocab, m.d_model, 128);
         for (Layer& L : M.layers) {
-            ok = ok && make_tensor_map_bf16(&L.tm_qkv, L.wqkv, M.n_qkv(), m.d_model, 128);
-            ok = ok && make_tensor_map_bf16(&L.tm_wo, L.wo, m.d_model, dq, 128);
-            ok = ok && make_tensor_map_bf16(&L.tm_gu, L.wgu, 2 * m.d_ffn, m.d_model, 128);
-            ok = ok && make_tensor_map_bf16(&L.tm_wd, L.wd, m.d_model, m.d_ffn, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_qkv, L.wqkv, M.n_qkv() + extra, m.d_model, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_wo, L.wo, m.d_model + extra, dq, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_gu, L.wgu, 2 * m.d_ffn + extra, m.d_model, 128);
+            ok = ok && make_tensor_map_bf16(&L.tm_wd, L.wd, m.d_model + extra, m.d_ffn, 128);
+            if (M.lora) {                                    // adapters start at zero: the base draft
+                const size_t n_lb = (size_t)cfg->lora_adapters * cfg->lora_rank * sizeof(bf16);
+                const size_t outs[4] = {(size_t)M.n_qkv(), (size_t)m.d_model, (size_t)2 * m.d_ffn, (size_t)m.d_model};
+                const size_t ins[4] = {(size_t)m.d_model, (size_t)dq, (size_t)m.d_model, (size_t)m.d_ffn};
+                void* mats[4] = {L.wqkv, L.wo, L.wgu, L.wd};
+                for (int k = 0; k < 4; ++k) {
+                    ok = ok && cudaMemsetAsync(L.lora_b[k], 0, n_lb * outs[k], st) == cudaSuccess;
+                    ok = ok && cudaMemsetAsync((char*)mats[k] + outs[k] * ins[k] * M.esz, 0, 128 * ins[k] * M.esz, st) == cudaSuccess;
+                }
+            }
         }
-        if (!ok) return fail(SD_ERR_CUDA);
+        if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
         // the persistent streaming kernel sees the layers of a matrix as one [layer][row][k] tensor
         const size_t stride = m.n_layers > 1 ? (size_t)((char*)M.layers[1].wqkv - (char*)M.layers[0].wqkv) : 0;
-        M.pass_ok = m.d_model % 64 == 0 && dq % 64 == 0 && m.d_ffn % 64 == 0 &&
+        M.pass_ok = !M.lora && m.d_model % 64 == 0 && dq % 64 == 0 && m.d_ffn % 64 == 0 &&
                     make_tensor_map_layers(&M.pmaps.m[MAT_QKV], M.layers[0].wqkv, M.n_qkv(), m.d_model, m.n_layers, stride) &&
                     make_tensor_map_layers(&M.pmaps.m[MAT_WO], M.layers[0].wo, m.d_model, dq, m.n_layers, stride) &&
                     make_tensor_map_layers(&M.pmaps.m[MAT_GU], M.layers[0].wgu, 2 * m.d_ffn, m.d_model, m.n_layers, stride) &&
@@ -865,6 +908,34 @@ sd_status sd_load_tensor(sd_ctx* c, int model_id, int kind, int layer, const voi
     }
     CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->st));
     if (!on_dev) CUDA_TRY(cudaStreamSynchronize(c->st));     // the host buffer may go away after the call
+    return SD_OK;
+}
+
+sd_status sd_load_lora(sd_ctx* c, int adapter, int layer, int mat, const void* a, const void* b, int on_dev) {
+    if (!c || !a || !b || mat < 0 || mat > 3) return SD_ERR_INVALID_ARG;
+    if (c->cfg.lora_adapters < 1) return SD_ERR_STATE;
+    Model& M = c->models[1];
+    const sd_model_desc& m = M.d;
+    if (adapter < 0 || adapter >= c->cfg.lora_adapters || layer < 0 || layer >= m.n_layers) return SD_ERR_INVALID_ARG;
+    Layer& L = M.layers[layer];
+    const size_t dq = (size_t)m.n_heads * m.head_dim, r = c->cfg.lora_rank, F = m.d_ffn;
+    const size_t outs[4] = {(size_t)M.n_qkv(), (size_t)m.d_model, 2 * F, (size_t)m.d_model};
+    const size_t ins[4] = {(size_t)m.d_model, dq, (size_t)m.d_model, F};
+    void* mats[4] = {L.wqkv, L.wo, L.wgu, L.wd};
+    const cudaMemcpyKind kd = on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    // A: rows adapter * r ... of the tile that follows the matrix's own rows
+    char* a_dst = (char*)mats[mat] + (outs[mat] + (size_t)adapter * r) * ins[mat] * sizeof(bf16);
+    CUDA_TRY(cudaMemcpyAsync(a_dst, a, r * ins[mat] * sizeof(bf16), kd, c->st));
+    // B: in the order of the GEMM's output features (gate / up rows interleaved in 64-row halves of a tile, as the weights are)
+    bf16* b_dst = L.lora_b[mat] + (size_t)adapter * outs[mat] * r;
+    if (mat == SD_LORA_GU) {
+        const size_t chunk = 64 * r * sizeof(bf16);
+        CUDA_TRY(cudaMemcpy2DAsync(b_dst, 2 * chunk, b, chunk, chunk, F / 64, kd, c->st));                                   // gate rows
+        CUDA_TRY(cudaMemcpy2DAsync((char*)b_dst + chunk, 2 * chunk, (const char*)b + F * r * sizeof(bf16), chunk, chunk, F / 64, kd, c->st));   // up rows
+    } else {
+        CUDA_TRY(cudaMemcpyAsync(b_dst, b, outs[mat] * r * sizeof(bf16), kd, c->st));
+    }
+    CUDA_TRY(cudaStreamSynchronize(c->st));
     return SD_OK;
 }
 
@@ -957,7 +1028,7 @@ sd_status sd_prefill(sd_ctx* c, const int32_t* seqs, int n_seq) {
         one.n = 1; one.ids[0] = s; one.out[0] = 0;
         for (int pass = 0; pass < 2; ++pass) {
             if (pass == 1 && c->cfg.n_drafts < 1) break;
-            Model& M = c->models[pass == 0 ? 0 : 1 + c->draft_id[s]];
+            Model& M = c->models[pass == 0 ? 0 : draft_model_index(c->cfg, c->draft_id[s])];
             for (int p0 = 0; p0 < n; p0 += SD_MAX_ROWS) {
                 const int rows = std::min(SD_MAX_ROWS, n - p0);
                 RowPlan plan{PLAN_PREFILL, rows, p0, 0, 0, nullptr, p0 + rows};
@@ -990,9 +1061,12 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
     bound = bound_bucket(bound + gamma) - gamma;
     CostScope cost(c, 0, gamma);
-    for (int k = 0; k < c->cfg.n_drafts; ++k) {             // programs of the persistent kernel exist before anything is captured
+    // with low-rank adapters every task runs on the one base draft: a single group, adapters picked row by row
+    const bool shared = c->cfg.lora_adapters > 0;
+    const int n_groups = shared ? 1 : c->cfg.n_drafts;
+    for (int k = 0; k < n_groups; ++k) {                    // programs of the persistent kernel exist before anything is captured
         int n = 0;
-        for (int i = 0; i < n_seq; ++i) n += c->draft_id[seqs[i]] == k;
+        for (int i = 0; i < n_seq; ++i) n += shared || c->draft_id[seqs[i]] == k;
         if (n == 0) continue;
         for (int s = 0; s < gamma; ++s) {
             if (s == 0) { RowPlan plan{PLAN_DRAFT_FIRST, 2, 0, 0, gamma, x_in, bound}; SD_TRY(prepare_pass(c, 1 + k, plan, 2 * n, LOGITS_LAST)); }
@@ -1000,11 +1074,11 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
         }
     }
     return run_graphed(c, key, [&]() -> sd_status {
-    for (int k = 0; k < c->cfg.n_drafts; ++k) {             // sequences grouped per routed draft
+    for (int k = 0; k < n_groups; ++k) {                    // sequences grouped per routed draft
         SeqList g = all;
         g.n = 0;
         for (int i = 0; i < n_seq; ++i)
-            if (c->draft_id[seqs[i]] == k) { g.ids[g.n] = seqs[i]; g.out[g.n] = i; ++g.n; }
+            if (shared || c->draft_id[seqs[i]] == k) { g.ids[g.n] = seqs[i]; g.out[g.n] = i; ++g.n; }
         if (g.n == 0) continue;
         Model& M = c->models[1 + k];
         for (int s = 0; s < gamma; ++s) {

@@ -25,6 +25,7 @@ struct StepShared {
     float scale[MB];                // 1/rms factor of the CTA's token rows
     float val[MB][TILE_N];          // exchange between the rows of the tile (rotary pairs, gate/up pairs)
     float wsum[MB][4];              // per-warp sums of squares
+    float lora_t[MB][32];           // x A^T of the CTA's token rows for their own adapters
 };
 
 // MB token rows x CB pieces are in flight together: (8, 8) for the verify rows, (2, 32) for one or
@@ -138,6 +139,49 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             for (int cc = 0; cc < CB; ++cc)                                   // the pieces are added in the order of their CTAs
 #pragma unroll
                 for (int i = 0; i < MB; ++i) v[i] += tmp[cc][i];
+        }
+    }
+    if (ep.lora_b) {                              // uniform: the low-rank update of this matrix
+        // t = x A^T sits in the GEMM's last tile; its pieces are summed like any tile's, by MB * r threads
+        const uint32_t tx = (uint32_t)g.n_tiles - 1u, xa = tx * KB, xb = xa + KB - 1;
+        const uint32_t x_first = ((xa + 1) * G + T - 1) / T - 1, x_last = ((xb + 1) * G + T - 1) / T - 1;
+        const uint32_t xj_first = tx - ((x_first * T) / G) / KB;
+        const int r = ep.lora_r;
+        for (int p = et; p < MB * r; p += 128) {
+            const int i = p / r, j = p % r;
+            float t = 0.f;
+            if (rows[i] >= 0) {
+                const int task = __ldcg(ep.lora_task + __ldcg(ep.row_slot + rows[i]));
+                if (task >= 0 && task < ep.lora_n) {
+                    for (uint32_t c = x_first; c <= x_last; ++c) {
+                        const uint32_t jj = c == x_first ? xj_first : 0u;
+                        t += __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)rows[i] * TILE_N + task * r + j);
+                    }
+                }
+            }
+            sh.lora_t[i][j] = t;
+        }
+        __syncthreads();
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < MB; ++i) {
+                if (rows[i] < 0) continue;
+                const int task = __ldcg(ep.lora_task + __ldcg(ep.row_slot + rows[i]));
+                if (task < 0 || task >= ep.lora_n) continue;
+                const bf16* b = ep.lora_b + ((size_t)task * g.n_out + n) * r;
+                float acc = 0.f;
+                for (int j = 0; j < r; j += 8) {                 // r is a multiple of 8: 16-byte pieces of the row of B
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(b + j));
+                    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __bfloat1622float2(h2[e]);
+                        acc = fmaf(sh.lora_t[i][j + 2 * e], f.x, acc);
+                        acc = fmaf(sh.lora_t[i][j + 2 * e + 1], f.y, acc);
+                    }
+                }
+                v[i] = fmaf(ep.lora_scale, acc, v[i]);
+            }
         }
     }
     if (ep.rs.ssq) {
@@ -295,6 +339,12 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     if (ep.mode == EPI_RESIDUAL && g.n_tiles > SSQ_STRIDE) return cudaErrorInvalidValue;
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
     if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
+    if (ep.lora_b) {                                   // the adapter's tile is complete only when the GEMM's grid is
+        if (ep.lora_r < 8 || ep.lora_r > 32 || (ep.lora_r & 7) || ep.lora_n * ep.lora_r > TILE_N || !ep.lora_task || !ep.row_slot ||
+            ep.mode == EPI_PLAIN || g.n_out % TILE_N || g.n_tiles != g.n_out / TILE_N + 1)
+            return cudaErrorInvalidValue;
+        arrive = nullptr;
+    }
     const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
     const int pieces = pieces_bound(g);
     if (ep.lo_off) {                                   // two-part activations: accumulator rows r and r + lo_off belong together

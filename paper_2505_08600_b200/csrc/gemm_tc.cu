@@ -289,14 +289,14 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages, bool prefill_all) {
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages, bool prefill_all, int extra_tiles) {
     GemmGeom g;
     g.lo_off = 0; g.m_real = m_tok; g.stamp = nullptr; g.pace_ns = 0;
     g.m_tok = m_tok;
     g.m_pad = (m_tok + 15) & ~15;
     g.n_out = n_out;
     g.K = K;
-    g.n_tiles = (n_out + TILE_N - 1) / TILE_N;
+    g.n_tiles = (n_out + TILE_N - 1) / TILE_N + extra_tiles;
     g.kb_per_tile = (K + TILE_K - 1) / TILE_K;
     const long long T = (long long)g.n_tiles * g.kb_per_tile;
     g.grid = (int)std::min<long long>(n_sm, T);

@@ -45,6 +45,13 @@ struct Epilogue {
     // the rows this step writes for the next GEMM are split the same way.  m_real = token rows (the GEMM saw lo_off + m_real).
     int lo_off, m_real;
     unsigned long long* stamp;       // optional time stamps of the step's launch (see LaunchStamp)
+    // Low-rank adapters (nullptr: none).  The GEMM's last output tile holds x A^T for every adapter (adapter a in its
+    // columns a * r ... a * r + r - 1); row i uses the adapter of its sequence, lora_task[row_slot[i]], and the step adds
+    // lora_scale * sum_j t[i][j] * lora_b[adapter][n][j] to output feature n before anything else.
+    const bf16* lora_b;              // [adapters][n_out][r], rows in the order of the GEMM's output features
+    const int32_t* lora_task;        // [slot]
+    int lora_r, lora_n;              // rank, adapters
+    float lora_scale;
     int ring_stages, prefill_all;    // GEMM before this step: cap on its stage ring (0: none) / request the whole ring before the dependency
     unsigned long long poll_ns;      // how long a tile's CTA watches its arrival word before it falls back to the grid dependency (0: 0.2 s)
     RowScale rs;                     // PLAIN, QKV_ROPE, SWIGLU: 1/rms factor of each token row
@@ -63,7 +70,8 @@ struct Epilogue {
 bool gemm_tc_supported(int m_tok, int n_out, int K);
 // max_stages > 0 caps the ring (a smaller ring leaves shared memory for CTAs of the kernel before, e.g. attention, so that
 // this GEMM's CTAs are resident and streaming while that kernel still runs); prefill_all: request the whole ring early.
-GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages = 0, bool prefill_all = false);
+// extra_tiles: 128-row tiles appended after the matrix's own (rounded up to whole tiles): rows of a low-rank adapter.
+GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages = 0, bool prefill_all = false, int extra_tiles = 0);
 size_t gemm_partials_bytes(const GemmGeom& g);
 bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int box_rows);
 // The GEMM proper: leaves the split accumulators in `partials` (gemm_partials_bytes()).

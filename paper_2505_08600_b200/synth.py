@@ -172,3 +172,17 @@ def make_mamba_classifier(vocab, d_model=128, d_state=16, d_conv=4, expand=2, n_
         w_out=n((d_model, Di), Di ** -0.5),
         w_fc=n((n_classes, d_model), 1.0), b_fc=n((n_classes,), 0.01),
     )
+
+
+def make_lora(dims, rank, task, seed=0, std=0.05, dtype="bf16"):
+    """One task's low-rank adapter for every layer of a draft: dict "qkv" / "wo" / "gu" / "wd" -> list over layers of
+    (A [rank][in], B [out][rank]), N(0, std) entries (with alpha / r = 2 and rank 16 the update B A has about the spread
+    of the N(0, 0.02) base weights, so tasks differ visibly), bf16 bit patterns unless dtype == 'f32'."""
+    d, F = dims["d_model"], dims["d_ffn"]
+    dq, dkv = dims["n_heads"] * dims["head_dim"], dims["n_kv_heads"] * dims["head_dim"]
+    shapes = {"qkv": (dq + 2 * dkv, d), "wo": (d, dq), "gu": (2 * F, d), "wd": (d, F)}
+    out = {}
+    for i, (name, (n_out, n_in)) in enumerate(shapes.items()):
+        out[name] = [(_normal((rank, n_in), seed, 600000 + task * 10000 + l * 16 + 2 * i, std, dtype),
+                      _normal((n_out, rank), seed, 600000 + task * 10000 + l * 16 + 2 * i + 1, std, dtype)) for l in range(dims["n_layers"])]
+    return out
