@@ -188,10 +188,24 @@ def setup(args, gamma_max, steps_per_phase):
         lens = [min(n, wl["max_ctx"] - need) for n in lens]          # the timed steps end at the config's cache size
     max_ctx = max(wl["max_ctx"], max(lens) + need)
 
-    ctx = sd.Context(tdims, cfg["drafts"], cfg["dtype"], B, max_ctx, max(gamma_max, 1), T, seed, clf_d_hidden=cfg["classifier"][1], device=dev)
-    for mid, dims in enumerate([tdims] + list(cfg["drafts"])):
+    lora = getattr(args, "lora", False)
+    drafts = [cfg["drafts"][0]] if lora else list(cfg["drafts"])       # --lora: one base draft + one rank-16 adapter per task
+    ctx = sd.Context(tdims, drafts, cfg["dtype"], B, max_ctx, max(gamma_max, 1), T, seed, clf_d_hidden=cfg["classifier"][1], device=dev,
+                     lora_adapters=len(cfg["drafts"]) if lora else 0, lora_rank=16 if lora else 0, lora_scale=2.0 if lora else 0.0)
+    for mid, dims in enumerate([tdims] + drafts):
         for name, l, tensor in device_weights(torch, dims, cfg["dtype"], 0, mid, dev):
             ctx.sd_load_tensor(mid, sd.TENSOR_KIND[name], l, tensor)
+    if lora:
+        dd = drafts[0]
+        dq, dkv = dd["n_heads"] * dd["head_dim"], dd["n_kv_heads"] * dd["head_dim"]
+        shapes = [(dq + 2 * dkv, dd["d_model"]), (dd["d_model"], dq), (2 * dd["d_ffn"], dd["d_model"]), (dd["d_model"], dd["d_ffn"])]
+        g = torch.Generator(device=dev); g.manual_seed(77)
+        for task in range(len(cfg["drafts"])):
+            for l in range(dd["n_layers"]):
+                for mat, (n_out, n_in) in enumerate(shapes):
+                    a = (torch.randn((16, n_in), generator=g, device=dev) * 0.05).to(torch.bfloat16).contiguous()
+                    b = (torch.randn((n_out, 16), generator=g, device=dev) * 0.05).to(torch.bfloat16).contiguous()
+                    ctx.sd_load_lora(task, l, mat, a, b)
     clf = synth.make_classifier(*cfg["classifier"], seed=0)
     ctx.sd_load_classifier(clf["w1"], clf["b1"], clf["w2"], clf["b2"])
     torch.cuda.synchronize()
@@ -411,7 +425,7 @@ def run_gpu(args):
               "verify_over_decode": ms_step / decode_ms,
               "eq1_speedup": {f"alpha={a}": eq1_speedup(a, gamma, c) for a in (0.6, 0.8)},
               "best_gamma": {f"alpha={a}": dict(zip(("gamma", "speedup"), sd.sd_best_gamma(a, c, 15))) for a in (0.6, 0.8)},
-              "routed_drafts": [int(r) for r in routed]}
+              "routed_drafts": [int(r) for r in routed], "drafts": "one base draft + low-rank adapters (rank 16)" if getattr(args, "lora", False) else "separate models"}
     status = ctx.sd_device_status()
 
     cpu = None
@@ -642,6 +656,7 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
+    ap.add_argument("--lora", action="store_true", help="drafts = one base draft + one low-rank adapter per task (sequences of all tasks share each draft pass)")
     ap.add_argument("--mamba", action="store_true", help="time the Mamba-based prompt classifier on 400 synthetic prompts and exit")
     ap.add_argument("--kmeans", action="store_true", help="time one K-means step over synthetic sentence vectors and exit")
     args = ap.parse_args()

@@ -281,9 +281,13 @@ class Context:
 
     # ---- loading
     def sd_load_lora(self, adapter, layer, mat, a, b):
-        """a [r][in], b [out][r]: numpy uint16 arrays of bf16 bit patterns."""
-        a = np.ascontiguousarray(a, dtype=np.uint16); b = np.ascontiguousarray(b, dtype=np.uint16)
-        _check(self.L.sd_load_lora(self.h, int(adapter), int(layer), int(mat), a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p), 0), "sd_load_lora")
+        """a [r][in], b [out][r]: numpy uint16 arrays of bf16 bit patterns, or contiguous torch.bfloat16 CUDA tensors."""
+        if isinstance(a, np.ndarray):
+            a = np.ascontiguousarray(a, dtype=np.uint16); b = np.ascontiguousarray(b, dtype=np.uint16)
+            pa, pb, dev = a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p), 0
+        else:
+            pa, pb, dev = _dp(a), _dp(b), 1
+        _check(self.L.sd_load_lora(self.h, int(adapter), int(layer), int(mat), pa, pb, dev), "sd_load_lora")
 
     def sd_load_tensor(self, model_id, kind, layer, src):
         """src: numpy array (host) or torch CUDA tensor, already in the model's dtype
