@@ -237,7 +237,7 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->act = B.take(4 * R * f_max);
     c->lin = (float*)B.take(sizeof(float) * R * lin_max);
     c->draft_logits = (float*)B.take(sizeof(float) * (size_t)SD_MAX_BATCH * ms[0].vocab);
-    c->row_slot = (int32_t*)B.take(sizeof(int32_t) * R);
+    c->row_slot = (int32_t*)B.take(sizeof(int32_t) * 2 * R);          // [row] slot, then [row] task of the slot (draft / adapter id)
     c->row_pos = (int32_t*)B.take(sizeof(int32_t) * R);
     c->attn_ws_bytes = 0;
     for (int i = 0; i < nm; ++i)
@@ -531,7 +531,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     }
     auto with_lora = [&](Epilogue& e, const Layer& L, int mat) {            // the adapters of this matrix, if the model has any
         if (!M.lora) return;
-        e.lora_b = L.lora_b[mat]; e.lora_task = c->S.draft_id; e.lora_r = c->cfg.lora_rank; e.lora_n = c->cfg.lora_adapters;
+        e.lora_b = L.lora_b[mat]; e.lora_task = c->row_slot + SD_MAX_ROWS; e.lora_r = c->cfg.lora_rank; e.lora_n = c->cfg.lora_adapters;
         e.lora_scale = c->cfg.lora_scale; e.row_slot = c->row_slot;
     };
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)

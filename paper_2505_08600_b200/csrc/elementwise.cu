@@ -37,7 +37,7 @@ __global__ void k_embed(SeqState S, SeqList list, RowPlan plan, const T* __restr
     }
     if (pos >= S.max_ctx) { if (threadIdx.x == 0) atomicOr(S.status, SD_DEV_BAD_POS); pos = -1; }
     if (tok < 0 || tok >= vocab) { if (threadIdx.x == 0) atomicOr(S.status, SD_DEV_BAD_TOKEN); tok = 0; }
-    if (threadIdx.x == 0) { row_slot[r] = slot; row_pos[r] = pos; }
+    if (threadIdx.x == 0) { row_slot[r] = slot; row_pos[r] = pos; row_slot[SD_MAX_ROWS + r] = S.draft_id[slot]; }      // (the row's task follows the slots)
     if (row_cos)                         // the row's rotary factors, so that the step after the QKV GEMM needs no dependent lookup
         for (int k = threadIdx.x; k < half; k += blockDim.x) {
             row_cos[(size_t)r * half + k] = pos >= 0 ? rcos[(size_t)pos * half + k] : 1.f;

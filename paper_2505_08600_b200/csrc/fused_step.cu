@@ -75,6 +75,21 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             sn[i] = (ok && rot) ? __ldcg(ep.rsin + (size_t)rows[i] * half + e) : 0.f;
         }
     }
+    int task[MB];                                 // the rows' adapters (part of the row plan: no wait needed)
+    uint4 braw[MB <= 2 ? MB : 1][MB <= 2 ? 4 : 1];  // one or two rows: their rows of B are requested before the wait as well
+    if (ep.lora_b) {
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            task[i] = rows[i] >= 0 ? __ldcg(ep.lora_task + rows[i]) : -1;
+            if (task[i] >= ep.lora_n) task[i] = -1;
+            if (MB <= 2 && live && task[i] >= 0) {
+                const bf16* b = ep.lora_b + ((size_t)task[i] * g.n_out + n) * ep.lora_r;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj)
+                    if (jj * 8 < ep.lora_r) braw[MB <= 2 ? i : 0][MB <= 2 ? jj : 0] = __ldg(reinterpret_cast<const uint4*>(b + jj * 8));
+            }
+        }
+    }
     // The pieces come from the GEMM before (the rows' sums of squares from kernels further back, long finished).
     // With arrival words the CTA starts as soon as its own tile is complete; otherwise when the GEMM's grid has retired.
     if (arrive) {
@@ -151,11 +166,11 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
             const int i = p / r, j = p % r;
             float t = 0.f;
             if (rows[i] >= 0) {
-                const int task = __ldcg(ep.lora_task + __ldcg(ep.row_slot + rows[i]));
-                if (task >= 0 && task < ep.lora_n) {
+                const int tk = __ldcg(ep.lora_task + rows[i]);
+                if (tk >= 0 && tk < ep.lora_n) {
                     for (uint32_t c = x_first; c <= x_last; ++c) {
                         const uint32_t jj = c == x_first ? xj_first : 0u;
-                        t += __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)rows[i] * TILE_N + task * r + j);
+                        t += __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)rows[i] * TILE_N + tk * r + j);
                     }
                 }
             }
@@ -165,13 +180,14 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         if (live) {
 #pragma unroll
             for (int i = 0; i < MB; ++i) {
-                if (rows[i] < 0) continue;
-                const int task = __ldcg(ep.lora_task + __ldcg(ep.row_slot + rows[i]));
-                if (task < 0 || task >= ep.lora_n) continue;
-                const bf16* b = ep.lora_b + ((size_t)task * g.n_out + n) * r;
+                if (rows[i] < 0 || task[i] < 0) continue;
+                const bf16* b = ep.lora_b + ((size_t)task[i] * g.n_out + n) * r;
                 float acc = 0.f;
-                for (int j = 0; j < r; j += 8) {                 // r is a multiple of 8: 16-byte pieces of the row of B
-                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(b + j));
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {                 // r is a multiple of 8, at most 32: 16-byte pieces of the row of B
+                    const int j = jj * 8;
+                    if (j >= r) break;
+                    const uint4 raw = MB <= 2 ? braw[MB <= 2 ? i : 0][MB <= 2 ? jj : 0] : __ldg(reinterpret_cast<const uint4*>(b + j));
                     const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -340,7 +356,7 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
     if (ep.mode == EPI_SWIGLU && (ep.F % 64)) return cudaErrorInvalidValue;
     if (ep.rs.ssq && ep.rs.n_parts > 64) return cudaErrorInvalidValue;
     if (ep.lora_b) {                                   // the adapter's tile is complete only when the GEMM's grid is
-        if (ep.lora_r < 8 || ep.lora_r > 32 || (ep.lora_r & 7) || ep.lora_n * ep.lora_r > TILE_N || !ep.lora_task || !ep.row_slot ||
+        if (ep.lora_r < 8 || ep.lora_r > 32 || (ep.lora_r & 7) || ep.lora_n * ep.lora_r > TILE_N || !ep.lora_task ||
             ep.mode == EPI_PLAIN || g.n_out % TILE_N || g.n_tiles != g.n_out / TILE_N + 1)
             return cudaErrorInvalidValue;
         arrive = nullptr;

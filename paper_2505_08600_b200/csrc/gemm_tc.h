@@ -46,10 +46,10 @@ struct Epilogue {
     int lo_off, m_real;
     unsigned long long* stamp;       // optional time stamps of the step's launch (see LaunchStamp)
     // Low-rank adapters (nullptr: none).  The GEMM's last output tile holds x A^T for every adapter (adapter a in its
-    // columns a * r ... a * r + r - 1); row i uses the adapter of its sequence, lora_task[row_slot[i]], and the step adds
+    // columns a * r ... a * r + r - 1); row i uses the adapter of its sequence, lora_task[i], and the step adds
     // lora_scale * sum_j t[i][j] * lora_b[adapter][n][j] to output feature n before anything else.
     const bf16* lora_b;              // [adapters][n_out][r], rows in the order of the GEMM's output features
-    const int32_t* lora_task;        // [slot]
+    const int32_t* lora_task;        // [row], written with the row plan by the pass's first kernel
     int lora_r, lora_n;              // rank, adapters
     float lora_scale;
     int ring_stages, prefill_all;    // GEMM before this step: cap on its stage ring (0: none) / request the whole ring before the dependency

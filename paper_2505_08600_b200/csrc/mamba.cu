@@ -65,42 +65,61 @@ k_mamba_in(MambaDims m, const int32_t* __restrict__ tokens, const int64_t* __res
     }
 }
 
-// Per token: causal depthwise convolution + SiLU, the projections to (r, B, C), the step size.
-__global__ void k_mamba_conv_proj(MambaDims m, int T, const int32_t* __restrict__ tok_pos /*position inside its prompt*/,
-                                  const float* __restrict__ u, const float* __restrict__ w_conv, const float* __restrict__ b_conv,
-                                  const float* __restrict__ w_x, const float* __restrict__ w_dt, const float* __restrict__ b_dt,
-                                  float* __restrict__ v, float* __restrict__ dt, float* __restrict__ bc) {
-    extern __shared__ float sm[];                        // v [Di], x_dbl [R + 2N]
+// Per tile of MB_CP_TILE tokens: causal depthwise convolution + SiLU, the projections to (r, B, C), the step size.
+// A tile shares every weight it reads (each row of W_x is read once per tile and used for all its tokens).
+constexpr int MB_CP_TILE = 8;
+__global__ void __launch_bounds__(256)
+k_mamba_conv_proj(MambaDims m, int T, const int32_t* __restrict__ tok_pos /*position inside its prompt*/,
+                  const float* __restrict__ u, const float* __restrict__ w_conv, const float* __restrict__ b_conv,
+                  const float* __restrict__ w_x, const float* __restrict__ w_dt, const float* __restrict__ b_dt,
+                  float* __restrict__ v, float* __restrict__ dt, float* __restrict__ bc) {
+    extern __shared__ float sm[];                        // v [tile][Di], x_dbl [tile][R + 2N]
+    const int n_x = m.R + 2 * m.N;
     float* v_s = sm;
-    float* xd_s = sm + m.Di;
-    const int t = blockIdx.x, pos = tok_pos[t];
-    for (int c = threadIdx.x; c < m.Di; c += blockDim.x) {
-        float acc = b_conv[c];
-        for (int j = 0; j < m.Kc; ++j) {
-            const int back = m.Kc - 1 - j;               // tap j looks `back` tokens back; nothing before the prompt's first token
-            if (back <= pos) acc = fmaf(w_conv[(size_t)c * m.Kc + j], u[(size_t)(t - back) * m.Di + c], acc);
+    float* xd_s = sm + MB_CP_TILE * m.Di;
+    const int t0 = blockIdx.x * MB_CP_TILE, nt = min(MB_CP_TILE, T - t0);
+    for (int idx = threadIdx.x; idx < MB_CP_TILE * m.Di; idx += blockDim.x) {
+        const int tt = idx / m.Di, c = idx % m.Di;
+        float val = 0.f;
+        if (tt < nt) {
+            const int t = t0 + tt, pos = tok_pos[t];
+            float acc = b_conv[c];
+            for (int j = 0; j < m.Kc; ++j) {
+                const int back = m.Kc - 1 - j;           // tap j looks `back` tokens back; nothing before the prompt's first token
+                if (back <= pos) acc = fmaf(w_conv[(size_t)c * m.Kc + j], u[(size_t)(t - back) * m.Di + c], acc);
+            }
+            val = silu_f(acc);
+            v[(size_t)t * m.Di + c] = val;
         }
-        const float val = silu_f(acc);
-        v_s[c] = val;
-        v[(size_t)t * m.Di + c] = val;
+        v_s[idx] = val;
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5, n_x = m.R + 2 * m.N;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     for (int o = warp; o < n_x; o += n_warps) {
-        float acc = 0.f;
-        for (int c = lane; c < m.Di; c += 32) acc = fmaf(w_x[(size_t)o * m.Di + c], v_s[c], acc);
+        float acc[MB_CP_TILE];
 #pragma unroll
-        for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-        if (lane == 0) {
-            xd_s[o] = acc;
-            if (o >= m.R) bc[(size_t)t * 2 * m.N + (o - m.R)] = acc;
+        for (int tt = 0; tt < MB_CP_TILE; ++tt) acc[tt] = 0.f;
+        for (int c = lane; c < m.Di; c += 32) {
+            const float w = w_x[(size_t)o * m.Di + c];
+#pragma unroll
+            for (int tt = 0; tt < MB_CP_TILE; ++tt) acc[tt] = fmaf(w, v_s[tt * m.Di + c], acc[tt]);
+        }
+#pragma unroll
+        for (int tt = 0; tt < MB_CP_TILE; ++tt) {
+#pragma unroll
+            for (int s = 16; s > 0; s >>= 1) acc[tt] += __shfl_xor_sync(0xffffffffu, acc[tt], s);
+            if (lane == 0 && tt < nt) {
+                xd_s[tt * n_x + o] = acc[tt];
+                if (o >= m.R) bc[(size_t)(t0 + tt) * 2 * m.N + (o - m.R)] = acc[tt];
+            }
         }
     }
     __syncthreads();
-    for (int c = threadIdx.x; c < m.Di; c += blockDim.x) {
+    for (int idx = threadIdx.x; idx < nt * m.Di; idx += blockDim.x) {
+        const int tt = idx / m.Di, c = idx % m.Di;
         float acc = b_dt[c];
-        for (int r = 0; r < m.R; ++r) acc = fmaf(w_dt[(size_t)c * m.R + r], xd_s[r], acc);
-        dt[(size_t)t * m.Di + c] = softplus_f(acc);
+        for (int r = 0; r < m.R; ++r) acc = fmaf(w_dt[(size_t)c * m.R + r], xd_s[tt * n_x + r], acc);
+        dt[(size_t)(t0 + tt) * m.Di + c] = softplus_f(acc);
     }
 }
 
@@ -292,8 +311,7 @@ extern "C" sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba
 
     k_mamba_in<<<(unsigned)((T + MB_TOK_TILE - 1) / MB_TOK_TILE), 256, (size_t)MB_TOK_TILE * m.D * 4, st>>>(
         m, tokens_dev, (const int64_t*)(base + L.tok_src), (int)T, w->embed, w->w_in, u, z);
-    const int conv_threads = m.Di >= 256 ? 256 : ((m.Di + 31) / 32) * 32;
-    k_mamba_conv_proj<<<(unsigned)T, conv_threads, (size_t)(m.Di + m.R + 2 * m.N) * 4, st>>>(
+    k_mamba_conv_proj<<<(unsigned)((T + MB_CP_TILE - 1) / MB_CP_TILE), 256, (size_t)MB_CP_TILE * (m.Di + m.R + 2 * m.N) * 4, st>>>(
         m, (int)T, (const int32_t*)(base + L.tok_pos), u, w->w_conv, w->b_conv, w->w_x, w->w_dt, w->b_dt, v, dt, bc);
     const dim3 sgrid((unsigned)n_chunks, (unsigned)((m.Di + 63) / 64));
     const float* start = nullptr;
