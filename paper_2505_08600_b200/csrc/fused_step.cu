@@ -32,7 +32,7 @@ struct StepShared {
 // two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) or (16, 2)
 // for many rows on few pieces.  MODE < 0: the step is read from ep.mode; with many row batches one
 // instantiation per step is used instead, whose lower register count lets more CTAs be resident.
-template <int MODE, int MB, int CB, bool HL = false>
+template <int MODE, int MB, int CB, bool HL = false, bool LORA = false>      // LORA: the matrix carries low-rank adapters
 __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials,
                                                     uint32_t* __restrict__ arrive, uint32_t* status) {
     __shared__ StepShared<MB> sh;
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     }
     int task[MB];                                 // the rows' adapters (part of the row plan: no wait needed)
     uint4 braw[MB <= 2 ? MB : 1][MB <= 2 ? 4 : 1];  // one or two rows: their rows of B are requested before the wait as well
-    if (ep.lora_b) {
+    if (LORA) {
 #pragma unroll
         for (int i = 0; i < MB; ++i) {
             task[i] = rows[i] >= 0 ? __ldcg(ep.lora_task + rows[i]) : -1;
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
                 for (int i = 0; i < MB; ++i) v[i] += tmp[cc][i];
         }
     }
-    if (ep.lora_b) {                              // uniform: the low-rank update of this matrix
+    if (LORA) {                                   // the low-rank update of this matrix
         // t = x A^T sits in the GEMM's last tile; its pieces are summed like any tile's, by MB * r threads
         const uint32_t tx = (uint32_t)g.n_tiles - 1u, xa = tx * KB, xb = xa + KB - 1;
         const uint32_t x_first = ((xa + 1) * G + T - 1) / T - 1, x_last = ((xb + 1) * G + T - 1) / T - 1;
@@ -295,12 +295,12 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     if (et == 0) stamp_pair(ep.stamp, ST_DONE_FIRST);
 }
 
-template <int MODE, bool HL>
+template <int MODE, bool HL, bool LORA>
 cudaError_t launch_many_rows(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status, int n_rows,
                              int pieces, int dependent, cudaStream_t st) {
     const dim3 grid(g.n_tiles, (n_rows + 15) / 16);
-    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2, HL>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
-    return launch_pdl(k_fused_step<MODE, 16, 4, HL>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    if (pieces <= 2) return launch_pdl(k_fused_step<MODE, 16, 2, HL, LORA>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    return launch_pdl(k_fused_step<MODE, 16, 4, HL, LORA>, grid, dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
 }  // namespace
@@ -329,20 +329,20 @@ bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
 
 namespace {
 
-template <bool HL>
+template <bool HL, bool LORA>
 cudaError_t launch_step(const GemmGeom& g, const Epilogue& ep, const float* partials, uint32_t* arrive, uint32_t* status, int n_rows, int pieces,
                         int dependent, cudaStream_t st) {
-    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32, HL>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    if (n_rows <= 2) return launch_pdl(k_fused_step<-1, 2, 32, HL, LORA>, dim3(g.n_tiles, 1), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
     if (n_rows > 8 && pieces <= 4) {
         switch (ep.mode) {
-        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
-        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU, HL>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_PLAIN: return launch_many_rows<EPI_PLAIN, HL, LORA>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_QKV_ROPE: return launch_many_rows<EPI_QKV_ROPE, HL, LORA>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_RESIDUAL: return launch_many_rows<EPI_RESIDUAL, HL, LORA>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        case EPI_SWIGLU: return launch_many_rows<EPI_SWIGLU, HL, LORA>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
         default: return cudaErrorInvalidValue;
         }
     }
-    return launch_pdl(k_fused_step<-1, 8, 8, HL>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
+    return launch_pdl(k_fused_step<-1, 8, 8, HL, LORA>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
 }  // namespace
@@ -367,9 +367,11 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
         // (the GEMM's epilogue has already added the two columns of a row: the pieces hold m_real merged rows)
         if (ep.m_real < 1 || ep.m_real > ep.lo_off || ep.m_real + ep.lo_off != g.m_tok || g.lo_off != ep.lo_off || g.m_real != ep.m_real) return cudaErrorInvalidValue;
         if (ep.lo_off != 8 && ep.lo_off != 16) return cudaErrorInvalidValue;
-        return launch_step<true>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+        return ep.lora_b ? launch_step<true, true>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st)
+                         : launch_step<true, false>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
     }
-    return launch_step<false>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
+    return ep.lora_b ? launch_step<false, true>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st)
+                     : launch_step<false, false>(g, ep, partials, arrive, status, n_rows, pieces, dependent, st);
 }
 
 }  // namespace sd
