@@ -1013,7 +1013,7 @@ sd_status sd_route_prompt_mamba(sd_ctx* c, const sd_mamba_desc* desc, const sd_m
     }
     // labels land in the scratch words the accept path uses for its counts (n_seq <= max_seqs of them)
     SD_TRY(sd_mamba_classify(desc, w, c->S.tokens, starts.data(), lens.data(), n_seq, nullptr, c->st_nacc, ws, ws_bytes, c->st));
-    c->launches += 5;
+    c->launches += 6;
     CUDA_TRY(cudaMemcpyAsync(labels.data(), c->st_nacc, sizeof(int32_t) * n_seq, cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
     return sd_route_prompt(c, seqs, n_seq, labels.data(), draft_out);

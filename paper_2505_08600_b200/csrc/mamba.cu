@@ -25,17 +25,31 @@ constexpr int MB_MAX_CONV = 8;
 
 struct MambaDims { int V, D, Di, N, R, Kc, K; };
 
-struct ChunkRec { int32_t prompt, tok0, n_tok, first; };     // tok0: index into the flattened token list; first: 1 for a prompt's first chunk
+struct ChunkRec { int32_t prompt, tok0, n_tok, pos0; };      // tok0: index into the flattened token list; pos0: position of the chunk's first token in its prompt
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplus_f(float x) { return x > 20.f ? x : log1pf(expf(x)); }
 
-// u, z = split(W_in E[token]) for a tile of tokens.  One thread per output feature (strided), the tile's embedding
-// rows in shared memory.
+// Where every flattened token comes from and its position in its prompt, from the chunk records (one CTA per chunk).
+__global__ void k_mamba_tables(const ChunkRec* __restrict__ chunks, const int64_t* __restrict__ starts, int64_t* __restrict__ tok_src,
+                               int32_t* __restrict__ tok_pos) {
+    const ChunkRec ch = chunks[blockIdx.x];
+    for (int i = threadIdx.x; i < ch.n_tok; i += blockDim.x) {
+        tok_src[ch.tok0 + i] = starts[ch.prompt] + ch.pos0 + i;
+        tok_pos[ch.tok0 + i] = ch.pos0 + i;
+    }
+}
+
+// u, z = split(W_in E[token]) for a tile of tokens.  One thread per output feature; the tile's embedding rows sit in
+// shared memory, and W_in passes through shared memory in blocks of 256 rows x 32 columns so that global loads are
+// coalesced (a warp reads 128 contiguous bytes of one row) and every thread then walks its own row without bank
+// conflicts (rows padded to 33 words).
 __global__ void __launch_bounds__(256)
 k_mamba_in(MambaDims m, const int32_t* __restrict__ tokens, const int64_t* __restrict__ tok_src, int T, const float* __restrict__ embed,
            const float* __restrict__ w_in, float* __restrict__ u, float* __restrict__ z) {
-    extern __shared__ float e_s[];                       // [MB_TOK_TILE][D]
+    extern __shared__ float in_smem[];
+    float* e_s = in_smem;                                // [MB_TOK_TILE][D]
+    float* w_s = in_smem + MB_TOK_TILE * m.D;            // [256][33]
     const int t0 = blockIdx.x * MB_TOK_TILE, nt = min(MB_TOK_TILE, T - t0);
     for (int i = threadIdx.x; i < MB_TOK_TILE * m.D; i += blockDim.x) {
         const int tt = i / m.D, d = i % m.D;
@@ -47,21 +61,32 @@ k_mamba_in(MambaDims m, const int32_t* __restrict__ tokens, const int64_t* __res
         }
         e_s[tt * m.D + d] = e;
     }
-    __syncthreads();
-    for (int j = threadIdx.x; j < 2 * m.Di; j += blockDim.x) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int j0 = 0; j0 < 2 * m.Di; j0 += 256) {
+        const int j = j0 + threadIdx.x;
         float acc[MB_TOK_TILE];
 #pragma unroll
         for (int tt = 0; tt < MB_TOK_TILE; ++tt) acc[tt] = 0.f;
-        const float* wr = w_in + (size_t)j * m.D;
-        for (int d = 0; d < m.D; ++d) {
-            const float w = wr[d];
+        for (int d0 = 0; d0 < m.D; d0 += 32) {
+            __syncthreads();                             // the previous block of W (and, the first time, e_s) is settled
+            for (int rr = warp; rr < 256; rr += 8) {     // warp per row: lanes along the row
+                const int row = j0 + rr;
+                w_s[rr * 33 + lane] = (row < 2 * m.Di && d0 + lane < m.D) ? w_in[(size_t)row * m.D + d0 + lane] : 0.f;
+            }
+            __syncthreads();
+            const int nd = min(32, m.D - d0);
+            for (int dd = 0; dd < nd; ++dd) {
+                const float w = w_s[threadIdx.x * 33 + dd];
 #pragma unroll
-            for (int tt = 0; tt < MB_TOK_TILE; ++tt) acc[tt] = fmaf(w, e_s[tt * m.D + d], acc[tt]);
+                for (int tt = 0; tt < MB_TOK_TILE; ++tt) acc[tt] = fmaf(w, e_s[tt * m.D + d0 + dd], acc[tt]);
+            }
         }
-        float* dst = j < m.Di ? u : z;
-        const int c = j < m.Di ? j : j - m.Di;
+        if (j < 2 * m.Di) {
+            float* dst = j < m.Di ? u : z;
+            const int c = j < m.Di ? j : j - m.Di;
 #pragma unroll
-        for (int tt = 0; tt < MB_TOK_TILE; ++tt) if (tt < nt) dst[(size_t)(t0 + tt) * m.Di + c] = acc[tt];
+            for (int tt = 0; tt < MB_TOK_TILE; ++tt) if (tt < nt) dst[(size_t)(t0 + tt) * m.Di + c] = acc[tt];
+        }
     }
 }
 
@@ -231,7 +256,7 @@ bool dims_ok(const sd_mamba_desc* d, MambaDims& m) {
     return true;
 }
 
-struct Layout { size_t u, z, v, dt, bc, end_state, decay, start_state, chunk_sum, tok_src, tok_pos, chunks, prompt_chunk0, lens, total; };
+struct Layout { size_t u, z, v, dt, bc, end_state, decay, start_state, chunk_sum, tok_src, tok_pos, chunks, prompt_chunk0, lens, starts, total; };
 
 Layout layout(const MambaDims& m, int64_t T, int64_t n_chunks, int n_prompts) {
     Layout L;
@@ -244,7 +269,7 @@ Layout layout(const MambaDims& m, int64_t T, int64_t n_chunks, int n_prompts) {
     L.chunk_sum = take((size_t)n_chunks * m.Di * 4);
     L.tok_src = take((size_t)T * 8); L.tok_pos = take((size_t)T * 4);
     L.chunks = take((size_t)n_chunks * sizeof(ChunkRec));
-    L.prompt_chunk0 = take((size_t)(n_prompts + 1) * 4); L.lens = take((size_t)n_prompts * 4);
+    L.prompt_chunk0 = take((size_t)(n_prompts + 1) * 4); L.lens = take((size_t)n_prompts * 4); L.starts = take((size_t)n_prompts * 8);
     L.total = o;
     return L;
 }
@@ -277,20 +302,18 @@ extern "C" sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba
     }
     if (T > (int64_t)1 << 30) return SD_ERR_CAPACITY;
     if (!workspace_dev || workspace_bytes < sd_mamba_workspace(desc, T, n_prompts)) return SD_ERR_CAPACITY;
-    // host tables: where every flattened token comes from, its position in its prompt, the chunks
-    std::vector<int64_t> tok_src((size_t)T);
-    std::vector<int32_t> tok_pos((size_t)T), prompt_chunk0((size_t)n_prompts + 1);
+    // host tables: the chunks of every prompt (the per-token tables are filled on the device from them)
+    std::vector<int32_t> prompt_chunk0((size_t)n_prompts + 1);
     std::vector<ChunkRec> chunks;
     int64_t t = 0;
     int max_len = 0;
     for (int i = 0; i < n_prompts; ++i) {
         prompt_chunk0[i] = (int32_t)chunks.size();
         max_len = lens_host[i] > max_len ? lens_host[i] : max_len;
-        for (int p = 0; p < lens_host[i]; ++p) {
-            if (p % MB_CHUNK == 0) chunks.push_back(ChunkRec{i, (int32_t)t, lens_host[i] - p < MB_CHUNK ? lens_host[i] - p : MB_CHUNK, p == 0});
-            tok_src[(size_t)t] = starts_host[i] + p;
-            tok_pos[(size_t)t] = p;
-            ++t;
+        for (int p = 0; p < lens_host[i]; p += MB_CHUNK) {
+            const int n = lens_host[i] - p < MB_CHUNK ? lens_host[i] - p : MB_CHUNK;
+            chunks.push_back(ChunkRec{i, (int32_t)t, n, p});
+            t += n;
         }
     }
     prompt_chunk0[n_prompts] = (int32_t)chunks.size();
@@ -299,9 +322,8 @@ extern "C" sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba
     char* base = (char*)workspace_dev;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     auto up = [&](size_t at, const void* src, size_t bytes) { return cudaMemcpyAsync(base + at, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess; };
-    if (!up(L.tok_src, tok_src.data(), (size_t)T * 8) || !up(L.tok_pos, tok_pos.data(), (size_t)T * 4) ||
-        !up(L.chunks, chunks.data(), (size_t)n_chunks * sizeof(ChunkRec)) || !up(L.prompt_chunk0, prompt_chunk0.data(), (size_t)(n_prompts + 1) * 4) ||
-        !up(L.lens, lens_host, (size_t)n_prompts * 4))
+    if (!up(L.chunks, chunks.data(), (size_t)n_chunks * sizeof(ChunkRec)) || !up(L.prompt_chunk0, prompt_chunk0.data(), (size_t)(n_prompts + 1) * 4) ||
+        !up(L.lens, lens_host, (size_t)n_prompts * 4) || !up(L.starts, starts_host, (size_t)n_prompts * 8))
         return SD_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SD_ERR_CUDA;      // the host tables above go out of scope
     float* u = (float*)(base + L.u); float* z = (float*)(base + L.z); float* v = (float*)(base + L.v); float* dt = (float*)(base + L.dt);
@@ -309,7 +331,10 @@ extern "C" sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba
     const ChunkRec* chunks_d = (const ChunkRec*)(base + L.chunks);
     const int32_t* pc0 = (const int32_t*)(base + L.prompt_chunk0);
 
-    k_mamba_in<<<(unsigned)((T + MB_TOK_TILE - 1) / MB_TOK_TILE), 256, (size_t)MB_TOK_TILE * m.D * 4, st>>>(
+    k_mamba_tables<<<(unsigned)n_chunks, 64, 0, st>>>(chunks_d, (const int64_t*)(base + L.starts), (int64_t*)(base + L.tok_src), (int32_t*)(base + L.tok_pos));
+    const size_t in_smem_bytes = ((size_t)MB_TOK_TILE * m.D + 256 * 33) * 4;      // up to 66 KB at d_model 512: above the default limit
+    if (cudaFuncSetAttribute(k_mamba_in, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)in_smem_bytes) != cudaSuccess) return SD_ERR_CUDA;
+    k_mamba_in<<<(unsigned)((T + MB_TOK_TILE - 1) / MB_TOK_TILE), 256, in_smem_bytes, st>>>(
         m, tokens_dev, (const int64_t*)(base + L.tok_src), (int)T, w->embed, w->w_in, u, z);
     k_mamba_conv_proj<<<(unsigned)((T + MB_CP_TILE - 1) / MB_CP_TILE), 256, (size_t)MB_CP_TILE * (m.Di + m.R + 2 * m.N) * 4, st>>>(
         m, (int)T, (const int32_t*)(base + L.tok_pos), u, w->w_conv, w->b_conv, w->w_x, w->w_dt, w->b_dt, v, dt, bc);

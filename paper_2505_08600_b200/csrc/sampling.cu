@@ -266,9 +266,18 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
             __syncthreads();
         }
         if (P.alpha_terms && j < gamma) {                       // Eq. 1's alpha for this slot: the draft is kept with probability sum_k min(p, q)
-            const float* qj = q + (size_t)j * V;
+            const float* __restrict__ qj = q + (size_t)j * V;
             float a = 0.f;
-            for (int k = threadIdx.x; k < V; k += blockDim.x) a += fminf(prob(j, li, k), qj[k]);
+            const int stride = blockDim.x;
+            int k = threadIdx.x;
+            for (; k + 3 * stride < V; k += 4 * stride) {             // four independent loads of q in flight per thread
+                const float q0 = __ldg(qj + k), q1 = __ldg(qj + k + stride), q2 = __ldg(qj + k + 2 * stride), q3 = __ldg(qj + k + 3 * stride);
+                a += fminf(prob(j, li, k), q0);
+                a += fminf(prob(j, li, k + stride), q1);
+                a += fminf(prob(j, li, k + 2 * stride), q2);
+                a += fminf(prob(j, li, k + 3 * stride), q3);
+            }
+            for (; k < V; k += stride) a += fminf(prob(j, li, k), __ldg(qj + k));
             a = block_sum(a, sh.red);
             if (threadIdx.x == 0) P.alpha_terms[(size_t)b * gamma + j] = a;
         }
