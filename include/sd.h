@@ -256,6 +256,8 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  *   SD_TUNE_ATTN_WARPS      4 or 8 warps per attention CTA (64 or 128 KB of shared memory at head_dim 128)
  *   SD_TUNE_PREFILL_STAGES  stages a weight GEMM requests at once before the kernel before it has finished
  *   SD_TUNE_PACE_NS         > 0: after those, one more stage every so many nanoseconds until that kernel has finished
+ *   SD_TUNE_MANY_ROWS_CB    4: the sixteen-row form of the step kernel requests up to four pieces of a tile per round
+ *                           (one round of loads, but 128-212 registers: two waves of CTAs); default: two per round
  *   SD_TUNE_ATTN_CLUSTER    1 or 2: at most this many CTAs of a cluster share one slice of a head's cache (default up to 4) */
 #define SD_TUNE_WO_STAGES 0
 #define SD_TUNE_WO_PREFILL_ALL 1
@@ -263,7 +265,8 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
 #define SD_TUNE_ATTN_CLUSTER 3
 #define SD_TUNE_PACE_NS 4
 #define SD_TUNE_PREFILL_STAGES 5
-#define SD_TUNE_COUNT 6
+#define SD_TUNE_MANY_ROWS_CB 6
+#define SD_TUNE_COUNT 7
 sd_status sd_tuning(sd_ctx* ctx, int knob, int value);
 
 #define SD_STAMP_WORDS 8

@@ -498,6 +498,7 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     g.pace_ns = c->tune[SD_TUNE_PACE_NS];
     if (c->tune[SD_TUNE_PREFILL_STAGES] >= 2) g.prefill = std::min(g.stages, c->tune[SD_TUNE_PREFILL_STAGES]);
     Epilogue eps = ep;
+    eps.many_rows_cb = c->tune[SD_TUNE_MANY_ROWS_CB];
     g.stamp = next_stamp(c, SD_STAMP_GEMM | (ep.mode << 8));
     eps.stamp = next_stamp(c, SD_STAMP_STEP | (ep.mode << 8));
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;

@@ -52,6 +52,7 @@ struct Epilogue {
     const int32_t* lora_task;        // [row], written with the row plan by the pass's first kernel
     int lora_r, lora_n;              // rank, adapters
     float lora_scale;
+    int many_rows_cb;                // many-row form of the step: 4 = request up to four pieces per round when a tile has more than two (default: two)
     int ring_stages, prefill_all;    // GEMM before this step: cap on its stage ring (0: none) / request the whole ring before the dependency
     unsigned long long poll_ns;      // how long a tile's CTA watches its arrival word before it falls back to the grid dependency (0: 0.2 s)
     RowScale rs;                     // PLAIN, QKV_ROPE, SWIGLU: 1/rms factor of each token row
