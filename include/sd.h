@@ -254,8 +254,10 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  *                           smaller ring its CTAs fit beside the attention kernel's and stream weights while it runs
  *   SD_TUNE_WO_PREFILL_ALL  1: the Wo GEMM requests its whole ring before attention has finished
  *   SD_TUNE_ATTN_WARPS      4 or 8 warps per attention CTA (64 or 128 KB of shared memory at head_dim 128)
- *   SD_TUNE_PREFILL_STAGES  stages a weight GEMM requests at once before the kernel before it has finished
- *   SD_TUNE_PACE_NS         > 0: after those, one more stage every so many nanoseconds until that kernel has finished
+ *   SD_TUNE_PREFILL_STAGES  stages a weight GEMM requests at once before the kernel before it has finished (default 4 for
+ *                           passes of up to 16 rows)
+ *   SD_TUNE_PACE_NS         after those, one more stage every so many nanoseconds until that kernel has finished
+ *                           (default 300); 1 = no pacing: seven stages at once, the rest when that kernel has finished
  *   SD_TUNE_MANY_ROWS_CB    4: the sixteen-row form of the step kernel requests up to four pieces of a tile per round
  *                           (one round of loads, but 128-212 registers: two waves of CTAs); default: two per round
  *   SD_TUNE_ATTN_CLUSTER    1 or 2: at most this many CTAs of a cluster share one slice of a head's cache (default up to 4) */

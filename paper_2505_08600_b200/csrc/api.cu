@@ -495,7 +495,8 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     if (ep.lo_off) rows += ep.lo_off;           // the input rows come in two bf16 parts: [x_hi rows][x_lo rows at + lo_off]
     GemmGeom g = gemm_geometry(rows, n_out, K, sm_count(), ep.ring_stages, ep.prefill_all != 0, ep.lora_b ? 1 : 0);
     if (ep.lo_off) { g.lo_off = ep.lo_off; g.m_real = ep.m_real; }
-    g.pace_ns = c->tune[SD_TUNE_PACE_NS];
+    if (c->tune[SD_TUNE_PACE_NS] == 1) { g.pace_ns = 0; g.prefill = g.m_pad > 16 ? g.stages : std::min(g.stages, 7); }
+    else if (c->tune[SD_TUNE_PACE_NS] > 1) g.pace_ns = c->tune[SD_TUNE_PACE_NS];
     if (c->tune[SD_TUNE_PREFILL_STAGES] >= 2) g.prefill = std::min(g.stages, c->tune[SD_TUNE_PREFILL_STAGES]);
     Epilogue eps = ep;
     eps.many_rows_cb = c->tune[SD_TUNE_MANY_ROWS_CB];

@@ -37,6 +37,8 @@ constexpr int NUM_THREADS = 224;
 constexpr int MAX_STAGES = 12;
 constexpr int RING_BYTES = 198 * 1024;          // stage ring of a CTA; the rest of the SM's shared memory is left to the fused-step CTAs
 constexpr int GEMM_PREFILL_BYTES = 120 * 1024;  // bytes per SM requested while the previous kernel is still at work (see the weight producer)
+constexpr int GEMM_PACED_PREFILL_STAGES = 4;    // ... or, with pacing: stages requested at once, the rest one by one
+constexpr int GEMM_PACE_NS = 300;
 constexpr int GEMM_STEADY_BYTES = 160 * 1024;   // bytes per SM kept in flight once the ring has been filled (measured best: 9 of 11 stages at 16 rows)
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }    // the four epilogue warps
@@ -309,7 +311,11 @@ GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages, bo
     g.steady = std::min(g.stages, std::max(2, (GEMM_STEADY_BYTES + stage_bytes - 1) / stage_bytes));
     // (measured: with more than 16 token rows the reduction kernel is bound by throughput, not latency, and the full run-ahead wins)
     g.prefill = g.m_pad > 16 ? g.stages : std::min(g.stages, std::max(2, (GEMM_PREFILL_BYTES + stage_bytes - 1) / stage_bytes));
-    if (prefill_all) g.prefill = g.stages;
+    if (g.m_pad <= 16) {            // few rows: four stages at once, then one more every 300 ns until the kernel before has finished
+        g.prefill = std::min(g.stages, GEMM_PACED_PREFILL_STAGES);      // (measured against 7 stages at once and none after: -0.7 % at 7B, -1 % at 1B)
+        g.pace_ns = GEMM_PACE_NS;
+    }
+    if (prefill_all) { g.prefill = g.stages; g.pace_ns = 0; }
     return g;
 }
 
