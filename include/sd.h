@@ -258,6 +258,7 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  *                           passes of up to 16 rows)
  *   SD_TUNE_PACE_NS         after those, one more stage every so many nanoseconds until that kernel has finished
  *                           (default 300); 1 = no pacing: seven stages at once, the rest when that kernel has finished
+ *   SD_TUNE_STEADY_STAGES   stages of the ring a weight GEMM keeps in use once the ring has been filled (default: 160 KB worth)
  *   SD_TUNE_MANY_ROWS_CB    4: the sixteen-row form of the step kernel requests up to four pieces of a tile per round
  *                           (one round of loads, but 128-212 registers: two waves of CTAs); default: two per round
  *   SD_TUNE_ATTN_CLUSTER    1 or 2: at most this many CTAs of a cluster share one slice of a head's cache (default up to 4) */
@@ -268,7 +269,8 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
 #define SD_TUNE_PACE_NS 4
 #define SD_TUNE_PREFILL_STAGES 5
 #define SD_TUNE_MANY_ROWS_CB 6
-#define SD_TUNE_COUNT 7
+#define SD_TUNE_STEADY_STAGES 7
+#define SD_TUNE_COUNT 8
 sd_status sd_tuning(sd_ctx* ctx, int knob, int value);
 
 #define SD_STAMP_WORDS 8

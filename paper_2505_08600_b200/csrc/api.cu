@@ -498,6 +498,7 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     if (c->tune[SD_TUNE_PACE_NS] == 1) { g.pace_ns = 0; g.prefill = g.m_pad > 16 ? g.stages : std::min(g.stages, 7); }
     else if (c->tune[SD_TUNE_PACE_NS] > 1) g.pace_ns = c->tune[SD_TUNE_PACE_NS];
     if (c->tune[SD_TUNE_PREFILL_STAGES] >= 2) g.prefill = std::min(g.stages, c->tune[SD_TUNE_PREFILL_STAGES]);
+    if (c->tune[SD_TUNE_STEADY_STAGES] >= 2) g.steady = std::min(g.stages, c->tune[SD_TUNE_STEADY_STAGES]);
     Epilogue eps = ep;
     eps.many_rows_cb = c->tune[SD_TUNE_MANY_ROWS_CB];
     g.stamp = next_stamp(c, SD_STAMP_GEMM | (ep.mode << 8));
