@@ -258,6 +258,9 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  *                           passes of up to 16 rows)
  *   SD_TUNE_PACE_NS         after those, one more stage every so many nanoseconds until that kernel has finished
  *                           (default 300); 1 = no pacing: seven stages at once, the rest when that kernel has finished
+ *   SD_TUNE_TILE_HANDOFF    1: a weight GEMM loads each k block of token rows as soon as the step kernel's CTA for that
+ *                           tile has written it (a word per tile, release / acquire) instead of waiting for the whole step
+ *                           kernel (passes of 3..16 rows).  Measured slower (+4 % on the 7B verify step): off by default
  *   SD_TUNE_STEADY_STAGES   stages of the ring a weight GEMM keeps in use once the ring has been filled (default: 160 KB worth)
  *   SD_TUNE_MANY_ROWS_CB    4: the sixteen-row form of the step kernel requests up to four pieces of a tile per round
  *                           (one round of loads, but 128-212 registers: two waves of CTAs); default: two per round
@@ -270,7 +273,8 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
 #define SD_TUNE_PREFILL_STAGES 5
 #define SD_TUNE_MANY_ROWS_CB 6
 #define SD_TUNE_STEADY_STAGES 7
-#define SD_TUNE_COUNT 8
+#define SD_TUNE_TILE_HANDOFF 8
+#define SD_TUNE_COUNT 9
 sd_status sd_tuning(sd_ctx* ctx, int knob, int value);
 
 #define SD_STAMP_WORDS 8

@@ -86,6 +86,11 @@ class AcceptArgs(C.Structure):
                 ("out_tok", C.c_void_p), ("cuda_stream", C.c_void_p)]
 
 
+# knobs of sd_tuning (see include/sd.h)
+(SD_TUNE_WO_STAGES, SD_TUNE_WO_PREFILL_ALL, SD_TUNE_ATTN_WARPS, SD_TUNE_ATTN_CLUSTER, SD_TUNE_PACE_NS, SD_TUNE_PREFILL_STAGES,
+ SD_TUNE_MANY_ROWS_CB, SD_TUNE_STEADY_STAGES, SD_TUNE_TILE_HANDOFF) = range(9)
+
+
 class SdError(RuntimeError):
     def __init__(self, status, where):
         self.status = status

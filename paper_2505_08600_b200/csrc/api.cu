@@ -62,6 +62,7 @@ enum Phase { PH_FREE = 0, PH_BEGUN = 1, PH_ROUTED = 2, PH_READY = 3 };
 }  // namespace
 
 constexpr int STAMP_CAP = 1024;                 // launches of one pass whose time stamps can be kept
+constexpr size_t XREADY_WORDS = 32768;          // readiness words of one pass (one per step kernel that feeds a GEMM and tile)
 constexpr size_t ARRIVE_WORDS = 65536;          // arrival words of one pass (the 13B target needs about 17,000)
 constexpr int PASS_ROWS_CAP = 32;               // most query rows of a pass on the persistent streaming kernel
 constexpr size_t PASS_REGION_BYTES = (size_t)64 << 20;      // each of the two workspace regions of that kernel
@@ -81,6 +82,10 @@ struct sd_ctx {
     float* ssq;                                 // [row][SSQ_STRIDE] pieces of sum h^2 for the folded RMSNorm
     uint32_t* gemm_arrive;                      // per GEMM of a pass and output tile: pieces that have arrived (zero between passes)
     size_t arrive_used;                         // words handed out to the GEMMs of the pass being enqueued
+    // per-tile readiness of token rows between a step kernel and the GEMM after it (zeroed at the start of a pass that uses them)
+    uint32_t* xready; size_t xready_used; bool xready_on;
+    struct XReady { uint32_t* words; int n_tiles; int shift; uint32_t need; };
+    XReady x_from;                              // what the most recent step kernel counts into (words == nullptr: nothing)
     float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
     // persistent streaming kernel (pass_stream.cu): packed input rows, workspace, programs
     // (everything CTAs of that kernel hand to one another is tagged 64-bit words; the whole block is cleared when tags are about to repeat)
@@ -258,6 +263,8 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
     c->gemm_arrive = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
     c->arrive_used = 0;
+    c->xready = (uint32_t*)B.take(sizeof(uint32_t) * XREADY_WORDS);
+    c->xready_used = 0;
     size_t half_max = 1;
     for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
     c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
@@ -501,6 +508,19 @@ sd_status gemm_tc(sd_ctx* c, const TensorMap& tw, const void* x, int rows, int n
     if (c->tune[SD_TUNE_STEADY_STAGES] >= 2) g.steady = std::min(g.stages, c->tune[SD_TUNE_STEADY_STAGES]);
     Epilogue eps = ep;
     eps.many_rows_cb = c->tune[SD_TUNE_MANY_ROWS_CB];
+    // token rows tile by tile: this GEMM watches the words the step kernel before it counts into (if that kernel wrote
+    // these rows), and its own step kernel gets words of its own when what it writes feeds the next GEMM
+    if (c->x_from.words && c->x_from.n_tiles >= ((g.kb_per_tile - 1) >> c->x_from.shift) + 1) {
+        g.xr = c->x_from.words; g.xr_shift = c->x_from.shift; g.xr_need = c->x_from.need;
+    }
+    c->x_from.words = nullptr;
+    const bool feeds_gemm = ep.mode == EPI_SWIGLU || (ep.mode == EPI_RESIDUAL && ep.gain_next != nullptr);
+    const int step_tiles = (n_out + 127) / 128;
+    if (c->xready_on && feeds_gemm && !ep.lora_b && c->xready_used + (size_t)step_tiles <= XREADY_WORDS) {
+        eps.xready = c->xready + c->xready_used;
+        c->xready_used += (size_t)step_tiles;
+        c->x_from = sd_ctx::XReady{eps.xready, step_tiles, ep.mode == EPI_SWIGLU ? 0 : 1, (uint32_t)fused_step_row_batches(g, ep)};
+    }
     g.stamp = next_stamp(c, SD_STAMP_GEMM | (ep.mode << 8));
     eps.stamp = next_stamp(c, SD_STAMP_STEP | (ep.mode << 8));
     if (gemm_partials_bytes(g) > c->partials_bytes) return SD_ERR_CAPACITY;
@@ -524,6 +544,13 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     const int d = m.d_model, H = m.n_heads, Hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ffn, dt = m.dtype;
     cudaStream_t st = c->st;
     c->arrive_used = 0;                          // the embedding kernel below is an ordinary launch: everything before it has finished
+    c->xready_used = 0;
+    c->x_from.words = nullptr;
+    // Off unless asked for: measured on the 7B verify step it loses 4 % (3.05 -> 3.18 ms).  The release / acquire / proxy
+    // fence chain from a step CTA to the copy of its tile costs more than the end of the step kernel and the release of its
+    // dependent do, and a CTA whose first k block belongs to a late tile stalls the loads queued behind it.
+    c->xready_on = c->tune[SD_TUNE_TILE_HANDOFF] == 1 && n_rows >= 3 && n_rows <= 16;
+    if (c->xready_on) CUDA_TRY(cudaMemsetAsync(c->xready, 0, sizeof(uint32_t) * XREADY_WORDS, st));
     // With 3..16 rows (the verify rows of one sequence) the 16 (or 32) columns of the MMA hold every activation twice over:
     // as bf16(x) and as bf16(x - bf16(x)), 8 (or 16) rows apart.  The weights stream once all the same, and the GEMMs'
     // inputs are no longer rounded to 8 bits of mantissa.
@@ -815,6 +842,7 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     c->two_part = true;
     c->cost_on = false; c->cost_depth = 0;
     c->stamps_on = false;
+    c->xready_on = false; c->x_from.words = nullptr;
     for (int i = 0; i < SD_TUNE_COUNT; ++i) c->tune[i] = 0;
     for (int i = 0; i < 3; ++i) { c->cost_ms[i] = 0.0; c->cost_units[i] = 0; }
     c->force_plain = false;

@@ -293,6 +293,10 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     default: break;
     }
     if (et == 0) stamp_pair(ep.stamp, ST_DONE_FIRST);
+    if (ep.xready) {                              // everything this CTA writes is written: the next GEMM may load the tile's columns
+        __syncthreads();                          // (orders the CTA's stores before thread 0's release, which is cumulative)
+        if (et == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ep.xready + tile) : "memory");
+    }
 }
 
 template <int MODE, bool HL, bool LORA>
@@ -321,6 +325,13 @@ int pieces_bound(const GemmGeom& g) {
 int rows_per_cta(int n_rows, int pieces) { return n_rows <= 2 ? 2 : (n_rows > 8 && pieces <= 4 ? 16 : 8); }
 
 }  // namespace
+
+int fused_step_row_batches(const GemmGeom& g, const Epilogue& ep) {
+    const int n_rows = ep.mode == EPI_PLAIN ? ep.n_out_rows : (ep.lo_off ? ep.m_real : g.m_tok);
+    if (n_rows <= 2) return 1;
+    const int mb = (n_rows > 8 && pieces_bound(g) <= 4) ? 16 : 8;
+    return (n_rows + mb - 1) / mb;
+}
 
 bool fused_step_polls(const GemmGeom& g, const Epilogue& ep) {
     // One batch of rows per tile (several would share a tile's word).  With one or two rows (draft and plain

@@ -43,12 +43,15 @@ constexpr int GEMM_STEADY_BYTES = 160 * 1024;   // bytes per SM kept in flight o
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }    // the four epilogue warps
 
+constexpr int XR_MAX_TILES = 512;      // most tiles of token rows a GEMM tracks one by one (beyond: it waits for the kernel before)
+
 struct Shared {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     int epi_abort;
     int dep_seen;            // the token-row producer is past its wait for the kernel before
+    unsigned char xr_ready[XR_MAX_TILES];      // tiles of the token rows seen complete (token-row producer warp only)
 };
 
 // Ring bookkeeping.  The first `stages` loads of a CTA fill the whole ring (run-ahead while the
@@ -190,7 +193,58 @@ k_gemm_streamk(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         }
     } else if (warp == 6) {
         // ------------------------------------------------------------------ token-row producer
-        if (lane == 0) {
+        const int n_src = g.xr ? ((g.kb_per_tile - 1) >> g.xr_shift) + 1 : 0;      // tiles the token rows were written in
+        if (g.xr && n_src <= XR_MAX_TILES) {
+            // The rows are handed over tile by tile: the step kernel before counts into a word per tile once a tile's rows
+            // are written, and a k block is loaded as soon as its tile's word is there; the whole warp watches words (a
+            // lane per tile, the tile needed next first), lane 0 issues the copies.
+            volatile unsigned char* ready = sh.xr_ready;
+            for (int t = lane; t < n_src; t += 32) ready[t] = 0;
+            __syncwarp();
+            uint64_t pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            RingPos rp;
+            int kb = u0 % g.kb_per_tile;
+            bool first = true, gave_up = false, stop = false;
+            for (uint32_t it = 0; it < n_units && !stop; ++it, rp.next(g.stages, g.steady)) {
+                const int tile = kb >> g.xr_shift;
+                if (!gave_up && !ready[tile]) {                                   // uniform: every lane reads the same byte
+                    const uint64_t t0 = global_ns();
+                    for (uint32_t spin = 0;; ++spin) {
+                        const int tl = tile + lane;
+                        if (tl < n_src && !ready[tl]) {
+                            uint32_t v;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(g.xr + tl) : "memory");
+                            if (v >= g.xr_need) ready[tl] = 1;
+                        }
+                        __syncwarp();
+                        if (ready[tile]) break;
+                        __nanosleep(40);
+                        if ((spin & 63u) == 63u && global_ns() - t0 > 200000000ull) {      // 0.2 s: not expected; wait for the whole kernel instead, and say so
+                            pdl_wait();
+                            if (lane == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
+                            gave_up = true;
+                            break;
+                        }
+                    }
+                    if (lane == 0) asm volatile("fence.proxy.async;" ::: "memory");      // rows written with ordinary stores, read by the bulk copy below
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    if (first) { *(volatile int*)&sh.dep_seen = 1; stamp_pair(g.stamp, ST_DEP_FIRST); }
+                    const int s = rp.stage;
+                    if (rp.use > 0u && !mbar_wait(smem_u32(&sh.empty[s]), (rp.use & 1u) ^ 1u, abort_flag)) stop = true;
+                    else {
+                        const uint32_t bar = smem_u32(&sh.full[s]);
+                        mbar_expect_tx(bar, x_bytes);
+                        tma_load_2d(tiles0 + s * stage_bytes + A_BYTES, &tm_x, kb * TILE_K, 0, bar, pol_keep);
+                    }
+                }
+                first = false;
+                stop = __shfl_sync(0xffffffffu, (int)stop, 0) != 0;
+                if (++kb == g.kb_per_tile) kb = 0;
+            }
+        } else if (lane == 0) {
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             pdl_wait();                                           // the token rows are the previous kernel's output
@@ -294,6 +348,7 @@ bool make_tensor_map_bf16(TensorMap* out, const void* base, int rows, int K, int
 GemmGeom gemm_geometry(int m_tok, int n_out, int K, int n_sm, int max_stages, bool prefill_all, int extra_tiles) {
     GemmGeom g;
     g.lo_off = 0; g.m_real = m_tok; g.stamp = nullptr; g.pace_ns = 0;
+    g.xr = nullptr; g.xr_shift = 0; g.xr_need = 0;
     g.m_tok = m_tok;
     g.m_pad = (m_tok + 15) & ~15;
     g.n_out = n_out;

@@ -19,6 +19,11 @@ struct GemmGeom {
     int steady;             // stages reused once the ring has been filled (<= stages)
     int prefill;            // weight tiles requested before the previous kernel has finished
     unsigned long long* stamp;   // optional time stamps of this launch (see LaunchStamp); nullptr: none
+    // Per-tile readiness of the token rows (nullptr: wait for the whole kernel before).  The step kernel that writes the
+    // rows counts one into xr[t] when its CTA for 128-row tile t (64 features of the activation: xr_shift 0; 128 columns
+    // of the normed residual: xr_shift 1) has written everything it writes; k block kb of this GEMM is loaded once
+    // xr[kb >> xr_shift] has reached xr_need (the step's row batches per tile).
+    const uint32_t* xr; int xr_shift; uint32_t xr_need;
     int pace_ns;            // > 0: past `prefill`, one more stage is requested every pace_ns until the kernel before has finished
     int lo_off, m_real;     // two-part input rows (see Epilogue::lo_off): the epilogue adds accumulator columns r and r + lo_off
                             // and leaves m_real merged rows in each piece; 0: every column is a row of its own
@@ -52,6 +57,7 @@ struct Epilogue {
     const int32_t* lora_task;        // [row], written with the row plan by the pass's first kernel
     int lora_r, lora_n;              // rank, adapters
     float lora_scale;
+    uint32_t* xready;                // non-null: words [tile] the step counts into when a CTA's outputs are written (see GemmGeom::xr)
     int many_rows_cb;                // many-row form of the step: 4 = request up to four pieces per round when a tile has more than two (default: two)
     int ring_stages, prefill_all;    // GEMM before this step: cap on its stage ring (0: none) / request the whole ring before the dependency
     unsigned long long poll_ns;      // how long a tile's CTA watches its arrival word before it falls back to the grid dependency (0: 0.2 s)
@@ -92,6 +98,7 @@ cudaError_t launch_fused_step(const GemmGeom& g, const Epilogue& ep, const float
                               int dependent, cudaStream_t st);
 // Whether launch_fused_step polls (and clears) the arrival words for this step; the GEMM must count exactly then.
 bool fused_step_polls(const GemmGeom& g, const Epilogue& ep);
+int fused_step_row_batches(const GemmGeom& g, const Epilogue& ep);      // CTAs of the step per output tile
 
 // Launch with the programmatic-dependent-launch attribute (or plainly when dependent == 0).
 template <typename... KArgs, typename... Args>

@@ -459,6 +459,31 @@ def test_capacity_and_state_errors_are_reported_on_the_host(sd):
     ctx.close()
 
 
+def test_tile_by_tile_hand_off_of_token_rows_gives_identical_results(sd):
+    """With SD_TUNE_TILE_HANDOFF the GEMMs load each k block of token rows as soon as the step kernel's CTA for that tile has
+    written it instead of waiting for the whole kernel: same arithmetic, so the teacher-forced run still matches the
+    oracle and the logits are bit for bit those of the default path; so are the other measurement knobs."""
+    V, gamma = 4096, 5
+    prompt = synth.make_prompt(V, 41, seed=12)
+    ref = None
+    for knobs in ({}, {sd.SD_TUNE_TILE_HANDOFF: 1}, {sd.SD_TUNE_PACE_NS: 1, sd.SD_TUNE_MANY_ROWS_CB: 4, sd.SD_TUNE_STEADY_STAGES: 8},
+                  {sd.SD_TUNE_WO_STAGES: 6, sd.SD_TUNE_WO_PREFILL_ALL: 1}):       # (the attention knobs change the order of its merges)
+        ctx, om = _build(sd, SMALL_BF16, [SMALL_BF16_DRAFT], "bf16", 1.0, 17, max_ctx=128)
+        for k, v in knobs.items():
+            ctx.sd_tuning(k, v)
+        _replay(sd, ctx, om, 0, prompt, gamma, 1.0, 17, 12, "bf16", min_agree=0.0)      # (few iterations: agreement counts are covered elsewhere)
+        x = torch.from_numpy(synth.make_prompt(V, gamma, seed=3).reshape(1, gamma).astype(np.int32)).to(DEV)
+        logits = torch.zeros((1, gamma + 1, V), dtype=torch.float32, device=DEV)
+        ctx.sd_verify([0], gamma, x, logits)
+        got = logits.cpu()
+        if ref is None:
+            ref = got
+        else:
+            assert torch.equal(got, ref), knobs
+        assert ctx.sd_device_status() == 0
+        ctx.close()
+
+
 def test_graph_replay_plain_path_and_fused_call_agree(sd):
     """The same iterations through (a) captured graphs, (b) kernel-by-kernel launches, (c) the plain
     CUDA-core kernels and (d) the one-call verify+accept+rollback give the same tokens; (a), (b) and
