@@ -260,7 +260,7 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  *                           (default 300); 1 = no pacing: seven stages at once, the rest when that kernel has finished
  *   SD_TUNE_TILE_HANDOFF    1: a weight GEMM loads each k block of token rows as soon as the step kernel's CTA for that
  *                           tile has written it (a word per tile, release / acquire) instead of waiting for the whole step
- *                           kernel (passes of 3..16 rows).  Measured slower (+4 % on the 7B verify step): off by default
+ *                           kernel (passes of 3..8 rows).  Measured slower (+4 % on the 7B verify step): off by default
  *   SD_TUNE_STEADY_STAGES   stages of the ring a weight GEMM keeps in use once the ring has been filled (default: 160 KB worth)
  *   SD_TUNE_MANY_ROWS_CB    4: the sixteen-row form of the step kernel requests up to four pieces of a tile per round
  *                           (one round of loads, but 128-212 registers: two waves of CTAs); default: two per round

@@ -549,7 +549,7 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
     // Off unless asked for: measured on the 7B verify step it loses 4 % (3.05 -> 3.18 ms).  The release / acquire / proxy
     // fence chain from a step CTA to the copy of its tile costs more than the end of the step kernel and the release of its
     // dependent do, and a CTA whose first k block belongs to a late tile stalls the loads queued behind it.
-    c->xready_on = c->tune[SD_TUNE_TILE_HANDOFF] == 1 && n_rows >= 3 && n_rows <= 16;
+    c->xready_on = c->tune[SD_TUNE_TILE_HANDOFF] == 1 && n_rows >= 3 && n_rows <= 8;
     if (c->xready_on) CUDA_TRY(cudaMemsetAsync(c->xready, 0, sizeof(uint32_t) * XREADY_WORDS, st));
     // With 3..16 rows (the verify rows of one sequence) the 16 (or 32) columns of the MMA hold every activation twice over:
     // as bf16(x) and as bf16(x - bf16(x)), 8 (or 16) rows apart.  The weights stream once all the same, and the GEMMs'

@@ -32,7 +32,9 @@ struct StepShared {
 // two rows (draft steps), where a tile of a small matrix is cut into many pieces, (16, 4) or (16, 2)
 // for many rows on few pieces.  MODE < 0: the step is read from ep.mode; with many row batches one
 // instantiation per step is used instead, whose lower register count lets more CTAs be resident.
-template <int MODE, int MB, int CB, bool HL = false, bool LORA = false>      // LORA: the matrix carries low-rank adapters
+// LORA: the matrix carries low-rank adapters.  XR: the CTA counts into a word of its tile when its outputs are written
+// (tile-by-tile hand-off of token rows to the next GEMM: an opt-in measurement path, compiled for the eight-row form only).
+template <int MODE, int MB, int CB, bool HL = false, bool LORA = false, bool XR = false>
 __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials,
                                                     uint32_t* __restrict__ arrive, uint32_t* status) {
     __shared__ StepShared<MB> sh;
@@ -293,7 +295,7 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     default: break;
     }
     if (et == 0) stamp_pair(ep.stamp, ST_DONE_FIRST);
-    if (ep.xready) {                              // everything this CTA writes is written: the next GEMM may load the tile's columns
+    if (XR && ep.xready) {                        // everything this CTA writes is written: the next GEMM may load the tile's columns
         __syncthreads();                          // (orders the CTA's stores before thread 0's release, which is cumulative)
         if (et == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ep.xready + tile) : "memory");
     }
@@ -356,6 +358,8 @@ cudaError_t launch_step(const GemmGeom& g, const Epilogue& ep, const float* part
         default: return cudaErrorInvalidValue;
         }
     }
+    if (ep.xready && !LORA)
+        return launch_pdl(k_fused_step<-1, 8, 8, HL, false, true>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
     return launch_pdl(k_fused_step<-1, 8, 8, HL, LORA>, dim3(g.n_tiles, (n_rows + 7) / 8), dim3(128), 0, st, dependent, g, ep, partials, arrive, status);
 }
 
