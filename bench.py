@@ -601,6 +601,44 @@ def run_mamba_bench(args):
                       "cpu_baseline": {"value": 1.0 / cpu_s, "unit": "prompts/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle", "sample": f"the first {done} prompts"}}))
 
 
+def run_prefill_bench(args):
+    """Prefill of one 512-token prompt of the configuration's target model (the contraction-bound regime): forward over the
+    prompt in batches of at most 256 rows through the same weight GEMM as the verify step, no logits.  The draft's prefill
+    runs in the same call and is timed with it; flops counted are the target's weight GEMMs only."""
+    env = setup(args, 1, 8)
+    torch, ctx, dev, cfg, seqs = (env[k] for k in ("torch", "ctx", "dev", "cfg", "seqs"))
+    t = cfg["target"]
+    n = env["lens"][0]
+    prompt = synth.make_prompt(t["vocab"], n, seed=3)
+    stream = torch.cuda.current_stream(dev)
+
+    def once():
+        ctx.sd_seq_begin(0, prompt, 0)
+        ctx.sd_route_prompt([0], forced_task=[0])
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.sd_prefill([0])
+        e1.record(stream); torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    for _ in range(3):
+        once()
+    K = max(3, min(args.steps, 10))
+    ms = sorted(once() for _ in range(K))[K // 2]
+    layer_params = synth.param_count(t, streamed_only=True) - t["vocab"] * t["d_model"]
+    flop = 2.0 * layer_params * (n - 1)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    peak = float(peaks.get("bf16_tflops", 1590.0))
+    print(json.dumps({"metric": "prefill_tokens_per_s", "unit": "tokens/s", "value": (n - 1) / (ms * 1e-3), "ms_per_step": ms, "n_gpus": 1, "steps": K,
+                      "dtype": cfg["dtype"], "data": "synthetic",
+                      "config": {"workload": f"{args.config}: prefill of one {n}-token prompt (target {t['n_layers']}x{t['d_model']} and its routed draft), rows in batches of <= 256"},
+                      "roofline": {"bound": "tensor", "achieved": flop / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s", "frac": flop / (ms * 1e-3) / 1e12 / peak,
+                                   "peak_kind": "of measured" if peaks else "of fallback", "traffic": None,
+                                   "note": "the draft's prefill and the attention over the prompt are inside the timed call; flops are the target's layer GEMMs"},
+                      "device_status": ctx.sd_device_status()}))
+    ctx.close()
+
+
 def run_accept_microbench(args):
     """Accept / reject / resample kernel alone at the 13B configuration's shape (8 sequences, gamma 8, vocab 32000):
     draft distributions are softmax(target_logits + N(0, sigma^2)) so that sigma sets the acceptance rate."""
@@ -657,6 +695,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
     ap.add_argument("--lora", action="store_true", help="drafts = one base draft + one low-rank adapter per task (sequences of all tasks share each draft pass)")
+    ap.add_argument("--prefill", action="store_true", help="time the prefill of one prompt of the configuration and exit")
     ap.add_argument("--mamba", action="store_true", help="time the Mamba-based prompt classifier on 400 synthetic prompts and exit")
     ap.add_argument("--kmeans", action="store_true", help="time one K-means step over synthetic sentence vectors and exit")
     args = ap.parse_args()
@@ -672,7 +711,7 @@ def main():
             argv[i + 1] = name
             rc = rc or subprocess.run(argv).returncode
         sys.exit(rc)
-    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep and not args.kmeans and not args.mamba:
+    if args.impl == "ours" and args.gpus > 1 and not launched and not args.accept_microbench and not args.gamma_sweep and not args.kmeans and not args.mamba and not args.prefill:
         # no launcher: this process starts the N replicas itself (one per GPU) and passes rank 0's line through
         rc, out = replicas.spawn_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
         sys.stdout.write(out)
@@ -683,6 +722,8 @@ def main():
         run_kmeans_bench(args)
     elif args.mamba:
         run_mamba_bench(args)
+    elif args.prefill:
+        run_prefill_bench(args)
     elif args.gamma_sweep:
         run_gamma_sweep(args)
     elif args.impl == "reference":
