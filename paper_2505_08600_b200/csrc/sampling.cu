@@ -151,10 +151,14 @@ __device__ __forceinline__ int softmax_sample_row(const float* __restrict__ l_gl
     for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, l[k]);
     m = block_max(m, sh.red);
     float s = 0.f;
-    for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) / T);
+    // one division each for 1/T and 1/sum, then multiplications: an IEEE division per element costs about as much as
+    // the exponential itself, and the result differs from e / sum by an ulp (the probability tolerance is 1e-3)
+    const float inv_T = 1.f / T;
+    for (int k = threadIdx.x; k < V; k += blockDim.x) s += expf((l[k] - m) * inv_T);
     s = block_sum(s, sh.red);
+    const float inv_s = 1.f / s;
     for (int k = threadIdx.x; k < V; k += blockDim.x) {
-        const float pk = expf((l[k] - m) / T) / s;
+        const float pk = expf((l[k] - m) * inv_T) * inv_s;
         probs[k] = pk;
         if (rowbuf) rowbuf[k] = pk;                      // the draw below reads the same fp32 values
     }
@@ -218,7 +222,7 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(16) float rowbuf[];            // one target row (when it fits): every pass over it reads shared memory
     __shared__ BlockScratch sh;
-    __shared__ float row_max[ACC_ROWS_PER_CTA], row_sum[ACC_ROWS_PER_CTA];
+    __shared__ float row_max[ACC_ROWS_PER_CTA], row_inv[ACC_ROWS_PER_CTA];      // max of the row's logits, 1 / sum of its exponentials
     __shared__ int row_arg[ACC_ROWS_PER_CTA];
     __shared__ int flag_sh[ACC_ROWS_PER_CTA];
     __shared__ int n_sh;
@@ -228,6 +232,7 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
     const int b = P.use_list ? P.list.out[i] : i;
     const int V = P.V, gamma = P.gamma;
     const float T = P.T;
+    const float inv_T = T > 0.f ? 1.f / T : 0.f;
     const float* tgt = P.target + (size_t)b * (gamma + 1) * V;
     const float* q = P.q + (size_t)b * gamma * V;
     const int32_t* x = P.x + (size_t)b * gamma;
@@ -243,7 +248,7 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
         if (logits && T == 0.f) return k == row_arg[li] ? 1.f : 0.f;
         const float v = val(j, k);
         if (!logits) return v;
-        return expf((v - row_max[li]) / T) / row_sum[li];
+        return expf((v - row_max[li]) * inv_T) * row_inv[li];      // (multiplications by 1/T and 1/sum: see softmax_sample_row)
     };
 
     for (int li = 0; li < ACC_ROWS_PER_CTA; ++li) {
@@ -259,9 +264,9 @@ __global__ void __launch_bounds__(1024) k_accept(AcceptParams P, int csize, int 
                 for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, val(j, k));
                 m = block_max(m, sh.red);
                 float sum = 0.f;
-                for (int k = threadIdx.x; k < V; k += blockDim.x) sum += expf((val(j, k) - m) / T);
+                for (int k = threadIdx.x; k < V; k += blockDim.x) sum += expf((val(j, k) - m) * inv_T);
                 sum = block_sum(sum, sh.red);
-                if (threadIdx.x == 0) { row_max[li] = m; row_sum[li] = sum; }
+                if (threadIdx.x == 0) { row_max[li] = m; row_inv[li] = 1.f / sum; }
             }
             __syncthreads();
         }
