@@ -564,6 +564,8 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         e.lora_b = L.lora_b[mat]; e.lora_task = c->row_slot + SD_MAX_ROWS; e.lora_r = c->cfg.lora_rank; e.lora_n = c->cfg.lora_adapters;
         e.lora_scale = c->cfg.lora_scale; e.row_slot = c->row_slot;
     };
+    int len_hint[SD_MAX_BATCH];                                             // context bounds of the pass's sequences, for attention's launch order
+    for (int i = 0; i < list.n && i < SD_MAX_BATCH; ++i) len_hint[i] = c->len_ub[list.ids[i]];
     const RowScale first{c->ssq, 1, 1.f / d, m.rms_eps};                    // sum of squares in one piece (after the embedding)
     const RowScale tiled{c->ssq, (d + 127) / 128, 1.f / d, m.rms_eps};      // ... in one piece per 128-wide tile of h
     LAUNCH(CAT_ELEMENTWISE, launch_embed(c->S, list, plan, n_rows, M.embed, dt, d, m.vocab, c->h, c->row_slot, c->row_pos,
@@ -582,7 +584,8 @@ sd_status forward_tc(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& pl
         SD_TRY(gemm_tc(c, L.tm_qkv, c->xn, n_rows, M.n_qkv(), d, e));
         LAUNCH(CAT_ATTENTION, launch_attention_split(c->q, kc, vc, c->attn, c->row_slot, c->row_pos, n_rows, plan.rows_per_seq, H, Hkv,
                                                      hd, c->cfg.max_ctx, plan.ctx_bound, c->attn_ws, c->attn_ws_bytes, 1, st, lo,
-                                                     next_stamp(c, SD_STAMP_ATTENTION), c->tune[SD_TUNE_ATTN_WARPS], c->tune[SD_TUNE_ATTN_CLUSTER]));
+                                                     next_stamp(c, SD_STAMP_ATTENTION), c->tune[SD_TUNE_ATTN_WARPS], c->tune[SD_TUNE_ATTN_CLUSTER],
+                                                     list.n > 1 ? len_hint : nullptr));
         memset(&e, 0, sizeof(e));
         e.lo_off = lo; e.m_real = n_rows;
         e.ring_stages = c->tune[SD_TUNE_WO_STAGES]; e.prefill_all = c->tune[SD_TUNE_WO_PREFILL_ALL];

@@ -35,6 +35,8 @@ struct AttnParams {
     int csize;          // CTAs of a thread-block cluster that share one slice (1, 2 or 4)
     int lo_off;         // > 0: the output is also written as a second bf16 part (x - bf16(x)) lo_off rows further down
     unsigned long long* stamp;   // optional time stamps of the launch (see LaunchStamp)
+    int use_order;               // sequences are taken in seq_order (longest context first: CTAs are handed out in grid order,
+    unsigned char seq_order[64]; // and the sequence that takes longest should not be the one that starts last)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
@@ -86,8 +88,10 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     const int split = blockIdx.x / CS, crank = blockIdx.x % CS, kvh = blockIdx.y;
     const int group = P.H / P.Hkv;
     const int bps = (P.rows_per_seq + P.rows_per_block - 1) / P.rows_per_block;     // query blocks per sequence
-    const int r0 = (blockIdx.z / bps) * P.rows_per_seq + (blockIdx.z % bps) * P.rows_per_block;
-    const int nr = min(P.rows_per_block, P.rows_per_seq - (int)(blockIdx.z % bps) * P.rows_per_block);
+    const int zseq = P.use_order ? (int)P.seq_order[blockIdx.z / bps] : (int)(blockIdx.z / bps);
+    const int zb = zseq * bps + (int)(blockIdx.z % bps);                             // query block this CTA works on
+    const int r0 = zseq * P.rows_per_seq + (zb % bps) * P.rows_per_block;
+    const int nr = min(P.rows_per_block, P.rows_per_seq - (zb % bps) * P.rows_per_block);
     const int nq = nr * group;
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5, gid = lane >> 2, tig = lane & 3;
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(sm_raw);
@@ -122,7 +126,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     // first position this pass appends for the block's sequence (its rows' positions rise; inactive rows are -1)
     int new_begin;
     {
-        const int seq_first = (blockIdx.z / bps) * P.rows_per_seq;
+        const int seq_first = zseq * P.rows_per_seq;
         const int fp = lane < min(P.rows_per_seq, 32) ? __ldcg(P.row_pos + seq_first + lane) : -1;
         int nb = fp >= 0 ? fp : 0x7fffffff;
 #pragma unroll
@@ -366,7 +370,7 @@ __global__ void __launch_bounds__(32 * NW) k_attn_mma(AttnParams P) {
     //      always in slice order, so the result does not depend on which slice that was
     __syncthreads();                                 // the block's writes are ordered before thread 0's release below
     if (t == 0) {
-        uint32_t* ctr = P.counters + (size_t)blockIdx.z * P.Hkv + kvh;
+        uint32_t* ctr = P.counters + (size_t)zb * P.Hkv + kvh;
         uint32_t old;
         asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
         const int last = old == (uint32_t)P.n_splits - 1u;
@@ -462,12 +466,21 @@ size_t attention_split_workspace(int rows, int H, int hd, int max_ctx) {
 cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc, void* out, const int32_t* row_slot,
                                    const int32_t* row_pos, int n_rows, int rows_per_seq, int H, int Hkv, int hd,
                                    int max_ctx, int ctx_bound, void* workspace, size_t workspace_bytes, int dependent,
-                                   cudaStream_t st, int lo_off, unsigned long long* stamp, int force_warps, int max_cluster) {
+                                   cudaStream_t st, int lo_off, unsigned long long* stamp, int force_warps, int max_cluster, const int* seq_len_hint) {
     if (n_rows <= 0) return cudaSuccess;
     ctx_bound = std::max(1, std::min(ctx_bound, max_ctx));
     AttnParams P;
     P.q = (const bf16*)q; P.kc = (const bf16*)kc; P.vc = (const bf16*)vc; P.out = (bf16*)out;
     P.row_slot = row_slot; P.row_pos = row_pos; P.lo_off = lo_off; P.stamp = stamp;
+    P.use_order = 0;
+    if (seq_len_hint && rows_per_seq >= 1 && n_rows / rows_per_seq > 1 && n_rows / rows_per_seq <= 64) {      // longest first
+        const int ns = n_rows / rows_per_seq;
+        int idx[64];
+        for (int i = 0; i < ns; ++i) idx[i] = i;
+        std::stable_sort(idx, idx + ns, [&](int a, int b) { return seq_len_hint[a] > seq_len_hint[b]; });
+        for (int i = 0; i < ns; ++i) P.seq_order[i] = (unsigned char)idx[i];
+        P.use_order = 1;
+    }
     if (rows_per_seq < 1 || n_rows % rows_per_seq || H / Hkv > NQ) return cudaErrorInvalidValue;
     P.n_rows = n_rows; P.rows_per_seq = rows_per_seq; P.H = H; P.Hkv = Hkv; P.max_ctx = max_ctx;
     P.rows_per_block = std::max(1, std::min(rows_per_seq, NQ / (H / Hkv)));

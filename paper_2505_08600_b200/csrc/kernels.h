@@ -52,7 +52,8 @@ cudaError_t launch_attention_split(const void* q, const void* kc, const void* vc
                                    cudaStream_t st, int lo_off = 0 /*> 0: also write out's second bf16 part, lo_off rows further down*/,
                                    unsigned long long* stamp = nullptr /*optional time stamps of the launch*/,
                                    int force_warps = 0 /*4 or 8: warps per CTA; 0: chosen from the number of work items*/,
-                                   int max_cluster = 0 /*1 or 2: at most this many CTAs share a slice; 0: up to 4*/);
+                                   int max_cluster = 0 /*1 or 2: at most this many CTAs share a slice; 0: up to 4*/,
+                                   const int* seq_len_hint = nullptr /*host, one per sequence: context lengths (bounds will do); longest sequences are started first*/);
 
 // ---- sampling.cu
 cudaError_t launch_philox(const uint32_t* ctr, int n, uint32_t k0, uint32_t k1, uint32_t* out, cudaStream_t st);
