@@ -118,7 +118,39 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
 
     if (et == 0) stamp_pair(ep.stamp, ST_DEP_FIRST);
 
-    // ---- one round of loads: sums of squares, residual / row plan / rotary factors, the pieces
+    // ---- one round of loads: (adapters: the pieces of x A^T,) sums of squares, residual / row plan / rotary factors, the pieces
+    // t = x A^T sits in the GEMM's last tile; its pieces are summed like any tile's, by MB * r threads.  The first four
+    // pieces of every sum are requested here, ahead of the tile's own pieces, so that both come back in the same round.
+    // (one or two rows only: with more rows per CTA the extra registers cost more than the round trip saves)
+    constexpr bool LPRE = LORA && MB <= 2;
+    constexpr int LNP = LPRE ? (MB * 32 + 127) / 128 : 1;
+    float tl[LNP][4];
+    uint32_t x_first = 0, x_last = 0, xj_first = 0;
+    auto lora_tile = [&]() {                      // which CTAs of the GEMM hold pieces of its last tile
+        const uint32_t tx = (uint32_t)g.n_tiles - 1u, xa = tx * KB, xb = xa + KB - 1;
+        x_first = ((xa + 1) * G + T - 1) / T - 1; x_last = ((xb + 1) * G + T - 1) / T - 1;
+        xj_first = tx - ((x_first * T) / G) / KB;
+    };
+    if (LPRE) {
+        lora_tile();
+        const int r = ep.lora_r;
+#pragma unroll
+        for (int pp = 0; pp < LNP; ++pp) {
+            const int p = et + pp * 128, i = p / r, j = p % r, row = m0 + i;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) tl[pp][cc] = 0.f;
+            if (LPRE && p < MB * r && row < n_rows) {
+                const int tk = __ldcg(ep.lora_task + row);
+                if (tk >= 0 && tk < ep.lora_n) {
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const uint32_t c = x_first + cc, jj = cc == 0 ? xj_first : 0u;
+                        if (c <= x_last) tl[pp][cc] = __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)row * TILE_N + tk * r + j);
+                    }
+                }
+            }
+        }
+    }
     float ssa[(MB + 3) / 4], ssb[(MB + 3) / 4];
     if (ep.rs.ssq) {                              // one warp per token row, one lane per piece of its sum of squares
 #pragma unroll
@@ -159,24 +191,37 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
         }
     }
     if (LORA) {                                   // the low-rank update of this matrix
-        // t = x A^T sits in the GEMM's last tile; its pieces are summed like any tile's, by MB * r threads
-        const uint32_t tx = (uint32_t)g.n_tiles - 1u, xa = tx * KB, xb = xa + KB - 1;
-        const uint32_t x_first = ((xa + 1) * G + T - 1) / T - 1, x_last = ((xb + 1) * G + T - 1) / T - 1;
-        const uint32_t xj_first = tx - ((x_first * T) / G) / KB;
         const int r = ep.lora_r;
-        for (int p = et; p < MB * r; p += 128) {
-            const int i = p / r, j = p % r;
-            float t = 0.f;
-            if (rows[i] >= 0) {
-                const int tk = __ldcg(ep.lora_task + rows[i]);
-                if (tk >= 0 && tk < ep.lora_n) {
-                    for (uint32_t c = x_first; c <= x_last; ++c) {
-                        const uint32_t jj = c == x_first ? xj_first : 0u;
-                        t += __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)rows[i] * TILE_N + tk * r + j);
+        if (!LPRE) {
+            lora_tile();
+            for (int p = et; p < MB * r; p += 128) {
+                const int i = p / r, j = p % r, row = m0 + i;
+                float t = 0.f;
+                if (row < n_rows) {
+                    const int tk = __ldcg(ep.lora_task + row);
+                    if (tk >= 0 && tk < ep.lora_n) {
+                        for (uint32_t c = x_first; c <= x_last; ++c) {
+                            const uint32_t jj = c == x_first ? xj_first : 0u;
+                            t += __ldcg(partials + ((size_t)c * g.max_seg + jj) * g.m_pad * TILE_N + (size_t)row * TILE_N + tk * r + j);
+                        }
                     }
                 }
+                sh.lora_t[i][j] = t;
             }
-            sh.lora_t[i][j] = t;
+        }
+#pragma unroll
+        for (int pp = 0; pp < LNP; ++pp) {
+            const int p = et + pp * 128, i = p / r, j = p % r, row = m0 + i;
+            if (LPRE && p < MB * r) {
+                float t = (tl[pp][0] + tl[pp][1]) + (tl[pp][2] + tl[pp][3]);
+                if (x_last > x_first + 3u && row < n_rows) {      // a tile cut into more than four pieces (small matrices on many SMs)
+                    const int tk = __ldcg(ep.lora_task + row);
+                    if (tk >= 0 && tk < ep.lora_n)
+                        for (uint32_t c = x_first + 4u; c <= x_last; ++c)
+                            t += __ldcg(partials + ((size_t)c * g.max_seg) * g.m_pad * TILE_N + (size_t)row * TILE_N + tk * r + j);
+                }
+                sh.lora_t[i][j] = t;
+            }
         }
         __syncthreads();
         if (live) {
