@@ -399,6 +399,23 @@ def run_gpu(args):
     ctx.sd_seq_read(0)
     rewind()
 
+    # ---- sustained: the same step for about two seconds (blocks of K steps from the same contexts), clocks sampled throughout
+    sustained = None
+    if world == 1 and args.sustained_s > 0:
+        sampler2 = ClockSampler(gpu_id)
+        blocks, tot_ms, t_end = 0, 0.0, time.perf_counter() + args.sustained_s
+        while time.perf_counter() < t_end:
+            rewind()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(K):
+                verify_step()
+            b.record(stream)
+            torch.cuda.synchronize()
+            tot_ms += a.elapsed_time(b); blocks += 1
+        sustained = {"ms_per_step": tot_ms / (blocks * K), "steps": blocks * K, "seconds": round(args.sustained_s, 1), "clocks": sampler2.stop()}
+        rewind()
+
     # ---- whole iterations and the cost ratio c of Eq. 1
     def timed(fn, n):
         torch.cuda.synchronize()
@@ -441,7 +458,7 @@ def run_gpu(args):
                        "context_at_end_of_timed_steps": n_ctx if B > 1 else n_ctx[0],
                        "l2": "weights (>= 2 GB per step) far exceed the 126 MB L2; no flush", "replicas": world,
                        "device_status": status},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, **extras,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "sustained": sustained, **extras,
         }))
     ctx.close()
     if world > 1:
@@ -693,6 +710,7 @@ def main():
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--profile-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-s", type=float, default=2.0, help="seconds of back-to-back verify steps for the sustained figure (0: skip)")
     ap.add_argument("--accept-microbench", action="store_true", help="time the accept kernel alone (sigma sweep) and exit")
     ap.add_argument("--lora", action="store_true", help="drafts = one base draft + one low-rank adapter per task (sequences of all tasks share each draft pass)")
     ap.add_argument("--prefill", action="store_true", help="time the prefill of one prompt of the configuration and exit")
