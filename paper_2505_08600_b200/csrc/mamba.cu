@@ -47,9 +47,9 @@ __global__ void k_mamba_tables(const ChunkRec* __restrict__ chunks, const int64_
 __global__ void __launch_bounds__(256)
 k_mamba_in(MambaDims m, const int32_t* __restrict__ tokens, const int64_t* __restrict__ tok_src, int T, const float* __restrict__ embed,
            const float* __restrict__ w_in, float* __restrict__ u, float* __restrict__ z) {
-    extern __shared__ float in_smem[];
+    extern __shared__ __align__(16) float in_smem[];
     float* e_s = in_smem;                                // [MB_TOK_TILE][D]
-    float* w_s = in_smem + MB_TOK_TILE * m.D;            // [256][33]
+    float* w_s = in_smem + MB_TOK_TILE * m.D;            // [256][36]: rows padded to 36 words (16-byte aligned, conflict-free float4 reads)
     const int t0 = blockIdx.x * MB_TOK_TILE, nt = min(MB_TOK_TILE, T - t0);
     for (int i = threadIdx.x; i < MB_TOK_TILE * m.D; i += blockDim.x) {
         const int tt = i / m.D, d = i % m.D;
@@ -71,14 +71,26 @@ k_mamba_in(MambaDims m, const int32_t* __restrict__ tokens, const int64_t* __res
             __syncthreads();                             // the previous block of W (and, the first time, e_s) is settled
             for (int rr = warp; rr < 256; rr += 8) {     // warp per row: lanes along the row
                 const int row = j0 + rr;
-                w_s[rr * 33 + lane] = (row < 2 * m.Di && d0 + lane < m.D) ? w_in[(size_t)row * m.D + d0 + lane] : 0.f;
+                w_s[rr * 36 + lane] = (row < 2 * m.Di && d0 + lane < m.D) ? w_in[(size_t)row * m.D + d0 + lane] : 0.f;
             }
             __syncthreads();
             const int nd = min(32, m.D - d0);
-            for (int dd = 0; dd < nd; ++dd) {
-                const float w = w_s[threadIdx.x * 33 + dd];
+            if ((m.D & 3) == 0) {                        // four columns at a time: one 16-byte read of W and of every token's embedding
+                for (int dd = 0; dd < nd; dd += 4) {
+                    const float4 w = *reinterpret_cast<const float4*>(w_s + threadIdx.x * 36 + dd);
 #pragma unroll
-                for (int tt = 0; tt < MB_TOK_TILE; ++tt) acc[tt] = fmaf(w, e_s[tt * m.D + d0 + dd], acc[tt]);
+                    for (int tt = 0; tt < MB_TOK_TILE; ++tt) {
+                        const float4 e = *reinterpret_cast<const float4*>(e_s + tt * m.D + d0 + dd);
+                        acc[tt] = fmaf(w.x, e.x, acc[tt]); acc[tt] = fmaf(w.y, e.y, acc[tt]);
+                        acc[tt] = fmaf(w.z, e.z, acc[tt]); acc[tt] = fmaf(w.w, e.w, acc[tt]);
+                    }
+                }
+            } else {
+                for (int dd = 0; dd < nd; ++dd) {
+                    const float w = w_s[threadIdx.x * 36 + dd];
+#pragma unroll
+                    for (int tt = 0; tt < MB_TOK_TILE; ++tt) acc[tt] = fmaf(w, e_s[tt * m.D + d0 + dd], acc[tt]);
+                }
             }
         }
         if (j < 2 * m.Di) {
@@ -332,7 +344,7 @@ extern "C" sd_status sd_mamba_classify(const sd_mamba_desc* desc, const sd_mamba
     const int32_t* pc0 = (const int32_t*)(base + L.prompt_chunk0);
 
     k_mamba_tables<<<(unsigned)n_chunks, 64, 0, st>>>(chunks_d, (const int64_t*)(base + L.starts), (int64_t*)(base + L.tok_src), (int32_t*)(base + L.tok_pos));
-    const size_t in_smem_bytes = ((size_t)MB_TOK_TILE * m.D + 256 * 33) * 4;      // up to 66 KB at d_model 512: above the default limit
+    const size_t in_smem_bytes = ((size_t)MB_TOK_TILE * m.D + 256 * 36) * 4;      // up to 66 KB at d_model 512: above the default limit
     if (cudaFuncSetAttribute(k_mamba_in, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)in_smem_bytes) != cudaSuccess) return SD_ERR_CUDA;
     k_mamba_in<<<(unsigned)((T + MB_TOK_TILE - 1) / MB_TOK_TILE), 256, in_smem_bytes, st>>>(
         m, tokens_dev, (const int64_t*)(base + L.tok_src), (int)T, w->embed, w->w_in, u, z);
