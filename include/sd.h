@@ -249,6 +249,12 @@ int sd_best_gamma(double alpha, double c, int gamma_max, double* speedup_out);
  * kinds_host[i] = SD_STAMP_GEMM / _STEP / _ATTENTION | (step after the GEMM: 0 plain, 1 QKV+rotary, 2 residual,
  * 3 SwiGLU) << 8; *n_out = records of the pass (may exceed cap).  Enabling changes the captured graphs' keys: the
  * first call afterwards captures anew.  A few atomics per CTA: for measurement, off by default. */
+/* Sequences routed to different draft models run their draft passes side by side (default, when the context has two or
+ * more separate draft models): every group after the first is enqueued on a stream of its own, forked from and joined
+ * back to the context's stream, with its own scratch memory from the arena.  on = 0: group after group on the
+ * context's stream. */
+sd_status sd_use_draft_streams(sd_ctx* ctx, int on);
+
 /* Measurement knobs of the kernel-per-matrix path (0 = the library's own choice).  Setting one drops the captured graphs.
  *   SD_TUNE_WO_STAGES       cap on the stage ring of the Wo GEMM (16 KB weight block + token rows per stage): with a
  *                           smaller ring its CTAs fit beside the attention kernel's and stream weights while it runs

@@ -120,6 +120,7 @@ _PROTOS = {
     "sd_verify_accept": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "sd_use_graphs": (_i, [_vp, _i]),
     "sd_tuning": (_i, [_vp, _i, _i]),
+    "sd_use_draft_streams": (_i, [_vp, _i]),
     "sd_launch_stamps": (_i, [_vp, _i]),
     "sd_launch_stamps_read": (_i, [_vp, _vp, _vp, _i, C.POINTER(C.c_int32)]),
     "sd_seq_alpha": (_i, [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
@@ -377,6 +378,9 @@ class Context:
         _check(self.L.sd_route_prompt_mamba(self.h, C.byref(clf.desc), C.byref(clf.w), seqs_a.ctypes.data_as(C.c_void_p), len(seqs),
                                             _dp(ws), need, out.ctypes.data_as(C.c_void_p)), "sd_route_prompt_mamba")
         return out
+
+    def sd_use_draft_streams(self, on):
+        _check(self.L.sd_use_draft_streams(self.h, int(on)), "sd_use_draft_streams")
 
     def sd_tuning(self, knob, value):
         _check(self.L.sd_tuning(self.h, int(knob), int(value)), "sd_tuning")

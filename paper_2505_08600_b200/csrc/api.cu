@@ -87,6 +87,18 @@ struct sd_ctx {
     struct XReady { uint32_t* words; int n_tiles; int shift; uint32_t need; };
     XReady x_from;                              // what the most recent step kernel counts into (words == nullptr: nothing)
     float* rope_row_cos; float* rope_row_sin;   // [row][head_dim/2] rotary factors of the pass's rows (their positions applied)
+    // Draft groups side by side: sequences routed to different draft models run their draft passes on streams of their own,
+    // each with a scratch set of its own (set 0 is the fields above; sets 1... are sized for the draft models only).
+    struct ScratchSet {
+        float* h; void* xn; void* q; void* attn; void* act; float* lin; float* draft_logits; int32_t* row_slot; int32_t* row_pos;
+        void* attn_ws; size_t attn_ws_bytes; float* partials; size_t partials_bytes; float* ssq; uint32_t* gemm_arrive; uint32_t* xready;
+        float* rope_row_cos; float* rope_row_sin;
+    };
+    std::vector<ScratchSet> sets;
+    std::vector<cudaStream_t> group_streams;    // streams of groups 1...
+    std::vector<cudaEvent_t> ev_join;
+    cudaEvent_t ev_fork;
+    bool groups_concurrent;
     // persistent streaming kernel (pass_stream.cu): packed input rows, workspace, programs
     // (everything CTAs of that kernel hand to one another is tagged 64-bit words; the whole block is cleared when tags are about to repeat)
     tagged_t* tg_h; tagged_t* tg_xn; tagged_t* tg_attn; tagged_t* tg_act; tagged_t* tg_q; tagged_t* tg_newkv; tagged_t* tg_ssq;
@@ -263,12 +275,50 @@ void layout(sd_ctx* c, const sd_model_desc* ms, Bump& B) {
     c->ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
     c->gemm_arrive = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
     c->arrive_used = 0;
-    c->xready = (uint32_t*)B.take(sizeof(uint32_t) * XREADY_WORDS);
-    c->xready_used = 0;
     size_t half_max = 1;
     for (int i = 0; i < nm; ++i) half_max = std::max(half_max, (size_t)ms[i].head_dim / 2);
     c->rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
     c->rope_row_sin = (float*)B.take(sizeof(float) * SD_MAX_ROWS * half_max);
+    c->xready = (uint32_t*)B.take(sizeof(uint32_t) * XREADY_WORDS);
+    c->xready_used = 0;
+    c->sets.clear();
+    c->sets.push_back(sd_ctx::ScratchSet{c->h, c->xn, c->q, c->attn, c->act, c->lin, c->draft_logits, c->row_slot, c->row_pos, c->attn_ws,
+                                         c->attn_ws_bytes, c->partials, c->partials_bytes, c->ssq, c->gemm_arrive, c->xready, c->rope_row_cos,
+                                         c->rope_row_sin});
+    if (cfg.n_drafts >= 2 && cfg.lora_adapters == 0) {       // one more scratch set per further draft group, sized for the drafts
+        int dd = 0, df = 0, dqm = 0, dlin = 0;
+        size_t dhalf = 1, d_ws = 0, d_part = 0;
+        for (int i = 1; i < nm; ++i) {
+            const sd_model_desc& m = ms[i];
+            const int dq = m.n_heads * m.head_dim, nqkv = (m.n_heads + 2 * m.n_kv_heads) * m.head_dim;
+            dd = std::max(dd, (int)m.d_model); df = std::max(df, (int)m.d_ffn); dqm = std::max(dqm, dq);
+            dlin = std::max(dlin, std::max(std::max(nqkv, 2 * (int)m.d_ffn), (int)m.d_model));
+            dhalf = std::max(dhalf, (size_t)m.head_dim / 2);
+            d_ws = std::max(d_ws, attention_split_supported(m.dtype, m.n_heads, m.n_kv_heads, m.head_dim)
+                                      ? attention_split_workspace((int)R, m.n_heads, m.head_dim, cfg.max_ctx)
+                                      : attention_workspace_bytes((int)R, m.n_heads, m.head_dim, cfg.max_ctx));
+            if (m.dtype == SD_BF16) {
+                const int shapes[5][2] = {{nqkv, m.d_model}, {m.d_model, dq}, {2 * m.d_ffn, m.d_model}, {m.d_model, m.d_ffn}, {m.vocab, m.d_model}};
+                for (auto& sh : shapes) d_part = std::max(d_part, gemm_partials_bytes(gemm_geometry(SD_MAX_ROWS, sh[0], sh[1], sm_count(), 0, false, 1)));
+            }
+        }
+        for (int k = 1; k < cfg.n_drafts; ++k) {
+            sd_ctx::ScratchSet s;
+            s.h = (float*)B.take(sizeof(float) * R * dd);
+            s.xn = B.take(4 * R * dd); s.q = B.take(4 * R * dqm); s.attn = B.take(4 * R * dqm); s.act = B.take(4 * R * df);
+            s.lin = (float*)B.take(sizeof(float) * R * dlin);
+            s.draft_logits = (float*)B.take(sizeof(float) * (size_t)SD_MAX_BATCH * ms[0].vocab);
+            s.row_slot = (int32_t*)B.take(sizeof(int32_t) * 2 * R); s.row_pos = (int32_t*)B.take(sizeof(int32_t) * R);
+            s.attn_ws_bytes = d_ws; s.attn_ws = B.take(d_ws);
+            s.partials_bytes = d_part; s.partials = (float*)B.take(d_part);
+            s.ssq = (float*)B.take(sizeof(float) * SD_MAX_ROWS * SSQ_STRIDE);
+            s.gemm_arrive = (uint32_t*)B.take(sizeof(uint32_t) * ARRIVE_WORDS);
+            s.xready = (uint32_t*)B.take(sizeof(uint32_t) * XREADY_WORDS);
+            s.rope_row_cos = (float*)B.take(sizeof(float) * SD_MAX_ROWS * dhalf);
+            s.rope_row_sin = (float*)B.take(sizeof(float) * SD_MAX_ROWS * dhalf);
+            c->sets.push_back(s);
+        }
+    }
     {   // persistent streaming kernel: tagged 64-bit words for up to PASS_ROWS_CAP rows (padded to a multiple of 16)
         const size_t rows_pad = (PASS_ROWS_CAP + 15) & ~15;
         int h_max = 1, hd_max = 8, kvd_max = 8;
@@ -488,6 +538,15 @@ sd_status forward(sd_ctx* c, Model& M, const SeqList& list, const RowPlan& plan,
     }
     CUDA_TRY(prof_mark(c, CAT_NONE));
     return SD_OK;
+}
+
+// Makes scratch set k the one the forward pass uses (pointers are read when a launch is enqueued).
+void use_set(sd_ctx* c, size_t k) {
+    const sd_ctx::ScratchSet& s = c->sets[k];
+    c->h = s.h; c->xn = s.xn; c->q = s.q; c->attn = s.attn; c->act = s.act; c->lin = s.lin; c->draft_logits = s.draft_logits;
+    c->row_slot = s.row_slot; c->row_pos = s.row_pos; c->attn_ws = s.attn_ws; c->attn_ws_bytes = s.attn_ws_bytes;
+    c->partials = s.partials; c->partials_bytes = s.partials_bytes; c->ssq = s.ssq; c->gemm_arrive = s.gemm_arrive; c->xready = s.xready;
+    c->rope_row_cos = s.rope_row_cos; c->rope_row_sin = s.rope_row_sin;
 }
 
 // The next record of the stamp buffer (nullptr when stamps are off or the buffer is full); kind: SD_STAMP_* | detail << 8.
@@ -813,7 +872,14 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     c->n_prompt.assign(cfg->max_seqs, 0);
     c->draft_id.assign(cfg->max_seqs, -1);
     cudaStream_t st = c->st;
-    auto fail = [&](sd_status s) { delete c; return s; };
+    auto fail = [&](sd_status s) {
+        for (cudaStream_t gs : c->group_streams) cudaStreamDestroy(gs);
+        for (cudaEvent_t e : c->ev_join) cudaEventDestroy(e);
+        if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+        delete c;
+        return s;
+    };
+    c->ev_fork = nullptr;
     // state starts at zero; rotary tables are computed here in double and stored as fp32
     if (cudaMemsetAsync(c->S.len, 0, (char*)c->S.status + sizeof(uint32_t) - (char*)c->S.len, st) != cudaSuccess) return fail(SD_ERR_CUDA);
     for (size_t i = 0; i < c->models.size(); ++i) {
@@ -835,7 +901,22 @@ sd_status sd_create(const sd_config* cfg, const sd_model_desc* models, void* cud
     if (cudaMemsetAsync(c->attn_ws, 0, std::min(c->attn_ws_bytes, (size_t)65536), st) != cudaSuccess ||
         cudaMemsetAsync(c->gemm_arrive, 0, sizeof(uint32_t) * ARRIVE_WORDS, st) != cudaSuccess)
         return fail(SD_ERR_CUDA);
+    for (size_t k = 1; k < c->sets.size(); ++k)
+        if (cudaMemsetAsync(c->sets[k].attn_ws, 0, std::min(c->sets[k].attn_ws_bytes, (size_t)65536), st) != cudaSuccess ||
+            cudaMemsetAsync(c->sets[k].gemm_arrive, 0, sizeof(uint32_t) * ARRIVE_WORDS, st) != cudaSuccess)
+            return fail(SD_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SD_ERR_CUDA);
+    c->groups_concurrent = c->sets.size() > 1;
+    c->ev_fork = nullptr;
+    if (c->sets.size() > 1) {
+        if (cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess) return fail(SD_ERR_CUDA);
+        for (size_t k = 1; k < c->sets.size(); ++k) {
+            cudaStream_t gs = nullptr; cudaEvent_t ge = nullptr;
+            if (cudaStreamCreateWithFlags(&gs, cudaStreamNonBlocking) != cudaSuccess || cudaEventCreateWithFlags(&ge, cudaEventDisableTiming) != cudaSuccess)
+                return fail(SD_ERR_CUDA);
+            c->group_streams.push_back(gs); c->ev_join.push_back(ge);
+        }
+    }
     if (cudaMemsetAsync(c->tg_begin, 0, c->tg_end - c->tg_begin, st) != cudaSuccess ||          // no word carries a tag a pass could expect
         cudaMemsetAsync(c->pass_epoch, 0, 2 * sizeof(uint32_t), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
@@ -898,6 +979,9 @@ sd_status sd_destroy(sd_ctx* c) {
     if (!c) return SD_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->st);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    for (cudaStream_t gs : c->group_streams) cudaStreamDestroy(gs);
+    for (cudaEvent_t e : c->ev_join) cudaEventDestroy(e);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     for (auto& m : c->cost_pending) { cudaEventDestroy(m.e0); cudaEventDestroy(m.e1); }
     for (cudaEvent_t e : c->cost_free) cudaEventDestroy(e);
     for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
@@ -1091,7 +1175,7 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
     int bound = 0;
     for (int i = 0; i < n_seq; ++i) bound = std::max(bound, c->len_ub[seqs[i]]);
     KeyBuilder key;
-    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows);
+    key.add(1).add_list(seqs, n_seq).add(gamma).add(x_in).add(x_dev).add(q_dev).add(bound_bucket(bound + gamma)).add(c->force_plain).add(c->stamps_on).add(c->pass_on).add(c->pass_drafts).add(c->pass_max_rows).add(c->groups_concurrent);
     for (int i = 0; i < n_seq; ++i) key.add(c->draft_id[seqs[i]]);
     bound = bound_bucket(bound + gamma) - gamma;
     CostScope cost(c, 0, gamma);
@@ -1108,12 +1192,34 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
         }
     }
     return run_graphed(c, key, [&]() -> sd_status {
+    // Groups of different draft models run side by side: every group after the first gets a stream and a scratch set of
+    // its own, forked from and joined back to the context's stream (inside a capture these become parallel branches).
+    int n_active = 0;
+    for (int k = 0; k < n_groups; ++k) {
+        bool any = false;
+        for (int i = 0; i < n_seq; ++i) any |= shared || c->draft_id[seqs[i]] == k;
+        n_active += any;
+    }
+    const bool side_by_side = c->groups_concurrent && n_active > 1 && !c->prof_on && !(c->pass_on && c->pass_drafts) &&
+                              (int)c->sets.size() >= n_active;
+    cudaStream_t main_st = c->st;
+    struct Restore {                                       // whatever happens below, the context ends on its own stream and scratch set
+        sd_ctx* c; cudaStream_t st;
+        ~Restore() { c->st = st; use_set(c, 0); }
+    } restore{c, main_st};
+    if (side_by_side) CUDA_TRY(cudaEventRecord(c->ev_fork, main_st));
+    int a = 0;                                             // index among the active groups
     for (int k = 0; k < n_groups; ++k) {                    // sequences grouped per routed draft
         SeqList g = all;
         g.n = 0;
         for (int i = 0; i < n_seq; ++i)
             if (shared || c->draft_id[seqs[i]] == k) { g.ids[g.n] = seqs[i]; g.out[g.n] = i; ++g.n; }
         if (g.n == 0) continue;
+        if (side_by_side && a > 0) {
+            use_set(c, (size_t)a);
+            c->st = c->group_streams[a - 1];
+            CUDA_TRY(cudaStreamWaitEvent(c->st, c->ev_fork, 0));
+        }
         Model& M = c->models[1 + k];
         for (int s = 0; s < gamma; ++s) {
             if (s == 0) {
@@ -1125,7 +1231,15 @@ sd_status sd_draft_steps_replay(sd_ctx* c, const int32_t* seqs, int n_seq, int g
             }
             LAUNCH(CAT_SAMPLING, launch_draft_sample(c->draft_logits, c->S, g, V, c->cfg.temperature, c->cfg.seed, s, gamma, q_dev, x_dev, c->st));
         }
+        if (side_by_side && a > 0) {
+            CUDA_TRY(cudaEventRecord(c->ev_join[a - 1], c->st));
+            c->st = main_st;
+            use_set(c, 0);
+        }
+        ++a;
     }
+    if (side_by_side)
+        for (int j = 1; j < a; ++j) CUDA_TRY(cudaStreamWaitEvent(main_st, c->ev_join[j - 1], 0));
     return SD_OK;
     });
 }
@@ -1376,6 +1490,12 @@ sd_status sd_seq_alpha(sd_ctx* c, int seq, double* alpha_sum_out, int64_t* judge
     CUDA_TRY(cudaMemcpyAsync(alpha_sum_out, c->S.alpha_sum + seq, sizeof(double), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaMemcpyAsync(judged_out, c->S.judged + seq, sizeof(int64_t), cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
+    return SD_OK;
+}
+
+sd_status sd_use_draft_streams(sd_ctx* c, int on) {
+    if (!c) return SD_ERR_INVALID_ARG;
+    c->groups_concurrent = on != 0 && c->sets.size() > 1;
     return SD_OK;
 }
 

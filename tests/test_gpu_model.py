@@ -331,6 +331,33 @@ def test_batched_ragged_sequences_match_single_sequence_runs(sd):
     ctx.close()
 
 
+def test_draft_groups_side_by_side_give_what_they_give_one_after_the_other(sd):
+    """Sequences routed to different draft models: their draft passes run on streams of their own by default; the drafts
+    and their distributions are bit for bit those of the group-after-group order, with and without captured graphs."""
+    V, gamma = 4096, 4
+    ctx, om = _build(sd, SMALL_BF16, [SMALL_BF16_DRAFT, SMALL_BF16_DRAFT, SMALL_BF16_DRAFT], "bf16", 1.0, 23, max_seqs=6, max_ctx=128)
+    prompts = [synth.make_prompt(V, n, seed=14, seq=i) for i, n in enumerate([17, 40, 33, 25, 58, 19])]
+    route = [2, 0, 1, 0, 2, 1]
+    outs = []
+    for graphs, streams in ((1, 1), (1, 0), (0, 1), (0, 0)):
+        ctx.sd_use_graphs(graphs); ctx.sd_use_draft_streams(streams)
+        for s, p in enumerate(prompts):
+            ctx.sd_seq_begin(s, p, 300 + s)
+        ctx.sd_route_prompt(list(range(6)), forced_task=route)
+        ctx.sd_prefill(list(range(6)))
+        x = torch.zeros((6, gamma), dtype=torch.int32, device=DEV); q = torch.zeros((6, gamma, V), dtype=torch.float32, device=DEV)
+        for _ in range(2):                                   # the second call replays the captured graph
+            ctx.sd_draft_steps(list(range(6)), gamma, x, q)
+        outs.append((x.cpu().clone(), q.cpu().clone()))
+    for x, q in outs[1:]:
+        assert torch.equal(x, outs[0][0]) and torch.equal(q, outs[0][1])
+    for s, p in enumerate(prompts):                          # and they are the oracle's
+        _, _, tr = oracle.spec_decode(om[0], om[1 + route[s]], p, gamma + 1, gamma, 1.0, 23, seq_id=300 + s, trace_iters=1, trace_probs=True)
+        assert np.abs(outs[0][1][s].numpy().astype(np.float64) - tr["q"][0]).max() <= TOL["bf16"]["probs"]
+    assert ctx.sd_device_status() == 0
+    ctx.close()
+
+
 def test_batch16_launch_configuration_at_full_width(sd):
     """The batched benchmark's launch configuration (16 sequences x (gamma + 1) = 96 verify rows in one call: wide-N
     GEMMs, fused steps in several row batches, the several-CTAs-per-SM form of attention, ragged contexts) at the
