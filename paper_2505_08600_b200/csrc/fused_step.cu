@@ -38,7 +38,6 @@ template <int MODE, int MB, int CB, bool HL = false, bool LORA = false, bool XR 
 __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, const float* __restrict__ partials,
                                                     uint32_t* __restrict__ arrive, uint32_t* status) {
     __shared__ StepShared<MB> sh;
-    __shared__ int tile_seen;
     const int mode = MODE < 0 ? ep.mode : MODE;
     pdl_launch_dependents();
     const int et = threadIdx.x, lane = et & 31, warp = et >> 5;
@@ -95,23 +94,20 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     // The pieces come from the GEMM before (the rows' sums of squares from kernels further back, long finished).
     // With arrival words the CTA starts as soon as its own tile is complete; otherwise when the GEMM's grid has retired.
     if (arrive) {
-        if (et == 0) {
-            const uint32_t need = i_last - i_first + 1u;
-            uint32_t seen = 0;
-            const uint64_t t0 = global_ns(), limit = ep.poll_ns ? ep.poll_ns : 200000000ull;
-            for (uint32_t spin = 0;; ++spin) {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrive + tile) : "memory");
-                if (seen >= need) break;
-                if ((spin & 63u) == 63u && global_ns() - t0 > limit) break;      // (0.2 s unless told otherwise): give up polling
-            }
-            tile_seen = seen >= need;
+        // every warp watches the tile's word for itself (one request per warp and poll): no barrier between the arrival
+        // of the last piece and the loads below
+        const uint32_t need = i_last - i_first + 1u;
+        uint32_t seen = 0;
+        const uint64_t t0 = global_ns(), limit = ep.poll_ns ? ep.poll_ns : 200000000ull;
+        for (uint32_t spin = 0;; ++spin) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrive + tile) : "memory");
+            if (seen >= need) break;
+            if ((spin & 63u) == 63u && global_ns() - t0 > limit) break;      // (0.2 s unless told otherwise): give up polling
         }
-        __syncthreads();
-        if (!tile_seen) {                          // not expected: wait for the whole grid instead, and say so
+        if (seen < need) {                         // not expected: wait for the whole grid instead, and say so
             pdl_wait();
-            if (et == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
+            if (lane == 0 && status) atomicOr(status, SD_DEV_WAIT_EXPIRED);
         }
-        if (et == 0) arrive[tile] = 0u;            // left at zero for the next GEMM (which starts counting only after this kernel has finished)
     } else {
         pdl_wait();
     }
@@ -340,6 +336,10 @@ __global__ void __launch_bounds__(128) k_fused_step(GemmGeom g, Epilogue ep, con
     default: break;
     }
     if (et == 0) stamp_pair(ep.stamp, ST_DONE_FIRST);
+    if (arrive) {                                 // left at zero for the next pass (every warp is past its polls by now)
+        __syncthreads();
+        if (et == 0) arrive[tile] = 0u;
+    }
     if (XR && ep.xready) {                        // everything this CTA writes is written: the next GEMM may load the tile's columns
         __syncthreads();                          // (orders the CTA's stores before thread 0's release, which is cumulative)
         if (et == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ep.xready + tile) : "memory");
